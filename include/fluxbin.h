@@ -1,0 +1,188 @@
+/*
+ * fluxbin.h -- C-ABI of the B200 (sm_100a) FluxBin decode linear layer.
+ *
+ * The layer computes  y = X * What^T  for a batch X of B activation vectors, where What is the
+ * multi-binary-base weight of the paper (Def. 3.1 / Eq. 3 with one row scale per group of g
+ * columns, plus the salient refinement of Eq. 9 on the columns listed in sal_idx):
+ *
+ *   What[i][j] = sum_{k<Kb} ar[k][i][j/g] * ac[k][j] * B[k][i][j]
+ *              + sum_{k<Ks} [j = sal_idx[v]] * asr[k][i][j/g] * ascd[k][v] * Bsd[k][i][v]
+ *
+ * evaluated the LUT way (Sec. 3.2, Eq. 10-15): column scales are fused into the activations
+ * (Eq. 11, Eq. 14), one table of 2^8 signed partial sums is built per 8-column sub-vector in
+ * shared memory, packed weight bytes index the tables (Eq. 15), row scales are applied per
+ * (row, group), and the salient columns are stored as dense "virtual columns" (VCM, Eq. 12-13)
+ * so the salient branch runs through the same lookup loop.
+ *
+ * Conventions
+ *   - M = output rows, N = input columns (the paper's M x N).
+ *   - All scales and activations are IEEE fp16 bit patterns (uint16_t).  Arithmetic is fp32.
+ *   - Bit 1 means +1, bit 0 means -1 (the 2b-1 of Eq. 14).
+ *   - "host" / "device" is stated for every pointer.  The library never allocates device
+ *     memory: packed weights, activations, outputs and workspace are owned by the caller.
+ *   - Every entry point returns a status; none throws, aborts or prints.
+ *   - Restrictions: N % 32 == 0, g % 32 == 0, N % g == 0, N <= 65536 (16-bit column index
+ *     metadata, as in the paper's storage model), 1 <= Kb <= 4, 0 <= Ks <= 4, M >= 1.
+ */
+#ifndef FLUXBIN_H
+#define FLUXBIN_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct fluxbin_weight fluxbin_weight_t; /* opaque host object describing one packed layer */
+
+typedef enum {
+    FLUXBIN_OK = 0,
+    FLUXBIN_ERR_NULL = 1,             /* a required pointer is NULL */
+    FLUXBIN_ERR_SHAPE = 2,            /* M/N/g violate the restrictions above */
+    FLUXBIN_ERR_RANGE = 3,            /* Kb, Ks, B or a leading dimension out of range */
+    FLUXBIN_ERR_SALIENT_MAP = 4,      /* sal_idx not strictly ascending or out of [0, N) */
+    FLUXBIN_ERR_BUFFER_TOO_SMALL = 5, /* packed buffer or workspace smaller than required */
+    FLUXBIN_ERR_ALIGNMENT = 6,        /* a device pointer is not 16-byte aligned */
+    FLUXBIN_ERR_UNSUPPORTED = 7,      /* valid request this build cannot run (e.g. wrong GPU) */
+    FLUXBIN_ERR_CUDA = 8,             /* a CUDA call failed; see fluxbin_last_cuda_error() */
+    FLUXBIN_ERR_FORMAT = 9            /* packed buffer does not carry a valid header */
+} fluxbin_status_t;
+
+/*
+ * One layer in canonical interchange layout (the problem statement of Sec. 3.2: parameter sets
+ * Theta_k = {B, ar, ac}, Phi_k = {Bs, asr, asc} and the salient set I_sal).  All pointers are
+ * HOST memory, borrowed for the duration of the call.
+ */
+typedef struct {
+    int32_t M, N;      /* output rows, input columns */
+    int32_t Kb, Ks;    /* global bases; extra bases on the salient columns (0 = no salient branch) */
+    int32_t g;         /* columns per row-scale group; g == N gives one scale per row */
+    int32_t n_sal;     /* number of salient columns, 0..N */
+    const uint32_t *bits;          /* [Kb][M][N/32]; bit (j%32) of word j/32 set <=> B[k][i][j] = +1 */
+    const uint16_t *row_scale;     /* [Kb][M][N/g] */
+    const uint16_t *col_scale;     /* [Kb][N] */
+    const int32_t  *sal_idx;       /* [n_sal] strictly ascending original column of virtual column v */
+    const uint32_t *sal_bits;      /* [Ks][M][ceil(n_sal/32)] dense VCM matrix Bsd (Eq. 12): virtual
+                                      column v is bit v%32 of word v/32; bits past n_sal must be 0 */
+    const uint16_t *sal_row_scale; /* [Ks][M][N/g]; virtual column v uses group sal_idx[v]/g */
+    const uint16_t *sal_col_scale; /* [Ks][n_sal] gathered column scale ascd (Eq. 13) */
+} fluxbin_layer_desc_t;
+
+/*
+ * Bytes of the private packed representation of a layer (bit-packed bases in the kernel's tiled
+ * order, row scales, fused column-scale/index table, salient map).  0 if the dimensions are
+ * invalid.  Reads the dimension fields and, when it is non-NULL, sal_idx (the salient padding
+ * depends on how the salient columns fall into row-scale groups); with sal_idx NULL the result
+ * is an upper bound over all salient maps of that size.  The figure is the storage model of the
+ * paper's appendix (S_base + S_sal) plus padding to the kernel's tiles.
+ */
+size_t fluxbin_packed_size(const fluxbin_layer_desc_t *desc);
+
+/*
+ * Validate a descriptor without packing it (dimension rules and the salient map).
+ */
+fluxbin_status_t fluxbin_validate(const fluxbin_layer_desc_t *desc);
+
+/*
+ * Pack into a HOST buffer of at least fluxbin_packed_size(desc) bytes (VCM, Def. 3.5: the
+ * salient columns become dense virtual columns; bits are re-tiled for the lookup kernel).
+ * Uses no GPU.  The result is position independent: copy it anywhere, then fluxbin_attach.
+ */
+fluxbin_status_t fluxbin_pack_host(const fluxbin_layer_desc_t *desc, void *h_packed, size_t bytes);
+
+/*
+ * Exact inverse of fluxbin_pack_host.  `out->M ... out->n_sal` are filled in; every non-NULL
+ * array pointer of `out` must address caller-allocated HOST memory of the canonical size and is
+ * written (the const qualifiers of the struct are ignored).  Bits, fp16 bit patterns and
+ * indices round-trip bit-exactly.
+ */
+fluxbin_status_t fluxbin_unpack_host(const void *h_packed, size_t bytes, fluxbin_layer_desc_t *out);
+
+/*
+ * Read only the dimensions (M, N, Kb, Ks, g, n_sal) of a packed HOST buffer; pointers untouched.
+ */
+fluxbin_status_t fluxbin_packed_dims(const void *h_packed, size_t bytes, fluxbin_layer_desc_t *out);
+
+/*
+ * Pack `desc` and copy the result into the caller-owned DEVICE buffer d_packed (16-byte aligned,
+ * d_bytes >= fluxbin_packed_size).  The copy is issued on `cuda_stream` (a cudaStream_t, NULL =
+ * default stream) and the stream is synchronised before returning.  On success *out receives a
+ * handle that borrows d_packed; release it with fluxbin_free (which never frees d_packed).
+ */
+fluxbin_status_t fluxbin_pack(const fluxbin_layer_desc_t *desc, void *d_packed, size_t d_bytes,
+                              void *cuda_stream, fluxbin_weight_t **out);
+
+/*
+ * Make a handle for a DEVICE buffer that already holds a packed layer (e.g. after relocating
+ * it).  `h_header` is HOST memory holding at least the first 256 bytes of that packed layer.
+ */
+fluxbin_status_t fluxbin_attach(const void *h_header, size_t header_bytes, void *d_packed, size_t d_bytes,
+                                fluxbin_weight_t **out);
+
+/*
+ * Copy the packed layer back from the device and unpack it (see fluxbin_unpack_host).
+ * Synchronises `cuda_stream`.
+ */
+fluxbin_status_t fluxbin_unpack(const fluxbin_weight_t *w, fluxbin_layer_desc_t *host_out, void *cuda_stream);
+
+/* Dimensions of a handle (pointers of `out` untouched). */
+fluxbin_status_t fluxbin_weight_dims(const fluxbin_weight_t *w, fluxbin_layer_desc_t *out);
+
+/*
+ * DEVICE workspace bytes fluxbin_linear needs for batch size B with this layer: fp32 split-K
+ * accumulators for up to 4 batch rows at a time plus one arrival counter per tile of output
+ * rows (stage (iii) "reduction" of Sec. 3.2).  The workspace must be zeroed once with
+ * fluxbin_workspace_init before its first use; every call leaves it zeroed again, so one
+ * workspace of the maximum size can serve any sequence of stream-ordered calls.
+ */
+size_t fluxbin_workspace_size(const fluxbin_weight_t *w, int32_t B);
+
+/* Zero a DEVICE workspace (asynchronous on cuda_stream). */
+fluxbin_status_t fluxbin_workspace_init(void *d_workspace, size_t bytes, void *cuda_stream);
+
+/*
+ * y[b][i] = sum_j What[i][j] * x[b][j]   for b < B, i < M          (Eq. 10, computed per Eq. 11-15)
+ *
+ *   d_x   DEVICE fp16 [B][ldx], ldx >= N, 16-byte aligned base
+ *   d_y   DEVICE [B][ldy], ldy >= M; fp32 if y_is_fp32 != 0 else fp16 (round-to-nearest-even of
+ *         the fp32 result); every y[b][0..M) is overwritten
+ *   d_workspace / ws_bytes   see fluxbin_workspace_size
+ *
+ * Asynchronous on cuda_stream; performs no allocation and no synchronisation, so calls can be
+ * captured into a CUDA graph.  B >= 1 arbitrary (processed in chunks of up to 4 vectors).  Calls
+ * sharing a workspace must be ordered on one stream.  Accumulation is fp32 with fp32 atomics
+ * across K slices, so results may differ in the last bits from run to run.
+ */
+fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint16_t *d_x, int32_t B, int64_t ldx,
+                                void *d_y, int32_t y_is_fp32, int64_t ldy,
+                                void *d_workspace, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Test hook for the LUT identity (Eq. 14): build the tables of table-set `pair` (32 tables:
+ * two runs of 16 consecutive 8-column sub-vectors) for activation row 0 of d_x exactly as the
+ * kernel does, and write them as fp32 [32][256] to DEVICE d_tables.  h_cols (HOST, may be NULL)
+ * receives the 32*8 source column indices and h_alpha the 32*8 fused column scales (fp16 bits)
+ * the tables were built from, in table order.
+ */
+fluxbin_status_t fluxbin_debug_tables(const fluxbin_weight_t *w, const uint16_t *d_x, int32_t pair,
+                                      float *d_tables, int32_t *h_cols, uint16_t *h_alpha, void *cuda_stream);
+
+/* Number of table sets (global + salient) of a layer; -1 on NULL. */
+int32_t fluxbin_num_table_sets(const fluxbin_weight_t *w);
+
+/* Kernel launches fluxbin_linear issues for this layer and batch size (for launch accounting). */
+int32_t fluxbin_num_launches(const fluxbin_weight_t *w, int32_t B);
+
+/* Release the host object (never touches device memory).  NULL is allowed. */
+void fluxbin_free(fluxbin_weight_t *w);
+
+const char *fluxbin_status_string(fluxbin_status_t s);
+
+/* The cudaError_t of the most recent FLUXBIN_ERR_CUDA on the calling thread (0 if none). */
+int fluxbin_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FLUXBIN_H */

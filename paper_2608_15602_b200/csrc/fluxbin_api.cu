@@ -1,0 +1,299 @@
+// C-ABI entry points that touch the GPU: pack-to-device, attach, unpack-from-device, workspace,
+// fluxbin_linear (launch only: no allocation, no synchronisation) and the table test hook.
+#include "fluxbin_internal.h"
+#include "fluxbin_kernel.cuh"
+
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+#include <new>
+
+using namespace fb;
+
+static thread_local int g_last_cuda_error = 0;
+
+static fluxbin_status_t cuda_fail(cudaError_t e)
+{
+    g_last_cuda_error = (int)e;
+    (void)cudaGetLastError();
+    return FLUXBIN_ERR_CUDA;
+}
+#define FB_CUDA(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return cuda_fail(e_); } while (0)
+
+extern "C" int fluxbin_last_cuda_error(void) { return g_last_cuda_error; }
+
+extern "C" const char *fluxbin_status_string(fluxbin_status_t s)
+{
+    switch (s) {
+    case FLUXBIN_OK: return "ok";
+    case FLUXBIN_ERR_NULL: return "null pointer";
+    case FLUXBIN_ERR_SHAPE: return "unsupported shape (need N%32==0, g%32==0, N%g==0, N<=65536, M>=1)";
+    case FLUXBIN_ERR_RANGE: return "argument out of range";
+    case FLUXBIN_ERR_SALIENT_MAP: return "salient map not strictly ascending in [0,N)";
+    case FLUXBIN_ERR_BUFFER_TOO_SMALL: return "buffer too small";
+    case FLUXBIN_ERR_ALIGNMENT: return "device pointer not 16-byte aligned";
+    case FLUXBIN_ERR_UNSUPPORTED: return "unsupported on this device/build";
+    case FLUXBIN_ERR_CUDA: return "CUDA error";
+    case FLUXBIN_ERR_FORMAT: return "not a packed FluxBin layer";
+    }
+    return "unknown status";
+}
+
+// ---- per-device one-time set-up: SM count, shared-memory opt-in, dynamic-smem base probe --------
+
+namespace {
+
+__device__ uint32_t g_smem_base_probe;
+
+struct DeviceInfo {
+    bool ready = false;
+    bool ok = false;
+    int num_sms = 0;
+};
+constexpr int kMaxDevices = 64;
+DeviceInfo g_dev[kMaxDevices];
+std::mutex g_dev_mutex;
+
+template <int S0, int S1, int BT> cudaError_t opt_in()
+{
+    return cudaFuncSetAttribute(fbk::fluxbin_linear_kernel<S0, S1, BT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)fbk::smem_bytes<BT>());
+}
+template <int BT> cudaError_t opt_in_bt()
+{
+    cudaError_t e;
+    if ((e = opt_in<16, 16, BT>()) != cudaSuccess) return e;
+    if ((e = opt_in<16, 1, BT>()) != cudaSuccess) return e;
+    if ((e = opt_in<8, 1, BT>()) != cudaSuccess) return e;
+    if ((e = opt_in<4, 1, BT>()) != cudaSuccess) return e;
+    return cudaSuccess;
+}
+
+fluxbin_status_t device_setup(int dev, int *num_sms)
+{
+    if (dev < 0 || dev >= kMaxDevices) return FLUXBIN_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
+    DeviceInfo &d = g_dev[dev];
+    if (!d.ready) {
+        int major = 0, sms = 0;
+        FB_CUDA(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+        FB_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        d.num_sms = sms;
+        d.ok = false;
+        if (major == 10) {
+            FB_CUDA(opt_in_bt<1>());
+            FB_CUDA(opt_in_bt<2>());
+            FB_CUDA(opt_in_bt<4>());
+            FB_CUDA(cudaFuncSetAttribute(fbk::fluxbin_debug_tables_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)fbk::smem_bytes<1>()));
+            FB_CUDA(cudaFuncSetAttribute(fbk::fluxbin_smem_base_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)fbk::smem_bytes<1>()));
+            // where does dynamic shared memory start?  the tables need the window below 0x10000
+            uint32_t *probe = nullptr;
+            FB_CUDA(cudaGetSymbolAddress((void **)&probe, g_smem_base_probe));
+            fbk::fluxbin_smem_base_kernel<<<1, 32, fbk::smem_bytes<1>(), 0>>>(probe);
+            FB_CUDA(cudaGetLastError());
+            uint32_t base = 0xffffffffu;
+            FB_CUDA(cudaMemcpy(&base, probe, sizeof(base), cudaMemcpyDeviceToHost));
+            d.ok = (base + fbk::kSmallBytes <= fbk::kTabBase);
+        }
+        d.ready = true;
+    }
+    if (num_sms) *num_sms = d.num_sms;
+    return d.ok ? FLUXBIN_OK : FLUXBIN_ERR_UNSUPPORTED;
+}
+
+fluxbin_status_t make_handle(const FbHeader &h, void *d_packed, size_t d_bytes, fluxbin_weight_t **out)
+{
+    if (((uintptr_t)d_packed & 15) != 0) return FLUXBIN_ERR_ALIGNMENT;
+    if (d_bytes < h.total_bytes) return FLUXBIN_ERR_BUFFER_TOO_SMALL;
+    int dev = 0, sms = 0;
+    FB_CUDA(cudaGetDevice(&dev));
+    fluxbin_status_t st = device_setup(dev, &sms);
+    if (st != FLUXBIN_OK) return st;
+    fluxbin_weight_t *w = new (std::nothrow) fluxbin_weight_t;
+    if (!w) return FLUXBIN_ERR_UNSUPPORTED;
+    w->h = h;
+    w->d_packed = d_packed;
+    w->d_bytes = d_bytes;
+    w->device = dev;
+    w->num_sms = sms;
+    w->tile_rb = 16;
+    if ((h.nrb + w->tile_rb - 1) / w->tile_rb > fbk::kMaxTiles) w->tile_rb = (h.nrb + fbk::kMaxTiles - 1) / fbk::kMaxTiles;
+    w->ntiles = (h.nrb + w->tile_rb - 1) / w->tile_rb;
+    *out = w;
+    return FLUXBIN_OK;
+}
+
+} // namespace
+
+extern "C" fluxbin_status_t fluxbin_pack(const fluxbin_layer_desc_t *desc, void *d_packed, size_t d_bytes,
+                                         void *cuda_stream, fluxbin_weight_t **out)
+{
+    if (!out || !d_packed) return FLUXBIN_ERR_NULL;
+    *out = nullptr;
+    fluxbin_status_t st = fluxbin_validate(desc);
+    if (st != FLUXBIN_OK) return st;
+    size_t bytes = fluxbin_packed_size(desc);
+    if (bytes == 0) return FLUXBIN_ERR_SHAPE;
+    if (d_bytes < bytes) return FLUXBIN_ERR_BUFFER_TOO_SMALL;
+    if (((uintptr_t)d_packed & 15) != 0) return FLUXBIN_ERR_ALIGNMENT;
+    void *host = std::malloc(bytes);
+    if (!host) return FLUXBIN_ERR_UNSUPPORTED;
+    st = fluxbin_pack_host(desc, host, bytes);
+    if (st == FLUXBIN_OK) {
+        FbHeader h;
+        std::memcpy(&h, host, sizeof(h));
+        cudaStream_t s = (cudaStream_t)cuda_stream;
+        cudaError_t e = cudaMemcpyAsync(d_packed, host, bytes, cudaMemcpyHostToDevice, s);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+        if (e != cudaSuccess) st = cuda_fail(e);
+        else st = make_handle(h, d_packed, d_bytes, out);
+    }
+    std::free(host);
+    return st;
+}
+
+extern "C" fluxbin_status_t fluxbin_attach(const void *h_header, size_t header_bytes, void *d_packed, size_t d_bytes,
+                                           fluxbin_weight_t **out)
+{
+    if (!out || !d_packed) return FLUXBIN_ERR_NULL;
+    *out = nullptr;
+    FbHeader h;
+    fluxbin_status_t st = check_header(h_header, header_bytes, h);
+    if (st != FLUXBIN_OK) return st;
+    return make_handle(h, d_packed, d_bytes, out);
+}
+
+extern "C" fluxbin_status_t fluxbin_unpack(const fluxbin_weight_t *w, fluxbin_layer_desc_t *host_out, void *cuda_stream)
+{
+    if (!w || !host_out) return FLUXBIN_ERR_NULL;
+    size_t bytes = (size_t)w->h.total_bytes;
+    void *host = std::malloc(bytes);
+    if (!host) return FLUXBIN_ERR_UNSUPPORTED;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    cudaError_t e = cudaMemcpyAsync(host, w->d_packed, bytes, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    fluxbin_status_t st = (e == cudaSuccess) ? fluxbin_unpack_host(host, bytes, host_out) : cuda_fail(e);
+    std::free(host);
+    return st;
+}
+
+extern "C" fluxbin_status_t fluxbin_weight_dims(const fluxbin_weight_t *w, fluxbin_layer_desc_t *out)
+{
+    if (!w || !out) return FLUXBIN_ERR_NULL;
+    out->M = w->h.M; out->N = w->h.N; out->Kb = w->h.Kb; out->Ks = w->h.Ks; out->g = w->h.g; out->n_sal = w->h.n_sal;
+    return FLUXBIN_OK;
+}
+
+extern "C" void fluxbin_free(fluxbin_weight_t *w) { delete w; }
+
+extern "C" int32_t fluxbin_num_table_sets(const fluxbin_weight_t *w) { return w ? w->h.npairs[0] + w->h.npairs[1] : -1; }
+
+extern "C" int32_t fluxbin_num_launches(const fluxbin_weight_t *w, int32_t B)
+{
+    if (!w || B < 1) return -1;
+    return (B + 3) / 4;      // chunks of up to 4 vectors (the last chunk runs as 1, 2 or 4)
+}
+
+// ---- workspace ----------------------------------------------------------------------------------
+
+static size_t acc_bytes(const fluxbin_weight_t *w, int bt) { return ((size_t)bt * w->h.Mpad * 4 + 255) / 256 * 256; }
+
+extern "C" size_t fluxbin_workspace_size(const fluxbin_weight_t *w, int32_t B)
+{
+    if (!w || B < 1) return 0;
+    int bt = B >= 3 ? 4 : B;
+    return acc_bytes(w, bt) + ((size_t)w->ntiles * 4 + 255) / 256 * 256;
+}
+
+extern "C" fluxbin_status_t fluxbin_workspace_init(void *d_workspace, size_t bytes, void *cuda_stream)
+{
+    if (!d_workspace) return FLUXBIN_ERR_NULL;
+    FB_CUDA(cudaMemsetAsync(d_workspace, 0, bytes, (cudaStream_t)cuda_stream));
+    return FLUXBIN_OK;
+}
+
+// ---- the layer ------------------------------------------------------------------------------------
+
+template <int S0, int S1, int BT>
+static cudaError_t launch(const fbk::LinearParams &p, int grid, cudaStream_t s)
+{
+    fbk::fluxbin_linear_kernel<S0, S1, BT><<<grid, fbk::kThreads, fbk::smem_bytes<BT>(), s>>>(p);
+    return cudaGetLastError();
+}
+
+template <int BT> static cudaError_t launch_bt(const fluxbin_weight_t *w, const fbk::LinearParams &p, int grid, cudaStream_t s)
+{
+    const int s0 = w->h.sps[0], s1 = w->h.sps[1];
+    if (s0 == 16 && s1 == 16) return launch<16, 16, BT>(p, grid, s);
+    if (s0 == 16) return launch<16, 1, BT>(p, grid, s);
+    if (s0 == 8) return launch<8, 1, BT>(p, grid, s);
+    return launch<4, 1, BT>(p, grid, s);
+}
+
+extern "C" fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint16_t *d_x, int32_t B, int64_t ldx,
+                                           void *d_y, int32_t y_is_fp32, int64_t ldy,
+                                           void *d_workspace, size_t ws_bytes, void *cuda_stream)
+{
+    if (!w || !d_x || !d_y || !d_workspace) return FLUXBIN_ERR_NULL;
+    if (B < 1 || ldx < w->h.N || ldy < w->h.M) return FLUXBIN_ERR_RANGE;
+    if ((((uintptr_t)d_x) & 15) || (((uintptr_t)d_y) & 15) || (((uintptr_t)d_workspace) & 15)) return FLUXBIN_ERR_ALIGNMENT;
+    if (ws_bytes < fluxbin_workspace_size(w, B)) return FLUXBIN_ERR_BUFFER_TOO_SMALL;
+    // a 16-segment salient region only exists with a single scale group, where sps[0] is 16 too
+    if (w->h.sps[1] == 16 && w->h.sps[0] != 16) return FLUXBIN_ERR_FORMAT;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+
+    fbk::LinearParams p;
+    p.packed = (const uint8_t *)w->d_packed;
+    p.ldx = ldx;
+    p.ldy = ldy;
+    p.y_fp32 = y_is_fp32 != 0;
+    p.M = w->h.M; p.Mpad = w->h.Mpad; p.nrb = w->h.nrb;
+    p.npairs[0] = w->h.npairs[0]; p.npairs[1] = w->h.npairs[1];
+    p.item_bytes[0] = w->h.item_bytes[0]; p.item_bytes[1] = w->h.item_bytes[1];
+    p.off_coldesc = w->h.off_coldesc; p.off_items[0] = w->h.off_items[0]; p.off_items[1] = w->h.off_items[1];
+    p.tile_rb = w->tile_rb; p.ntiles = w->ntiles;
+    p.acc = (float *)d_workspace;
+    const int bt_ws = B >= 3 ? 4 : B;
+    p.tickets = (unsigned *)((uint8_t *)d_workspace + acc_bytes(w, bt_ws));
+
+    const long long items = (long long)(p.npairs[0] + p.npairs[1]) * p.nrb;
+    const int grid = (int)(items < w->num_sms ? items : w->num_sms);
+
+    const size_t ysz = y_is_fp32 ? 4 : 2;
+    for (int b0 = 0; b0 < B; b0 += 4) {
+        const int nb = (B - b0 < 4) ? B - b0 : 4;
+        p.x = d_x + (int64_t)b0 * ldx;
+        p.y = (uint8_t *)d_y + (size_t)b0 * ldy * ysz;
+        p.nb = nb;
+        cudaError_t e;
+        if (nb == 1) e = launch_bt<1>(w, p, grid, s);
+        else if (nb == 2) e = launch_bt<2>(w, p, grid, s);
+        else e = launch_bt<4>(w, p, grid, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    return FLUXBIN_OK;
+}
+
+extern "C" fluxbin_status_t fluxbin_debug_tables(const fluxbin_weight_t *w, const uint16_t *d_x, int32_t pair,
+                                                 float *d_tables, int32_t *h_cols, uint16_t *h_alpha, void *cuda_stream)
+{
+    if (!w || !d_x || !d_tables) return FLUXBIN_ERR_NULL;
+    const int np = w->h.npairs[0] + w->h.npairs[1];
+    if (pair < 0 || pair >= np) return FLUXBIN_ERR_RANGE;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    const uint8_t *desc = (const uint8_t *)w->d_packed + w->h.off_coldesc + (size_t)pair * FB_PAIR_DESC_BYTES;
+    fbk::fluxbin_debug_tables_kernel<<<1, fbk::kThreads, fbk::smem_bytes<1>(), s>>>(desc, d_x, d_tables);
+    FB_CUDA(cudaGetLastError());
+    if (h_cols || h_alpha) {
+        uint16_t tmp[512];
+        FB_CUDA(cudaMemcpyAsync(tmp, desc, sizeof(tmp), cudaMemcpyDeviceToHost, s));
+        FB_CUDA(cudaStreamSynchronize(s));
+        for (int i = 0; i < 256; ++i) {
+            if (h_cols) h_cols[i] = tmp[2 * i];
+            if (h_alpha) h_alpha[i] = tmp[2 * i + 1];
+        }
+    }
+    return FLUXBIN_OK;
+}

@@ -1,0 +1,222 @@
+"""ctypes binding of the FluxBin C-ABI (include/fluxbin.h).  Argument marshalling only.
+
+Every step of the layer runs in the CUDA library; there is no Python or CPU fallback.  The
+library must have been built (python -m paper_2608_15602_b200.build); loading fails loudly
+otherwise.  Device buffers are passed as integer addresses (e.g. torch.Tensor.data_ptr()).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+from .build import LIB_PATH
+
+STATUS_OK = 0
+
+
+class FluxBinError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = _lib().fluxbin_status_string(status).decode()
+        extra = f" (cudaError {_lib().fluxbin_last_cuda_error()})" if status == 8 else ""
+        super().__init__(f"{where}: {msg}{extra}")
+
+
+class LayerDesc(ctypes.Structure):
+    _fields_ = [("M", ctypes.c_int32), ("N", ctypes.c_int32), ("Kb", ctypes.c_int32), ("Ks", ctypes.c_int32),
+                ("g", ctypes.c_int32), ("n_sal", ctypes.c_int32),
+                ("bits", ctypes.c_void_p), ("row_scale", ctypes.c_void_p), ("col_scale", ctypes.c_void_p),
+                ("sal_idx", ctypes.c_void_p), ("sal_bits", ctypes.c_void_p), ("sal_row_scale", ctypes.c_void_p),
+                ("sal_col_scale", ctypes.c_void_p)]
+
+
+EXPORTS = ["fluxbin_packed_size", "fluxbin_validate", "fluxbin_pack_host", "fluxbin_unpack_host",
+           "fluxbin_packed_dims", "fluxbin_pack", "fluxbin_attach", "fluxbin_unpack", "fluxbin_weight_dims",
+           "fluxbin_workspace_size", "fluxbin_workspace_init", "fluxbin_linear", "fluxbin_debug_tables",
+           "fluxbin_num_table_sets", "fluxbin_num_launches", "fluxbin_free", "fluxbin_status_string",
+           "fluxbin_last_cuda_error"]
+
+_LIB = None
+
+
+def _lib():
+    global _LIB
+    if _LIB is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2608_15602_b200.build` "
+                              "(there is no CPU fallback)")
+        lib = ctypes.CDLL(LIB_PATH)
+        vp, sz, i32, i64 = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int32, ctypes.c_int64
+        dp = ctypes.POINTER(LayerDesc)
+        lib.fluxbin_packed_size.restype, lib.fluxbin_packed_size.argtypes = sz, [dp]
+        lib.fluxbin_validate.restype, lib.fluxbin_validate.argtypes = ctypes.c_int, [dp]
+        lib.fluxbin_pack_host.restype, lib.fluxbin_pack_host.argtypes = ctypes.c_int, [dp, vp, sz]
+        lib.fluxbin_unpack_host.restype, lib.fluxbin_unpack_host.argtypes = ctypes.c_int, [vp, sz, dp]
+        lib.fluxbin_packed_dims.restype, lib.fluxbin_packed_dims.argtypes = ctypes.c_int, [vp, sz, dp]
+        lib.fluxbin_pack.restype, lib.fluxbin_pack.argtypes = ctypes.c_int, [dp, vp, sz, vp, ctypes.POINTER(vp)]
+        lib.fluxbin_attach.restype, lib.fluxbin_attach.argtypes = ctypes.c_int, [vp, sz, vp, sz, ctypes.POINTER(vp)]
+        lib.fluxbin_unpack.restype, lib.fluxbin_unpack.argtypes = ctypes.c_int, [vp, dp, vp]
+        lib.fluxbin_weight_dims.restype, lib.fluxbin_weight_dims.argtypes = ctypes.c_int, [vp, dp]
+        lib.fluxbin_workspace_size.restype, lib.fluxbin_workspace_size.argtypes = sz, [vp, i32]
+        lib.fluxbin_workspace_init.restype, lib.fluxbin_workspace_init.argtypes = ctypes.c_int, [vp, sz, vp]
+        lib.fluxbin_linear.restype = ctypes.c_int
+        lib.fluxbin_linear.argtypes = [vp, vp, i32, i64, vp, i32, i64, vp, sz, vp]
+        lib.fluxbin_debug_tables.restype = ctypes.c_int
+        lib.fluxbin_debug_tables.argtypes = [vp, vp, i32, vp, vp, vp, vp]
+        lib.fluxbin_num_table_sets.restype, lib.fluxbin_num_table_sets.argtypes = i32, [vp]
+        lib.fluxbin_num_launches.restype, lib.fluxbin_num_launches.argtypes = i32, [vp, i32]
+        lib.fluxbin_free.restype, lib.fluxbin_free.argtypes = None, [vp]
+        lib.fluxbin_status_string.restype, lib.fluxbin_status_string.argtypes = ctypes.c_char_p, [ctypes.c_int]
+        lib.fluxbin_last_cuda_error.restype, lib.fluxbin_last_cuda_error.argtypes = ctypes.c_int, []
+        if hasattr(lib, "fluxbin_linear_noalloc"):
+            lib.fluxbin_linear_noalloc.restype = ctypes.c_int
+            lib.fluxbin_linear_noalloc.argtypes = [vp, vp, i32, i64, vp, i32, i64, vp]
+        _LIB = lib
+    return _LIB
+
+
+def library():
+    """The loaded ctypes library (for symbol checks)."""
+    return _lib()
+
+
+def _check(status: int, where: str):
+    if status != STATUS_OK:
+        raise FluxBinError(status, where)
+
+
+def _ptr(a):
+    return None if a is None or a.size == 0 else a.ctypes.data
+
+
+def make_desc(L) -> LayerDesc:
+    """LayerDesc borrowing the numpy arrays of a canonical layer object (keep `L` alive)."""
+    return LayerDesc(L.M, L.N, L.Kb, L.Ks, L.g, L.n_sal, _ptr(L.bits), _ptr(L.row_scale), _ptr(L.col_scale),
+                     _ptr(L.sal_idx), _ptr(L.sal_bits), _ptr(L.sal_row_scale), _ptr(L.sal_col_scale))
+
+
+def status_string(status: int) -> str:
+    return _lib().fluxbin_status_string(status).decode()
+
+
+def validate(L) -> int:
+    d = make_desc(L)
+    return int(_lib().fluxbin_validate(ctypes.byref(d)))
+
+
+def packed_size(L, with_map: bool = True) -> int:
+    d = make_desc(L)
+    if not with_map:
+        d.sal_idx = None
+    return int(_lib().fluxbin_packed_size(ctypes.byref(d)))
+
+
+def pack_host(L) -> np.ndarray:
+    """Packed layer as a uint8 numpy array (host)."""
+    n = packed_size(L)
+    if n == 0:
+        _check(validate(L) or 2, "fluxbin_packed_size")
+    buf = np.empty(n, np.uint8)
+    d = make_desc(L)
+    _check(_lib().fluxbin_pack_host(ctypes.byref(d), buf.ctypes.data, n), "fluxbin_pack_host")
+    return buf
+
+
+def _empty_canonical(M, N, Kb, Ks, g, n_sal):
+    from types import SimpleNamespace
+    ng, nws = N // g, (n_sal + 31) // 32
+    return SimpleNamespace(
+        M=M, N=N, Kb=Kb, Ks=Ks, g=g, n_sal=n_sal,
+        bits=np.zeros((Kb, M, N // 32), np.uint32), row_scale=np.zeros((Kb, M, ng), np.uint16),
+        col_scale=np.zeros((Kb, N), np.uint16), sal_idx=np.zeros(n_sal, np.int32),
+        sal_bits=np.zeros((Ks, M, nws), np.uint32), sal_row_scale=np.zeros((Ks, M, ng), np.uint16),
+        sal_col_scale=np.zeros((Ks, n_sal), np.uint16))
+
+
+def unpack_host(buf: np.ndarray):
+    """Inverse of pack_host: a namespace with the canonical arrays."""
+    d = LayerDesc()
+    _check(_lib().fluxbin_packed_dims(buf.ctypes.data, buf.size, ctypes.byref(d)), "fluxbin_packed_dims")
+    out = _empty_canonical(d.M, d.N, d.Kb, d.Ks, d.g, d.n_sal)
+    dd = make_desc(out)
+    _check(_lib().fluxbin_unpack_host(buf.ctypes.data, buf.size, ctypes.byref(dd)), "fluxbin_unpack_host")
+    return out
+
+
+class Weight:
+    """A packed layer resident in device memory (the caller's buffer) plus its handle."""
+
+    def __init__(self, handle: int, dims, buffer=None):
+        self.handle = handle
+        self.M, self.N, self.Kb, self.Ks, self.g, self.n_sal = dims
+        self.buffer = buffer          # keeps the caller's device tensor alive, if given
+
+    def close(self):
+        if self.handle:
+            _lib().fluxbin_free(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def workspace_size(self, B: int) -> int:
+        return int(_lib().fluxbin_workspace_size(self.handle, B))
+
+    def num_table_sets(self) -> int:
+        return int(_lib().fluxbin_num_table_sets(self.handle))
+
+    def num_launches(self, B: int) -> int:
+        return int(_lib().fluxbin_num_launches(self.handle, B))
+
+
+def pack(L, d_packed: int, d_bytes: int, stream: int = 0, buffer=None) -> Weight:
+    """fluxbin_pack: pack canonical layer L into the device buffer at address d_packed."""
+    d = make_desc(L)
+    h = ctypes.c_void_p()
+    _check(_lib().fluxbin_pack(ctypes.byref(d), d_packed, d_bytes, stream, ctypes.byref(h)), "fluxbin_pack")
+    return Weight(h.value, (L.M, L.N, L.Kb, L.Ks if L.n_sal else 0, L.g, L.n_sal if L.Ks else 0), buffer)
+
+
+def attach(header: np.ndarray, d_packed: int, d_bytes: int, buffer=None) -> Weight:
+    h = ctypes.c_void_p()
+    _check(_lib().fluxbin_attach(header.ctypes.data, header.size, d_packed, d_bytes, ctypes.byref(h)), "fluxbin_attach")
+    d = LayerDesc()
+    _check(_lib().fluxbin_weight_dims(h.value, ctypes.byref(d)), "fluxbin_weight_dims")
+    return Weight(h.value, (d.M, d.N, d.Kb, d.Ks, d.g, d.n_sal), buffer)
+
+
+def unpack(w: Weight, stream: int = 0):
+    out = _empty_canonical(w.M, w.N, w.Kb, w.Ks, w.g, w.n_sal)
+    dd = make_desc(out)
+    _check(_lib().fluxbin_unpack(w.handle, ctypes.byref(dd), stream), "fluxbin_unpack")
+    return out
+
+
+def workspace_init(d_ws: int, nbytes: int, stream: int = 0):
+    _check(_lib().fluxbin_workspace_init(d_ws, nbytes, stream), "fluxbin_workspace_init")
+
+
+def linear(w: Weight, d_x: int, B: int, ldx: int, d_y: int, y_is_fp32: bool, ldy: int, d_ws: int, ws_bytes: int,
+           stream: int = 0):
+    """fluxbin_linear: y[B][ldy] = x[B][ldx] * What^T on `stream` (asynchronous)."""
+    _check(_lib().fluxbin_linear(w.handle, d_x, B, ldx, d_y, 1 if y_is_fp32 else 0, ldy, d_ws, ws_bytes, stream),
+           "fluxbin_linear")
+
+
+def linear_status(w: Weight, d_x, B, ldx, d_y, y_is_fp32, ldy, d_ws, ws_bytes, stream=0) -> int:
+    """Same call, returning the raw status (for argument-validation tests)."""
+    return int(_lib().fluxbin_linear(w.handle if w else None, d_x, B, ldx, d_y, 1 if y_is_fp32 else 0, ldy, d_ws,
+                                     ws_bytes, stream))
+
+
+def debug_tables(w: Weight, d_x: int, pair: int, d_tables: int, stream: int = 0):
+    cols = np.zeros(256, np.int32)
+    alpha = np.zeros(256, np.uint16)
+    _check(_lib().fluxbin_debug_tables(w.handle, d_x, pair, d_tables, cols.ctypes.data, alpha.ctypes.data, stream),
+           "fluxbin_debug_tables")
+    return cols, alpha
