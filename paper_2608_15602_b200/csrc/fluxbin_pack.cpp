@@ -55,6 +55,10 @@ void salient_svecs(const fluxbin_layer_desc_t *d, int sps1, std::vector<SalSvec>
     }
 }
 
+// Salient units carry one scale per row only when the layer has a single row-scale group and the
+// global region is in that format too (g a multiple of 128); otherwise one scale per sub-vector.
+static int salient_sps(int N, int g) { return (N / g == 1 && g % 128 == 0) ? 16 : 1; }
+
 static int item_bytes_for(int sps) { return FB_ITEM_BITS_BYTES + 32 * 2 * (32 / sps); }
 
 // Fill every header field.  n_svec < 0 selects the upper bound (salient map unknown).
@@ -71,7 +75,7 @@ static void make_header(const fluxbin_layer_desc_t *d, int n_svec, int n_dead, F
     h.nrb = h.Mpad / 32;
     int ng = d->N / d->g;
     h.sps[0] = gcd_int(d->g, 128) / 8;
-    h.sps[1] = (ng == 1) ? 16 : 1;
+    h.sps[1] = salient_sps(d->N, d->g);
     int nblk = (d->N + 127) / 128;
     h.nunits[0] = nblk * d->Kb;
     h.npairs[0] = (h.nunits[0] + 1) / 2;
@@ -184,7 +188,7 @@ extern "C" size_t fluxbin_packed_size(const fluxbin_layer_desc_t *d)
     FbHeader h;
     if (d->Ks > 0 && d->n_sal > 0 && d->sal_idx) {
         if (validate_salient(d) != FLUXBIN_OK) return 0;
-        int sps1 = (d->N / d->g == 1) ? 16 : 1;
+        int sps1 = salient_sps(d->N, d->g);
         std::vector<SalSvec> sv;
         std::vector<int> dead;
         salient_svecs(d, sps1, sv);
@@ -212,7 +216,7 @@ extern "C" fluxbin_status_t fluxbin_pack_host(const fluxbin_layer_desc_t *d, voi
     if (st != FLUXBIN_OK) return st;
     if (!h_packed) return FLUXBIN_ERR_NULL;
 
-    const int sps1 = (d->N / d->g == 1) ? 16 : 1;
+    const int sps1 = salient_sps(d->N, d->g);
     std::vector<SalSvec> sv;
     std::vector<int> dead;
     salient_svecs(d, sps1, sv);

@@ -1,0 +1,57 @@
+"""Device-resident FluxBin linear layer: torch owns the memory and the stream, the C-ABI library
+does all the work (argument marshalling only on this side)."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import fluxbin
+
+
+def _stream_ptr(stream=None) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return int(s.cuda_stream)
+
+
+class Workspace:
+    """Zero-initialised scratch for fluxbin_linear; any number of stream-ordered calls may share it."""
+
+    def __init__(self, nbytes: int, device="cuda"):
+        self.nbytes = max(256, int(nbytes))
+        self.tensor = torch.empty(self.nbytes, dtype=torch.uint8, device=device)
+        fluxbin.workspace_init(self.tensor.data_ptr(), self.nbytes, _stream_ptr())
+
+
+class FluxBinLinear:
+    """y = x @ What^T for a packed layer held in a torch uint8 CUDA tensor."""
+
+    def __init__(self, L, device="cuda", packed: np.ndarray | None = None):
+        """Pack canonical layer `L` (synth.Linear-like) into device memory.  If `packed` (the result
+        of fluxbin.pack_host) is given it is uploaded as is and a handle attached."""
+        self.device = torch.device(device)
+        if packed is None:
+            nbytes = fluxbin.packed_size(L)
+            self.buffer = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+            self.weight = fluxbin.pack(L, self.buffer.data_ptr(), nbytes, _stream_ptr(), buffer=self.buffer)
+        else:
+            self.buffer = torch.from_numpy(packed).to(self.device)
+            self.weight = fluxbin.attach(packed[:256], self.buffer.data_ptr(), packed.size, buffer=self.buffer)
+        self.M, self.N = self.weight.M, self.weight.N
+        self.packed_bytes = int(self.buffer.numel())
+
+    def workspace(self, B: int) -> Workspace:
+        return Workspace(self.weight.workspace_size(B), self.device)
+
+    def forward(self, x: torch.Tensor, ws: Workspace, out: torch.Tensor | None = None, fp32_out: bool = False,
+                stream=None) -> torch.Tensor:
+        """x: fp16 [B][>=N] (row stride = x.stride(0)); returns y [B][M] (fp16, or fp32 if fp32_out)."""
+        assert x.dtype == torch.float16 and x.is_cuda and x.dim() == 2 and x.stride(1) == 1
+        B = x.shape[0]
+        if out is None:
+            out = torch.empty((B, self.M), dtype=torch.float32 if fp32_out else torch.float16, device=x.device)
+        fluxbin.linear(self.weight, x.data_ptr(), B, x.stride(0), out.data_ptr(), out.dtype == torch.float32,
+                       out.stride(0), ws.tensor.data_ptr(), ws.nbytes, _stream_ptr(stream))
+        return out
+
+    def unpack(self):
+        return fluxbin.unpack(self.weight, _stream_ptr())

@@ -71,6 +71,13 @@ def _rng(seed: int, linear_id: int, tensor: str) -> np.random.Generator:
     return np.random.Generator(np.random.Philox(key=int(key), counter=[0, 0, 0, ctr]))
 
 
+def _random_words(rng: np.random.Generator, shape) -> np.ndarray:
+    """Uniform uint32 words straight from the raw Philox stream (fast path for GBs of bits)."""
+    n = int(np.prod(shape))
+    raw = rng.bit_generator.random_raw((n + 1) // 2)
+    return raw.view(np.uint32)[:n].reshape(shape)
+
+
 def _half_bits(a: np.ndarray) -> np.ndarray:
     return np.ascontiguousarray(a.astype(np.float16)).view(np.uint16)
 
@@ -112,13 +119,13 @@ def make_linear(seed: int, linear_id: int, M: int, N: int, Kb: int = 2, Ks: int 
     n_sal = int(sal_idx.size)
     ng = N // g
 
-    bits = _rng(seed, linear_id, "bits").integers(0, 1 << 32, size=(Kb, M, N // 32), dtype=np.uint32)
+    bits = _random_words(_rng(seed, linear_id, "bits"), (Kb, M, N // 32))
     row_scale = _abs_normal_fp16(_rng(seed, linear_id, "row_scale"), 0.0, 0.02, (Kb, M, ng))
     col_scale = _abs_normal_fp16(_rng(seed, linear_id, "col_scale"), 1.0, 0.1, (Kb, N))
 
     nw = (n_sal + 31) // 32
     if Ks > 0 and n_sal > 0:
-        sal_bits = _rng(seed, linear_id, "sal_bits").integers(0, 1 << 32, size=(Ks, M, nw), dtype=np.uint32)
+        sal_bits = np.ascontiguousarray(_random_words(_rng(seed, linear_id, "sal_bits"), (Ks, M, nw)))
         tail = n_sal % 32
         if tail:
             sal_bits[:, :, -1] &= np.uint32((1 << tail) - 1)
