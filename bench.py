@@ -1,0 +1,370 @@
+#!/usr/bin/env python
+"""Benchmark of the FluxBin decode linear stack on B200 (one JSON line on stdout).
+
+Workload (N=1): the Llama-2-70B-shaped stack of decode linears -- 80 layers x {q, k, v, o, gate,
+up, down}, 2 global bases + 1 extra base on a seeded random 5 % of the input columns, g = 128,
+batch 1, fp16 activations, every linear with its own input, all 560 packed layers resident in HBM
+at once (about 21 GB, far larger than L2, so every step streams the weights from HBM).  A "step" is
+one forward token: one fluxbin_linear call per linear, replayed from a CUDA graph.
+
+value = algorithmic bytes moved per second over all GPUs (GB/s); us_per_layer and us_per_linear
+carry the latency side of the metric.  With --gpus N the N ranks run independent replicas (the
+path has no exchange step): weak scaling, no collective on the data path.
+
+--impl reference times the CPU oracle (oracle/) on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import concurrent.futures as cf
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2608_15602_b200 import synth  # noqa: E402
+
+METRIC = "decode_linear_stack_effective_hbm_gbps_batch1"
+UNIT = "GB/s"
+
+
+def algorithmic_bytes(M, N, Kb, Ks, g, n_sal, B):
+    """Bytes the method must move for one call (storage model of the paper's appendix + fp16 x, y):
+    bits, row scales per (row, group, base), column scales, 16-bit salient indices, activations."""
+    w = Kb * M * N // 8 + 2 * Kb * M * (N // g) + 2 * Kb * N
+    if Ks > 0 and n_sal > 0:
+        w += Ks * M * ((n_sal + 7) // 8) + 2 * Ks * M * (N // g) + 2 * Ks * n_sal + 2 * n_sal
+    return w + 2 * B * N + 2 * B * M
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0}, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons sampled every 200 ms while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.rows = []
+        self.proc = None
+        self.index = index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "200", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([t.strip() for t in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        self.thread.join(timeout=2)
+        sm, smax, reasons = [], [], set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); smax.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def stack_spec(config: int, layers: int | None):
+    lins, nl = synth.config_linears(config)
+    if layers is not None:
+        nl = layers
+    return lins, nl
+
+
+def cpu_oracle_sample(config: int, B: int, max_linears: int = 7):
+    """Time the oracle as it stands on the linears of layer 0 (bounded sample); returns
+    (GB/s of algorithmic bytes, seconds, bytes, cores, description)."""
+    import oracle
+    lins, _ = synth.config_linears(config)
+    n = min(max_linears, len(lins))
+    tot_b, tot_t = 0, 0.0
+    for li in range(n):
+        L = synth.make_config_linear(config, 0, li)
+        x = synth.make_config_activations(config, 0, li, B)
+        t0 = time.perf_counter()
+        oracle.linear_direct(L, x)
+        tot_t += time.perf_counter() - t0
+        tot_b += algorithmic_bytes(L.M, L.N, L.Kb, L.Ks, L.g, L.n_sal, B)
+    return tot_b / tot_t / 1e9, tot_t, tot_b, oracle.num_threads(), f"layer 0 of the stack ({n} linears, B={B})"
+
+
+def run_reference(args, rank):
+    """--impl reference: the CPU oracle on the host cores, each step a bounded sample."""
+    if rank != 0:
+        return
+    vals = []
+    for i in range(args.warmup + args.steps):
+        gbps, t, b, cores, sample = cpu_oracle_sample(args.config, args.batch, max_linears=args.ref_linears)
+        if i >= args.warmup:
+            vals.append((gbps, t))
+    gbps = statistics.mean(v[0] for v in vals)
+    ms = statistics.mean(v[1] for v in vals) * 1e3
+    line = {"impl": "reference", "metric": METRIC, "value": gbps, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"config {args.config}: sample = {sample}", "batch": args.batch},
+            "cpu_baseline": {"value": gbps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": gbps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=4, help="workload: 4 = Llama-2-70B-shaped stack")
+    ap.add_argument("--layers", type=int, default=None, help="override the number of layers (profiling only)")
+    ap.add_argument("--batch", type=int, default=1)
+    ap.add_argument("--g", type=int, default=128)
+    ap.add_argument("--no-graph", action="store_true", help="plain launches instead of a CUDA graph replay")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ref-linears", type=int, default=7)
+    ap.add_argument("--per-linear", action="store_true", help="also print per-linear timings to stderr")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2608_15602_b200 import build as fb_build
+    fb_build.build()
+    from paper_2608_15602_b200 import fluxbin, layer as fb_layer
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    B = args.batch
+    lins, nl = stack_spec(args.config, args.layers)
+    jobs = [(layer, li) for layer in range(nl) for li in range(len(lins))]
+
+    # ---- build the resident stack: generate (threads) -> pack on the host -> upload ----------------
+    t_setup = time.perf_counter()
+    def gen(job):
+        layer, li = job
+        return job, synth.make_config_linear(args.config, layer, li, g=args.g), \
+            synth.make_config_activations(args.config, layer, li, B)
+
+    linears, xs_host, alg_bytes = [], [], []
+    nthreads = max(1, min(16, (os.cpu_count() or 4) - 1))
+    with cf.ThreadPoolExecutor(nthreads) as ex:
+        window = []
+        it = iter(jobs)
+        for _ in range(2 * nthreads):
+            j = next(it, None)
+            if j is not None:
+                window.append(ex.submit(gen, j))
+        while window:
+            job, L, x = window.pop(0).result()
+            j = next(it, None)
+            if j is not None:
+                window.append(ex.submit(gen, j))
+            lin = fb_layer.FluxBinLinear(L)
+            linears.append(lin)
+            xs_host.append(x)
+            alg_bytes.append(algorithmic_bytes(L.M, L.N, L.Kb, L.Ks, L.g, L.n_sal, B))
+            del L
+    setup_s = time.perf_counter() - t_setup
+
+    # activations / outputs: one arena each (device) + pinned host mirrors for the end-to-end leg
+    n_in = sum(l.N for l in linears) * B
+    n_out = sum(l.M for l in linears) * B
+    x_host = torch.empty(n_in, dtype=torch.float16).pin_memory()
+    y_host = torch.empty(n_out, dtype=torch.float16).pin_memory()
+    off = 0
+    for l, x in zip(linears, xs_host):
+        x_host[off:off + B * l.N] = torch.from_numpy(x.view(np.float16).reshape(-1))
+        off += B * l.N
+    x_dev = torch.empty(n_in, dtype=torch.float16, device="cuda")
+    y_dev = torch.empty(n_out, dtype=torch.float16, device="cuda")
+    x_dev.copy_(x_host)
+    ws = fb_layer.Workspace(max(l.weight.workspace_size(B) for l in linears))
+    views = []
+    ox = oy = 0
+    for l in linears:
+        views.append((l, x_dev[ox:ox + B * l.N].view(B, l.N), y_dev[oy:oy + B * l.M].view(B, l.M)))
+        ox += B * l.N
+        oy += B * l.M
+    launches_per_step = sum(l.weight.num_launches(B) for l in linears)
+    packed_bytes = sum(l.packed_bytes for l in linears)
+
+    stream = torch.cuda.Stream()
+
+    def issue_all():
+        for l, xv, yv in views:
+            l.forward(xv, ws, out=yv, stream=stream)
+
+    graph = None
+    with torch.cuda.stream(stream):
+        issue_all()                                   # first call per device does the one-time set-up
+        stream.synchronize()
+        if not args.no_graph:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                issue_all()
+
+    def step():
+        if graph is not None:
+            graph.replay()
+        else:
+            issue_all()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing --------------------------------------------------------------------
+    with torch.cuda.stream(stream):
+        for _ in range(max(3, args.warmup)):
+            step()
+        barrier()
+        sampler = ClockSampler(local_rank)
+        sampler.start()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+        ev[0].record(stream)
+        for i in range(args.steps):
+            step()
+            ev[i + 1].record(stream)
+        barrier()
+        clocks = sampler.stop()
+    step_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
+    total_ms = ev[0].elapsed_time(ev[-1])
+
+    # ---- end to end: pinned host x -> device, the stack, y -> pinned host, every step ---------------
+    with torch.cuda.stream(stream):
+        for _ in range(2):
+            x_dev.copy_(x_host, non_blocking=True); step(); y_host.copy_(y_dev, non_blocking=True)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.steps):
+            x_dev.copy_(x_host, non_blocking=True)
+            step()
+            y_host.copy_(y_dev, non_blocking=True)
+        e1.record(stream)
+        barrier()
+    e2e_ms = e0.elapsed_time(e1)
+
+    # ---- optional per-linear timing (plain launches, rotating over the layers so L2 stays cold) -----
+    per_linear = None
+    if args.per_linear and rank == 0:
+        per_linear = {}
+        nlin = len(lins)
+        with torch.cuda.stream(stream):
+            for li, (name, M, N) in enumerate(lins):
+                idxs = [layer * nlin + li for layer in range(nl)]
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                reps = 3
+                for r in range(reps + 1):
+                    if r == 1:
+                        a.record(stream)
+                    for i in idxs:
+                        l, xv, yv = views[i]
+                        l.forward(xv, ws, out=yv, stream=stream)
+                b.record(stream)
+                stream.synchronize()
+                us = a.elapsed_time(b) * 1e3 / (reps * len(idxs))
+                per_linear[f"{name}_{M}x{N}"] = {"us": round(us, 2), "GBps": round(alg_bytes[li] / us / 1e3, 1)}
+        print(json.dumps({"per_linear_plain_launches": per_linear}), file=sys.stderr)
+
+    # ---- max over ranks, aggregate ------------------------------------------------------------------
+    t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms = float(t[0]), float(t[1])
+    bytes_per_step = sum(alg_bytes)
+    ms_per_step = total_ms / args.steps
+    value = world * bytes_per_step / (ms_per_step * 1e-3) / 1e9
+    e2e_value = world * bytes_per_step / (e2e_ms / args.steps * 1e-3) / 1e9
+
+    if rank == 0:
+        peaks, peak_kind = measured_peaks()
+        peak = float(peaks["hbm_gbs"])
+        achieved = bytes_per_step / (ms_per_step * 1e-3) / 1e9     # one GPU's kernels
+        traffic = None
+        tpath = os.path.join(ROOT, "profiles", "dram_traffic.json")
+        if os.path.exists(tpath):
+            with open(tpath) as f:
+                tj = json.load(f)
+            # ncu DRAM bytes per algorithmic byte of the captured launch, scaled to a mean launch of this run
+            traffic = tj.get("dram_bytes_per_algorithmic_byte", None)
+            if traffic is not None:
+                traffic = traffic * bytes_per_step / launches_per_step
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"config {args.config}: Llama-2-70B-shaped decode linear stack" if args.config == 4
+                       else f"config {args.config}", "layers": nl, "linears_per_step": len(linears), "batch": B,
+                       "Kb": 2, "Ks": 0 if args.config == 0 else 1, "salient_frac": 0.0 if args.config == 0 else 0.05,
+                       "g": args.g, "packed_bytes_resident": packed_bytes, "algorithmic_bytes_per_step": bytes_per_step,
+                       "l2": "inputs larger than L2 (weights streamed once per step)" if packed_bytes > 4e8
+                       else "working set fits L2: L2-warm number",
+                       "launch": "cuda graph replay" if graph is not None else "plain launches",
+                       "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
+            "us_per_layer": ms_per_step * 1e3 / nl, "us_per_linear": ms_per_step * 1e3 / len(linears),
+            "frac_of_8TBps": achieved / 8000.0,
+            "step_ms_min_median_max": [min(step_ms), statistics.median(step_ms), max(step_ms)],
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": traffic, "peak_source": f"{peak_kind} (torch copy, read+write)",
+                         "kernel": "fluxbin_linear_kernel", "per": "mean over the launches of one step"},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(x_host.numel() * 2),
+                    "d2h_bytes_per_step": int(y_host.numel() * 2), "ms_per_step": e2e_ms / args.steps},
+            "gpu_launches": launches_per_step * args.steps,
+            "clocks": clocks, "setup_s": round(setup_s, 1),
+        }
+        if not args.no_cpu_baseline:
+            gbps, tsec, nbytes, cores, sample = cpu_oracle_sample(args.config, B)
+            line["cpu_baseline"] = {"value": gbps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
+                                    "seconds": round(tsec, 2)}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

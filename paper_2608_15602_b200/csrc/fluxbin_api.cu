@@ -95,7 +95,7 @@ fluxbin_status_t device_setup(int dev, int *num_sms)
             FB_CUDA(cudaGetLastError());
             uint32_t base = 0xffffffffu;
             FB_CUDA(cudaMemcpy(&base, probe, sizeof(base), cudaMemcpyDeviceToHost));
-            d.ok = (base + fbk::kSmallBytes <= fbk::kTabBase);
+            d.ok = (base <= fbk::kTabBase);
         }
         d.ready = true;
     }
@@ -217,19 +217,29 @@ extern "C" fluxbin_status_t fluxbin_workspace_init(void *d_workspace, size_t byt
 // ---- the layer ------------------------------------------------------------------------------------
 
 template <int S0, int S1, int BT>
-static cudaError_t launch(const fbk::LinearParams &p, int grid, cudaStream_t s)
+static cudaError_t launch(const fbk::LinearParams &p, int num_sms, long long items, cudaStream_t s)
 {
-    fbk::fluxbin_linear_kernel<S0, S1, BT><<<grid, fbk::kThreads, fbk::smem_bytes<BT>(), s>>>(p);
+    static int occ = 0;     // resident CTAs per SM of this instantiation (same on every B200)
+    if (occ == 0) {
+        int o = 0;
+        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, fbk::fluxbin_linear_kernel<S0, S1, BT>,
+                                                                      fbk::kThreads, fbk::smem_bytes<BT>());
+        if (e != cudaSuccess) return e;
+        occ = o > 0 ? o : 1;
+    }
+    long long grid = (long long)num_sms * occ;
+    if (items < grid) grid = items;
+    fbk::fluxbin_linear_kernel<S0, S1, BT><<<(int)grid, fbk::kThreads, fbk::smem_bytes<BT>(), s>>>(p);
     return cudaGetLastError();
 }
 
-template <int BT> static cudaError_t launch_bt(const fluxbin_weight_t *w, const fbk::LinearParams &p, int grid, cudaStream_t s)
+template <int BT> static cudaError_t launch_bt(const fluxbin_weight_t *w, const fbk::LinearParams &p, long long items, cudaStream_t s)
 {
-    const int s0 = w->h.sps[0], s1 = w->h.sps[1];
-    if (s0 == 16 && s1 == 16) return launch<16, 16, BT>(p, grid, s);
-    if (s0 == 16) return launch<16, 1, BT>(p, grid, s);
-    if (s0 == 8) return launch<8, 1, BT>(p, grid, s);
-    return launch<4, 1, BT>(p, grid, s);
+    const int s0 = w->h.sps[0], s1 = w->h.sps[1], n = w->num_sms;
+    if (s0 == 16 && s1 == 16) return launch<16, 16, BT>(p, n, items, s);
+    if (s0 == 16) return launch<16, 1, BT>(p, n, items, s);
+    if (s0 == 8) return launch<8, 1, BT>(p, n, items, s);
+    return launch<4, 1, BT>(p, n, items, s);
 }
 
 extern "C" fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint16_t *d_x, int32_t B, int64_t ldx,
@@ -259,7 +269,6 @@ extern "C" fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint
     p.tickets = (unsigned *)((uint8_t *)d_workspace + acc_bytes(w, bt_ws));
 
     const long long items = (long long)(p.npairs[0] + p.npairs[1]) * p.nrb;
-    const int grid = (int)(items < w->num_sms ? items : w->num_sms);
 
     const size_t ysz = y_is_fp32 ? 4 : 2;
     for (int b0 = 0; b0 < B; b0 += 4) {
@@ -268,9 +277,9 @@ extern "C" fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint
         p.y = (uint8_t *)d_y + (size_t)b0 * ldy * ysz;
         p.nb = nb;
         cudaError_t e;
-        if (nb == 1) e = launch_bt<1>(w, p, grid, s);
-        else if (nb == 2) e = launch_bt<2>(w, p, grid, s);
-        else e = launch_bt<4>(w, p, grid, s);
+        if (nb == 1) e = launch_bt<1>(w, p, items, s);
+        else if (nb == 2) e = launch_bt<2>(w, p, items, s);
+        else e = launch_bt<4>(w, p, items, s);
         if (e != cudaSuccess) return cuda_fail(e);
     }
     return FLUXBIN_OK;

@@ -1,22 +1,29 @@
 // FluxBin decode linear layer: the LUT GEMV kernel for sm_100a (no tensor cores: the path is a
 // table-lookup GEMV bound by HBM and by the shared-memory lookup rate).
 //
-// One persistent CTA per SM.  The work of a layer is the list of items (pair, row block): a pair
-// is one table set (32 tables = two units of 16 sub-vectors), a row block is 32 output rows.
-// Items are ordered pair-major and cut into equal contiguous shares, so a CTA builds the tables
-// of one or two pairs (stage (i), Eq. 14, column scale fused per Eq. 11) and then streams the
-// weight bytes of a long run of rows through them (stage (ii), Eq. 15).  Row scales are applied
-// per (row, segment) in registers and the per-row partial sums of this K slice are added to an
-// fp32 accumulator in global memory (stage (iii)); the CTA that completes a tile of rows -- found
-// with one arrival counter per tile, never by waiting -- converts the tile to the output type and
-// re-zeroes the accumulator.
+// Persistent CTAs, two or three per SM.  The work of a layer is the list of items (pair, row
+// block): a pair is one table set (32 tables = two units of 16 sub-vectors), a row block is 32
+// output rows.  Items are ordered pair-major and cut into equal contiguous shares, so a CTA
+// builds the tables of one or two pairs (stage (i), Eq. 14, column scale fused per Eq. 11) and
+// streams the weight bytes of a long run of rows through them (stage (ii), Eq. 15).  Row scales
+// are applied per (row, segment) in registers and the per-row partial sums of this K slice are
+// added to an fp32 accumulator in global memory (stage (iii)); the CTA that completes a tile of
+// rows -- found with one arrival counter per tile, never by waiting -- converts the tile to the
+// output type and re-zeroes the accumulator.
 //
-// Shared-memory table layout: entry p of table slot sigma lives at shared-window address
-// 0x10000 + p*256 + sigma*4*BT  (BT = batch vectors per launch, their entries side by side; for
-// BT = 4 the two units of a pair get separate 64 KB planes at 0x10000 and 0x20000).
-// A lane at step s reads slot  lane ^ s, so the 32 lanes of a warp always hit 32 different slots:
-// every lookup is bank-conflict free by construction, and the packer has stored each lane's
-// weight bytes in exactly that order, so the byte of step s sits at a compile-time position.
+// Weight stream: every item is one contiguous block of memory.  A lane pulls its 32 weight bytes
+// and its row scales straight into registers with 128-bit loads (staging them in shared memory
+// would add traffic to the port the lookups saturate); one lane per warp runs a bulk L2 prefetch
+// a few items ahead so those loads find their lines in L2.
+//
+// Shared-memory table layout: entry p of table slot sigma lives at  kTabBase + p*256 + sigma*4*BT
+// (BT = batch vectors per launch, their entries side by side; for BT = 4 the two units of a pair
+// get separate 64 KB planes).  A lane at step s reads slot  lane ^ s, so the 32 lanes of a warp
+// always hit 32 different slots: every lookup is bank-conflict free by construction, and the
+// packer has stored each lane's weight bytes in exactly that order, so the byte of step s sits at
+// a compile-time position.  For BT = 1 the whole address is formed by ONE byte-permute (table
+// index into byte 1, the lane's pre-packed slot offset into byte 0) and the table base rides in
+// the load's immediate: 3 instructions per lookup (PRMT, LDS, FADD).
 #pragma once
 
 #include <cuda_fp16.h>
@@ -27,10 +34,10 @@
 
 namespace fbk {
 
-constexpr int kThreads = 512;
+constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxTiles = 1024;
-constexpr uint32_t kSmallBytes = 256 * 4 * 4 + kMaxTiles * 4;   // scale-fusion scratch + tile counters
+constexpr int kPrefetchItems = 4;   // L2 prefetch distance, in items of one warp
 
 struct LinearParams {
     const uint8_t *packed;
@@ -49,24 +56,20 @@ struct LinearParams {
     int tile_rb, ntiles;
 };
 
-// The tables start at shared-window address 0x10000 so that the address of entry p of a slot is
-// (lane constant) | p << 8 with the p byte dropped in by one PRMT and nothing to add.
-constexpr uint32_t kTabBase = 0x10000u;
+// The tables start at this shared-window address.  It is a compile-time constant so that it can
+// ride in the immediate field of every table load; dynamic shared memory starts below it (1 KB is
+// reserved by the system at the bottom of the window; the host probes the actual start once).
+constexpr uint32_t kTabBase = 0x800u;
 
 template <int BT> struct TabCfg {
     static constexpr int kTableBytes = (BT == 4) ? 131072 : 65536;
-    // address bits of slot sigma at step 0 (table base included); entry p adds p << 8
+    static constexpr int kSmallBytes = 256 * BT * 4 + kMaxTiles * 4;   // scale-fusion scratch + tile counters
+    // offset of slot sigma from the table base at step 0; entry p adds p << 8
     __host__ __device__ static constexpr uint32_t lane_const(uint32_t sigma)
     {
-        return BT == 1 ? (kTabBase | sigma * 4u)
-             : BT == 2 ? (kTabBase | sigma * 8u)
-                       : ((kTabBase << (sigma >> 4)) | ((sigma & 15u) * 16u));
+        return BT == 1 ? sigma * 4u : BT == 2 ? sigma * 8u : (((sigma >> 4) << 16) | ((sigma & 15u) * 16u));
     }
-    // lane_const(lane ^ s) == lane_const(lane) ^ step_const(s)
-    __host__ __device__ static constexpr uint32_t step_const(uint32_t s)
-    {
-        return BT == 1 ? s * 4u : BT == 2 ? s * 8u : (((s >> 4) ? 0x30000u : 0u) | ((s & 15u) * 16u));
-    }
+    // lane_const(lane ^ s) == lane_const(lane) ^ lane_const(s)
 };
 
 __device__ __forceinline__ float h2f(uint32_t bits16) { return __half2float(__ushort_as_half((unsigned short)bits16)); }
@@ -99,18 +102,22 @@ template <> struct Vec<4> { float v[4]; };
 template <int BT> __device__ __forceinline__ Vec<BT> lds_entry(uint32_t addr)
 {
     Vec<BT> r;
-    if constexpr (BT == 1) asm volatile("ld.shared.f32 %0, [%1];" : "=f"(r.v[0]) : "r"(addr));
-    else if constexpr (BT == 2) asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];" : "=f"(r.v[0]), "=f"(r.v[1]) : "r"(addr));
-    else asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
-                      : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3]) : "r"(addr));
+    // addr is an offset from the table base; the base is the immediate
+    if constexpr (BT == 1) asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(r.v[0]) : "r"(addr), "n"(kTabBase));
+    else if constexpr (BT == 2)
+        asm volatile("ld.shared.v2.f32 {%0,%1}, [%2+%3];" : "=f"(r.v[0]), "=f"(r.v[1]) : "r"(addr), "n"(kTabBase));
+    else asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4+%5];"
+                      : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3]) : "r"(addr), "n"(kTabBase));
     return r;
 }
 
 template <int BT> __device__ __forceinline__ void sts_entry(uint32_t addr, const float *v)
 {
-    if constexpr (BT == 1) asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v[0]));
-    else if constexpr (BT == 2) asm volatile("st.shared.v2.f32 [%0], {%1,%2};" ::"r"(addr), "f"(v[0]), "f"(v[1]));
-    else asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]));
+    if constexpr (BT == 1) asm volatile("st.shared.f32 [%0+%2], %1;" ::"r"(addr), "f"(v[0]), "n"(kTabBase) : "memory");
+    else if constexpr (BT == 2)
+        asm volatile("st.shared.v2.f32 [%0+%3], {%1,%2};" ::"r"(addr), "f"(v[0]), "f"(v[1]), "n"(kTabBase) : "memory");
+    else asm volatile("st.shared.v4.f32 [%0+%5], {%1,%2,%3,%4};" ::"r"(addr), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]),
+                      "n"(kTabBase) : "memory");
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -135,31 +142,35 @@ __device__ __forceinline__ void build_tables(const uint8_t *pair_desc, const uin
     }
     __syncthreads();
     const int lane = tid & 31, warp = tid >> 5;
-    constexpr int PW = 256 / kWarps;          // table entries per warp: p = warp*PW + q
-    constexpr int LOW = (PW == 16) ? 4 : (PW == 32) ? 5 : 3;
-    static_assert((1 << LOW) == PW, "warps per CTA must be 8, 16 or 32");
+    constexpr int PW = 256 / kWarps;          // table entries per warp: p = warp*PW + ...
+    static_assert(PW % 16 == 0, "at most 16 warps per CTA");
     float a[8][BT];
 #pragma unroll
     for (int n = 0; n < 8; ++n)
 #pragma unroll
         for (int b = 0; b < BT; ++b) a[n][b] = abuf[(lane * 8 + n) * BT + b];
-    float v[PW][BT];
+    // 16 entries at a time: the high four index bits fix a base value, the low four are enumerated
+    // by doubling (entry p | 2^n = entry p + 2 a_n), one add per entry
+#pragma unroll 1
+    for (int p0 = warp * PW; p0 < (warp + 1) * PW; p0 += 16) {
+        float v[16][BT];
 #pragma unroll
-    for (int b = 0; b < BT; ++b) {
-        float base = 0.f;
+        for (int b = 0; b < BT; ++b) {
+            float base = 0.f;
 #pragma unroll
-        for (int n = 7; n >= LOW; --n) base += ((warp * PW) >> n & 1) ? a[n][b] : -a[n][b];
+            for (int n = 7; n >= 4; --n) base += ((p0 >> n) & 1) ? a[n][b] : -a[n][b];
 #pragma unroll
-        for (int n = LOW - 1; n >= 0; --n) base -= a[n][b];
-        v[0][b] = base;
+            for (int n = 3; n >= 0; --n) base -= a[n][b];
+            v[0][b] = base;
 #pragma unroll
-        for (int n = 0; n < LOW; ++n)
+            for (int n = 0; n < 4; ++n)
 #pragma unroll
-            for (int q = 0; q < (1 << n); ++q) v[q | (1 << n)][b] = v[q][b] + 2.f * a[n][b];
+                for (int q = 0; q < (1 << n); ++q) v[q | (1 << n)][b] = v[q][b] + 2.f * a[n][b];
+        }
+#pragma unroll
+        for (int q = 0; q < 16; ++q)
+            sts_entry<BT>(TabCfg<BT>::lane_const((uint32_t)lane) | ((uint32_t)(p0 + q) << 8), v[q]);
     }
-#pragma unroll
-    for (int q = 0; q < PW; ++q)
-        sts_entry<BT>(TabCfg<BT>::lane_const((uint32_t)lane) | ((uint32_t)(warp * PW + q) << 8), v[q]);
     __syncthreads();
 }
 
@@ -189,8 +200,43 @@ template <int SPS> __device__ __forceinline__ void load_item(ItemRegs<SPS> &r, c
     }
 }
 
+// PRMT with the full selector: bit 3 of a nibble replicates the sign bit of the selected byte
+// (the __byte_perm intrinsic masks that bit away, so the instruction is spelled out).
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
+{
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+
+// One bulk request that pulls `bytes` (a multiple of 16) starting at p into L2.
+__device__ __forceinline__ void prefetch_l2(const void *p, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
+
+// Lane constants of the lookup address.  BT == 1: eight registers holding, byte by byte, the slot
+// offset (lane ^ s) * 4 of each of the 32 steps, so that PRMT can drop it into byte 0 of the address.
+template <int BT> struct LaneAddr {
+    uint32_t c[(BT == 1) ? 8 : 1];
+    __device__ __forceinline__ void init(int lane)
+    {
+        if constexpr (BT == 1) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                uint32_t v = 0;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) v |= (uint32_t)(((lane ^ (4 * q + k)) * 4) & 0xff) << (8 * k);
+                c[q] = v;
+            }
+        } else {
+            c[0] = TabCfg<BT>::lane_const((uint32_t)lane);
+        }
+    }
+};
+
 template <int SPS, int BT>
-__device__ __forceinline__ void compute_item(const ItemRegs<SPS> &r, uint32_t tab_lane, float (&out)[BT])
+__device__ __forceinline__ void compute_item(const ItemRegs<SPS> &r, const LaneAddr<BT> &la, float (&out)[BT])
 {
     constexpr int NSEG = 32 / SPS;
     const uint32_t w[8] = {r.b0.x, r.b0.y, r.b0.z, r.b0.w, r.b1.x, r.b1.y, r.b1.z, r.b1.w};
@@ -204,9 +250,16 @@ __device__ __forceinline__ void compute_item(const ItemRegs<SPS> &r, uint32_t ta
 #pragma unroll
         for (int q = 0; q < SPS; ++q) {
             const int s = j * SPS + q;
-            // table index byte -> p << 8; the rest of the address is (lane constant) xor (step constant)
-            uint32_t idx = __byte_perm(w[s >> 2], 0u, 0x4404u | ((uint32_t)(s & 3) << 4));
-            uint32_t addr = idx | (tab_lane ^ TabCfg<BT>::step_const((uint32_t)s));
+            const uint32_t k = (uint32_t)(s & 3);
+            uint32_t addr;
+            if constexpr (BT == 1) {
+                // byte 1 <- weight byte k (table index p), byte 0 <- packed slot offset k, bytes 2,3 <- 0
+                // (sign replication of the offset byte, which is < 128)
+                addr = prmt(w[s >> 2], la.c[s >> 2], ((0xCu | k) << 12) | ((0xCu | k) << 8) | (k << 4) | (4u | k));
+            } else {
+                uint32_t idx = __byte_perm(w[s >> 2], 0u, 0x4404u | (k << 4));
+                addr = idx | (la.c[0] ^ TabCfg<BT>::lane_const((uint32_t)s));
+            }
             Vec<BT> e = lds_entry<BT>(addr);
 #pragma unroll
             for (int b = 0; b < BT; ++b) {
@@ -219,21 +272,31 @@ __device__ __forceinline__ void compute_item(const ItemRegs<SPS> &r, uint32_t ta
     }
 }
 
-template <int SPS, int BT>
-__device__ __forceinline__ void process_rows(const uint8_t *pair_items, int item_bytes, int rb_lo, int rb_hi,
-                                             float *acc, int Mpad)
+// First L2 prefetches of a run of row blocks (issued before the tables are built).
+__device__ __forceinline__ void prefetch_run_head(const uint8_t *pair_items, int item_bytes, int rb_lo, int rb_hi)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const uint32_t tab_lane = TabCfg<BT>::lane_const((uint32_t)lane);
+    if (lane < kPrefetchItems) {
+        int rb = rb_lo + warp + lane * kWarps;
+        if (rb < rb_hi) prefetch_l2(pair_items + (int64_t)rb * item_bytes, (uint32_t)item_bytes);
+    }
+}
+
+template <int SPS, int BT>
+__device__ __forceinline__ void process_rows(const uint8_t *pair_items, int item_bytes, int rb_lo, int rb_hi,
+                                             const LaneAddr<BT> &la, float *acc, int Mpad)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     int rb = rb_lo + warp;
     if (rb >= rb_hi) return;
     ItemRegs<SPS> cur, nxt;
     load_item<SPS>(cur, pair_items + (int64_t)rb * item_bytes, lane);
     for (; rb < rb_hi; rb += kWarps) {
-        const int rbn = rb + kWarps;
+        const int rbn = rb + kWarps, rbp = rb + kPrefetchItems * kWarps;
+        if (lane == 0 && rbp < rb_hi) prefetch_l2(pair_items + (int64_t)rbp * item_bytes, (uint32_t)item_bytes);
         if (rbn < rb_hi) load_item<SPS>(nxt, pair_items + (int64_t)rbn * item_bytes, lane);
         float out[BT];
-        compute_item<SPS, BT>(cur, tab_lane, out);
+        compute_item<SPS, BT>(cur, la, out);
 #pragma unroll
         for (int b = 0; b < BT; ++b) atomicAdd(acc + (int64_t)b * Mpad + rb * 32 + lane, out[b]);
         cur = nxt;
@@ -241,16 +304,20 @@ __device__ __forceinline__ void process_rows(const uint8_t *pair_items, int item
 }
 
 template <int SPS0, int SPS1, int BT>
-__global__ void __launch_bounds__(kThreads, 1) fluxbin_linear_kernel(const __grid_constant__ LinearParams P)
+__global__ void __launch_bounds__(kThreads, (BT == 4) ? 1 : 2) fluxbin_linear_kernel(const __grid_constant__ LinearParams P)
 {
-    // dynamic shared memory: [base, 0x10000) holds the small buffers, [0x10000, ...) the tables
+    // dynamic shared memory: [kTabBase, +tables) at a fixed window address, small buffers after it
     extern __shared__ __align__(16) uint8_t smem[];
-    float *abuf = (float *)smem;
+    const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem);
+    if (smem_base > kTabBase) return;                                    // the host probes this first
+    uint8_t *small = smem + (kTabBase - smem_base) + TabCfg<BT>::kTableBytes;
+    float *abuf = (float *)small;
     int *tile_cnt = (int *)(abuf + 256 * BT);
     const int tid = threadIdx.x;
-    if ((uint32_t)__cvta_generic_to_shared(smem) + kSmallBytes > kTabBase) return;   // host probes this first
 
     for (int t = tid; t < P.ntiles; t += kThreads) tile_cnt[t] = 0;
+    LaneAddr<BT> la;
+    la.init(tid & 31);
 
     // equal shares of the item list, weighted by item bytes
     const long long I0 = (long long)P.npairs[0] * P.nrb, I1 = (long long)P.npairs[1] * P.nrb;
@@ -273,13 +340,14 @@ __global__ void __launch_bounds__(kThreads, 1) fluxbin_linear_kernel(const __gri
         const int pair = (int)(local / P.nrb), rb_lo = (int)(local % P.nrb);
         const long long seg_end = min(end, cur - rb_lo + P.nrb);
         const int rb_hi = rb_lo + (int)(seg_end - cur);
+        const uint8_t *items = P.packed + P.off_items[region] + (size_t)pair * P.nrb * P.item_bytes[region];
+        prefetch_run_head(items, P.item_bytes[region], rb_lo, rb_hi);      // weights start moving now
 
         __syncthreads();     // previous segment's lookups are done before the tables are overwritten
         const uint8_t *desc = P.packed + P.off_coldesc + (size_t)((region ? P.npairs[0] : 0) + pair) * FB_PAIR_DESC_BYTES;
         build_tables<BT>(desc, P.x, P.ldx, P.nb, abuf);
-        const uint8_t *items = P.packed + P.off_items[region] + (size_t)pair * P.nrb * P.item_bytes[region];
-        if (region == 0) process_rows<SPS0, BT>(items, P.item_bytes[0], rb_lo, rb_hi, P.acc, P.Mpad);
-        else process_rows<SPS1, BT>(items, P.item_bytes[1], rb_lo, rb_hi, P.acc, P.Mpad);
+        if (region == 0) process_rows<SPS0, BT>(items, P.item_bytes[0], rb_lo, rb_hi, la, P.acc, P.Mpad);
+        else process_rows<SPS1, BT>(items, P.item_bytes[1], rb_lo, rb_hi, la, P.acc, P.Mpad);
 
         // how many items this CTA contributed to each tile of rows
         const int t_lo = rb_lo / P.tile_rb, t_hi = (rb_hi - 1) / P.tile_rb;
@@ -328,13 +396,13 @@ __global__ void __launch_bounds__(kThreads, 1)
 fluxbin_debug_tables_kernel(const uint8_t *pair_desc, const uint16_t *x, float *out)
 {
     extern __shared__ __align__(16) uint8_t smem[];
-    float *abuf = (float *)smem;
-    const uint32_t base = (uint32_t)__cvta_generic_to_shared(smem);
-    if (base + kSmallBytes > kTabBase) return;
-    build_tables<1>(pair_desc, x, 0, 1, abuf);
+    const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem);
+    if (smem_base > kTabBase) return;
+    uint8_t *tables = smem + (kTabBase - smem_base);
+    build_tables<1>(pair_desc, x, 0, 1, (float *)(tables + TabCfg<1>::kTableBytes));
     for (int i = threadIdx.x; i < 32 * 256; i += kThreads) {
         uint32_t sigma = i >> 8, p = i & 255;
-        out[i] = *(const float *)(smem + ((TabCfg<1>::lane_const(sigma) | (p << 8)) - base));
+        out[i] = *(const float *)(tables + (TabCfg<1>::lane_const(sigma) | (p << 8)));
     }
 }
 
@@ -345,7 +413,8 @@ __global__ void fluxbin_smem_base_kernel(uint32_t *out)
     if (threadIdx.x == 0) *out = (uint32_t)__cvta_generic_to_shared(smem);
 }
 
-// dynamic shared memory to request: everything up to the end of the tables, as if the window began at 0
-template <int BT> constexpr size_t smem_bytes() { return kTabBase + TabCfg<BT>::kTableBytes; }
+// dynamic shared memory to request: everything up to the end of the small buffers, as if the
+// window began at 0 (the system-reserved bytes below the dynamic start are over-counted on purpose)
+template <int BT> constexpr size_t smem_bytes() { return kTabBase + TabCfg<BT>::kTableBytes + TabCfg<BT>::kSmallBytes; }
 
 } // namespace fbk

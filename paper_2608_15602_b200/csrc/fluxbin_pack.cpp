@@ -162,6 +162,21 @@ static inline unsigned extract_bits(const uint32_t *row, int bit, int w)
     return (unsigned)(((lo | (hi << 32)) >> (bit & 31)) & ((1u << w) - 1u));
 }
 
+// out byte c = in byte c ^ m for the 16 bytes held in (lo, hi), little-endian.
+static inline void xor_permute16(uint64_t &lo, uint64_t &hi, int m)
+{
+    if (m & 8) { uint64_t t = lo; lo = hi; hi = t; }
+    if (m & 4) { lo = (lo << 32) | (lo >> 32); hi = (hi << 32) | (hi >> 32); }
+    if (m & 2) {
+        lo = ((lo & 0x0000ffff0000ffffull) << 16) | ((lo >> 16) & 0x0000ffff0000ffffull);
+        hi = ((hi & 0x0000ffff0000ffffull) << 16) | ((hi >> 16) & 0x0000ffff0000ffffull);
+    }
+    if (m & 1) {
+        lo = ((lo & 0x00ff00ff00ff00ffull) << 8) | ((lo >> 8) & 0x00ff00ff00ff00ffull);
+        hi = ((hi & 0x00ff00ff00ff00ffull) << 8) | ((hi >> 8) & 0x00ff00ff00ff00ffull);
+    }
+}
+
 static inline void deposit_bits(uint32_t *row, int bit, int w, unsigned val)
 {
     for (int n = 0; n < w; ++n)
@@ -271,33 +286,39 @@ extern "C" fluxbin_status_t fluxbin_pack_host(const fluxbin_layer_desc_t *d, voi
                 const int row = rb * 32 + l;
                 const bool live = row < M;
                 // the 16 table indices of this row for both units, in sub-vector order
-                uint8_t src[2][16];
-                uint16_t segscale[2][16];   // row scale per sub-vector (replicated over a segment)
-                for (int u = 0; u < 2; ++u)
-                    for (int t = 0; t < 16; ++t) {
-                        uint8_t b = 0;
-                        uint16_t s16 = 0;
-                        if (live && us[u].valid && !us[u].salient) {
-                            int col0 = us[u].blk * 128 + t * 8;
-                            if (col0 < N) {
-                                const uint32_t *r = d->bits + ((size_t)us[u].k * M + row) * nw;
-                                b = (uint8_t)(r[col0 >> 5] >> (col0 & 31));
-                                s16 = d->row_scale[((size_t)us[u].k * M + row) * ng + col0 / g];
-                            }
-                        } else if (live && us[u].valid) {
-                            int s = us[u].blk + t;
-                            if (s < (int)sv.size()) {
-                                const uint32_t *r = d->sal_bits + ((size_t)us[u].k * M + row) * nws;
-                                b = (uint8_t)extract_bits(r, sv[s].vstart, sv[s].w);
-                                s16 = d->sal_row_scale[((size_t)us[u].k * M + row) * ng + sv[s].G];
-                            }
+                alignas(16) uint8_t src[2][16];
+                uint16_t segscale[2][16];   // row scale per sub-vector (only segment starts are read)
+                for (int u = 0; u < 2; ++u) {
+                    std::memset(src[u], 0, 16);
+                    std::memset(segscale[u], 0, sizeof(segscale[u]));
+                    if (!live || !us[u].valid) continue;
+                    if (!us[u].salient) {
+                        const int colb = us[u].blk * 128;
+                        const int nbytes = std::min(16, (N - colb) / 8);   // N % 32 == 0
+                        const uint8_t *r = (const uint8_t *)(d->bits + ((size_t)us[u].k * M + row) * nw);
+                        std::memcpy(src[u], r + colb / 8, nbytes);         // little-endian words: byte = 8 columns
+                        const uint16_t *rs = d->row_scale + ((size_t)us[u].k * M + row) * ng;
+                        for (int t = 0; t < nbytes; t += sps) segscale[u][t] = rs[(colb + t * 8) / g];
+                    } else {
+                        const uint32_t *r = d->sal_bits + ((size_t)us[u].k * M + row) * nws;
+                        const uint16_t *rs = d->sal_row_scale + ((size_t)us[u].k * M + row) * ng;
+                        for (int t = 0; t < 16 && us[u].blk + t < (int)sv.size(); ++t) {
+                            const SalSvec &q = sv[us[u].blk + t];
+                            src[u][t] = (uint8_t)extract_bits(r, q.vstart, q.w);
+                            segscale[u][t] = rs[q.G];
                         }
-                        src[u][t] = b;
-                        segscale[u][t] = s16;
                     }
-                for (int s = 0; s < 32; ++s) {
-                    int sigma = l ^ s;
-                    item[(s >> 4) * 512 + l * 16 + (s & 15)] = src[sigma >> 4][sigma & 15];
+                }
+                // lane l reads slot l ^ s at step s: unit u sits in half u ^ (l >> 4), and inside the
+                // half the byte of sub-vector t sits at position t ^ (l & 15)
+                for (int u = 0; u < 2; ++u) {
+                    uint64_t lo, hi;
+                    std::memcpy(&lo, src[u], 8);
+                    std::memcpy(&hi, src[u] + 8, 8);
+                    xor_permute16(lo, hi, l & 15);
+                    uint8_t *dst = item + (u ^ (l >> 4)) * 512 + l * 16;
+                    std::memcpy(dst, &lo, 8);
+                    std::memcpy(dst + 8, &hi, 8);
                 }
                 for (int j = 0; j < nseg; ++j) {
                     // the segment is the aligned block of sps sub-vectors around slot l ^ (j*sps); its
