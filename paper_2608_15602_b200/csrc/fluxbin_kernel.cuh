@@ -63,7 +63,7 @@ constexpr uint32_t kTabBase = 0x800u;
 
 template <int BT> struct TabCfg {
     static constexpr int kTableBytes = (BT == 4) ? 131072 : 65536;
-    static constexpr int kSmallBytes = 256 * BT * 4 + kMaxTiles * 4;   // scale-fusion scratch + tile counters
+    static constexpr int kSmallBytes = 256 * BT * 4 + (2 * kMaxTiles + 4) * 4;   // scale-fusion scratch, tile counters, done list
     // offset of slot sigma from the table base at step 0; entry p adds p << 8
     __host__ __device__ static constexpr uint32_t lane_const(uint32_t sigma)
     {
@@ -282,25 +282,46 @@ __device__ __forceinline__ void prefetch_run_head(const uint8_t *pair_items, int
     }
 }
 
+template <int SPS> struct ItemBytes { static constexpr int value = FB_ITEM_BITS_BYTES + 64 * (32 / SPS); };
+
 template <int SPS, int BT>
-__device__ __forceinline__ void process_rows(const uint8_t *pair_items, int item_bytes, int rb_lo, int rb_hi,
+__device__ __forceinline__ void finish_item(const ItemRegs<SPS> &r, const LaneAddr<BT> &la, float *accp, int Mpad)
+{
+    float out[BT];
+    compute_item<SPS, BT>(r, la, out);
+#pragma unroll
+    for (int b = 0; b < BT; ++b) atomicAdd(accp + (int64_t)b * Mpad, out[b]);
+}
+
+// Row blocks rb_lo + warp, + kWarps, ... of one pair.  Two register sets alternate so that the
+// loads of the next item are in flight while the current one is looked up; lane 0 keeps a bulk L2
+// prefetch kPrefetchItems iterations ahead.
+template <int SPS, int BT>
+__device__ __forceinline__ void process_rows(const uint8_t *pair_items, int rb_lo, int rb_hi,
                                              const LaneAddr<BT> &la, float *acc, int Mpad)
 {
+    constexpr int IB = ItemBytes<SPS>::value;
+    constexpr int STRIDE = kWarps * IB;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    int rb = rb_lo + warp;
-    if (rb >= rb_hi) return;
-    ItemRegs<SPS> cur, nxt;
-    load_item<SPS>(cur, pair_items + (int64_t)rb * item_bytes, lane);
-    for (; rb < rb_hi; rb += kWarps) {
-        const int rbn = rb + kWarps, rbp = rb + kPrefetchItems * kWarps;
-        if (lane == 0 && rbp < rb_hi) prefetch_l2(pair_items + (int64_t)rbp * item_bytes, (uint32_t)item_bytes);
-        if (rbn < rb_hi) load_item<SPS>(nxt, pair_items + (int64_t)rbn * item_bytes, lane);
-        float out[BT];
-        compute_item<SPS, BT>(cur, la, out);
-#pragma unroll
-        for (int b = 0; b < BT; ++b) atomicAdd(acc + (int64_t)b * Mpad + rb * 32 + lane, out[b]);
-        cur = nxt;
+    const int first = rb_lo + warp;
+    if (first >= rb_hi) return;
+    const int n = (rb_hi - first + kWarps - 1) / kWarps;          // iterations of this warp
+    const uint8_t *p = pair_items + (int64_t)first * IB;           // item of iteration i: p + i*STRIDE
+    float *accp = acc + first * 32 + lane;
+    ItemRegs<SPS> ra, rb;
+    load_item<SPS>(ra, p, lane);
+    int i = 0;
+    for (; i + 1 < n; i += 2) {
+        if (lane == 0 && i + kPrefetchItems < n) prefetch_l2(p + (int64_t)kPrefetchItems * STRIDE, IB);
+        load_item<SPS>(rb, p + STRIDE, lane);
+        finish_item<SPS, BT>(ra, la, accp, Mpad);
+        if (lane == 0 && i + 1 + kPrefetchItems < n) prefetch_l2(p + (int64_t)(kPrefetchItems + 1) * STRIDE, IB);
+        if (i + 2 < n) load_item<SPS>(ra, p + 2 * STRIDE, lane);
+        finish_item<SPS, BT>(rb, la, accp + kWarps * 32, Mpad);
+        p += 2 * STRIDE;
+        accp += 2 * kWarps * 32;
     }
+    if (i < n) finish_item<SPS, BT>(ra, la, accp, Mpad);
 }
 
 template <int SPS0, int SPS1, int BT>
@@ -346,8 +367,8 @@ __global__ void __launch_bounds__(kThreads, (BT == 4) ? 1 : 2) fluxbin_linear_ke
         __syncthreads();     // previous segment's lookups are done before the tables are overwritten
         const uint8_t *desc = P.packed + P.off_coldesc + (size_t)((region ? P.npairs[0] : 0) + pair) * FB_PAIR_DESC_BYTES;
         build_tables<BT>(desc, P.x, P.ldx, P.nb, abuf);
-        if (region == 0) process_rows<SPS0, BT>(items, P.item_bytes[0], rb_lo, rb_hi, la, P.acc, P.Mpad);
-        else process_rows<SPS1, BT>(items, P.item_bytes[1], rb_lo, rb_hi, la, P.acc, P.Mpad);
+        if (region == 0) process_rows<SPS0, BT>(items, rb_lo, rb_hi, la, P.acc, P.Mpad);
+        else process_rows<SPS1, BT>(items, rb_lo, rb_hi, la, P.acc, P.Mpad);
 
         // how many items this CTA contributed to each tile of rows
         const int t_lo = rb_lo / P.tile_rb, t_hi = (rb_hi - 1) / P.tile_rb;
@@ -362,6 +383,7 @@ __global__ void __launch_bounds__(kThreads, (BT == 4) ? 1 : 2) fluxbin_linear_ke
     __threadfence();
     __syncthreads();
     const int npairs = P.npairs[0] + P.npairs[1];
+    int *done_list = tile_cnt + kMaxTiles;        // tiles this CTA completed, then their count
     for (int t = tid; t < P.ntiles; t += kThreads) {
         int c = tile_cnt[t];
         int last = 0;
@@ -373,22 +395,52 @@ __global__ void __launch_bounds__(kThreads, (BT == 4) ? 1 : 2) fluxbin_linear_ke
         tile_cnt[t] = last;
     }
     __syncthreads();
-    for (int t = 0; t < P.ntiles; ++t) {
-        if (!tile_cnt[t]) continue;
-        __threadfence();
-        const int r0 = t * P.tile_rb * 32, r1 = min(P.Mpad, r0 + P.tile_rb * 32);
-        for (int idx = tid; idx < (r1 - r0) * BT; idx += kThreads) {
-            const int b = idx / (r1 - r0), r = r0 + idx % (r1 - r0);
-            float *a = P.acc + (int64_t)b * P.Mpad + r;
-            float v = __ldcg(a);
-            __stcg(a, 0.f);
-            if (r < P.M && b < P.nb) {
-                if (P.y_fp32) ((float *)P.y)[(int64_t)b * P.ldy + r] = v;
-                else ((__half *)P.y)[(int64_t)b * P.ldy + r] = __float2half_rn(v);
+    if (tid < 32) {                                // warp 0 compacts the completed tiles into a list
+        int cnt = 0;
+        for (int base = 0; base < P.ntiles; base += 32) {
+            int t = base + tid;
+            int f = (t < P.ntiles) ? tile_cnt[t] : 0;
+            unsigned m = __ballot_sync(0xffffffffu, f);
+            if (f) done_list[cnt + __popc(m & ((1u << tid) - 1u))] = t;
+            cnt += __popc(m);
+        }
+        if (tid == 0) done_list[kMaxTiles] = cnt;
+    }
+    __syncthreads();
+    const int ndone = done_list[kMaxTiles];
+    if (ndone == 0) return;
+    __threadfence();
+    // all rows of all completed tiles in one flat loop, four independent loads in flight per thread
+    const int rpt = P.tile_rb * 32;
+    const int total = ndone * rpt * BT;
+    for (int base = tid; base < total; base += 4 * kThreads) {
+        float v[4];
+        float *a[4];
+        int row[4], bb[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            int idx = base + u * kThreads;
+            a[u] = nullptr;
+            if (idx < total) {
+                int li = idx / (rpt * BT), rem = idx - li * (rpt * BT);
+                bb[u] = rem / rpt;
+                row[u] = done_list[li] * rpt + (rem - bb[u] * rpt);
+                if (row[u] < P.Mpad) a[u] = P.acc + (int64_t)bb[u] * P.Mpad + row[u];
             }
         }
-        if (tid == 0) P.tickets[t] = 0;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) if (a[u]) v[u] = __ldcg(a[u]);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (!a[u]) continue;
+            __stcg(a[u], 0.f);
+            if (row[u] < P.M && bb[u] < P.nb) {
+                if (P.y_fp32) ((float *)P.y)[(int64_t)bb[u] * P.ldy + row[u]] = v[u];
+                else ((__half *)P.y)[(int64_t)bb[u] * P.ldy + row[u]] = __float2half_rn(v[u]);
+            }
+        }
     }
+    for (int li = tid; li < ndone; li += kThreads) P.tickets[done_list[li]] = 0;
 }
 
 // Test hook: build one table set exactly as the kernel does and write it out as [32][256] fp32.
