@@ -7,7 +7,7 @@ import subprocess
 _PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_PKG, "csrc")
 LIB_DIR = os.path.join(_PKG, "lib")
-LIB_PATH = os.path.join(LIB_DIR, "libfluxbin.so")
+LIB_PATH = os.environ.get("FLUXBIN_LIB") or os.path.join(LIB_DIR, "libfluxbin.so")
 SOURCES = ["fluxbin_api.cu", "fluxbin_pack.cpp", "fluxbin_noalloc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC,-fopenmp", "-shared"]
@@ -33,7 +33,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     os.makedirs(LIB_DIR, exist_ok=True)
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     tmp = LIB_PATH + f".tmp{os.getpid()}"
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + _sources()
+    extra = os.environ.get("FLUXBIN_NVCC_EXTRA", "").split()       # e.g. -DFB_TRACE for the instrumented build
+    cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + _sources()
     subprocess.check_call(cmd)
     os.replace(tmp, LIB_PATH)
     return LIB_PATH

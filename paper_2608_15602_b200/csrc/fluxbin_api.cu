@@ -259,9 +259,12 @@ extern "C" fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint
     p.ldx = ldx;
     p.ldy = ldy;
     p.y_fp32 = y_is_fp32 != 0;
-    p.M = w->h.M; p.Mpad = w->h.Mpad; p.nrb = w->h.nrb;
+    p.M = w->h.M; p.N = w->h.N; p.Kb = w->h.Kb; p.Mpad = w->h.Mpad; p.nrb = w->h.nrb;
     p.npairs[0] = w->h.npairs[0]; p.npairs[1] = w->h.npairs[1];
     p.item_bytes[0] = w->h.item_bytes[0]; p.item_bytes[1] = w->h.item_bytes[1];
+    // measured: a per-sub-vector-scale item (3072 B) takes about 1.5x the time of a 1152-byte item
+    p.item_cost[0] = 2;
+    p.item_cost[1] = (w->h.sps[1] == w->h.sps[0]) ? 2 : 3;
     p.off_coldesc = w->h.off_coldesc; p.off_items[0] = w->h.off_items[0]; p.off_items[1] = w->h.off_items[1];
     p.tile_rb = w->tile_rb; p.ntiles = w->ntiles;
     p.acc = (float *)d_workspace;
@@ -306,3 +309,11 @@ extern "C" fluxbin_status_t fluxbin_debug_tables(const fluxbin_weight_t *w, cons
     }
     return FLUXBIN_OK;
 }
+
+#ifdef FB_TRACE
+// Instrumented build only: copy the per-CTA phase timestamps of the last launch to the host.
+extern "C" int fluxbin_debug_trace(unsigned long long *h_out)
+{
+    return (int)cudaMemcpyFromSymbol(h_out, fbk::g_fb_trace, sizeof(unsigned long long) * 1024 * 8);
+}
+#endif

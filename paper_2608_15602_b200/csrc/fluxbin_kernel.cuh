@@ -37,7 +37,7 @@ namespace fbk {
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxTiles = 1024;
-constexpr int kPrefetchItems = 4;   // L2 prefetch distance, in items of one warp
+constexpr int kPrefetchItems = 6;   // L2 prefetch distance, in items of one warp
 
 struct LinearParams {
     const uint8_t *packed;
@@ -49,9 +49,10 @@ struct LinearParams {
     int nb;              // live batch rows (<= BT)
     float *acc;          // [BT][Mpad] split-K accumulators, zero on entry and on exit
     unsigned *tickets;   // [ntiles] arrival counters, zero on entry and on exit
-    int M, Mpad, nrb;
+    int M, N, Kb, Mpad, nrb;
     int npairs[2];
     int item_bytes[2];
+    int item_cost[2];    // relative time of one item of each region (work split)
     unsigned long long off_coldesc, off_items[2];
     int tile_rb, ntiles;
 };
@@ -127,18 +128,29 @@ template <int BT> __device__ __forceinline__ void sts_entry(uint32_t addr, const
 // ---------------------------------------------------------------------------------------------
 template <int BT>
 __device__ __forceinline__ void build_tables(const uint8_t *pair_desc, const uint16_t *x, int64_t ldx, int nb,
-                                             float *abuf)
+                                             float *abuf, int col0_a, int col0_b, int ncols)
 {
     const int tid = threadIdx.x;
     if (tid < 256) {
-        uint32_t e = __ldg((const uint32_t *)pair_desc + tid);   // {u16 column, fp16 alpha} of (slot tid/8, n tid%8)
-        uint32_t col = e & 0xffffu;
-        float al = h2f(e >> 16);
+        // {u16 column, fp16 alpha} of (slot tid/8, n tid%8).  For a global pair the column is also
+        // known from the pair's position, so x and alpha are fetched side by side, not in a chain.
+        float xv[BT];
+        uint32_t e;
+        if (col0_a >= 0) {       // first unit of the pair: slots 0..15, second unit: slots 16..31
+            const uint32_t col = (uint32_t)(tid < 128 ? col0_a : col0_b) + (uint32_t)(tid & 127);
+            const bool live = col < (uint32_t)ncols;          // padded columns carry alpha = 0
 #pragma unroll
-        for (int b = 0; b < BT; ++b) {
-            float xv = (b < nb) ? h2f(__ldg(x + (int64_t)b * ldx + col)) : 0.f;
-            abuf[tid * BT + b] = xv * al;     // exact in fp32: two 11-bit significands
+            for (int b = 0; b < BT; ++b) xv[b] = (b < nb && live) ? h2f(__ldg(x + (int64_t)b * ldx + col)) : 0.f;
+            e = __ldg((const uint32_t *)pair_desc + tid);
+        } else {
+            e = __ldg((const uint32_t *)pair_desc + tid);
+            const uint32_t col = e & 0xffffu;
+#pragma unroll
+            for (int b = 0; b < BT; ++b) xv[b] = (b < nb) ? h2f(__ldg(x + (int64_t)b * ldx + col)) : 0.f;
         }
+        const float al = h2f(e >> 16);
+#pragma unroll
+        for (int b = 0; b < BT; ++b) abuf[tid * BT + b] = xv[b] * al;     // exact in fp32: two 11-bit significands
     }
     __syncthreads();
     const int lane = tid & 31, warp = tid >> 5;
@@ -288,41 +300,83 @@ template <int SPS, int BT>
 __device__ __forceinline__ void finish_item(const ItemRegs<SPS> &r, const LaneAddr<BT> &la, float *accp, int Mpad)
 {
     float out[BT];
+#if defined(FB_EXP) && (FB_EXP == 1 || FB_EXP == 3)      // experiment: memory side only (no lookups)
+#pragma unroll
+    for (int b = 0; b < BT; ++b) out[b] = __uint_as_float((r.b0.x ^ r.b0.y ^ r.b0.z ^ r.b0.w ^ r.b1.x ^ r.b1.y ^ r.b1.z ^ r.b1.w ^ r.sc[0]) & 0x3fffffffu);
+#else
     compute_item<SPS, BT>(r, la, out);
+#endif
+#if defined(FB_EXP) && FB_EXP == 3      // experiment: memory side only, no reduction traffic either
+    float sink = 0.f;
+#pragma unroll
+    for (int b = 0; b < BT; ++b) sink += __uint_as_float((r.b0.x ^ r.b0.y ^ r.b0.z ^ r.b0.w ^ r.b1.x ^ r.b1.y ^ r.b1.z ^ r.b1.w ^ r.sc[0]) & 0x3fffffffu);
+    if (sink == 12345.f) atomicAdd(accp, sink);
+    return;
+#endif
 #pragma unroll
     for (int b = 0; b < BT; ++b) atomicAdd(accp + (int64_t)b * Mpad, out[b]);
 }
 
-// Row blocks rb_lo + warp, + kWarps, ... of one pair.  Two register sets alternate so that the
-// loads of the next item are in flight while the current one is looked up; lane 0 keeps a bulk L2
-// prefetch kPrefetchItems iterations ahead.
+// Row blocks rb_lo + warp, + kWarps, ... of one pair.  DEPTH register sets rotate so that the
+// loads of the next DEPTH-1 items are in flight while the current one is looked up (the loads hit
+// L2, whose latency is about one item's worth of work per warp); lane 0 keeps a bulk L2 prefetch
+// kPrefetchItems iterations ahead.
 template <int SPS, int BT>
 __device__ __forceinline__ void process_rows(const uint8_t *pair_items, int rb_lo, int rb_hi,
                                              const LaneAddr<BT> &la, float *acc, int Mpad)
 {
     constexpr int IB = ItemBytes<SPS>::value;
     constexpr int STRIDE = kWarps * IB;
+    constexpr int DEPTH = 2;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int first = rb_lo + warp;
     if (first >= rb_hi) return;
     const int n = (rb_hi - first + kWarps - 1) / kWarps;          // iterations of this warp
     const uint8_t *p = pair_items + (int64_t)first * IB;           // item of iteration i: p + i*STRIDE
     float *accp = acc + first * 32 + lane;
-    ItemRegs<SPS> ra, rb;
-    load_item<SPS>(ra, p, lane);
-    int i = 0;
-    for (; i + 1 < n; i += 2) {
-        if (lane == 0 && i + kPrefetchItems < n) prefetch_l2(p + (int64_t)kPrefetchItems * STRIDE, IB);
-        load_item<SPS>(rb, p + STRIDE, lane);
-        finish_item<SPS, BT>(ra, la, accp, Mpad);
-        if (lane == 0 && i + 1 + kPrefetchItems < n) prefetch_l2(p + (int64_t)(kPrefetchItems + 1) * STRIDE, IB);
-        if (i + 2 < n) load_item<SPS>(ra, p + 2 * STRIDE, lane);
-        finish_item<SPS, BT>(rb, la, accp + kWarps * 32, Mpad);
-        p += 2 * STRIDE;
-        accp += 2 * kWarps * 32;
+    ItemRegs<SPS> r[DEPTH];
+#pragma unroll
+    for (int d = 0; d < DEPTH - 1; ++d)
+        if (d < n) load_item<SPS>(r[d], p + d * STRIDE, lane);
+    for (int i = 0; i < n; i += DEPTH) {
+#pragma unroll
+        for (int d = 0; d < DEPTH; ++d) {
+            if (i + d < n) {
+#if defined(FB_EXP) && FB_EXP == 2
+                if (false)
+#else
+                if (lane == 0 && i + d + kPrefetchItems < n)
+#endif
+                    prefetch_l2(p + (int64_t)(d + kPrefetchItems) * STRIDE, IB);
+#if defined(FB_EXP) && FB_EXP == 2      // experiment: lookup side only (every warp re-reads its first items)
+                if (i + d + DEPTH - 1 < n && i < DEPTH)
+#else
+                if (i + d + DEPTH - 1 < n)
+#endif
+                    load_item<SPS>(r[(d + DEPTH - 1) % DEPTH], p + (int64_t)(d + DEPTH - 1) * STRIDE, lane);
+                finish_item<SPS, BT>(r[d], la, accp + d * (kWarps * 32), Mpad);
+            }
+        }
+        p += DEPTH * STRIDE;
+        accp += DEPTH * kWarps * 32;
     }
-    if (i < n) finish_item<SPS, BT>(ra, la, accp, Mpad);
 }
+
+#ifdef FB_TRACE
+// Instrumented build only: per-CTA phase timestamps (globaltimer, ns) for the cycle breakdown.
+__device__ unsigned long long g_fb_trace[1024][8];
+__device__ __forceinline__ void trace(int slot)
+{
+    if (threadIdx.x == 0 && blockIdx.x < 1024) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        g_fb_trace[blockIdx.x][slot] = t;
+    }
+}
+#define FB_TRACE_AT(slot) trace(slot)
+#else
+#define FB_TRACE_AT(slot)
+#endif
 
 template <int SPS0, int SPS1, int BT>
 __global__ void __launch_bounds__(kThreads, (BT == 4) ? 1 : 2) fluxbin_linear_kernel(const __grid_constant__ LinearParams P)
@@ -336,13 +390,14 @@ __global__ void __launch_bounds__(kThreads, (BT == 4) ? 1 : 2) fluxbin_linear_ke
     int *tile_cnt = (int *)(abuf + 256 * BT);
     const int tid = threadIdx.x;
 
+    FB_TRACE_AT(0);
     for (int t = tid; t < P.ntiles; t += kThreads) tile_cnt[t] = 0;
     LaneAddr<BT> la;
     la.init(tid & 31);
 
-    // equal shares of the item list, weighted by item bytes
+    // equal shares of the item list, weighted by the relative cost of an item of each region
     const long long I0 = (long long)P.npairs[0] * P.nrb, I1 = (long long)P.npairs[1] * P.nrb;
-    const long long w0 = P.item_bytes[0], w1 = P.item_bytes[1];
+    const long long w0 = P.item_cost[0], w1 = P.item_cost[1];
     const long long T0 = I0 * w0, T = T0 + I1 * w1;
     auto first_item = [&](long long pos) -> long long {
         if (pos <= 0) return 0;
@@ -366,7 +421,8 @@ __global__ void __launch_bounds__(kThreads, (BT == 4) ? 1 : 2) fluxbin_linear_ke
 
         __syncthreads();     // previous segment's lookups are done before the tables are overwritten
         const uint8_t *desc = P.packed + P.off_coldesc + (size_t)((region ? P.npairs[0] : 0) + pair) * FB_PAIR_DESC_BYTES;
-        build_tables<BT>(desc, P.x, P.ldx, P.nb, abuf);
+        build_tables<BT>(desc, P.x, P.ldx, P.nb, abuf, region ? -1 : (2 * pair) / P.Kb * 128,
+                         (2 * pair + 1) / P.Kb * 128, P.N);
         if (region == 0) process_rows<SPS0, BT>(items, rb_lo, rb_hi, la, P.acc, P.Mpad);
         else process_rows<SPS1, BT>(items, rb_lo, rb_hi, la, P.acc, P.Mpad);
 
@@ -380,8 +436,10 @@ __global__ void __launch_bounds__(kThreads, (BT == 4) ? 1 : 2) fluxbin_linear_ke
     }
 
     // Stage (iii): publish, take a ticket per touched tile; the last arrival finishes the tile.
+    FB_TRACE_AT(2);
     __threadfence();
     __syncthreads();
+    FB_TRACE_AT(3);
     const int npairs = P.npairs[0] + P.npairs[1];
     int *done_list = tile_cnt + kMaxTiles;        // tiles this CTA completed, then their count
     for (int t = tid; t < P.ntiles; t += kThreads) {
@@ -408,39 +466,50 @@ __global__ void __launch_bounds__(kThreads, (BT == 4) ? 1 : 2) fluxbin_linear_ke
     }
     __syncthreads();
     const int ndone = done_list[kMaxTiles];
+    FB_TRACE_AT(4);
     if (ndone == 0) return;
     __threadfence();
-    // all rows of all completed tiles in one flat loop, four independent loads in flight per thread
-    const int rpt = P.tile_rb * 32;
-    const int total = ndone * rpt * BT;
-    for (int base = tid; base < total; base += 4 * kThreads) {
-        float v[4];
-        float *a[4];
-        int row[4], bb[4];
+    // all rows of all completed tiles in one flat loop of 4-row groups, eight 128-bit loads in
+    // flight per thread (the accumulators live in L2; one round trip serves ~8K rows per CTA)
+    const int gpt = P.tile_rb * 8;                 // 4-row groups per tile
+    const int total = ndone * gpt * BT;
+    constexpr int U = 8;
+    for (int base = tid; base < total; base += U * kThreads) {
+        float4 v[U];
+        float *a[U];
+        int row[U], bb[U];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < U; ++u) {
             int idx = base + u * kThreads;
             a[u] = nullptr;
             if (idx < total) {
-                int li = idx / (rpt * BT), rem = idx - li * (rpt * BT);
-                bb[u] = rem / rpt;
-                row[u] = done_list[li] * rpt + (rem - bb[u] * rpt);
+                int li = idx / (gpt * BT), rem = idx - li * (gpt * BT);
+                bb[u] = rem / gpt;
+                row[u] = (done_list[li] * gpt + (rem - bb[u] * gpt)) * 4;
                 if (row[u] < P.Mpad) a[u] = P.acc + (int64_t)bb[u] * P.Mpad + row[u];
             }
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) if (a[u]) v[u] = __ldcg(a[u]);
+        for (int u = 0; u < U; ++u) if (a[u]) v[u] = __ldcg((const float4 *)a[u]);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < U; ++u) {
             if (!a[u]) continue;
-            __stcg(a[u], 0.f);
-            if (row[u] < P.M && bb[u] < P.nb) {
-                if (P.y_fp32) ((float *)P.y)[(int64_t)bb[u] * P.ldy + row[u]] = v[u];
-                else ((__half *)P.y)[(int64_t)bb[u] * P.ldy + row[u]] = __float2half_rn(v[u]);
+            __stcg((float4 *)a[u], make_float4(0.f, 0.f, 0.f, 0.f));
+            if (bb[u] >= P.nb) continue;
+            const float e[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                if (row[u] + k >= P.M) break;
+                if (P.y_fp32) ((float *)P.y)[(int64_t)bb[u] * P.ldy + row[u] + k] = e[k];
+                else ((__half *)P.y)[(int64_t)bb[u] * P.ldy + row[u] + k] = __float2half_rn(e[k]);
             }
         }
     }
     for (int li = tid; li < ndone; li += kThreads) P.tickets[done_list[li]] = 0;
+    FB_TRACE_AT(5);
+#ifdef FB_TRACE
+    if (tid == 0 && blockIdx.x < 1024) g_fb_trace[blockIdx.x][6] = ndone;
+#endif
 }
 
 // Test hook: build one table set exactly as the kernel does and write it out as [32][256] fp32.
@@ -451,7 +520,7 @@ fluxbin_debug_tables_kernel(const uint8_t *pair_desc, const uint16_t *x, float *
     const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem);
     if (smem_base > kTabBase) return;
     uint8_t *tables = smem + (kTabBase - smem_base);
-    build_tables<1>(pair_desc, x, 0, 1, (float *)(tables + TabCfg<1>::kTableBytes));
+    build_tables<1>(pair_desc, x, 0, 1, (float *)(tables + TabCfg<1>::kTableBytes), -1, -1, 0);
     for (int i = threadIdx.x; i < 32 * 256; i += kThreads) {
         uint32_t sigma = i >> 8, p = i & 255;
         out[i] = *(const float *)(tables + (TabCfg<1>::lane_const(sigma) | (p << 8)));
