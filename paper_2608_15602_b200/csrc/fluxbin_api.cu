@@ -217,7 +217,7 @@ extern "C" fluxbin_status_t fluxbin_workspace_init(void *d_workspace, size_t byt
 // ---- the layer ------------------------------------------------------------------------------------
 
 template <int S0, int S1, int BT>
-static cudaError_t launch(const fbk::LinearParams &p, int num_sms, long long items, cudaStream_t s)
+static cudaError_t launch(const fbk::LaunchParams &p, int num_sms, long long items, cudaStream_t s)
 {
     static int occ = 0;     // resident CTAs per SM of this instantiation (same on every B200)
     if (occ == 0) {
@@ -233,13 +233,39 @@ static cudaError_t launch(const fbk::LinearParams &p, int num_sms, long long ite
     return cudaGetLastError();
 }
 
-template <int BT> static cudaError_t launch_bt(const fluxbin_weight_t *w, const fbk::LinearParams &p, long long items, cudaStream_t s)
+template <int BT> static cudaError_t launch_bt(int s0, int s1, int num_sms, const fbk::LaunchParams &p, long long items, cudaStream_t s)
 {
-    const int s0 = w->h.sps[0], s1 = w->h.sps[1], n = w->num_sms;
-    if (s0 == 16 && s1 == 16) return launch<16, 16, BT>(p, n, items, s);
-    if (s0 == 16) return launch<16, 1, BT>(p, n, items, s);
-    if (s0 == 8) return launch<8, 1, BT>(p, n, items, s);
-    return launch<4, 1, BT>(p, n, items, s);
+    if (s0 == 16 && s1 == 16) return launch<16, 16, BT>(p, num_sms, items, s);
+    if (s0 == 16) return launch<16, 1, BT>(p, num_sms, items, s);
+    if (s0 == 8) return launch<8, 1, BT>(p, num_sms, items, s);
+    return launch<4, 1, BT>(p, num_sms, items, s);
+}
+
+// Measured on B200: an item with one row scale per sub-vector (3072 bytes) takes about 1.5x the
+// time of a 1152-byte item.
+static void item_costs(const FbHeader &h, int cost[2])
+{
+    cost[0] = 2;
+    cost[1] = (h.sps[1] == h.sps[0]) ? 2 : 3;
+}
+
+static long long entry_cost(const FbHeader &h)
+{
+    int c[2];
+    item_costs(h, c);
+    return ((long long)h.npairs[0] * c[0] + (long long)h.npairs[1] * c[1]) * h.nrb;
+}
+
+static void fill_entry(fbk::LinearEntry &E, const fluxbin_weight_t *w, const uint16_t *x, int64_t ldx, void *y, int64_t ldy,
+                       float *acc, unsigned *tickets, long long cost_begin)
+{
+    E.packed = (const uint8_t *)w->d_packed;
+    E.x = x; E.y = y; E.acc = acc; E.tickets = tickets;
+    E.ldx = ldx; E.ldy = ldy; E.cost_begin = cost_begin;
+    E.off_coldesc = w->h.off_coldesc; E.off_items[0] = w->h.off_items[0]; E.off_items[1] = w->h.off_items[1];
+    E.M = w->h.M; E.N = w->h.N; E.Kb = w->h.Kb; E.Mpad = w->h.Mpad; E.nrb = w->h.nrb;
+    E.npairs[0] = w->h.npairs[0]; E.npairs[1] = w->h.npairs[1];
+    E.tile_rb = w->tile_rb; E.ntiles = w->ntiles; E.reserved = 0;
 }
 
 extern "C" fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint16_t *d_x, int32_t B, int64_t ldx,
@@ -254,35 +280,26 @@ extern "C" fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint
     if (w->h.sps[1] == 16 && w->h.sps[0] != 16) return FLUXBIN_ERR_FORMAT;
     cudaStream_t s = (cudaStream_t)cuda_stream;
 
-    fbk::LinearParams p;
-    p.packed = (const uint8_t *)w->d_packed;
-    p.ldx = ldx;
-    p.ldy = ldy;
+    fbk::LaunchParams p;
+    p.table = nullptr;
+    p.n = 1;
     p.y_fp32 = y_is_fp32 != 0;
-    p.M = w->h.M; p.N = w->h.N; p.Kb = w->h.Kb; p.Mpad = w->h.Mpad; p.nrb = w->h.nrb;
-    p.npairs[0] = w->h.npairs[0]; p.npairs[1] = w->h.npairs[1];
-    p.item_bytes[0] = w->h.item_bytes[0]; p.item_bytes[1] = w->h.item_bytes[1];
-    // measured: a per-sub-vector-scale item (3072 B) takes about 1.5x the time of a 1152-byte item
-    p.item_cost[0] = 2;
-    p.item_cost[1] = (w->h.sps[1] == w->h.sps[0]) ? 2 : 3;
-    p.off_coldesc = w->h.off_coldesc; p.off_items[0] = w->h.off_items[0]; p.off_items[1] = w->h.off_items[1];
-    p.tile_rb = w->tile_rb; p.ntiles = w->ntiles;
-    p.acc = (float *)d_workspace;
+    item_costs(w->h, p.item_cost);
+    p.total_cost = entry_cost(w->h);
     const int bt_ws = B >= 3 ? 4 : B;
-    p.tickets = (unsigned *)((uint8_t *)d_workspace + acc_bytes(w, bt_ws));
-
-    const long long items = (long long)(p.npairs[0] + p.npairs[1]) * p.nrb;
+    float *acc = (float *)d_workspace;
+    unsigned *tickets = (unsigned *)((uint8_t *)d_workspace + acc_bytes(w, bt_ws));
+    const long long items = (long long)(w->h.npairs[0] + w->h.npairs[1]) * w->h.nrb;
 
     const size_t ysz = y_is_fp32 ? 4 : 2;
     for (int b0 = 0; b0 < B; b0 += 4) {
         const int nb = (B - b0 < 4) ? B - b0 : 4;
-        p.x = d_x + (int64_t)b0 * ldx;
-        p.y = (uint8_t *)d_y + (size_t)b0 * ldy * ysz;
+        fill_entry(p.single, w, d_x + (int64_t)b0 * ldx, ldx, (uint8_t *)d_y + (size_t)b0 * ldy * ysz, ldy, acc, tickets, 0);
         p.nb = nb;
         cudaError_t e;
-        if (nb == 1) e = launch_bt<1>(w, p, items, s);
-        else if (nb == 2) e = launch_bt<2>(w, p, items, s);
-        else e = launch_bt<4>(w, p, items, s);
+        if (nb == 1) e = launch_bt<1>(w->h.sps[0], w->h.sps[1], w->num_sms, p, items, s);
+        else if (nb == 2) e = launch_bt<2>(w->h.sps[0], w->h.sps[1], w->num_sms, p, items, s);
+        else e = launch_bt<4>(w->h.sps[0], w->h.sps[1], w->num_sms, p, items, s);
         if (e != cudaSuccess) return cuda_fail(e);
     }
     return FLUXBIN_OK;

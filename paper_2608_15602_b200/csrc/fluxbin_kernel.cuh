@@ -1,15 +1,17 @@
 // FluxBin decode linear layer: the LUT GEMV kernel for sm_100a (no tensor cores: the path is a
 // table-lookup GEMV bound by HBM and by the shared-memory lookup rate).
 //
-// Persistent CTAs, two or three per SM.  The work of a layer is the list of items (pair, row
-// block): a pair is one table set (32 tables = two units of 16 sub-vectors), a row block is 32
-// output rows.  Items are ordered pair-major and cut into equal contiguous shares, so a CTA
-// builds the tables of one or two pairs (stage (i), Eq. 14, column scale fused per Eq. 11) and
-// streams the weight bytes of a long run of rows through them (stage (ii), Eq. 15).  Row scales
-// are applied per (row, segment) in registers and the per-row partial sums of this K slice are
-// added to an fp32 accumulator in global memory (stage (iii)); the CTA that completes a tile of
-// rows -- found with one arrival counter per tile, never by waiting -- converts the tile to the
-// output type and re-zeroes the accumulator.
+// One launch runs a list of layers ("entries": one for fluxbin_linear, many for a plan).  Persistent
+// CTAs, several per SM.  The work of an entry is its list of items (pair, row block): a pair is one
+// table set (32 tables = two units of 16 sub-vectors), a row block is 32 output rows.  The items
+// of all entries, in order, are cut into equal contiguous shares (by cost), so a CTA builds the
+// tables of one or two pairs (stage (i), Eq. 14, column scale fused per Eq. 11) and streams the
+// weight bytes of a long run of rows through them (stage (ii), Eq. 15).  Row scales are applied
+// per (row, segment) in registers and the per-row partial sums of this K slice are added to an
+// fp32 accumulator in global memory (stage (iii)); the CTA that completes a tile of rows -- found
+// with one arrival counter per tile, never by waiting -- converts the tile to the output type and
+// re-zeroes the accumulator.  With many entries in one launch the start-up and reduction tails of
+// one layer overlap the streaming of the next.
 //
 // Weight stream: every item is one contiguous block of memory.  A lane pulls its 32 weight bytes
 // and its row scales straight into registers with 128-bit loads (staging them in shared memory
@@ -37,24 +39,36 @@ namespace fbk {
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxTiles = 1024;
-constexpr int kPrefetchItems = 6;   // L2 prefetch distance, in items of one warp
+#ifndef FB_DEPTH
+#define FB_DEPTH 3
+#endif
+constexpr int kDepth = FB_DEPTH;    // register sets (items in flight per warp) in the main loop
+constexpr int kPrefetchTrips = 2;   // L2 prefetch distance in loop trips (one trip = kDepth items per warp)
 
-struct LinearParams {
+// One layer of a launch.
+struct LinearEntry {
     const uint8_t *packed;
-    const uint16_t *x;
-    int64_t ldx;
-    void *y;
-    int64_t ldy;
-    int y_fp32;
-    int nb;              // live batch rows (<= BT)
-    float *acc;          // [BT][Mpad] split-K accumulators, zero on entry and on exit
-    unsigned *tickets;   // [ntiles] arrival counters, zero on entry and on exit
+    const uint16_t *x;       // [B][ldx] fp16
+    void *y;                 // [B][ldy] fp16 or fp32
+    float *acc;              // [BT][Mpad] split-K accumulators, zero on entry and on exit
+    unsigned *tickets;       // [ntiles] arrival counters, zero on entry and on exit
+    long long ldx, ldy;
+    long long cost_begin;    // summed cost of the entries before this one
+    unsigned long long off_coldesc, off_items[2];
     int M, N, Kb, Mpad, nrb;
     int npairs[2];
-    int item_bytes[2];
-    int item_cost[2];    // relative time of one item of each region (work split)
-    unsigned long long off_coldesc, off_items[2];
     int tile_rb, ntiles;
+    int reserved;
+};
+
+struct LaunchParams {
+    const LinearEntry *table;   // device table of n entries; nullptr: the single entry below
+    LinearEntry single;
+    long long total_cost;
+    int n;
+    int nb;                     // live batch rows (<= BT)
+    int y_fp32;
+    int item_cost[2];           // relative time of one item of each region (work split)
 };
 
 // The tables start at this shared-window address.  It is a compile-time constant so that it can
@@ -64,14 +78,17 @@ constexpr uint32_t kTabBase = 0x800u;
 
 template <int BT> struct TabCfg {
     static constexpr int kTableBytes = (BT == 4) ? 131072 : 65536;
-    static constexpr int kSmallBytes = 256 * BT * 4 + (2 * kMaxTiles + 4) * 4;   // scale-fusion scratch, tile counters, done list
-    // offset of slot sigma from the table base at step 0; entry p adds p << 8
+    // scale-fusion scratch, tile counters (+ count of completed tiles), work range, copy of the current entry
+    static constexpr int kSmallBytes = 256 * BT * 4 + (kMaxTiles + 4) * 4 + 32 + 128;
+    // offset of slot sigma from the table base at step 0; entry p adds p << 8.
+    // lane_const(lane ^ s) == lane_const(lane) ^ lane_const(s)
     __host__ __device__ static constexpr uint32_t lane_const(uint32_t sigma)
     {
         return BT == 1 ? sigma * 4u : BT == 2 ? sigma * 8u : (((sigma >> 4) << 16) | ((sigma & 15u) * 16u));
     }
-    // lane_const(lane ^ s) == lane_const(lane) ^ lane_const(s)
 };
+
+template <int SPS> struct ItemBytes { static constexpr int value = FB_ITEM_BITS_BYTES + 64 * (32 / SPS); };
 
 __device__ __forceinline__ float h2f(uint32_t bits16) { return __half2float(__ushort_as_half((unsigned short)bits16)); }
 
@@ -121,17 +138,33 @@ template <int BT> __device__ __forceinline__ void sts_entry(uint32_t addr, const
                       "n"(kTabBase) : "memory");
 }
 
+// PRMT with the full selector: bit 3 of a nibble replicates the sign bit of the selected byte
+// (the __byte_perm intrinsic masks that bit away, so the instruction is spelled out).
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
+{
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+
+// One bulk request that pulls `bytes` (a multiple of 16) starting at p into L2.
+__device__ __forceinline__ void prefetch_l2(const void *p, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
+
 // ---------------------------------------------------------------------------------------------
 // Stage (i): LUT building with scale fusion (Eq. 14 with a_n = x[col_n] * alpha_c[col_n], Eq. 11;
 // for salient tables col_n = sal_idx[v] and alpha = gathered scale, Eq. 13).
 // abuf: shared scratch of 32*8*BT floats.  Ends with the tables visible to the whole CTA.
+// col0_a / col0_b: first column of the pair's two units for a global pair, -1 for a salient pair.
 // ---------------------------------------------------------------------------------------------
 template <int BT>
 __device__ __forceinline__ void build_tables(const uint8_t *pair_desc, const uint16_t *x, int64_t ldx, int nb,
                                              float *abuf, int col0_a, int col0_b, int ncols)
 {
     const int tid = threadIdx.x;
-    if (tid < 256) {
+    {
         // {u16 column, fp16 alpha} of (slot tid/8, n tid%8).  For a global pair the column is also
         // known from the pair's position, so x and alpha are fetched side by side, not in a chain.
         float xv[BT];
@@ -155,7 +188,7 @@ __device__ __forceinline__ void build_tables(const uint8_t *pair_desc, const uin
     __syncthreads();
     const int lane = tid & 31, warp = tid >> 5;
     constexpr int PW = 256 / kWarps;          // table entries per warp: p = warp*PW + ...
-    static_assert(PW % 16 == 0, "at most 16 warps per CTA");
+    static_assert(kThreads == 256 && PW % 16 == 0, "the builder maps one thread to one table column");
     float a[8][BT];
 #pragma unroll
     for (int n = 0; n < 8; ++n)
@@ -195,36 +228,22 @@ template <int SPS> struct ItemRegs {
     uint32_t sc[(SPS == 16) ? 1 : (SPS == 8) ? 2 : (SPS == 4) ? 4 : 16];
 };
 
-template <int SPS> __device__ __forceinline__ void load_item(ItemRegs<SPS> &r, const uint8_t *item, int lane)
+// pl = item + lane*16 (weight bytes), ps = item + 1024 + lane*(scale bytes per lane, at most 16);
+// `off` is a compile-time byte offset added to both (the stride to a later item).
+template <int SPS> __device__ __forceinline__ void load_item(ItemRegs<SPS> &r, const uint8_t *pl, const uint8_t *ps, int off)
 {
-    r.b0 = ldg_stream_v4(item + lane * 16);
-    r.b1 = ldg_stream_v4(item + 512 + lane * 16);
-    const uint8_t *s = item + FB_ITEM_BITS_BYTES;
-    if constexpr (SPS == 16) r.sc[0] = ldg_stream_u32(s + lane * 4);
-    else if constexpr (SPS == 8) { uint2 t = ldg_stream_v2(s + lane * 8); r.sc[0] = t.x; r.sc[1] = t.y; }
-    else if constexpr (SPS == 4) { uint4 t = ldg_stream_v4(s + lane * 16); r.sc[0] = t.x; r.sc[1] = t.y; r.sc[2] = t.z; r.sc[3] = t.w; }
+    r.b0 = ldg_stream_v4(pl + off);
+    r.b1 = ldg_stream_v4(pl + off + 512);
+    if constexpr (SPS == 16) r.sc[0] = ldg_stream_u32(ps + off);
+    else if constexpr (SPS == 8) { uint2 t = ldg_stream_v2(ps + off); r.sc[0] = t.x; r.sc[1] = t.y; }
+    else if constexpr (SPS == 4) { uint4 t = ldg_stream_v4(ps + off); r.sc[0] = t.x; r.sc[1] = t.y; r.sc[2] = t.z; r.sc[3] = t.w; }
     else {
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-            uint4 t = ldg_stream_v4(s + q * 512 + lane * 16);
+            uint4 t = ldg_stream_v4(ps + off + q * 512);
             r.sc[4 * q] = t.x; r.sc[4 * q + 1] = t.y; r.sc[4 * q + 2] = t.z; r.sc[4 * q + 3] = t.w;
         }
     }
-}
-
-// PRMT with the full selector: bit 3 of a nibble replicates the sign bit of the selected byte
-// (the __byte_perm intrinsic masks that bit away, so the instruction is spelled out).
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
-{
-    uint32_t d;
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
-    return d;
-}
-
-// One bulk request that pulls `bytes` (a multiple of 16) starting at p into L2.
-__device__ __forceinline__ void prefetch_l2(const void *p, uint32_t bytes)
-{
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
 }
 
 // Lane constants of the lookup address.  BT == 1: eight registers holding, byte by byte, the slot
@@ -284,81 +303,71 @@ __device__ __forceinline__ void compute_item(const ItemRegs<SPS> &r, const LaneA
     }
 }
 
-// First L2 prefetches of a run of row blocks (issued before the tables are built).
-__device__ __forceinline__ void prefetch_run_head(const uint8_t *pair_items, int item_bytes, int rb_lo, int rb_hi)
-{
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (lane < kPrefetchItems) {
-        int rb = rb_lo + warp + lane * kWarps;
-        if (rb < rb_hi) prefetch_l2(pair_items + (int64_t)rb * item_bytes, (uint32_t)item_bytes);
-    }
-}
-
-template <int SPS> struct ItemBytes { static constexpr int value = FB_ITEM_BITS_BYTES + 64 * (32 / SPS); };
-
 template <int SPS, int BT>
 __device__ __forceinline__ void finish_item(const ItemRegs<SPS> &r, const LaneAddr<BT> &la, float *accp, int Mpad)
 {
     float out[BT];
-#if defined(FB_EXP) && (FB_EXP == 1 || FB_EXP == 3)      // experiment: memory side only (no lookups)
-#pragma unroll
-    for (int b = 0; b < BT; ++b) out[b] = __uint_as_float((r.b0.x ^ r.b0.y ^ r.b0.z ^ r.b0.w ^ r.b1.x ^ r.b1.y ^ r.b1.z ^ r.b1.w ^ r.sc[0]) & 0x3fffffffu);
-#else
     compute_item<SPS, BT>(r, la, out);
-#endif
-#if defined(FB_EXP) && FB_EXP == 3      // experiment: memory side only, no reduction traffic either
-    float sink = 0.f;
-#pragma unroll
-    for (int b = 0; b < BT; ++b) sink += __uint_as_float((r.b0.x ^ r.b0.y ^ r.b0.z ^ r.b0.w ^ r.b1.x ^ r.b1.y ^ r.b1.z ^ r.b1.w ^ r.sc[0]) & 0x3fffffffu);
-    if (sink == 12345.f) atomicAdd(accp, sink);
+#if defined(FB_EXP) && (FB_EXP == 4 || FB_EXP == 5)     // experiment: no reduction traffic
+    if (out[0] == 12345.678f) atomicAdd(accp, out[0]);
     return;
 #endif
 #pragma unroll
     for (int b = 0; b < BT; ++b) atomicAdd(accp + (int64_t)b * Mpad, out[b]);
 }
 
-// Row blocks rb_lo + warp, + kWarps, ... of one pair.  DEPTH register sets rotate so that the
-// loads of the next DEPTH-1 items are in flight while the current one is looked up (the loads hit
-// L2, whose latency is about one item's worth of work per warp); lane 0 keeps a bulk L2 prefetch
-// kPrefetchItems iterations ahead.
+// Row blocks rb_lo + warp, + kWarps, ... of one pair.  kDepth register sets rotate so that the
+// loads of the next kDepth-1 items are in flight while the current one is looked up (enough bytes
+// in flight per SM to cover the L2 latency at full HBM rate).  A trip of the steady loop handles
+// kDepth items with every address a pointer plus an immediate; each warp also bulk-prefetches,
+// kPrefetchTrips trips ahead, its share of the kDepth*kWarps items the CTA reads per trip.
 template <int SPS, int BT>
 __device__ __forceinline__ void process_rows(const uint8_t *pair_items, int rb_lo, int rb_hi,
                                              const LaneAddr<BT> &la, float *acc, int Mpad)
 {
     constexpr int IB = ItemBytes<SPS>::value;
-    constexpr int STRIDE = kWarps * IB;
-    constexpr int DEPTH = 2;
+    constexpr int STRIDE = kWarps * IB;                   // bytes between a warp's consecutive items
+    constexpr int SB = (SPS == 16) ? 4 : (SPS == 8) ? 8 : 16;   // scale bytes per lane (per plane)
+    constexpr int D = (SPS == 1) ? 1 : (BT == 4) ? 2 : kDepth;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int first = rb_lo + warp;
     if (first >= rb_hi) return;
-    const int n = (rb_hi - first + kWarps - 1) / kWarps;          // iterations of this warp
-    const uint8_t *p = pair_items + (int64_t)first * IB;           // item of iteration i: p + i*STRIDE
+    const int n = (rb_hi - first + kWarps - 1) / kWarps;  // items of this warp
+    const uint8_t *pl = pair_items + (int64_t)first * IB + lane * 16;
+    const uint8_t *ps = pair_items + (int64_t)first * IB + FB_ITEM_BITS_BYTES + lane * SB;
+    // this warp's prefetch window inside the block of D*kWarps items the CTA consumes per trip
+    const uint8_t *pp = pair_items + (int64_t)(rb_lo + D * warp) * IB + (int64_t)kPrefetchTrips * D * STRIDE;
+    const uint8_t *pend = pair_items + (int64_t)rb_hi * IB;
     float *accp = acc + first * 32 + lane;
-    ItemRegs<SPS> r[DEPTH];
+
+    ItemRegs<SPS> r[D];
 #pragma unroll
-    for (int d = 0; d < DEPTH - 1; ++d)
-        if (d < n) load_item<SPS>(r[d], p + d * STRIDE, lane);
-    for (int i = 0; i < n; i += DEPTH) {
+    for (int d = 0; d < D - 1; ++d)
+        if (d < n) load_item<SPS>(r[d], pl, ps, d * STRIDE);
+    // items t .. t+D-1 are looked up while items t+D-1 .. t+2D-2 are loaded (warp-uniform guards)
+    for (int t = 0; t < n; t += D) {
+        if (lane == 0 && pp + D * IB <= pend) prefetch_l2(pp, D * IB);
 #pragma unroll
-        for (int d = 0; d < DEPTH; ++d) {
-            if (i + d < n) {
-#if defined(FB_EXP) && FB_EXP == 2
-                if (false)
-#else
-                if (lane == 0 && i + d + kPrefetchItems < n)
-#endif
-                    prefetch_l2(p + (int64_t)(d + kPrefetchItems) * STRIDE, IB);
-#if defined(FB_EXP) && FB_EXP == 2      // experiment: lookup side only (every warp re-reads its first items)
-                if (i + d + DEPTH - 1 < n && i < DEPTH)
-#else
-                if (i + d + DEPTH - 1 < n)
-#endif
-                    load_item<SPS>(r[(d + DEPTH - 1) % DEPTH], p + (int64_t)(d + DEPTH - 1) * STRIDE, lane);
-                finish_item<SPS, BT>(r[d], la, accp + d * (kWarps * 32), Mpad);
-            }
+        for (int d = 0; d < D; ++d) {
+            if (t + d + D - 1 < n) load_item<SPS>(r[(d + D - 1) % D], pl, ps, (d + D - 1) * STRIDE);
+            if (t + d < n) finish_item<SPS, BT>(r[d], la, accp + d * (kWarps * 32), Mpad);
         }
-        p += DEPTH * STRIDE;
-        accp += DEPTH * kWarps * 32;
+        pl += D * STRIDE;
+        ps += D * STRIDE;
+        pp += D * STRIDE;
+        accp += D * kWarps * 32;
+    }
+}
+
+// First L2 prefetches of a run of row blocks (issued before the tables are built): the first
+// kPrefetchTrips blocks of D*kWarps items, one D-item request per lane.
+__device__ __forceinline__ void prefetch_run_head(const uint8_t *pair_items, int item_bytes, int D, int rb_lo, int rb_hi)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane < kPrefetchTrips) {
+        int rb = rb_lo + lane * D * kWarps + D * warp;
+        int cnt = min(D, rb_hi - rb);
+        if (cnt > 0) prefetch_l2(pair_items + (int64_t)rb * item_bytes, (uint32_t)(cnt * item_bytes));
     }
 }
 
@@ -378,86 +387,32 @@ __device__ __forceinline__ void trace(int slot)
 #define FB_TRACE_AT(slot)
 #endif
 
-template <int SPS0, int SPS1, int BT>
-__global__ void __launch_bounds__(kThreads, (BT == 4) ? 1 : 2) fluxbin_linear_kernel(const __grid_constant__ LinearParams P)
+// Stage (iii) for the entry a CTA has just finished contributing to: publish, take a ticket per
+// touched tile of rows; whoever arrives last at a tile converts it and re-zeroes the accumulator.
+template <int BT>
+__device__ __forceinline__ void reduce_and_store(const LinearEntry &E, int nb, int y_fp32, int *tile_cnt, int *done_list)
 {
-    // dynamic shared memory: [kTabBase, +tables) at a fixed window address, small buffers after it
-    extern __shared__ __align__(16) uint8_t smem[];
-    const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem);
-    if (smem_base > kTabBase) return;                                    // the host probes this first
-    uint8_t *small = smem + (kTabBase - smem_base) + TabCfg<BT>::kTableBytes;
-    float *abuf = (float *)small;
-    int *tile_cnt = (int *)(abuf + 256 * BT);
     const int tid = threadIdx.x;
-
-    FB_TRACE_AT(0);
-    for (int t = tid; t < P.ntiles; t += kThreads) tile_cnt[t] = 0;
-    LaneAddr<BT> la;
-    la.init(tid & 31);
-
-    // equal shares of the item list, weighted by the relative cost of an item of each region
-    const long long I0 = (long long)P.npairs[0] * P.nrb, I1 = (long long)P.npairs[1] * P.nrb;
-    const long long w0 = P.item_cost[0], w1 = P.item_cost[1];
-    const long long T0 = I0 * w0, T = T0 + I1 * w1;
-    auto first_item = [&](long long pos) -> long long {
-        if (pos <= 0) return 0;
-        if (pos >= T) return I0 + I1;
-        long long i = (pos + w0 - 1) / w0;
-        if (i < I0) return i;
-        long long r = pos - T0;
-        return I0 + (r <= 0 ? 0 : (r + w1 - 1) / w1);
-    };
-    long long cur = first_item(T * (long long)blockIdx.x / gridDim.x);
-    const long long end = first_item(T * (long long)(blockIdx.x + 1) / gridDim.x);
-
-    while (cur < end) {
-        const int region = cur >= I0;
-        const long long local = region ? cur - I0 : cur;
-        const int pair = (int)(local / P.nrb), rb_lo = (int)(local % P.nrb);
-        const long long seg_end = min(end, cur - rb_lo + P.nrb);
-        const int rb_hi = rb_lo + (int)(seg_end - cur);
-        const uint8_t *items = P.packed + P.off_items[region] + (size_t)pair * P.nrb * P.item_bytes[region];
-        prefetch_run_head(items, P.item_bytes[region], rb_lo, rb_hi);      // weights start moving now
-
-        __syncthreads();     // previous segment's lookups are done before the tables are overwritten
-        const uint8_t *desc = P.packed + P.off_coldesc + (size_t)((region ? P.npairs[0] : 0) + pair) * FB_PAIR_DESC_BYTES;
-        build_tables<BT>(desc, P.x, P.ldx, P.nb, abuf, region ? -1 : (2 * pair) / P.Kb * 128,
-                         (2 * pair + 1) / P.Kb * 128, P.N);
-        if (region == 0) process_rows<SPS0, BT>(items, rb_lo, rb_hi, la, P.acc, P.Mpad);
-        else process_rows<SPS1, BT>(items, rb_lo, rb_hi, la, P.acc, P.Mpad);
-
-        // how many items this CTA contributed to each tile of rows
-        const int t_lo = rb_lo / P.tile_rb, t_hi = (rb_hi - 1) / P.tile_rb;
-        for (int t = t_lo + tid; t <= t_hi; t += kThreads) {
-            int lo = max(rb_lo, t * P.tile_rb), hi = min(rb_hi, (t + 1) * P.tile_rb);
-            tile_cnt[t] += hi - lo;          // one thread per tile, segments are serial: no race
-        }
-        cur = seg_end;
-    }
-
-    // Stage (iii): publish, take a ticket per touched tile; the last arrival finishes the tile.
-    FB_TRACE_AT(2);
     __threadfence();
     __syncthreads();
-    FB_TRACE_AT(3);
-    const int npairs = P.npairs[0] + P.npairs[1];
-    int *done_list = tile_cnt + kMaxTiles;        // tiles this CTA completed, then their count
-    for (int t = tid; t < P.ntiles; t += kThreads) {
+    const int npairs = E.npairs[0] + E.npairs[1];
+    for (int t = tid; t < E.ntiles; t += kThreads) {
         int c = tile_cnt[t];
         int last = 0;
         if (c > 0) {
-            int rbs = min(P.tile_rb, P.nrb - t * P.tile_rb);
-            unsigned old = atomicAdd(P.tickets + t, (unsigned)c);
+            int rbs = min(E.tile_rb, E.nrb - t * E.tile_rb);
+            unsigned old = atomicAdd(E.tickets + t, (unsigned)c);
             last = (old + (unsigned)c == (unsigned)(npairs * rbs));
         }
         tile_cnt[t] = last;
     }
     __syncthreads();
-    if (tid < 32) {                                // warp 0 compacts the completed tiles into a list
+    if (tid < 32) {                                // warp 0 compacts the completed tiles into a list, in place:
+                                                   // a tile's slot in the list never lies beyond its own index
         int cnt = 0;
-        for (int base = 0; base < P.ntiles; base += 32) {
+        for (int base = 0; base < E.ntiles; base += 32) {
             int t = base + tid;
-            int f = (t < P.ntiles) ? tile_cnt[t] : 0;
+            int f = (t < E.ntiles) ? tile_cnt[t] : 0;
             unsigned m = __ballot_sync(0xffffffffu, f);
             if (f) done_list[cnt + __popc(m & ((1u << tid) - 1u))] = t;
             cnt += __popc(m);
@@ -466,50 +421,147 @@ __global__ void __launch_bounds__(kThreads, (BT == 4) ? 1 : 2) fluxbin_linear_ke
     }
     __syncthreads();
     const int ndone = done_list[kMaxTiles];
-    FB_TRACE_AT(4);
-    if (ndone == 0) return;
-    __threadfence();
-    // all rows of all completed tiles in one flat loop of 4-row groups, eight 128-bit loads in
-    // flight per thread (the accumulators live in L2; one round trip serves ~8K rows per CTA)
-    const int gpt = P.tile_rb * 8;                 // 4-row groups per tile
-    const int total = ndone * gpt * BT;
-    constexpr int U = 8;
-    for (int base = tid; base < total; base += U * kThreads) {
-        float4 v[U];
-        float *a[U];
-        int row[U], bb[U];
+    if (ndone > 0) {
+        __threadfence();
+        // all rows of all completed tiles in one flat loop of 4-row groups, four 128-bit loads in
+        // flight per thread (the accumulators live in L2; one round trip serves ~8K rows per CTA)
+        const int gpt = E.tile_rb * 8;                 // 4-row groups per tile
+        const int total = ndone * gpt * BT;
+        constexpr int U = 4;
+        for (int base = tid; base < total; base += U * kThreads) {
+            float4 v[U];
+            float *a[U];
+            int row[U], bb[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            int idx = base + u * kThreads;
-            a[u] = nullptr;
-            if (idx < total) {
-                int li = idx / (gpt * BT), rem = idx - li * (gpt * BT);
-                bb[u] = rem / gpt;
-                row[u] = (done_list[li] * gpt + (rem - bb[u] * gpt)) * 4;
-                if (row[u] < P.Mpad) a[u] = P.acc + (int64_t)bb[u] * P.Mpad + row[u];
+            for (int u = 0; u < U; ++u) {
+                int idx = base + u * kThreads;
+                a[u] = nullptr;
+                if (idx < total) {
+                    int li = idx / (gpt * BT), rem = idx - li * (gpt * BT);
+                    bb[u] = rem / gpt;
+                    row[u] = (done_list[li] * gpt + (rem - bb[u] * gpt)) * 4;
+                    if (row[u] < E.Mpad) a[u] = E.acc + (int64_t)bb[u] * E.Mpad + row[u];
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) if (a[u]) v[u] = __ldcg((const float4 *)a[u]);
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (!a[u]) continue;
+                __stcg((float4 *)a[u], make_float4(0.f, 0.f, 0.f, 0.f));
+                if (bb[u] >= nb) continue;
+                const float e[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    if (row[u] + k >= E.M) break;
+                    if (y_fp32) ((float *)E.y)[(int64_t)bb[u] * E.ldy + row[u] + k] = e[k];
+                    else ((__half *)E.y)[(int64_t)bb[u] * E.ldy + row[u] + k] = __float2half_rn(e[k]);
+                }
             }
         }
-#pragma unroll
-        for (int u = 0; u < U; ++u) if (a[u]) v[u] = __ldcg((const float4 *)a[u]);
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            if (!a[u]) continue;
-            __stcg((float4 *)a[u], make_float4(0.f, 0.f, 0.f, 0.f));
-            if (bb[u] >= P.nb) continue;
-            const float e[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                if (row[u] + k >= P.M) break;
-                if (P.y_fp32) ((float *)P.y)[(int64_t)bb[u] * P.ldy + row[u] + k] = e[k];
-                else ((__half *)P.y)[(int64_t)bb[u] * P.ldy + row[u] + k] = __float2half_rn(e[k]);
-            }
-        }
+        for (int li = tid; li < ndone; li += kThreads) E.tickets[done_list[li]] = 0;
     }
-    for (int li = tid; li < ndone; li += kThreads) P.tickets[done_list[li]] = 0;
-    FB_TRACE_AT(5);
-#ifdef FB_TRACE
-    if (tid == 0 && blockIdx.x < 1024) g_fb_trace[blockIdx.x][6] = ndone;
+    __syncthreads();       // done_list / tile_cnt are reused by the next entry
+}
+
+#ifndef FB_MINB
+#define FB_MINB 2
 #endif
+template <int SPS0, int SPS1, int BT>
+__global__ void __launch_bounds__(kThreads, (BT == 4) ? 1 : (BT == 2) ? 2 : FB_MINB)
+fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
+{
+    // dynamic shared memory: [kTabBase, +tables) at a fixed window address, small buffers after it
+    extern __shared__ __align__(16) uint8_t smem[];
+    const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem);
+    if (smem_base > kTabBase) return;                                    // the host probes this first
+    uint8_t *small = smem + (kTabBase - smem_base) + TabCfg<BT>::kTableBytes;
+    float *abuf = (float *)small;
+    int *tile_cnt = (int *)(abuf + 256 * BT);
+    int *done_list = tile_cnt;                     // compacted in place over the counters
+    int *range = tile_cnt + kMaxTiles + 4;        // [0]: first item, [1]: end item of this CTA in the entry
+    LinearEntry *Es = (LinearEntry *)(range + 8);  // the current entry, copied once (128 bytes)
+    static_assert(sizeof(LinearEntry) == 128, "entry copy below moves 32 words");
+    const int tid = threadIdx.x;
+    FB_TRACE_AT(0);
+
+    LaneAddr<BT> la;
+    la.init(tid & 31);
+
+    // this CTA's share [lo, hi) of the summed item cost of all entries
+    const long long lo = P.total_cost * (long long)blockIdx.x / gridDim.x;
+    const long long hi = P.total_cost * (long long)(blockIdx.x + 1) / gridDim.x;
+    const long long w0 = P.item_cost[0], w1 = P.item_cost[1];
+
+    // first entry that reaches past lo (CTA-uniform binary search over the prefix sums)
+    int e = 0;
+    if (P.table) {
+        int a = 0, b = P.n - 1;
+        while (a < b) {
+            int m = (a + b + 1) >> 1;
+            if (__ldg(&P.table[m].cost_begin) <= lo) a = m; else b = m - 1;
+        }
+        e = a;
+    }
+
+    for (; e < P.n; ++e) {
+        const LinearEntry *src = P.table ? P.table + e : &P.single;
+        if (src->cost_begin >= hi) break;
+        if (tid < 32) ((uint32_t *)Es)[tid] = ((const uint32_t *)src)[tid];
+        __syncthreads();
+        const LinearEntry &E = *Es;
+        const int I0 = E.npairs[0] * E.nrb, I1 = E.npairs[1] * E.nrb;
+        if (tid == 0) {
+            // items of this entry whose start cost lies in [lo, hi): costs are i*w0, then T0 + j*w1
+            const long long T0 = (long long)I0 * w0, T = T0 + (long long)I1 * w1;
+            auto first_item = [&](long long pos) -> int {
+                if (pos <= 0) return 0;
+                if (pos >= T) return I0 + I1;
+                long long i = (pos + w0 - 1) / w0;
+                if (i < I0) return (int)i;
+                long long r = pos - T0;
+                return I0 + (int)(r <= 0 ? 0 : (r + w1 - 1) / w1);
+            };
+            range[0] = first_item(lo - E.cost_begin);
+            range[1] = first_item(hi - E.cost_begin);
+        }
+        for (int t = tid; t < E.ntiles; t += kThreads) tile_cnt[t] = 0;
+        __syncthreads();
+        int cur = range[0];
+        const int end = range[1];
+        __syncthreads();                           // range[] is rewritten for the next entry
+        if (cur >= end) continue;
+
+        while (cur < end) {
+            const int region = cur >= I0;
+            const int local = region ? cur - I0 : cur;
+            const int pair = local / E.nrb, rb_lo = local - pair * E.nrb;
+            const int seg_end = min(end, cur - rb_lo + E.nrb);
+            const int rb_hi = rb_lo + (seg_end - cur);
+            const int ib = region ? ItemBytes<SPS1>::value : ItemBytes<SPS0>::value;
+            const uint8_t *items = E.packed + E.off_items[region] + (size_t)pair * E.nrb * ib;
+            prefetch_run_head(items, ib, (region ? SPS1 : SPS0) == 1 ? 1 : BT == 4 ? 2 : kDepth, rb_lo, rb_hi);   // weights start moving now
+
+            __syncthreads();     // previous segment's lookups are done before the tables are overwritten
+            const uint8_t *desc = E.packed + E.off_coldesc + (size_t)((region ? E.npairs[0] : 0) + pair) * FB_PAIR_DESC_BYTES;
+            build_tables<BT>(desc, E.x, E.ldx, P.nb, abuf, region ? -1 : (2 * pair) / E.Kb * 128,
+                             (2 * pair + 1) / E.Kb * 128, E.N);
+            FB_TRACE_AT(1);
+            if (region == 0) process_rows<SPS0, BT>(items, rb_lo, rb_hi, la, E.acc, E.Mpad);
+            else process_rows<SPS1, BT>(items, rb_lo, rb_hi, la, E.acc, E.Mpad);
+
+            // how many items this CTA contributed to each tile of rows
+            const int t_lo = rb_lo / E.tile_rb, t_hi = (rb_hi - 1) / E.tile_rb;
+            for (int t = t_lo + tid; t <= t_hi; t += kThreads) {
+                int a = max(rb_lo, t * E.tile_rb), b = min(rb_hi, (t + 1) * E.tile_rb);
+                tile_cnt[t] += b - a;            // one thread per tile, segments are serial: no race
+            }
+            cur = seg_end;
+        }
+        FB_TRACE_AT(2);
+        reduce_and_store<BT>(E, P.nb, P.y_fp32, tile_cnt, done_list);
+        FB_TRACE_AT(3);
+    }
 }
 
 // Test hook: build one table set exactly as the kernel does and write it out as [32][256] fp32.
