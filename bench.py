@@ -151,6 +151,11 @@ def main():
     ap.add_argument("--batch", type=int, default=1)
     ap.add_argument("--g", type=int, default=128)
     ap.add_argument("--no-graph", action="store_true", help="plain launches instead of a CUDA graph replay")
+    ap.add_argument("--launch", default="group", choices=["linear", "group", "layer", "stack"],
+                    help="linear: one fluxbin_linear call per linear; group: one plan per set of linears that "
+                         "depend on nothing inside the set ({q,k,v}, {o}, {gate,up}, {down}); layer: one plan per "
+                         "layer; stack: one plan for the whole stack (valid because the workload gives every "
+                         "linear its own input)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ref-linears", type=int, default=7)
     ap.add_argument("--per-linear", action="store_true", help="also print per-linear timings to stderr")
@@ -227,14 +232,35 @@ def main():
         views.append((l, x_dev[ox:ox + B * l.N].view(B, l.N), y_dev[oy:oy + B * l.M].view(B, l.M)))
         ox += B * l.N
         oy += B * l.M
-    launches_per_step = sum(l.weight.num_launches(B) for l in linears)
     packed_bytes = sum(l.packed_bytes for l in linears)
-
     stream = torch.cuda.Stream()
 
+    # how the linears of a step are grouped into launches
+    nlin = len(lins)
+    names = [n for n, _, _ in lins]
+    if args.launch == "linear":
+        groups = None
+    elif args.launch == "group":
+        dep_sets = [["q", "k", "v"], ["o"], ["gate", "up"], ["down"]] if "gate" in names else [[n] for n in names]
+        groups = [[layer * nlin + names.index(n) for n in ds] for layer in range(nl) for ds in dep_sets]
+    elif args.launch == "layer":
+        groups = [[layer * nlin + li for li in range(nlin)] for layer in range(nl)]
+    else:
+        groups = [list(range(len(linears)))]
+    plans = None
+    if groups is not None:
+        plans = [fb_layer.FluxBinPlan([views[i] for i in g]) for g in groups]
+        launches_per_step = sum(p.num_launches() for p in plans)
+    else:
+        launches_per_step = sum(l.weight.num_launches(B) for l in linears)
+
     def issue_all():
-        for l, xv, yv in views:
-            l.forward(xv, ws, out=yv, stream=stream)
+        if plans is not None:
+            for p in plans:
+                p.run(stream=stream)
+        else:
+            for l, xv, yv in views:
+                l.forward(xv, ws, out=yv, stream=stream)
 
     graph = None
     with torch.cuda.stream(stream):
@@ -343,7 +369,8 @@ def main():
                        "g": args.g, "packed_bytes_resident": packed_bytes, "algorithmic_bytes_per_step": bytes_per_step,
                        "l2": "inputs larger than L2 (weights streamed once per step)" if packed_bytes > 4e8
                        else "working set fits L2: L2-warm number",
-                       "launch": "cuda graph replay" if graph is not None else "plain launches",
+                       "launch": ("cuda graph replay" if graph is not None else "plain launches") + f", {args.launch}: "
+                       f"{launches_per_step} kernel launches per step",
                        "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
             "us_per_layer": ms_per_step * 1e3 / nl, "us_per_linear": ms_per_step * 1e3 / len(linears),
             "frac_of_8TBps": achieved / 8000.0,

@@ -177,6 +177,51 @@ int32_t fluxbin_num_launches(const fluxbin_weight_t *w, int32_t B);
 /* Release the host object (never touches device memory).  NULL is allowed. */
 void fluxbin_free(fluxbin_weight_t *w);
 
+/*
+ * A plan runs a fixed list of layers -- each with its own x and y -- in ONE persistent launch:
+ * y_l = X_l * What_l^T for l < n (Eq. 10 for every layer).  The paper removes launch overhead from
+ * its decode step by replaying all kernels from a CUDA graph (Experimental Setup); a plan goes one
+ * step further and lets the table build and the split-K reduction of one layer overlap the weight
+ * stream of the next.  Layers of a plan are independent: no member may read another member's
+ * output (q/k/v or gate/up of a decoder layer qualify; so does any batch of unrelated layers).
+ * Members may share an input.  All members must be of one row-scale format class -- g a multiple of
+ * 128 with several groups per row; g == N (one scale per row) a multiple of 128; or one common
+ * g < 128 -- otherwise FLUXBIN_ERR_UNSUPPORTED (members without salient columns only need to agree
+ * on the class of their global bases).
+ *
+ *   w, d_x, ldx, d_y, ldy   HOST arrays of n handles / DEVICE pointers / leading dimensions
+ *   d_table                 DEVICE buffer of fluxbin_plan_table_bytes(n, B) bytes, 16-byte aligned;
+ *                           written here (stream synchronised) and read by every run
+ *   d_workspace             DEVICE buffer of fluxbin_plan_workspace_bytes(...) bytes, zeroed once
+ *                           with fluxbin_workspace_init before the first run; runs leave it zeroed
+ * The pointers are captured at creation; all buffers must outlive the plan.
+ */
+typedef struct fluxbin_plan fluxbin_plan_t;
+
+size_t fluxbin_plan_table_bytes(int32_t n, int32_t B);
+
+size_t fluxbin_plan_workspace_bytes(int32_t n, const fluxbin_weight_t *const *w, int32_t B);
+
+fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_t *const *w,
+                                     const uint16_t *const *d_x, const int64_t *ldx,
+                                     void *const *d_y, const int64_t *ldy,
+                                     int32_t B, int32_t y_is_fp32,
+                                     void *d_table, size_t table_bytes,
+                                     void *d_workspace, size_t ws_bytes,
+                                     void *cuda_stream, fluxbin_plan_t **out);
+
+/*
+ * Launch the plan on cuda_stream: asynchronous, no allocation, no synchronisation (capturable).
+ * Runs of plans that share a workspace must be ordered on one stream.
+ */
+fluxbin_status_t fluxbin_plan_run(const fluxbin_plan_t *plan, void *cuda_stream);
+
+/* Kernel launches one fluxbin_plan_run issues (one per chunk of up to 4 batch vectors); -1 on NULL. */
+int32_t fluxbin_plan_num_launches(const fluxbin_plan_t *plan);
+
+/* Release the host object (never touches device memory).  NULL is allowed. */
+void fluxbin_plan_free(fluxbin_plan_t *plan);
+
 const char *fluxbin_status_string(fluxbin_status_t s);
 
 /* The cudaError_t of the most recent FLUXBIN_ERR_CUDA on the calling thread (0 if none). */

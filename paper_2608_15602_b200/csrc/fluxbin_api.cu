@@ -277,7 +277,7 @@ extern "C" fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint
     if ((((uintptr_t)d_x) & 15) || (((uintptr_t)d_y) & 15) || (((uintptr_t)d_workspace) & 15)) return FLUXBIN_ERR_ALIGNMENT;
     if (ws_bytes < fluxbin_workspace_size(w, B)) return FLUXBIN_ERR_BUFFER_TOO_SMALL;
     // a 16-segment salient region only exists with a single scale group, where sps[0] is 16 too
-    if (w->h.sps[1] == 16 && w->h.sps[0] != 16) return FLUXBIN_ERR_FORMAT;
+    if (w->h.npairs[1] > 0 && w->h.sps[1] == 16 && w->h.sps[0] != 16) return FLUXBIN_ERR_FORMAT;
     cudaStream_t s = (cudaStream_t)cuda_stream;
 
     fbk::LaunchParams p;
@@ -297,13 +297,141 @@ extern "C" fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint
         fill_entry(p.single, w, d_x + (int64_t)b0 * ldx, ldx, (uint8_t *)d_y + (size_t)b0 * ldy * ysz, ldy, acc, tickets, 0);
         p.nb = nb;
         cudaError_t e;
-        if (nb == 1) e = launch_bt<1>(w->h.sps[0], w->h.sps[1], w->num_sms, p, items, s);
-        else if (nb == 2) e = launch_bt<2>(w->h.sps[0], w->h.sps[1], w->num_sms, p, items, s);
-        else e = launch_bt<4>(w->h.sps[0], w->h.sps[1], w->num_sms, p, items, s);
+        const int s1 = w->h.npairs[1] > 0 ? w->h.sps[1] : 1;
+        if (nb == 1) e = launch_bt<1>(w->h.sps[0], s1, w->num_sms, p, items, s);
+        else if (nb == 2) e = launch_bt<2>(w->h.sps[0], s1, w->num_sms, p, items, s);
+        else e = launch_bt<4>(w->h.sps[0], s1, w->num_sms, p, items, s);
         if (e != cudaSuccess) return cuda_fail(e);
     }
     return FLUXBIN_OK;
 }
+
+// ---- plans: many layers in one persistent launch -------------------------------------------------
+
+struct fluxbin_plan {
+    int n, B, y_fp32, nchunks;
+    int sps0, sps1, num_sms;
+    long long total_cost, items;
+    int item_cost[2];
+    const fbk::LinearEntry *d_table;     // [nchunks][n]
+};
+
+static size_t entry_ws_bytes(const fluxbin_weight_t *w, int bt)
+{
+    return acc_bytes(w, bt) + ((size_t)w->ntiles * 4 + 255) / 256 * 256;
+}
+
+extern "C" size_t fluxbin_plan_table_bytes(int32_t n, int32_t B)
+{
+    if (n < 1 || B < 1) return 0;
+    return (size_t)n * sizeof(fbk::LinearEntry) * (size_t)((B + 3) / 4);
+}
+
+extern "C" size_t fluxbin_plan_workspace_bytes(int32_t n, const fluxbin_weight_t *const *w, int32_t B)
+{
+    if (n < 1 || B < 1 || !w) return 0;
+    const int bt = B >= 3 ? 4 : B;
+    size_t total = 0;
+    for (int i = 0; i < n; ++i) {
+        if (!w[i]) return 0;
+        total += entry_ws_bytes(w[i], bt);
+    }
+    return total;
+}
+
+extern "C" fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_t *const *w,
+                                                const uint16_t *const *d_x, const int64_t *ldx,
+                                                void *const *d_y, const int64_t *ldy,
+                                                int32_t B, int32_t y_is_fp32,
+                                                void *d_table, size_t table_bytes,
+                                                void *d_workspace, size_t ws_bytes,
+                                                void *cuda_stream, fluxbin_plan_t **out)
+{
+    if (!out) return FLUXBIN_ERR_NULL;
+    *out = nullptr;
+    if (!w || !d_x || !ldx || !d_y || !ldy || !d_table || !d_workspace) return FLUXBIN_ERR_NULL;
+    if (n < 1 || B < 1) return FLUXBIN_ERR_RANGE;
+    if ((((uintptr_t)d_table) & 15) || (((uintptr_t)d_workspace) & 15)) return FLUXBIN_ERR_ALIGNMENT;
+    if (table_bytes < fluxbin_plan_table_bytes(n, B)) return FLUXBIN_ERR_BUFFER_TOO_SMALL;
+    int sps1 = 0;
+    for (int i = 0; i < n; ++i) {
+        if (!w[i] || !d_x[i] || !d_y[i]) return FLUXBIN_ERR_NULL;
+        if (ldx[i] < w[i]->h.N || ldy[i] < w[i]->h.M) return FLUXBIN_ERR_RANGE;
+        if ((((uintptr_t)d_x[i]) & 15) || (((uintptr_t)d_y[i]) & 15)) return FLUXBIN_ERR_ALIGNMENT;
+        if (w[i]->h.sps[0] != w[0]->h.sps[0]) return FLUXBIN_ERR_UNSUPPORTED;
+        if (w[i]->h.npairs[1] > 0) {          // the salient format only matters where there is a salient region
+            if (w[i]->h.sps[1] == 16 && w[i]->h.sps[0] != 16) return FLUXBIN_ERR_FORMAT;
+            if (sps1 != 0 && w[i]->h.sps[1] != sps1) return FLUXBIN_ERR_UNSUPPORTED;
+            sps1 = w[i]->h.sps[1];
+        }
+    }
+    if (sps1 == 0) sps1 = 1;
+    if (ws_bytes < fluxbin_plan_workspace_bytes(n, w, B)) return FLUXBIN_ERR_BUFFER_TOO_SMALL;
+
+    const int nchunks = (B + 3) / 4, bt = B >= 3 ? 4 : B;
+    const size_t ysz = y_is_fp32 ? 4 : 2;
+    fbk::LinearEntry *host = (fbk::LinearEntry *)std::malloc(sizeof(fbk::LinearEntry) * (size_t)n * nchunks);
+    if (!host) return FLUXBIN_ERR_UNSUPPORTED;
+    long long cost = 0, items = 0;
+    for (int c = 0; c < nchunks; ++c) {
+        uint8_t *ws = (uint8_t *)d_workspace;
+        cost = 0;
+        items = 0;
+        for (int i = 0; i < n; ++i) {
+            float *acc = (float *)ws;
+            unsigned *tickets = (unsigned *)(ws + acc_bytes(w[i], bt));
+            fill_entry(host[(size_t)c * n + i], w[i], d_x[i] + (int64_t)c * 4 * ldx[i], ldx[i],
+                       (uint8_t *)d_y[i] + (size_t)c * 4 * ldy[i] * ysz, ldy[i], acc, tickets, cost);
+            cost += ((long long)w[i]->h.npairs[0] * 2 + (long long)w[i]->h.npairs[1] * ((sps1 == w[0]->h.sps[0]) ? 2 : 3)) * w[i]->h.nrb;
+            items += (long long)(w[i]->h.npairs[0] + w[i]->h.npairs[1]) * w[i]->h.nrb;
+            ws += entry_ws_bytes(w[i], bt);
+        }
+    }
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    cudaError_t e = cudaMemcpyAsync(d_table, host, sizeof(fbk::LinearEntry) * (size_t)n * nchunks, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    std::free(host);
+    if (e != cudaSuccess) return cuda_fail(e);
+
+    fluxbin_plan *p = new (std::nothrow) fluxbin_plan;
+    if (!p) return FLUXBIN_ERR_UNSUPPORTED;
+    p->n = n; p->B = B; p->y_fp32 = y_is_fp32 != 0; p->nchunks = nchunks;
+    p->sps0 = w[0]->h.sps[0]; p->sps1 = sps1; p->num_sms = w[0]->num_sms;
+    p->total_cost = cost; p->items = items;
+    p->item_cost[0] = 2;
+    p->item_cost[1] = (sps1 == p->sps0) ? 2 : 3;
+    p->d_table = (const fbk::LinearEntry *)d_table;
+    *out = p;
+    return FLUXBIN_OK;
+}
+
+extern "C" fluxbin_status_t fluxbin_plan_run(const fluxbin_plan_t *plan, void *cuda_stream)
+{
+    if (!plan) return FLUXBIN_ERR_NULL;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    fbk::LaunchParams p;
+    std::memset(&p.single, 0, sizeof(p.single));
+    p.n = plan->n;
+    p.y_fp32 = plan->y_fp32;
+    p.item_cost[0] = plan->item_cost[0];
+    p.item_cost[1] = plan->item_cost[1];
+    p.total_cost = plan->total_cost;
+    for (int c = 0; c < plan->nchunks; ++c) {
+        const int nb = (plan->B - 4 * c < 4) ? plan->B - 4 * c : 4;
+        p.table = plan->d_table + (size_t)c * plan->n;
+        p.nb = nb;
+        cudaError_t e;
+        if (nb == 1) e = launch_bt<1>(plan->sps0, plan->sps1, plan->num_sms, p, plan->items, s);
+        else if (nb == 2) e = launch_bt<2>(plan->sps0, plan->sps1, plan->num_sms, p, plan->items, s);
+        else e = launch_bt<4>(plan->sps0, plan->sps1, plan->num_sms, p, plan->items, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    return FLUXBIN_OK;
+}
+
+extern "C" int32_t fluxbin_plan_num_launches(const fluxbin_plan_t *plan) { return plan ? plan->nchunks : -1; }
+
+extern "C" void fluxbin_plan_free(fluxbin_plan_t *plan) { delete plan; }
 
 extern "C" fluxbin_status_t fluxbin_debug_tables(const fluxbin_weight_t *w, const uint16_t *d_x, int32_t pair,
                                                  float *d_tables, int32_t *h_cols, uint16_t *h_alpha, void *cuda_stream)

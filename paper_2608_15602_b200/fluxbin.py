@@ -36,7 +36,8 @@ EXPORTS = ["fluxbin_packed_size", "fluxbin_validate", "fluxbin_pack_host", "flux
            "fluxbin_packed_dims", "fluxbin_pack", "fluxbin_attach", "fluxbin_unpack", "fluxbin_weight_dims",
            "fluxbin_workspace_size", "fluxbin_workspace_init", "fluxbin_linear", "fluxbin_debug_tables",
            "fluxbin_num_table_sets", "fluxbin_num_launches", "fluxbin_free", "fluxbin_status_string",
-           "fluxbin_last_cuda_error"]
+           "fluxbin_last_cuda_error", "fluxbin_plan_table_bytes", "fluxbin_plan_workspace_bytes",
+           "fluxbin_plan_create", "fluxbin_plan_run", "fluxbin_plan_num_launches", "fluxbin_plan_free"]
 
 _LIB = None
 
@@ -70,6 +71,16 @@ def _lib():
         lib.fluxbin_free.restype, lib.fluxbin_free.argtypes = None, [vp]
         lib.fluxbin_status_string.restype, lib.fluxbin_status_string.argtypes = ctypes.c_char_p, [ctypes.c_int]
         lib.fluxbin_last_cuda_error.restype, lib.fluxbin_last_cuda_error.argtypes = ctypes.c_int, []
+        lib.fluxbin_plan_table_bytes.restype, lib.fluxbin_plan_table_bytes.argtypes = sz, [i32, i32]
+        lib.fluxbin_plan_workspace_bytes.restype = sz
+        lib.fluxbin_plan_workspace_bytes.argtypes = [i32, ctypes.POINTER(vp), i32]
+        lib.fluxbin_plan_create.restype = ctypes.c_int
+        lib.fluxbin_plan_create.argtypes = [i32, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(i64),
+                                            ctypes.POINTER(vp), ctypes.POINTER(i64), i32, i32, vp, sz, vp, sz, vp,
+                                            ctypes.POINTER(vp)]
+        lib.fluxbin_plan_run.restype, lib.fluxbin_plan_run.argtypes = ctypes.c_int, [vp, vp]
+        lib.fluxbin_plan_num_launches.restype, lib.fluxbin_plan_num_launches.argtypes = i32, [vp]
+        lib.fluxbin_plan_free.restype, lib.fluxbin_plan_free.argtypes = None, [vp]
         if hasattr(lib, "fluxbin_linear_noalloc"):
             lib.fluxbin_linear_noalloc.restype = ctypes.c_int
             lib.fluxbin_linear_noalloc.argtypes = [vp, vp, i32, i64, vp, i32, i64, vp]
@@ -220,3 +231,59 @@ def debug_tables(w: Weight, d_x: int, pair: int, d_tables: int, stream: int = 0)
     _check(_lib().fluxbin_debug_tables(w.handle, d_x, pair, d_tables, cols.ctypes.data, alpha.ctypes.data, stream),
            "fluxbin_debug_tables")
     return cols, alpha
+
+
+class Plan:
+    """Handle of fluxbin_plan_create: n layers, each with its own x and y, run in one launch."""
+
+    def __init__(self, handle: int, keep):
+        self.handle = handle
+        self._keep = keep            # weights and buffers the plan points into
+
+    def run(self, stream: int = 0):
+        _check(_lib().fluxbin_plan_run(self.handle, stream), "fluxbin_plan_run")
+
+    def num_launches(self) -> int:
+        return int(_lib().fluxbin_plan_num_launches(self.handle))
+
+    def close(self):
+        if self.handle:
+            _lib().fluxbin_plan_free(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def _arr(ctype, values):
+    return (ctype * len(values))(*values)
+
+
+def plan_table_bytes(n: int, B: int) -> int:
+    return int(_lib().fluxbin_plan_table_bytes(n, B))
+
+
+def plan_workspace_bytes(weights, B: int) -> int:
+    hs = _arr(ctypes.c_void_p, [w.handle for w in weights])
+    return int(_lib().fluxbin_plan_workspace_bytes(len(weights), hs, B))
+
+
+def plan_create_status(weights, d_x, ldx, d_y, ldy, B, y_is_fp32, d_table, table_bytes, d_ws, ws_bytes, stream=0):
+    """fluxbin_plan_create returning (status, handle)."""
+    n = len(weights)
+    h = ctypes.c_void_p()
+    st = _lib().fluxbin_plan_create(n, _arr(ctypes.c_void_p, [w.handle for w in weights]),
+                                    _arr(ctypes.c_void_p, list(d_x)), _arr(ctypes.c_int64, list(ldx)),
+                                    _arr(ctypes.c_void_p, list(d_y)), _arr(ctypes.c_int64, list(ldy)),
+                                    B, 1 if y_is_fp32 else 0, d_table, table_bytes, d_ws, ws_bytes, stream,
+                                    ctypes.byref(h))
+    return int(st), h.value
+
+
+def plan_create(weights, d_x, ldx, d_y, ldy, B, y_is_fp32, d_table, table_bytes, d_ws, ws_bytes, stream=0, keep=None):
+    st, h = plan_create_status(weights, d_x, ldx, d_y, ldy, B, y_is_fp32, d_table, table_bytes, d_ws, ws_bytes, stream)
+    _check(st, "fluxbin_plan_create")
+    return Plan(h, (list(weights), keep))

@@ -1,0 +1,115 @@
+"""GPU parity of plans (many layers in one persistent launch) against the CPU oracle."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2608_15602_b200 import synth
+from test_gpu_parity import check, layer_of
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def fb():
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_2608_15602_b200 import build
+    build.build()
+    from paper_2608_15602_b200 import layer
+    return layer
+
+
+def make_members(fb, specs, B, fp32, shared_x=False):
+    members, wants = [], []
+    x_shared = None
+    for i, (M, N, Kb, Ks, g, n_sal) in enumerate(specs):
+        L = layer_of(100 + i, M, N, Kb, Ks, g, n_sal)
+        if shared_x and x_shared is not None:
+            x = x_shared
+        else:
+            x = synth.make_activations(7, i, B, N)
+            x_shared = x
+        lin = fb.FluxBinLinear(L)
+        xt = torch.from_numpy(x.view(np.float16)).cuda()
+        yt = torch.full((B, M), float("nan"), dtype=torch.float32 if fp32 else torch.float16, device="cuda")
+        members.append((lin, xt, yt))
+        wants.append(oracle.linear_direct(L, x))
+    return members, wants
+
+
+SPECS = [(300, 1024, 2, 1, 128, 51), (33, 256, 2, 0, 128, 0), (1000, 2048, 2, 2, 128, 100), (64, 256, 3, 1, 128, 7),
+         (2100, 384, 2, 1, 128, 19), (1, 128, 1, 0, 128, 0)]
+
+
+@pytest.mark.parametrize("B", [1, 2, 3, 6])
+@pytest.mark.parametrize("fp32", [True, False])
+def test_plan_of_mixed_shapes(fb, B, fp32):
+    members, wants = make_members(fb, SPECS, B, fp32)
+    plan = fb.FluxBinPlan(members)
+    assert plan.num_launches() == (B + 3) // 4
+    for rep in range(2):                                   # second run reuses the self-cleaning workspace
+        for _, _, y in members:
+            y.fill_(float("nan"))
+        plan.run()
+        torch.cuda.synchronize()
+        assert int(plan.ws.tensor.count_nonzero()) == 0, "workspace must be left zeroed"
+        for (lin, _, y), want in zip(members, wants):
+            got = y.float().cpu().numpy()
+            if fp32:
+                check(got, want, f"plan member M={lin.M} rep {rep}")
+            else:
+                ulp = np.spacing(np.abs(want).astype(np.float16)).astype(np.float64)
+                rms = np.sqrt(np.mean(want ** 2))
+                assert np.all(np.abs(got - want) <= 1.01 * ulp + 5e-3 * np.maximum(np.abs(want), 1e-2 * rms))
+
+
+def test_plan_members_sharing_one_input(fb):
+    """q/k/v-style: three layers reading the same activation vector."""
+    specs = [(512, 1024, 2, 1, 128, 51), (128, 1024, 2, 1, 128, 51), (128, 1024, 2, 1, 128, 51)]
+    members, wants = make_members(fb, specs, 1, True, shared_x=True)
+    x0 = members[0][1]
+    members = [(lin, x0, y) for lin, _, y in members]
+    plan = fb.FluxBinPlan(members)
+    plan.run()
+    torch.cuda.synchronize()
+    for (lin, _, y), want in zip(members, wants):
+        check(y.cpu().numpy(), want, "shared input")
+
+
+def test_plan_equals_single_calls_on_a_70b_layer(fb):
+    """All seven linears of one Llama-2-70B-shaped layer in one plan vs. the oracle (batch 1)."""
+    members, wants = [], []
+    for li in range(7):
+        L = synth.make_config_linear(4, 1, li)
+        x = synth.make_config_activations(4, 1, li, 1)
+        lin = fb.FluxBinLinear(L)
+        members.append((lin, torch.from_numpy(x.view(np.float16)).cuda(),
+                        torch.empty((1, L.M), dtype=torch.float32, device="cuda")))
+        wants.append(oracle.linear_direct(L, x))
+        del L
+    plan = fb.FluxBinPlan(members)
+    plan.run()
+    torch.cuda.synchronize()
+    for (lin, _, y), want in zip(members, wants):
+        check(y.cpu().numpy(), want, f"70B member {lin.M}x{lin.N}")
+
+
+def test_plan_rejects_mixed_scale_formats_and_bad_buffers(fb):
+    from paper_2608_15602_b200 import fluxbin
+    a = fb.FluxBinLinear(layer_of(1, 64, 256, 2, 0, 128, 0))
+    b = fb.FluxBinLinear(layer_of(2, 64, 256, 2, 0, 64, 0))       # row-scale groups of 64: other format class
+    x = torch.zeros((1, 256), dtype=torch.float16, device="cuda")
+    ya = torch.zeros((1, 64), dtype=torch.float16, device="cuda")
+    yb = torch.zeros((1, 64), dtype=torch.float16, device="cuda")
+    table = torch.zeros(1024, dtype=torch.uint8, device="cuda")
+    ws = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+    args = ([x.data_ptr()] * 2, [256, 256], [ya.data_ptr(), yb.data_ptr()], [64, 64], 1, False)
+    st, _ = fluxbin.plan_create_status([a.weight, b.weight], *args, table.data_ptr(), 1024, ws.data_ptr(), 1 << 16)
+    assert st == 7
+    st, _ = fluxbin.plan_create_status([a.weight, a.weight], *args, table.data_ptr(), 100, ws.data_ptr(), 1 << 16)
+    assert st == 5
+    st, _ = fluxbin.plan_create_status([a.weight, a.weight], *args, table.data_ptr(), 1024, ws.data_ptr(), 64)
+    assert st == 5
+    st, h = fluxbin.plan_create_status([a.weight, a.weight], *args, table.data_ptr(), 1024, ws.data_ptr(), 1 << 16)
+    assert st == 0
+    fluxbin.library().fluxbin_plan_free(h)
