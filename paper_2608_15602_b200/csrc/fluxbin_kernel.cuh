@@ -40,7 +40,7 @@ constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxTiles = 1024;
 #ifndef FB_DEPTH
-#define FB_DEPTH 3
+#define FB_DEPTH 2
 #endif
 constexpr int kDepth = FB_DEPTH;    // register sets (items in flight per warp) in the main loop
 constexpr int kPrefetchTrips = 2;   // L2 prefetch distance in loop trips (one trip = kDepth items per warp)
@@ -266,6 +266,24 @@ template <int BT> struct LaneAddr {
     }
 };
 
+// Two fp32 lanes in one 64-bit register and one add for both (sm_100 packed fp32 pipe).
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi)
+{
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void add2(unsigned long long &acc, unsigned long long v)
+{
+    asm("add.rn.f32x2 %0, %0, %1;" : "+l"(acc) : "l"(v));
+}
+__device__ __forceinline__ float sum2(unsigned long long v)
+{
+    float lo, hi;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+    return lo + hi;
+}
+
 template <int SPS, int BT>
 __device__ __forceinline__ void compute_item(const ItemRegs<SPS> &r, const LaneAddr<BT> &la, float (&out)[BT])
 {
@@ -275,31 +293,53 @@ __device__ __forceinline__ void compute_item(const ItemRegs<SPS> &r, const LaneA
     for (int b = 0; b < BT; ++b) out[b] = 0.f;
 #pragma unroll
     for (int j = 0; j < NSEG; ++j) {
-        float s0[BT], s1[BT];
+        float seg[BT];
+        if constexpr (BT == 1 && SPS >= 4) {
+            // lookups in pairs: PRMT, LDS, PRMT, LDS, one packed add -- 2.5 issue slots per lookup
+            unsigned long long a0 = 0ull, a1 = 0ull;
 #pragma unroll
-        for (int b = 0; b < BT; ++b) { s0[b] = 0.f; s1[b] = 0.f; }
+            for (int q = 0; q < SPS; q += 2) {
+                float v[2];
 #pragma unroll
-        for (int q = 0; q < SPS; ++q) {
-            const int s = j * SPS + q;
-            const uint32_t k = (uint32_t)(s & 3);
-            uint32_t addr;
-            if constexpr (BT == 1) {
-                // byte 1 <- weight byte k (table index p), byte 0 <- packed slot offset k, bytes 2,3 <- 0
-                // (sign replication of the offset byte, which is < 128)
-                addr = prmt(w[s >> 2], la.c[s >> 2], ((0xCu | k) << 12) | ((0xCu | k) << 8) | (k << 4) | (4u | k));
-            } else {
-                uint32_t idx = __byte_perm(w[s >> 2], 0u, 0x4404u | (k << 4));
-                addr = idx | (la.c[0] ^ TabCfg<BT>::lane_const((uint32_t)s));
+                for (int h = 0; h < 2; ++h) {
+                    const int s = j * SPS + q + h;
+                    const uint32_t k = (uint32_t)(s & 3);
+                    // byte 1 <- weight byte k (table index p), byte 0 <- packed slot offset k, bytes 2,3 <- 0
+                    // (sign replication of the offset byte, which is < 128)
+                    uint32_t addr = prmt(w[s >> 2], la.c[s >> 2], ((0xCu | k) << 12) | ((0xCu | k) << 8) | (k << 4) | (4u | k));
+                    v[h] = lds_entry<1>(addr).v[0];
+                }
+                if (q & 2) add2(a1, pack2(v[0], v[1])); else add2(a0, pack2(v[0], v[1]));
             }
-            Vec<BT> e = lds_entry<BT>(addr);
+            add2(a0, a1);
+            seg[0] = sum2(a0);
+        } else {
+            float s0[BT], s1[BT];
 #pragma unroll
-            for (int b = 0; b < BT; ++b) {
-                if (q & 1) s1[b] += e.v[b]; else s0[b] += e.v[b];
+            for (int b = 0; b < BT; ++b) { s0[b] = 0.f; s1[b] = 0.f; }
+#pragma unroll
+            for (int q = 0; q < SPS; ++q) {
+                const int s = j * SPS + q;
+                const uint32_t k = (uint32_t)(s & 3);
+                uint32_t addr;
+                if constexpr (BT == 1) {
+                    addr = prmt(w[s >> 2], la.c[s >> 2], ((0xCu | k) << 12) | ((0xCu | k) << 8) | (k << 4) | (4u | k));
+                } else {
+                    uint32_t idx = __byte_perm(w[s >> 2], 0u, 0x4404u | (k << 4));
+                    addr = idx | (la.c[0] ^ TabCfg<BT>::lane_const((uint32_t)s));
+                }
+                Vec<BT> e = lds_entry<BT>(addr);
+#pragma unroll
+                for (int b = 0; b < BT; ++b) {
+                    if (q & 1) s1[b] += e.v[b]; else s0[b] += e.v[b];
+                }
             }
+#pragma unroll
+            for (int b = 0; b < BT; ++b) seg[b] = s0[b] + s1[b];
         }
         float scale = h2f((r.sc[j >> 1] >> ((j & 1) * 16)) & 0xffffu);
 #pragma unroll
-        for (int b = 0; b < BT; ++b) out[b] = fmaf(scale, s0[b] + s1[b], out[b]);
+        for (int b = 0; b < BT; ++b) out[b] = fmaf(scale, seg[b], out[b]);
     }
 }
 
@@ -465,7 +505,7 @@ __device__ __forceinline__ void reduce_and_store(const LinearEntry &E, int nb, i
 }
 
 #ifndef FB_MINB
-#define FB_MINB 2
+#define FB_MINB 3
 #endif
 template <int SPS0, int SPS1, int BT>
 __global__ void __launch_bounds__(kThreads, (BT == 4) ? 1 : (BT == 2) ? 2 : FB_MINB)
