@@ -5,7 +5,12 @@ Workload (N=1): the Llama-2-70B-shaped stack of decode linears -- 80 layers x {q
 up, down}, 2 global bases + 1 extra base on a seeded random 5 % of the input columns, g = 128,
 batch 1, fp16 activations, every linear with its own input, all 560 packed layers resident in HBM
 at once (about 21 GB, far larger than L2, so every step streams the weights from HBM).  A "step" is
-one forward token: one fluxbin_linear call per linear, replayed from a CUDA graph.
+one forward token.  --launch says how its 560 linears are launched (replayed from a CUDA graph):
+  stack   one fluxbin_plan launch for the whole step (default; the workload gives every linear its own
+          input, so all 560 are independent and the persistent kernel streams them back to back)
+  layer   one plan per layer (80 launches)
+  group   one plan per set of linears a decoder could run together: {q,k,v} {o} {gate,up} {down} (320)
+  linear  one fluxbin_linear call per linear (560)
 
 value = algorithmic bytes moved per second over all GPUs (GB/s); us_per_layer and us_per_linear
 carry the latency side of the metric.  With --gpus N the N ranks run independent replicas (the
@@ -54,7 +59,7 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """nvidia-smi clocks and throttle reasons sampled every 200 ms while the timed region runs."""
+    """nvidia-smi clocks and throttle reasons sampled every 50 ms while the timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
@@ -67,7 +72,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "200", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+                                          "-lms", "50", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except OSError:
@@ -102,21 +107,22 @@ def stack_spec(config: int, layers: int | None):
     return lins, nl
 
 
-def cpu_oracle_sample(config: int, B: int, max_linears: int = 7):
-    """Time the oracle as it stands on the linears of layer 0 (bounded sample); returns
+def cpu_oracle_sample(config: int, B: int, max_linears: int = 28):
+    """Time the oracle as it stands on the first linears of the stack (bounded sample); returns
     (GB/s of algorithmic bytes, seconds, bytes, cores, description)."""
     import oracle
-    lins, _ = synth.config_linears(config)
-    n = min(max_linears, len(lins))
+    lins, nl = synth.config_linears(config)
+    n = min(max_linears, len(lins) * nl)
     tot_b, tot_t = 0, 0.0
-    for li in range(n):
-        L = synth.make_config_linear(config, 0, li)
-        x = synth.make_config_activations(config, 0, li, B)
+    for i in range(n):
+        layer, li = divmod(i, len(lins))
+        L = synth.make_config_linear(config, layer, li)
+        x = synth.make_config_activations(config, layer, li, B)
         t0 = time.perf_counter()
         oracle.linear_direct(L, x)
         tot_t += time.perf_counter() - t0
         tot_b += algorithmic_bytes(L.M, L.N, L.Kb, L.Ks, L.g, L.n_sal, B)
-    return tot_b / tot_t / 1e9, tot_t, tot_b, oracle.num_threads(), f"layer 0 of the stack ({n} linears, B={B})"
+    return tot_b / tot_t / 1e9, tot_t, tot_b, oracle.num_threads(), f"first {n} linears of the stack (B={B})"
 
 
 def run_reference(args, rank):
@@ -143,7 +149,7 @@ def run_reference(args, rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=4, help="workload: 4 = Llama-2-70B-shaped stack")
@@ -151,13 +157,13 @@ def main():
     ap.add_argument("--batch", type=int, default=1)
     ap.add_argument("--g", type=int, default=128)
     ap.add_argument("--no-graph", action="store_true", help="plain launches instead of a CUDA graph replay")
-    ap.add_argument("--launch", default="group", choices=["linear", "group", "layer", "stack"],
+    ap.add_argument("--launch", default="stack", choices=["linear", "group", "layer", "stack"],
                     help="linear: one fluxbin_linear call per linear; group: one plan per set of linears that "
                          "depend on nothing inside the set ({q,k,v}, {o}, {gate,up}, {down}); layer: one plan per "
                          "layer; stack: one plan for the whole stack (valid because the workload gives every "
                          "linear its own input)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--ref-linears", type=int, default=7)
+    ap.add_argument("--ref-linears", type=int, default=7, help="linears per step of --impl reference")
     ap.add_argument("--per-linear", action="store_true", help="also print per-linear timings to stderr")
     args = ap.parse_args()
 

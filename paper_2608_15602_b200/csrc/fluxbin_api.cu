@@ -241,19 +241,23 @@ template <int BT> static cudaError_t launch_bt(int s0, int s1, int num_sms, cons
     return launch<4, 1, BT>(p, num_sms, items, s);
 }
 
-// Measured on B200: an item with one row scale per sub-vector (3072 bytes) takes about 1.5x the
-// time of a 1152-byte item.
-static void item_costs(const FbHeader &h, int cost[2])
+// Work-split cost model, measured on B200 in units of half a 1152-byte item (about 50 ns per CTA):
+// an item with one row scale per sub-vector (3072 bytes) takes about 1.5x a plain item; building one
+// table set (two dependent loads, 8K table entries, two barriers) takes about as long as 18 items.
+constexpr int kBuildCost = 36;
+
+static void item_costs(int sps0, int sps1, int cost[2])
 {
     cost[0] = 2;
-    cost[1] = (h.sps[1] == h.sps[0]) ? 2 : 3;
+    cost[1] = (sps1 == sps0) ? 2 : 3;
 }
 
-static long long entry_cost(const FbHeader &h)
+static long long entry_cost(const FbHeader &h, int sps1)
 {
     int c[2];
-    item_costs(h, c);
-    return ((long long)h.npairs[0] * c[0] + (long long)h.npairs[1] * c[1]) * h.nrb;
+    item_costs(h.sps[0], sps1, c);
+    return (long long)h.npairs[0] * (kBuildCost + (long long)h.nrb * c[0]) +
+           (long long)h.npairs[1] * (kBuildCost + (long long)h.nrb * c[1]);
 }
 
 static void fill_entry(fbk::LinearEntry &E, const fluxbin_weight_t *w, const uint16_t *x, int64_t ldx, void *y, int64_t ldy,
@@ -284,8 +288,10 @@ extern "C" fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint
     p.table = nullptr;
     p.n = 1;
     p.y_fp32 = y_is_fp32 != 0;
-    item_costs(w->h, p.item_cost);
-    p.total_cost = entry_cost(w->h);
+    const int sps1_eff = w->h.npairs[1] > 0 ? w->h.sps[1] : 1;
+    item_costs(w->h.sps[0], sps1_eff, p.item_cost);
+    p.build_cost = kBuildCost;
+    p.total_cost = entry_cost(w->h, sps1_eff);
     const int bt_ws = B >= 3 ? 4 : B;
     float *acc = (float *)d_workspace;
     unsigned *tickets = (unsigned *)((uint8_t *)d_workspace + acc_bytes(w, bt_ws));
@@ -382,7 +388,7 @@ extern "C" fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_
             unsigned *tickets = (unsigned *)(ws + acc_bytes(w[i], bt));
             fill_entry(host[(size_t)c * n + i], w[i], d_x[i] + (int64_t)c * 4 * ldx[i], ldx[i],
                        (uint8_t *)d_y[i] + (size_t)c * 4 * ldy[i] * ysz, ldy[i], acc, tickets, cost);
-            cost += ((long long)w[i]->h.npairs[0] * 2 + (long long)w[i]->h.npairs[1] * ((sps1 == w[0]->h.sps[0]) ? 2 : 3)) * w[i]->h.nrb;
+            cost += entry_cost(w[i]->h, sps1);
             items += (long long)(w[i]->h.npairs[0] + w[i]->h.npairs[1]) * w[i]->h.nrb;
             ws += entry_ws_bytes(w[i], bt);
         }
@@ -398,8 +404,7 @@ extern "C" fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_
     p->n = n; p->B = B; p->y_fp32 = y_is_fp32 != 0; p->nchunks = nchunks;
     p->sps0 = w[0]->h.sps[0]; p->sps1 = sps1; p->num_sms = w[0]->num_sms;
     p->total_cost = cost; p->items = items;
-    p->item_cost[0] = 2;
-    p->item_cost[1] = (sps1 == p->sps0) ? 2 : 3;
+    item_costs(p->sps0, sps1, p->item_cost);
     p->d_table = (const fbk::LinearEntry *)d_table;
     *out = p;
     return FLUXBIN_OK;
@@ -415,6 +420,7 @@ extern "C" fluxbin_status_t fluxbin_plan_run(const fluxbin_plan_t *plan, void *c
     p.y_fp32 = plan->y_fp32;
     p.item_cost[0] = plan->item_cost[0];
     p.item_cost[1] = plan->item_cost[1];
+    p.build_cost = kBuildCost;
     p.total_cost = plan->total_cost;
     for (int c = 0; c < plan->nchunks; ++c) {
         const int nb = (plan->B - 4 * c < 4) ? plan->B - 4 * c : 4;

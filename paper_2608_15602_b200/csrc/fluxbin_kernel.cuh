@@ -69,6 +69,7 @@ struct LaunchParams {
     int nb;                     // live batch rows (<= BT)
     int y_fp32;
     int item_cost[2];           // relative time of one item of each region (work split)
+    int build_cost;             // relative time of building one table set
 };
 
 // The tables start at this shared-window address.  It is a compile-time constant so that it can
@@ -552,15 +553,20 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
         const LinearEntry &E = *Es;
         const int I0 = E.npairs[0] * E.nrb, I1 = E.npairs[1] * E.nrb;
         if (tid == 0) {
-            // items of this entry whose start cost lies in [lo, hi): costs are i*w0, then T0 + j*w1
-            const long long T0 = (long long)I0 * w0, T = T0 + (long long)I1 * w1;
+            // Cost line of this entry: every pair costs build_cost + nrb * item_cost of its region.
+            // The CTA owns the items whose start lies in [lo, hi); a cut inside a pair's build part
+            // goes to that pair's first row block.
+            const long long Pc0 = P.build_cost + (long long)E.nrb * w0, Pc1 = P.build_cost + (long long)E.nrb * w1;
+            const long long T0 = (long long)E.npairs[0] * Pc0, T = T0 + (long long)E.npairs[1] * Pc1;
             auto first_item = [&](long long pos) -> int {
                 if (pos <= 0) return 0;
                 if (pos >= T) return I0 + I1;
-                long long i = (pos + w0 - 1) / w0;
-                if (i < I0) return (int)i;
-                long long r = pos - T0;
-                return I0 + (int)(r <= 0 ? 0 : (r + w1 - 1) / w1);
+                const bool reg1 = pos >= T0;
+                const long long rel = reg1 ? pos - T0 : pos, Pc = reg1 ? Pc1 : Pc0, w = reg1 ? w1 : w0;
+                const long long pair = rel / Pc, within = rel - pair * Pc - P.build_cost;
+                long long rb = within <= 0 ? 0 : (within + w - 1) / w;
+                if (rb > E.nrb) rb = E.nrb;
+                return (reg1 ? I0 : 0) + (int)(pair * E.nrb + rb);
             };
             range[0] = first_item(lo - E.cost_begin);
             range[1] = first_item(hi - E.cost_begin);
