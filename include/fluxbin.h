@@ -159,6 +159,37 @@ fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint16_t *d_x, 
                                 void *d_workspace, size_t ws_bytes, void *cuda_stream);
 
 /*
+ * fluxbin_linear for callers that may not allocate device memory.  (The paper has no counterpart:
+ * this is a convenience of this library.)
+ *
+ * Who needs it: code that runs as a guest inside someone else's process -- an inference-server
+ * backend, a plug-in, a callback on a latency-critical path -- and is handed its input and output
+ * buffers but has no allocator of its own: the host application fixed the memory budget at start-up,
+ * forbids cudaMalloc (it can synchronise the whole device and can fail once memory is fragmented),
+ * and offers no per-call scratch.  Such a caller cannot provide the workspace fluxbin_linear asks for.
+ *
+ * Same arguments and result as fluxbin_linear, minus the workspace: the split-K accumulators and
+ * arrival counters live in a fixed 1 MiB array inside the library image (fluxbin_noalloc_capacity();
+ * every GPU that loads the library holds it until the process exits).  The call allocates nothing --
+ * no cudaMalloc, no cudaFree, no allocating library routine.
+ *
+ *   - Layers whose fluxbin_workspace_size(w, B) exceeds the capacity (more than about 65,000 output
+ *     rows at batch >= 3, 262,000 at batch 1) are rejected with FLUXBIN_ERR_BUFFER_TOO_SMALL.
+ *   - The first call on each device looks up the device address of the array (with that device
+ *     current) and keeps it; make that first call before any stream capture begins.  The current
+ *     device must be the one that holds the layer, else FLUXBIN_ERR_UNSUPPORTED.
+ *   - All calls on a device share the one array, which keeps the previous call's contents: each call
+ *     clears the part it uses (cudaMemsetAsync on cuda_stream) before its kernel runs.  Two calls that
+ *     overlap on the GPU (issued on different streams, or from several host threads at once) race
+ *     on it and give wrong results; order them on one stream.
+ */
+fluxbin_status_t fluxbin_linear_noalloc(const fluxbin_weight_t *w, const uint16_t *d_x, int32_t B, int64_t ldx,
+                                        void *d_y, int32_t y_is_fp32, int64_t ldy, void *cuda_stream);
+
+/* Bytes of the fixed scratch array behind fluxbin_linear_noalloc. */
+size_t fluxbin_noalloc_capacity(void);
+
+/*
  * Test hook for the LUT identity (Eq. 14): build the tables of table-set `pair` (32 tables:
  * two runs of 16 consecutive 8-column sub-vectors) for activation row 0 of d_x exactly as the
  * kernel does, and write them as fp32 [32][256] to DEVICE d_tables.  h_cols (HOST, may be NULL)

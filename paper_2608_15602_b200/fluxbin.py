@@ -37,7 +37,8 @@ EXPORTS = ["fluxbin_packed_size", "fluxbin_validate", "fluxbin_pack_host", "flux
            "fluxbin_workspace_size", "fluxbin_workspace_init", "fluxbin_linear", "fluxbin_debug_tables",
            "fluxbin_num_table_sets", "fluxbin_num_launches", "fluxbin_free", "fluxbin_status_string",
            "fluxbin_last_cuda_error", "fluxbin_plan_table_bytes", "fluxbin_plan_workspace_bytes",
-           "fluxbin_plan_create", "fluxbin_plan_run", "fluxbin_plan_num_launches", "fluxbin_plan_free"]
+           "fluxbin_plan_create", "fluxbin_plan_run", "fluxbin_plan_num_launches", "fluxbin_plan_free",
+           "fluxbin_linear_noalloc", "fluxbin_noalloc_capacity"]
 
 _LIB = None
 
@@ -81,9 +82,9 @@ def _lib():
         lib.fluxbin_plan_run.restype, lib.fluxbin_plan_run.argtypes = ctypes.c_int, [vp, vp]
         lib.fluxbin_plan_num_launches.restype, lib.fluxbin_plan_num_launches.argtypes = i32, [vp]
         lib.fluxbin_plan_free.restype, lib.fluxbin_plan_free.argtypes = None, [vp]
-        if hasattr(lib, "fluxbin_linear_noalloc"):
-            lib.fluxbin_linear_noalloc.restype = ctypes.c_int
-            lib.fluxbin_linear_noalloc.argtypes = [vp, vp, i32, i64, vp, i32, i64, vp]
+        lib.fluxbin_linear_noalloc.restype = ctypes.c_int
+        lib.fluxbin_linear_noalloc.argtypes = [vp, vp, i32, i64, vp, i32, i64, vp]
+        lib.fluxbin_noalloc_capacity.restype, lib.fluxbin_noalloc_capacity.argtypes = sz, []
         _LIB = lib
     return _LIB
 
@@ -223,6 +224,19 @@ def linear_status(w: Weight, d_x, B, ldx, d_y, y_is_fp32, ldy, d_ws, ws_bytes, s
     """Same call, returning the raw status (for argument-validation tests)."""
     return int(_lib().fluxbin_linear(w.handle if w else None, d_x, B, ldx, d_y, 1 if y_is_fp32 else 0, ldy, d_ws,
                                      ws_bytes, stream))
+
+
+def linear_noalloc_status(w: Weight, d_x: int, B: int, ldx: int, d_y: int, y_is_fp32: bool, ldy: int, stream: int = 0) -> int:
+    """fluxbin_linear_noalloc (no workspace argument: the scratch is a fixed array inside the library)."""
+    return int(_lib().fluxbin_linear_noalloc(w.handle if w else None, d_x, B, ldx, d_y, 1 if y_is_fp32 else 0, ldy, stream))
+
+
+def linear_noalloc(w: Weight, d_x: int, B: int, ldx: int, d_y: int, y_is_fp32: bool, ldy: int, stream: int = 0):
+    _check(linear_noalloc_status(w, d_x, B, ldx, d_y, y_is_fp32, ldy, stream), "fluxbin_linear_noalloc")
+
+
+def noalloc_capacity() -> int:
+    return int(_lib().fluxbin_noalloc_capacity())
 
 
 def debug_tables(w: Weight, d_x: int, pair: int, d_tables: int, stream: int = 0):
