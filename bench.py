@@ -343,14 +343,12 @@ def main():
         print(json.dumps({"per_linear_plain_launches": per_linear}), file=sys.stderr)
 
     # ---- max over ranks, aggregate ------------------------------------------------------------------
-    t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms, e2e_ms = float(t[0]), float(t[1])
+    from paper_2608_15602_b200 import dist_util
+    total_ms, e2e_ms = dist_util.max_over_ranks([total_ms, e2e_ms], device="cuda")
     bytes_per_step = sum(alg_bytes)
     ms_per_step = total_ms / args.steps
-    value = world * bytes_per_step / (ms_per_step * 1e-3) / 1e9
-    e2e_value = world * bytes_per_step / (e2e_ms / args.steps * 1e-3) / 1e9
+    value = dist_util.replica_throughput(bytes_per_step, ms_per_step, world)
+    e2e_value = dist_util.replica_throughput(bytes_per_step, e2e_ms / args.steps, world)
 
     if rank == 0:
         peaks, peak_kind = measured_peaks()

@@ -157,34 +157,45 @@ __device__ __forceinline__ void prefetch_l2(const void *p, uint32_t bytes)
 // ---------------------------------------------------------------------------------------------
 // Stage (i): LUT building with scale fusion (Eq. 14 with a_n = x[col_n] * alpha_c[col_n], Eq. 11;
 // for salient tables col_n = sal_idx[v] and alpha = gathered scale, Eq. 13).
-// abuf: shared scratch of 32*8*BT floats.  Ends with the tables visible to the whole CTA.
+// abuf: shared scratch of 32*8*BT floats.  build_tables ends with the tables visible to the whole CTA.
 // col0_a / col0_b: first column of the pair's two units for a global pair, -1 for a salient pair.
 // ---------------------------------------------------------------------------------------------
+// The two values a thread contributes to a table set: x of its column (per batch vector) and the
+// fused column scale.
+template <int BT> struct BuildInput {
+    float xv[BT];
+    uint32_t e;        // {u16 column, fp16 alpha}
+};
+
 template <int BT>
-__device__ __forceinline__ void build_tables(const uint8_t *pair_desc, const uint16_t *x, int64_t ldx, int nb,
-                                             float *abuf, int col0_a, int col0_b, int ncols)
+__device__ __forceinline__ void fetch_build_input(BuildInput<BT> &in, const uint8_t *pair_desc, const uint16_t *x,
+                                                  int64_t ldx, int nb, int col0_a, int col0_b, int ncols)
+{
+    const int tid = threadIdx.x;
+    // {u16 column, fp16 alpha} of (slot tid/8, n tid%8).  For a global pair the column is also known
+    // from the pair's position, so x and alpha are fetched side by side, not in a chain.
+    if (col0_a >= 0) {       // first unit of the pair: slots 0..15, second unit: slots 16..31
+        const uint32_t col = (uint32_t)(tid < 128 ? col0_a : col0_b) + (uint32_t)(tid & 127);
+        const bool live = col < (uint32_t)ncols;          // padded columns carry alpha = 0
+#pragma unroll
+        for (int b = 0; b < BT; ++b) in.xv[b] = (b < nb && live) ? h2f(__ldg(x + (int64_t)b * ldx + col)) : 0.f;
+        in.e = __ldg((const uint32_t *)pair_desc + tid);
+    } else {
+        in.e = __ldg((const uint32_t *)pair_desc + tid);
+        const uint32_t col = in.e & 0xffffu;
+#pragma unroll
+        for (int b = 0; b < BT; ++b) in.xv[b] = (b < nb) ? h2f(__ldg(x + (int64_t)b * ldx + col)) : 0.f;
+    }
+}
+
+template <int BT>
+__device__ __forceinline__ void build_tables(const BuildInput<BT> &in, float *abuf)
 {
     const int tid = threadIdx.x;
     {
-        // {u16 column, fp16 alpha} of (slot tid/8, n tid%8).  For a global pair the column is also
-        // known from the pair's position, so x and alpha are fetched side by side, not in a chain.
-        float xv[BT];
-        uint32_t e;
-        if (col0_a >= 0) {       // first unit of the pair: slots 0..15, second unit: slots 16..31
-            const uint32_t col = (uint32_t)(tid < 128 ? col0_a : col0_b) + (uint32_t)(tid & 127);
-            const bool live = col < (uint32_t)ncols;          // padded columns carry alpha = 0
+        const float al = h2f(in.e >> 16);
 #pragma unroll
-            for (int b = 0; b < BT; ++b) xv[b] = (b < nb && live) ? h2f(__ldg(x + (int64_t)b * ldx + col)) : 0.f;
-            e = __ldg((const uint32_t *)pair_desc + tid);
-        } else {
-            e = __ldg((const uint32_t *)pair_desc + tid);
-            const uint32_t col = e & 0xffffu;
-#pragma unroll
-            for (int b = 0; b < BT; ++b) xv[b] = (b < nb) ? h2f(__ldg(x + (int64_t)b * ldx + col)) : 0.f;
-        }
-        const float al = h2f(e >> 16);
-#pragma unroll
-        for (int b = 0; b < BT; ++b) abuf[tid * BT + b] = xv[b] * al;     // exact in fp32: two 11-bit significands
+        for (int b = 0; b < BT; ++b) abuf[tid * BT + b] = in.xv[b] * al;     // exact in fp32: two 11-bit significands
     }
     __syncthreads();
     const int lane = tid & 31, warp = tid >> 5;
@@ -578,6 +589,15 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
         __syncthreads();                           // range[] is rewritten for the next entry
         if (cur >= end) continue;
 
+        // a segment = the CTA's row blocks of one pair
+        auto fetch_for = [&](int item, BuildInput<BT> &in) {
+            const int region = item >= I0;
+            const int pair = (region ? item - I0 : item) / E.nrb;
+            const uint8_t *desc = E.packed + E.off_coldesc + (size_t)((region ? E.npairs[0] : 0) + pair) * FB_PAIR_DESC_BYTES;
+            fetch_build_input<BT>(in, desc, E.x, E.ldx, P.nb, region ? -1 : (2 * pair) / E.Kb * 128,
+                                  (2 * pair + 1) / E.Kb * 128, E.N);
+        };
+        BuildInput<BT> bin;
         while (cur < end) {
             const int region = cur >= I0;
             const int local = region ? cur - I0 : cur;
@@ -589,9 +609,10 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
             prefetch_run_head(items, ib, (region ? SPS1 : SPS0) == 1 ? 1 : BT == 4 ? 2 : kDepth, rb_lo, rb_hi);   // weights start moving now
 
             __syncthreads();     // previous segment's lookups are done before the tables are overwritten
-            const uint8_t *desc = E.packed + E.off_coldesc + (size_t)((region ? E.npairs[0] : 0) + pair) * FB_PAIR_DESC_BYTES;
-            build_tables<BT>(desc, E.x, E.ldx, P.nb, abuf, region ? -1 : (2 * pair) / E.Kb * 128,
-                             (2 * pair + 1) / E.Kb * 128, E.N);
+            // (fetching the next pair's inputs here, ahead of the lookups, was measured 15 % slower: the
+            // two extra live registers push the lookup loop over the 80-register budget of 3 CTAs per SM)
+            fetch_for(cur, bin);
+            build_tables<BT>(bin, abuf);
             FB_TRACE_AT(1);
             if (region == 0) process_rows<SPS0, BT>(items, rb_lo, rb_hi, la, E.acc, E.Mpad);
             else process_rows<SPS1, BT>(items, rb_lo, rb_hi, la, E.acc, E.Mpad);
@@ -618,7 +639,9 @@ fluxbin_debug_tables_kernel(const uint8_t *pair_desc, const uint16_t *x, float *
     const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem);
     if (smem_base > kTabBase) return;
     uint8_t *tables = smem + (kTabBase - smem_base);
-    build_tables<1>(pair_desc, x, 0, 1, (float *)(tables + TabCfg<1>::kTableBytes), -1, -1, 0);
+    BuildInput<1> bin;
+    fetch_build_input<1>(bin, pair_desc, x, 0, 1, -1, -1, 0);
+    build_tables<1>(bin, (float *)(tables + TabCfg<1>::kTableBytes));
     for (int i = threadIdx.x; i < 32 * 256; i += kThreads) {
         uint32_t sigma = i >> 8, p = i & 255;
         out[i] = *(const float *)(tables + (TabCfg<1>::lane_const(sigma) | (p << 8)));
