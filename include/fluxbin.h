@@ -131,7 +131,7 @@ fluxbin_status_t fluxbin_weight_dims(const fluxbin_weight_t *w, fluxbin_layer_de
 
 /*
  * DEVICE workspace bytes fluxbin_linear needs for batch size B with this layer: fp32 split-K
- * accumulators for up to 4 batch rows at a time plus one arrival counter per tile of output
+ * accumulators for up to 2 batch rows at a time plus one arrival counter per tile of output
  * rows (stage (iii) "reduction" of Sec. 3.2).  The workspace must be zeroed once with
  * fluxbin_workspace_init before its first use; every call leaves it zeroed again, so one
  * workspace of the maximum size can serve any sequence of stream-ordered calls.
@@ -150,7 +150,7 @@ fluxbin_status_t fluxbin_workspace_init(void *d_workspace, size_t bytes, void *c
  *   d_workspace / ws_bytes   see fluxbin_workspace_size
  *
  * Asynchronous on cuda_stream; performs no allocation and no synchronisation, so calls can be
- * captured into a CUDA graph.  B >= 1 arbitrary (processed in chunks of up to 4 vectors).  Calls
+ * captured into a CUDA graph.  B >= 1 arbitrary (processed in chunks of up to 2 vectors).  Calls
  * sharing a workspace must be ordered on one stream.  Accumulation is fp32 with fp32 atomics
  * across K slices, so results may differ in the last bits from run to run.
  */
@@ -173,8 +173,8 @@ fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint16_t *d_x, 
  * every GPU that loads the library holds it until the process exits).  The call allocates nothing --
  * no cudaMalloc, no cudaFree, no allocating library routine.
  *
- *   - Layers whose fluxbin_workspace_size(w, B) exceeds the capacity (more than about 65,000 output
- *     rows at batch >= 3, 262,000 at batch 1) are rejected with FLUXBIN_ERR_BUFFER_TOO_SMALL.
+ *   - Layers whose fluxbin_workspace_size(w, B) exceeds the capacity (more than about 130,000 output
+ *     rows at batch >= 2, 260,000 at batch 1) are rejected with FLUXBIN_ERR_BUFFER_TOO_SMALL.
  *   - The first call on each device looks up the device address of the array (with that device
  *     current) and keeps it; make that first call before any stream capture begins.  The current
  *     device must be the one that holds the layer, else FLUXBIN_ERR_UNSUPPORTED.
@@ -247,7 +247,7 @@ fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_t *const *w
  */
 fluxbin_status_t fluxbin_plan_run(const fluxbin_plan_t *plan, void *cuda_stream);
 
-/* Kernel launches one fluxbin_plan_run issues (one per chunk of up to 4 batch vectors); -1 on NULL. */
+/* Kernel launches one fluxbin_plan_run issues (one per chunk of up to 2 batch vectors); -1 on NULL. */
 int32_t fluxbin_plan_num_launches(const fluxbin_plan_t *plan);
 
 /* Release the host object (never touches device memory).  NULL is allowed. */

@@ -83,7 +83,6 @@ fluxbin_status_t device_setup(int dev, int *num_sms)
         if (major == 10) {
             FB_CUDA(opt_in_bt<1>());
             FB_CUDA(opt_in_bt<2>());
-            FB_CUDA(opt_in_bt<4>());
             FB_CUDA(cudaFuncSetAttribute(fbk::fluxbin_debug_tables_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)fbk::smem_bytes<1>()));
             FB_CUDA(cudaFuncSetAttribute(fbk::fluxbin_smem_base_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -190,10 +189,17 @@ extern "C" void fluxbin_free(fluxbin_weight_t *w) { delete w; }
 
 extern "C" int32_t fluxbin_num_table_sets(const fluxbin_weight_t *w) { return w ? w->h.npairs[0] + w->h.npairs[1] : -1; }
 
+// Batch vectors per launch: B is processed in chunks of two (the last chunk may hold one).  Measured
+// on B200: two passes with two vectors' table entries side by side (LDS.64, 3 CTAs per SM) beat one
+// pass with four (LDS.128, 128 KB of tables, 1 CTA per SM) by 12 % -- both are shared-memory bound.
+static int chunk_size() { return 2; }
+static int num_chunks(int B) { return (B + chunk_size() - 1) / chunk_size(); }
+static int ws_bt(int B) { return B == 1 ? 1 : 2; }
+
 extern "C" int32_t fluxbin_num_launches(const fluxbin_weight_t *w, int32_t B)
 {
     if (!w || B < 1) return -1;
-    return (B + 3) / 4;      // chunks of up to 4 vectors (the last chunk runs as 1, 2 or 4)
+    return num_chunks(B);
 }
 
 // ---- workspace ----------------------------------------------------------------------------------
@@ -203,7 +209,7 @@ static size_t acc_bytes(const fluxbin_weight_t *w, int bt) { return ((size_t)bt 
 extern "C" size_t fluxbin_workspace_size(const fluxbin_weight_t *w, int32_t B)
 {
     if (!w || B < 1) return 0;
-    int bt = B >= 3 ? 4 : B;
+    int bt = ws_bt(B);
     return acc_bytes(w, bt) + ((size_t)w->ntiles * 4 + 255) / 256 * 256;
 }
 
@@ -292,21 +298,21 @@ extern "C" fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint
     item_costs(w->h.sps[0], sps1_eff, p.item_cost);
     p.build_cost = kBuildCost;
     p.total_cost = entry_cost(w->h, sps1_eff);
-    const int bt_ws = B >= 3 ? 4 : B;
+    const int bt_ws = ws_bt(B);
     float *acc = (float *)d_workspace;
     unsigned *tickets = (unsigned *)((uint8_t *)d_workspace + acc_bytes(w, bt_ws));
     const long long items = (long long)(w->h.npairs[0] + w->h.npairs[1]) * w->h.nrb;
 
     const size_t ysz = y_is_fp32 ? 4 : 2;
-    for (int b0 = 0; b0 < B; b0 += 4) {
-        const int nb = (B - b0 < 4) ? B - b0 : 4;
+    const int CH = chunk_size();
+    for (int b0 = 0; b0 < B; b0 += CH) {
+        const int nb = (B - b0 < CH) ? B - b0 : CH;
         fill_entry(p.single, w, d_x + (int64_t)b0 * ldx, ldx, (uint8_t *)d_y + (size_t)b0 * ldy * ysz, ldy, acc, tickets, 0);
         p.nb = nb;
         cudaError_t e;
         const int s1 = w->h.npairs[1] > 0 ? w->h.sps[1] : 1;
         if (nb == 1) e = launch_bt<1>(w->h.sps[0], s1, w->num_sms, p, items, s);
-        else if (nb == 2) e = launch_bt<2>(w->h.sps[0], s1, w->num_sms, p, items, s);
-        else e = launch_bt<4>(w->h.sps[0], s1, w->num_sms, p, items, s);
+        else e = launch_bt<2>(w->h.sps[0], s1, w->num_sms, p, items, s);
         if (e != cudaSuccess) return cuda_fail(e);
     }
     return FLUXBIN_OK;
@@ -330,13 +336,13 @@ static size_t entry_ws_bytes(const fluxbin_weight_t *w, int bt)
 extern "C" size_t fluxbin_plan_table_bytes(int32_t n, int32_t B)
 {
     if (n < 1 || B < 1) return 0;
-    return (size_t)n * sizeof(fbk::LinearEntry) * (size_t)((B + 3) / 4);
+    return (size_t)n * sizeof(fbk::LinearEntry) * (size_t)num_chunks(B);
 }
 
 extern "C" size_t fluxbin_plan_workspace_bytes(int32_t n, const fluxbin_weight_t *const *w, int32_t B)
 {
     if (n < 1 || B < 1 || !w) return 0;
-    const int bt = B >= 3 ? 4 : B;
+    const int bt = ws_bt(B);
     size_t total = 0;
     for (int i = 0; i < n; ++i) {
         if (!w[i]) return 0;
@@ -374,7 +380,7 @@ extern "C" fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_
     if (sps1 == 0) sps1 = 1;
     if (ws_bytes < fluxbin_plan_workspace_bytes(n, w, B)) return FLUXBIN_ERR_BUFFER_TOO_SMALL;
 
-    const int nchunks = (B + 3) / 4, bt = B >= 3 ? 4 : B;
+    const int nchunks = num_chunks(B), bt = ws_bt(B), CH = chunk_size();
     const size_t ysz = y_is_fp32 ? 4 : 2;
     fbk::LinearEntry *host = (fbk::LinearEntry *)std::malloc(sizeof(fbk::LinearEntry) * (size_t)n * nchunks);
     if (!host) return FLUXBIN_ERR_UNSUPPORTED;
@@ -386,8 +392,8 @@ extern "C" fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_
         for (int i = 0; i < n; ++i) {
             float *acc = (float *)ws;
             unsigned *tickets = (unsigned *)(ws + acc_bytes(w[i], bt));
-            fill_entry(host[(size_t)c * n + i], w[i], d_x[i] + (int64_t)c * 4 * ldx[i], ldx[i],
-                       (uint8_t *)d_y[i] + (size_t)c * 4 * ldy[i] * ysz, ldy[i], acc, tickets, cost);
+            fill_entry(host[(size_t)c * n + i], w[i], d_x[i] + (int64_t)c * CH * ldx[i], ldx[i],
+                       (uint8_t *)d_y[i] + (size_t)c * CH * ldy[i] * ysz, ldy[i], acc, tickets, cost);
             cost += entry_cost(w[i]->h, sps1);
             items += (long long)(w[i]->h.npairs[0] + w[i]->h.npairs[1]) * w[i]->h.nrb;
             ws += entry_ws_bytes(w[i], bt);
@@ -423,13 +429,13 @@ extern "C" fluxbin_status_t fluxbin_plan_run(const fluxbin_plan_t *plan, void *c
     p.build_cost = kBuildCost;
     p.total_cost = plan->total_cost;
     for (int c = 0; c < plan->nchunks; ++c) {
-        const int nb = (plan->B - 4 * c < 4) ? plan->B - 4 * c : 4;
+        const int CH = chunk_size();
+        const int nb = (plan->B - CH * c < CH) ? plan->B - CH * c : CH;
         p.table = plan->d_table + (size_t)c * plan->n;
         p.nb = nb;
         cudaError_t e;
         if (nb == 1) e = launch_bt<1>(plan->sps0, plan->sps1, plan->num_sms, p, plan->items, s);
-        else if (nb == 2) e = launch_bt<2>(plan->sps0, plan->sps1, plan->num_sms, p, plan->items, s);
-        else e = launch_bt<4>(plan->sps0, plan->sps1, plan->num_sms, p, plan->items, s);
+        else e = launch_bt<2>(plan->sps0, plan->sps1, plan->num_sms, p, plan->items, s);
         if (e != cudaSuccess) return cuda_fail(e);
     }
     return FLUXBIN_OK;

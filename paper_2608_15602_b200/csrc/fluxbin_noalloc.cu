@@ -8,8 +8,8 @@
 #include <cuda_runtime.h>
 #include <mutex>
 
-// Scratch shared by every call on a device.  1 MiB covers any layer with up to 65,000 output rows at
-// any batch size (262,000 rows at batch 1); each GPU that loads the library holds it until exit.
+// Scratch shared by every call on a device.  1 MiB covers any layer with up to 130,000 output rows at
+// any batch size (260,000 rows at batch 1); each GPU that loads the library holds it until exit.
 #define FLUXBIN_NOALLOC_SCRATCH_BYTES (1u << 20)
 static __device__ __align__(256) unsigned char g_fluxbin_noalloc_scratch[FLUXBIN_NOALLOC_SCRATCH_BYTES];
 

@@ -55,12 +55,12 @@ def test_noalloc_rejects_layers_beyond_the_fixed_scratch():
     from paper_2608_15602_b200 import fluxbin, layer
     cap = fluxbin.noalloc_capacity()
     assert cap == 1 << 20
-    L = synth.make_linear(5, 5, 70000, 32, 1, 0, 32)                             # 70,000 rows: needs > 1 MiB at batch 4
+    L = synth.make_linear(5, 5, 140000, 32, 1, 0, 32)                            # 140,000 rows: needs > 1 MiB at batch 2
     lin = layer.FluxBinLinear(L)
-    assert lin.weight.workspace_size(4) > cap
-    x = torch.zeros((4, 32), dtype=torch.float16, device="cuda")
-    y = torch.zeros((4, 70000), dtype=torch.float16, device="cuda")
-    st = fluxbin.linear_noalloc_status(lin.weight, x.data_ptr(), 4, 32, y.data_ptr(), False, 70000)
+    assert lin.weight.workspace_size(2) > cap
+    x = torch.zeros((2, 32), dtype=torch.float16, device="cuda")
+    y = torch.zeros((2, 140000), dtype=torch.float16, device="cuda")
+    st = fluxbin.linear_noalloc_status(lin.weight, x.data_ptr(), 2, 32, y.data_ptr(), False, 140000)
     assert st == 5 and "too small" in fluxbin.status_string(st)
-    assert fluxbin.linear_noalloc_status(lin.weight, x.data_ptr(), 1, 32, y.data_ptr(), False, 70000) == 0   # batch 1 fits
+    assert fluxbin.linear_noalloc_status(lin.weight, x.data_ptr(), 1, 32, y.data_ptr(), False, 140000) == 0  # batch 1 fits
     torch.cuda.synchronize()
