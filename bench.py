@@ -155,7 +155,7 @@ def main():
     ap.add_argument("--config", type=int, default=4, help="workload: 4 = Llama-2-70B-shaped stack")
     ap.add_argument("--layers", type=int, default=None, help="override the number of layers (profiling only)")
     ap.add_argument("--batch", type=int, default=1)
-    ap.add_argument("--g", type=int, default=128)
+    ap.add_argument("--g", type=int, default=128, help="columns per row-scale group; 0 = one scale per row (g = N)")
     ap.add_argument("--no-graph", action="store_true", help="plain launches instead of a CUDA graph replay")
     ap.add_argument("--launch", default="stack", choices=["linear", "group", "layer", "stack"],
                     help="linear: one fluxbin_linear call per linear; group: one plan per set of linears that "
@@ -195,7 +195,7 @@ def main():
     t_setup = time.perf_counter()
     def gen(job):
         layer, li = job
-        return job, synth.make_config_linear(args.config, layer, li, g=args.g), \
+        return job, synth.make_config_linear(args.config, layer, li, g=(args.g or lins[li][2])), \
             synth.make_config_activations(args.config, layer, li, B)
 
     linears, xs_host, alg_bytes = [], [], []
@@ -370,7 +370,7 @@ def main():
             "config": {"workload": f"config {args.config}: Llama-2-70B-shaped decode linear stack" if args.config == 4
                        else f"config {args.config}", "layers": nl, "linears_per_step": len(linears), "batch": B,
                        "Kb": 2, "Ks": 0 if args.config == 0 else 1, "salient_frac": 0.0 if args.config == 0 else 0.05,
-                       "g": args.g, "packed_bytes_resident": packed_bytes, "algorithmic_bytes_per_step": bytes_per_step,
+                       "g": args.g or "N", "packed_bytes_resident": packed_bytes, "algorithmic_bytes_per_step": bytes_per_step,
                        "l2": "inputs larger than L2 (weights streamed once per step)" if packed_bytes > 4e8
                        else "working set fits L2: L2-warm number",
                        "launch": ("cuda graph replay" if graph is not None else "plain launches") + f", {args.launch}: "

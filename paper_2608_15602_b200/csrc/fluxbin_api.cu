@@ -210,7 +210,7 @@ extern "C" size_t fluxbin_workspace_size(const fluxbin_weight_t *w, int32_t B)
 {
     if (!w || B < 1) return 0;
     int bt = ws_bt(B);
-    return acc_bytes(w, bt) + ((size_t)w->ntiles * 4 + 255) / 256 * 256;
+    return acc_bytes(w, bt) + ((size_t)w->ntiles * 4 + 255) / 256 * 256 + 256;    // + the launch counters
 }
 
 extern "C" fluxbin_status_t fluxbin_workspace_init(void *d_workspace, size_t bytes, void *cuda_stream)
@@ -235,7 +235,19 @@ static cudaError_t launch(const fbk::LaunchParams &p, int num_sms, long long ite
     }
     long long grid = (long long)num_sms * occ;
     if (items < grid) grid = items;
-    fbk::fluxbin_linear_kernel<S0, S1, BT><<<(int)grid, fbk::kThreads, fbk::smem_bytes<BT>(), s>>>(p);
+    // Launches with enough work deal 90 % of it out statically and cut the rest into three small
+    // shares per CTA (each worth >= ~200 items), drawn dynamically; small launches stay static.
+    fbk::LaunchParams q = p;
+    constexpr int dyn_pct = 10, dyn_k = 3;
+    const long long rest = p.total_cost * dyn_pct / 100;
+    if (dyn_pct > 0 && dyn_k > 0 && rest / (grid * dyn_k) >= 400) {
+        q.static_cost = p.total_cost - rest;
+        q.nshares = (int)(grid * (1 + dyn_k));
+    } else {
+        q.static_cost = p.total_cost;
+        q.nshares = (int)grid;
+    }
+    fbk::fluxbin_linear_kernel<S0, S1, BT><<<(int)grid, fbk::kThreads, fbk::smem_bytes<BT>(), s>>>(q);
     return cudaGetLastError();
 }
 
@@ -248,14 +260,17 @@ template <int BT> static cudaError_t launch_bt(int s0, int s1, int num_sms, cons
 }
 
 // Work-split cost model, measured on B200 in units of half a 1152-byte item (about 50 ns per CTA):
-// an item with one row scale per sub-vector (3072 bytes) takes about 1.5x a plain item; building one
+// an item with one row scale per sub-vector (3072 bytes) takes about 2x a plain item; building one
 // table set (two dependent loads, 8K table entries, two barriers) takes about as long as 18 items.
 constexpr int kBuildCost = 36;
+// The reduction epilogue a CTA runs when it leaves an entry (fence, tickets, read-back of the tiles it
+// completed): a fixed part plus a part that grows with the rows to convert.
+static long long epilogue_cost(const FbHeader &h) { return 80 + h.Mpad / 128; }
 
 static void item_costs(int sps0, int sps1, int cost[2])
 {
     cost[0] = 2;
-    cost[1] = (sps1 == sps0) ? 2 : 3;
+    cost[1] = (sps1 == sps0) ? 2 : 4;
 }
 
 static long long entry_cost(const FbHeader &h, int sps1)
@@ -263,7 +278,7 @@ static long long entry_cost(const FbHeader &h, int sps1)
     int c[2];
     item_costs(h.sps[0], sps1, c);
     return (long long)h.npairs[0] * (kBuildCost + (long long)h.nrb * c[0]) +
-           (long long)h.npairs[1] * (kBuildCost + (long long)h.nrb * c[1]);
+           (long long)h.npairs[1] * (kBuildCost + (long long)h.nrb * c[1]) + epilogue_cost(h);
 }
 
 static void fill_entry(fbk::LinearEntry &E, const fluxbin_weight_t *w, const uint16_t *x, int64_t ldx, void *y, int64_t ldy,
@@ -301,6 +316,7 @@ extern "C" fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint
     const int bt_ws = ws_bt(B);
     float *acc = (float *)d_workspace;
     unsigned *tickets = (unsigned *)((uint8_t *)d_workspace + acc_bytes(w, bt_ws));
+    p.counters = (unsigned *)((uint8_t *)d_workspace + acc_bytes(w, bt_ws) + ((size_t)w->ntiles * 4 + 255) / 256 * 256);
     const long long items = (long long)(w->h.npairs[0] + w->h.npairs[1]) * w->h.nrb;
 
     const size_t ysz = y_is_fp32 ? 4 : 2;
@@ -326,6 +342,7 @@ struct fluxbin_plan {
     long long total_cost, items;
     int item_cost[2];
     const fbk::LinearEntry *d_table;     // [nchunks][n]
+    unsigned *d_counters;
 };
 
 static size_t entry_ws_bytes(const fluxbin_weight_t *w, int bt)
@@ -348,7 +365,7 @@ extern "C" size_t fluxbin_plan_workspace_bytes(int32_t n, const fluxbin_weight_t
         if (!w[i]) return 0;
         total += entry_ws_bytes(w[i], bt);
     }
-    return total;
+    return total + 256;      // + the launch counters
 }
 
 extern "C" fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_t *const *w,
@@ -412,6 +429,7 @@ extern "C" fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_
     p->total_cost = cost; p->items = items;
     item_costs(p->sps0, sps1, p->item_cost);
     p->d_table = (const fbk::LinearEntry *)d_table;
+    p->d_counters = (unsigned *)((uint8_t *)d_workspace + fluxbin_plan_workspace_bytes(n, w, B) - 256);
     *out = p;
     return FLUXBIN_OK;
 }
@@ -428,6 +446,7 @@ extern "C" fluxbin_status_t fluxbin_plan_run(const fluxbin_plan_t *plan, void *c
     p.item_cost[1] = plan->item_cost[1];
     p.build_cost = kBuildCost;
     p.total_cost = plan->total_cost;
+    p.counters = plan->d_counters;
     for (int c = 0; c < plan->nchunks; ++c) {
         const int CH = chunk_size();
         const int nb = (plan->B - CH * c < CH) ? plan->B - CH * c : CH;

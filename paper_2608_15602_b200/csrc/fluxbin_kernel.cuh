@@ -19,8 +19,8 @@
 // a few items ahead so those loads find their lines in L2.
 //
 // Shared-memory table layout: entry p of table slot sigma lives at  kTabBase + p*256 + sigma*4*BT
-// (BT = batch vectors per launch, their entries side by side; for BT = 4 the two units of a pair
-// get separate 64 KB planes).  A lane at step s reads slot  lane ^ s, so the 32 lanes of a warp
+// (BT = 1 or 2 batch vectors per launch, their entries side by side).  A lane at step s reads slot
+// lane ^ s, so the 32 lanes of a warp
 // always hit 32 different slots: every lookup is bank-conflict free by construction, and the
 // packer has stored each lane's weight bytes in exactly that order, so the byte of step s sits at
 // a compile-time position.  For BT = 1 the whole address is formed by ONE byte-permute (table
@@ -43,7 +43,13 @@ constexpr int kMaxTiles = 1024;
 #define FB_DEPTH 2
 #endif
 constexpr int kDepth = FB_DEPTH;    // register sets (items in flight per warp) in the main loop
-constexpr int kPrefetchTrips = 2;   // L2 prefetch distance in loop trips (one trip = kDepth items per warp)
+#ifndef FB_PF
+#define FB_PF 1
+#endif
+// L2 prefetch distance in loop trips (one trip = kDepth items per warp).  Measured: 1 trip 5.40 TB/s,
+// 2 trips 5.26, 3 trips 4.21, 8 trips 3.58 in a stripped copy of the loop -- far prefetches compete with
+// the demand loads instead of helping them.
+constexpr int kPrefetchTrips = FB_PF;
 
 // One layer of a launch.
 struct LinearEntry {
@@ -70,6 +76,9 @@ struct LaunchParams {
     int y_fp32;
     int item_cost[2];           // relative time of one item of each region (work split)
     int build_cost;             // relative time of building one table set
+    long long static_cost;      // part of the cost line dealt out as one share per CTA
+    int nshares;                // grid size + number of small shares drawn dynamically from the rest
+    unsigned *counters;         // [2] share counter and exit counter, zero on entry and on exit
 };
 
 // The tables start at this shared-window address.  It is a compile-time constant so that it can
@@ -78,14 +87,14 @@ struct LaunchParams {
 constexpr uint32_t kTabBase = 0x800u;
 
 template <int BT> struct TabCfg {
-    static constexpr int kTableBytes = (BT == 4) ? 131072 : 65536;
+    static constexpr int kTableBytes = 65536;
     // scale-fusion scratch, tile counters (+ count of completed tiles), work range, copy of the current entry
     static constexpr int kSmallBytes = 256 * BT * 4 + (kMaxTiles + 4) * 4 + 32 + 128;
     // offset of slot sigma from the table base at step 0; entry p adds p << 8.
     // lane_const(lane ^ s) == lane_const(lane) ^ lane_const(s)
     __host__ __device__ static constexpr uint32_t lane_const(uint32_t sigma)
     {
-        return BT == 1 ? sigma * 4u : BT == 2 ? sigma * 8u : (((sigma >> 4) << 16) | ((sigma & 15u) * 16u));
+        return BT == 1 ? sigma * 4u : sigma * 8u;
     }
 };
 
@@ -116,27 +125,20 @@ __device__ __forceinline__ uint32_t ldg_stream_u32(const void *p)
 template <int BT> struct Vec;
 template <> struct Vec<1> { float v[1]; };
 template <> struct Vec<2> { float v[2]; };
-template <> struct Vec<4> { float v[4]; };
 
 template <int BT> __device__ __forceinline__ Vec<BT> lds_entry(uint32_t addr)
 {
     Vec<BT> r;
     // addr is an offset from the table base; the base is the immediate
     if constexpr (BT == 1) asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(r.v[0]) : "r"(addr), "n"(kTabBase));
-    else if constexpr (BT == 2)
-        asm volatile("ld.shared.v2.f32 {%0,%1}, [%2+%3];" : "=f"(r.v[0]), "=f"(r.v[1]) : "r"(addr), "n"(kTabBase));
-    else asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4+%5];"
-                      : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3]) : "r"(addr), "n"(kTabBase));
+    else asm volatile("ld.shared.v2.f32 {%0,%1}, [%2+%3];" : "=f"(r.v[0]), "=f"(r.v[1]) : "r"(addr), "n"(kTabBase));
     return r;
 }
 
 template <int BT> __device__ __forceinline__ void sts_entry(uint32_t addr, const float *v)
 {
     if constexpr (BT == 1) asm volatile("st.shared.f32 [%0+%2], %1;" ::"r"(addr), "f"(v[0]), "n"(kTabBase) : "memory");
-    else if constexpr (BT == 2)
-        asm volatile("st.shared.v2.f32 [%0+%3], {%1,%2};" ::"r"(addr), "f"(v[0]), "f"(v[1]), "n"(kTabBase) : "memory");
-    else asm volatile("st.shared.v4.f32 [%0+%5], {%1,%2,%3,%4};" ::"r"(addr), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]),
-                      "n"(kTabBase) : "memory");
+    else asm volatile("st.shared.v2.f32 [%0+%3], {%1,%2};" ::"r"(addr), "f"(v[0]), "f"(v[1]), "n"(kTabBase) : "memory");
 }
 
 // PRMT with the full selector: bit 3 of a nibble replicates the sign bit of the selected byte
@@ -278,24 +280,6 @@ template <int BT> struct LaneAddr {
     }
 };
 
-// Two fp32 lanes in one 64-bit register and one add for both (sm_100 packed fp32 pipe).
-__device__ __forceinline__ unsigned long long pack2(float lo, float hi)
-{
-    unsigned long long r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ void add2(unsigned long long &acc, unsigned long long v)
-{
-    asm("add.rn.f32x2 %0, %0, %1;" : "+l"(acc) : "l"(v));
-}
-__device__ __forceinline__ float sum2(unsigned long long v)
-{
-    float lo, hi;
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-    return lo + hi;
-}
-
 template <int SPS, int BT>
 __device__ __forceinline__ void compute_item(const ItemRegs<SPS> &r, const LaneAddr<BT> &la, float (&out)[BT])
 {
@@ -306,26 +290,8 @@ __device__ __forceinline__ void compute_item(const ItemRegs<SPS> &r, const LaneA
 #pragma unroll
     for (int j = 0; j < NSEG; ++j) {
         float seg[BT];
-        if constexpr (BT == 1 && SPS >= 4) {
-            // lookups in pairs: PRMT, LDS, PRMT, LDS, one packed add -- 2.5 issue slots per lookup
-            unsigned long long a0 = 0ull, a1 = 0ull;
-#pragma unroll
-            for (int q = 0; q < SPS; q += 2) {
-                float v[2];
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const int s = j * SPS + q + h;
-                    const uint32_t k = (uint32_t)(s & 3);
-                    // byte 1 <- weight byte k (table index p), byte 0 <- packed slot offset k, bytes 2,3 <- 0
-                    // (sign replication of the offset byte, which is < 128)
-                    uint32_t addr = prmt(w[s >> 2], la.c[s >> 2], ((0xCu | k) << 12) | ((0xCu | k) << 8) | (k << 4) | (4u | k));
-                    v[h] = lds_entry<1>(addr).v[0];
-                }
-                if (q & 2) add2(a1, pack2(v[0], v[1])); else add2(a0, pack2(v[0], v[1]));
-            }
-            add2(a0, a1);
-            seg[0] = sum2(a0);
-        } else {
+        {
+            // (a packed add.f32x2 for two lookups was measured 2 % slower: the pairing costs a MOV per lookup)
             float s0[BT], s1[BT];
 #pragma unroll
             for (int b = 0; b < BT; ++b) { s0[b] = 0.f; s1[b] = 0.f; }
@@ -360,10 +326,6 @@ __device__ __forceinline__ void finish_item(const ItemRegs<SPS> &r, const LaneAd
 {
     float out[BT];
     compute_item<SPS, BT>(r, la, out);
-#if defined(FB_EXP) && (FB_EXP == 4 || FB_EXP == 5)     // experiment: no reduction traffic
-    if (out[0] == 12345.678f) atomicAdd(accp, out[0]);
-    return;
-#endif
 #pragma unroll
     for (int b = 0; b < BT; ++b) atomicAdd(accp + (int64_t)b * Mpad, out[b]);
 }
@@ -380,7 +342,7 @@ __device__ __forceinline__ void process_rows(const uint8_t *pair_items, int rb_l
     constexpr int IB = ItemBytes<SPS>::value;
     constexpr int STRIDE = kWarps * IB;                   // bytes between a warp's consecutive items
     constexpr int SB = (SPS == 16) ? 4 : (SPS == 8) ? 8 : 16;   // scale bytes per lane (per plane)
-    constexpr int D = (SPS == 1) ? 1 : (BT == 4) ? 2 : kDepth;
+    constexpr int D = (SPS == 1) ? 1 : kDepth;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int first = rb_lo + warp;
     if (first >= rb_hi) return;
@@ -520,7 +482,7 @@ __device__ __forceinline__ void reduce_and_store(const LinearEntry &E, int nb, i
 #define FB_MINB 3
 #endif
 template <int SPS0, int SPS1, int BT>
-__global__ void __launch_bounds__(kThreads, (BT == 4) ? 1 : (BT == 2) ? 2 : FB_MINB)
+__global__ void __launch_bounds__(kThreads, (BT == 2) ? 2 : FB_MINB)
 fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
 {
     // dynamic shared memory: [kTabBase, +tables) at a fixed window address, small buffers after it
@@ -540,10 +502,24 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
     LaneAddr<BT> la;
     la.init(tid & 31);
 
-    // this CTA's share [lo, hi) of the summed item cost of all entries
-    const long long lo = P.total_cost * (long long)blockIdx.x / gridDim.x;
-    const long long hi = P.total_cost * (long long)(blockIdx.x + 1) / gridDim.x;
     const long long w0 = P.item_cost[0], w1 = P.item_cost[1];
+
+    // The first P.static_cost of the cost line is cut into one big share per CTA; the rest into small
+    // shares that CTAs draw from a counter when they finish (no CTA waits for another).  Co-resident
+    // CTAs do not progress at the same speed (the warp schedulers favour the older ones), so the
+    // quick ones pick up the small shares and the SM stays fully occupied until the end.
+    const int G = (int)gridDim.x;
+    for (int share = blockIdx.x; share < P.nshares;) {
+    long long lo, hi;
+    if (share < G) {
+        lo = P.static_cost * (long long)share / G;
+        hi = P.static_cost * (long long)(share + 1) / G;
+    } else {
+        const long long rest = P.total_cost - P.static_cost;
+        const int j = share - G, nj = P.nshares - G;
+        lo = P.static_cost + rest * (long long)j / nj;
+        hi = P.static_cost + rest * (long long)(j + 1) / nj;
+    }
 
     // first entry that reaches past lo (CTA-uniform binary search over the prefix sums)
     int e = 0;
@@ -606,7 +582,7 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
             const int rb_hi = rb_lo + (seg_end - cur);
             const int ib = region ? ItemBytes<SPS1>::value : ItemBytes<SPS0>::value;
             const uint8_t *items = E.packed + E.off_items[region] + (size_t)pair * E.nrb * ib;
-            prefetch_run_head(items, ib, (region ? SPS1 : SPS0) == 1 ? 1 : BT == 4 ? 2 : kDepth, rb_lo, rb_hi);   // weights start moving now
+            prefetch_run_head(items, ib, (region ? SPS1 : SPS0) == 1 ? 1 : kDepth, rb_lo, rb_hi);   // weights start moving now
 
             __syncthreads();     // previous segment's lookups are done before the tables are overwritten
             // (fetching the next pair's inputs here, ahead of the lookups, was measured 15 % slower: the
@@ -628,6 +604,17 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
         FB_TRACE_AT(2);
         reduce_and_store<BT>(E, P.nb, P.y_fp32, tile_cnt, done_list);
         FB_TRACE_AT(3);
+    }
+        if (P.nshares <= (int)gridDim.x) break;    // one share per CTA: nothing to draw
+        if (tid == 0) range[2] = (int)gridDim.x + (int)atomicAdd(P.counters, 1u);
+        __syncthreads();
+        share = range[2];
+        __syncthreads();
+    }
+    // the last CTA to leave puts the two launch counters back to zero for the next launch
+    if (P.nshares > (int)gridDim.x && tid == 0) {
+        unsigned old = atomicAdd(P.counters + 1, 1u);
+        if (old == gridDim.x - 1) { P.counters[0] = 0u; P.counters[1] = 0u; }
     }
 }
 
