@@ -28,6 +28,8 @@ def _stale() -> bool:
 
 def build(force: bool = False, verbose: bool = False) -> str:
     """Compile libfluxbin.so if it is missing or older than its sources; returns its path."""
+    if not force and os.environ.get("FLUXBIN_LIB") and os.path.exists(LIB_PATH):
+        return LIB_PATH          # an explicitly chosen library is used as it is
     if not force and not _stale():
         return LIB_PATH
     os.makedirs(LIB_DIR, exist_ok=True)

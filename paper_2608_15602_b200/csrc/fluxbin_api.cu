@@ -56,8 +56,13 @@ std::mutex g_dev_mutex;
 
 template <int S0, int S1, int BT> cudaError_t opt_in()
 {
-    return cudaFuncSetAttribute(fbk::fluxbin_linear_kernel<S0, S1, BT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)fbk::smem_bytes<BT>());
+    cudaError_t e = cudaFuncSetAttribute(fbk::fluxbin_linear_kernel<S0, S1, BT, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)fbk::smem_bytes<BT>());
+    if (e != cudaSuccess) return e;
+    if constexpr (BT == 1)
+        e = cudaFuncSetAttribute(fbk::fluxbin_linear_kernel<S0, S1, BT, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)fbk::smem_bytes<BT>());
+    return e;
 }
 template <int BT> cudaError_t opt_in_bt()
 {
@@ -223,12 +228,12 @@ extern "C" fluxbin_status_t fluxbin_workspace_init(void *d_workspace, size_t byt
 // ---- the layer ------------------------------------------------------------------------------------
 
 template <int S0, int S1, int BT>
-static cudaError_t launch(const fbk::LaunchParams &p, int num_sms, long long items, cudaStream_t s)
+static cudaError_t launch(const fbk::LaunchParams &p, int num_sms, long long items, long long couple_cost, cudaStream_t s)
 {
     static int occ = 0;     // resident CTAs per SM of this instantiation (same on every B200)
     if (occ == 0) {
         int o = 0;
-        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, fbk::fluxbin_linear_kernel<S0, S1, BT>,
+        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, fbk::fluxbin_linear_kernel<S0, S1, BT, 1>,
                                                                       fbk::kThreads, fbk::smem_bytes<BT>());
         if (e != cudaSuccess) return e;
         occ = o > 0 ? o : 1;
@@ -247,17 +252,30 @@ static cudaError_t launch(const fbk::LaunchParams &p, int num_sms, long long ite
         q.static_cost = p.total_cost;
         q.nshares = (int)grid;
     }
-    fbk::fluxbin_linear_kernel<S0, S1, BT><<<(int)grid, fbk::kThreads, fbk::smem_bytes<BT>(), s>>>(q);
+    // two pairs per row block (half the reduction traffic) when every layer allows it (couple_cost > 0:
+    // even pair counts everywhere) and a CTA's share spans several whole couples
+    bool couples = false;
+    if constexpr (BT == 1) couples = couple_cost > 0 && q.static_cost / grid >= 2 * couple_cost;
+    if constexpr (BT == 1) {
+        if (couples) fbk::fluxbin_linear_kernel<S0, S1, BT, 2><<<(int)grid, fbk::kThreads, fbk::smem_bytes<BT>(), s>>>(q);
+        else fbk::fluxbin_linear_kernel<S0, S1, BT, 1><<<(int)grid, fbk::kThreads, fbk::smem_bytes<BT>(), s>>>(q);
+    } else {
+        fbk::fluxbin_linear_kernel<S0, S1, BT, 1><<<(int)grid, fbk::kThreads, fbk::smem_bytes<BT>(), s>>>(q);
+    }
     return cudaGetLastError();
 }
 
-template <int BT> static cudaError_t launch_bt(int s0, int s1, int num_sms, const fbk::LaunchParams &p, long long items, cudaStream_t s)
+// couple_cost: cost of the largest couple of global pairs over the layers of the launch, or 0 when
+// some layer has an odd number of global pairs (then the one-pair kernel runs).
+template <int BT> static cudaError_t launch_bt(int s0, int s1, int num_sms, const fbk::LaunchParams &p, long long items,
+                                               long long couple_cost, cudaStream_t s)
 {
-    if (s0 == 16 && s1 == 16) return launch<16, 16, BT>(p, num_sms, items, s);
-    if (s0 == 16) return launch<16, 1, BT>(p, num_sms, items, s);
-    if (s0 == 8) return launch<8, 1, BT>(p, num_sms, items, s);
-    return launch<4, 1, BT>(p, num_sms, items, s);
+    if (s0 == 16 && s1 == 16) return launch<16, 16, BT>(p, num_sms, items, couple_cost, s);
+    if (s0 == 16) return launch<16, 1, BT>(p, num_sms, items, couple_cost, s);
+    if (s0 == 8) return launch<8, 1, BT>(p, num_sms, items, couple_cost, s);
+    return launch<4, 1, BT>(p, num_sms, items, couple_cost, s);
 }
+
 
 // Work-split cost model, measured on B200 in units of half a 1152-byte item (about 50 ns per CTA):
 // an item with one row scale per sub-vector (3072 bytes) takes about 2x a plain item; building one
@@ -266,6 +284,12 @@ constexpr int kBuildCost = 36;
 // The reduction epilogue a CTA runs when it leaves an entry (fence, tickets, read-back of the tiles it
 // completed): a fixed part plus a part that grows with the rows to convert.
 static long long epilogue_cost(const FbHeader &h) { return 80 + h.Mpad / 128; }
+
+static long long couple_cost_of(const FbHeader &h)
+{
+    if (h.npairs[0] < 2 || (h.npairs[0] & 1)) return 0;
+    return 2 * (kBuildCost + (long long)h.nrb * 2);
+}
 
 static void item_costs(int sps0, int sps1, int cost[2])
 {
@@ -327,8 +351,8 @@ extern "C" fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint
         p.nb = nb;
         cudaError_t e;
         const int s1 = w->h.npairs[1] > 0 ? w->h.sps[1] : 1;
-        if (nb == 1) e = launch_bt<1>(w->h.sps[0], s1, w->num_sms, p, items, s);
-        else e = launch_bt<2>(w->h.sps[0], s1, w->num_sms, p, items, s);
+        if (nb == 1) e = launch_bt<1>(w->h.sps[0], s1, w->num_sms, p, items, couple_cost_of(w->h), s);
+        else e = launch_bt<2>(w->h.sps[0], s1, w->num_sms, p, items, 0, s);
         if (e != cudaSuccess) return cuda_fail(e);
     }
     return FLUXBIN_OK;
@@ -339,7 +363,7 @@ extern "C" fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint
 struct fluxbin_plan {
     int n, B, y_fp32, nchunks;
     int sps0, sps1, num_sms;
-    long long total_cost, items;
+    long long total_cost, items, couple_cost;
     int item_cost[2];
     const fbk::LinearEntry *d_table;     // [nchunks][n]
     unsigned *d_counters;
@@ -427,6 +451,16 @@ extern "C" fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_
     p->n = n; p->B = B; p->y_fp32 = y_is_fp32 != 0; p->nchunks = nchunks;
     p->sps0 = w[0]->h.sps[0]; p->sps1 = sps1; p->num_sms = w[0]->num_sms;
     p->total_cost = cost; p->items = items;
+    p->couple_cost = 0;
+    {
+        bool all_even = true;
+        for (int i = 0; i < n; ++i) {
+            long long c = couple_cost_of(w[i]->h);
+            if (c == 0) all_even = false;
+            if (c > p->couple_cost) p->couple_cost = c;
+        }
+        if (!all_even) p->couple_cost = 0;
+    }
     item_costs(p->sps0, sps1, p->item_cost);
     p->d_table = (const fbk::LinearEntry *)d_table;
     p->d_counters = (unsigned *)((uint8_t *)d_workspace + fluxbin_plan_workspace_bytes(n, w, B) - 256);
@@ -453,8 +487,8 @@ extern "C" fluxbin_status_t fluxbin_plan_run(const fluxbin_plan_t *plan, void *c
         p.table = plan->d_table + (size_t)c * plan->n;
         p.nb = nb;
         cudaError_t e;
-        if (nb == 1) e = launch_bt<1>(plan->sps0, plan->sps1, plan->num_sms, p, plan->items, s);
-        else e = launch_bt<2>(plan->sps0, plan->sps1, plan->num_sms, p, plan->items, s);
+        if (nb == 1) e = launch_bt<1>(plan->sps0, plan->sps1, plan->num_sms, p, plan->items, plan->couple_cost, s);
+        else e = launch_bt<2>(plan->sps0, plan->sps1, plan->num_sms, p, plan->items, 0, s);
         if (e != cudaSuccess) return cuda_fail(e);
     }
     return FLUXBIN_OK;

@@ -126,11 +126,12 @@ template <int BT> struct Vec;
 template <> struct Vec<1> { float v[1]; };
 template <> struct Vec<2> { float v[2]; };
 
-template <int BT> __device__ __forceinline__ Vec<BT> lds_entry(uint32_t addr)
+// HALF selects the table set inside the 256-byte p-rows: slots 0..31 or (BT == 1 only) slots 32..63.
+template <int BT, int HALF> __device__ __forceinline__ Vec<BT> lds_entry(uint32_t addr)
 {
     Vec<BT> r;
-    // addr is an offset from the table base; the base is the immediate
-    if constexpr (BT == 1) asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(r.v[0]) : "r"(addr), "n"(kTabBase));
+    // addr is an offset from the table base; base and half ride in the immediate
+    if constexpr (BT == 1) asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(r.v[0]) : "r"(addr), "n"(kTabBase + HALF * 128));
     else asm volatile("ld.shared.v2.f32 {%0,%1}, [%2+%3];" : "=f"(r.v[0]), "=f"(r.v[1]) : "r"(addr), "n"(kTabBase));
     return r;
 }
@@ -191,7 +192,7 @@ __device__ __forceinline__ void fetch_build_input(BuildInput<BT> &in, const uint
 }
 
 template <int BT>
-__device__ __forceinline__ void build_tables(const BuildInput<BT> &in, float *abuf)
+__device__ __forceinline__ void build_tables(const BuildInput<BT> &in, float *abuf, uint32_t half_off = 0)
 {
     const int tid = threadIdx.x;
     {
@@ -228,7 +229,7 @@ __device__ __forceinline__ void build_tables(const BuildInput<BT> &in, float *ab
         }
 #pragma unroll
         for (int q = 0; q < 16; ++q)
-            sts_entry<BT>(TabCfg<BT>::lane_const((uint32_t)lane) | ((uint32_t)(p0 + q) << 8), v[q]);
+            sts_entry<BT>(half_off | TabCfg<BT>::lane_const((uint32_t)lane) | ((uint32_t)(p0 + q) << 8), v[q]);
     }
     __syncthreads();
 }
@@ -280,7 +281,7 @@ template <int BT> struct LaneAddr {
     }
 };
 
-template <int SPS, int BT>
+template <int SPS, int BT, int HALF = 0>
 __device__ __forceinline__ void compute_item(const ItemRegs<SPS> &r, const LaneAddr<BT> &la, float (&out)[BT])
 {
     constexpr int NSEG = 32 / SPS;
@@ -306,7 +307,7 @@ __device__ __forceinline__ void compute_item(const ItemRegs<SPS> &r, const LaneA
                     uint32_t idx = __byte_perm(w[s >> 2], 0u, 0x4404u | (k << 4));
                     addr = idx | (la.c[0] ^ TabCfg<BT>::lane_const((uint32_t)s));
                 }
-                Vec<BT> e = lds_entry<BT>(addr);
+                Vec<BT> e = lds_entry<BT, HALF>(addr);
 #pragma unroll
                 for (int b = 0; b < BT; ++b) {
                     if (q & 1) s1[b] += e.v[b]; else s0[b] += e.v[b];
@@ -370,6 +371,44 @@ __device__ __forceinline__ void process_rows(const uint8_t *pair_items, int rb_l
         ps += D * STRIDE;
         pp += D * STRIDE;
         accp += D * kWarps * 32;
+    }
+}
+
+// The same for TWO pairs whose table sets are resident together (slots 0..31 and 32..63, BT == 1):
+// for every row block the lane looks up the item of the first pair, then the item of the second
+// (items_b = the second pair's items), adds the two row sums and issues ONE reduction -- half the
+// atomic traffic and half the per-item bookkeeping.  One item is always in flight ahead.
+template <int SPS>
+__device__ __forceinline__ void process_rows2(const uint8_t *items_a, const uint8_t *items_b, int rb_lo, int rb_hi,
+                                              const LaneAddr<1> &la, float *acc)
+{
+    constexpr int IB = ItemBytes<SPS>::value;
+    constexpr int STRIDE = kWarps * IB;
+    constexpr int SB = (SPS == 16) ? 4 : (SPS == 8) ? 8 : 16;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int first = rb_lo + warp;
+    if (first >= rb_hi) return;
+    const int n = (rb_hi - first + kWarps - 1) / kWarps;
+    const int64_t o_l = (int64_t)first * IB + lane * 16, o_s = (int64_t)first * IB + FB_ITEM_BITS_BYTES + lane * SB;
+    const uint8_t *pla = items_a + o_l, *psa = items_a + o_s;
+    const uint8_t *plb = items_b + o_l, *psb = items_b + o_s;
+    // the CTA reads kWarps items of each pair per trip; lanes 0 and 1 of every warp prefetch the
+    // warp's own item of the trip kPrefetchTrips + 1 ahead in the first and the second pair
+    const uint8_t *pp = (lane == 0 ? items_a : items_b) + (int64_t)first * IB + (int64_t)(kPrefetchTrips + 1) * STRIDE;
+    float *accp = acc + first * 32 + lane;
+
+    ItemRegs<SPS> ra, rb;
+    load_item<SPS>(ra, pla, psa, 0);
+    for (int t = 0; t < n; ++t) {
+        if (lane < 2 && t + kPrefetchTrips + 1 < n) prefetch_l2(pp, IB);
+        load_item<SPS>(rb, plb, psb, 0);
+        float oa[1], ob[1];
+        compute_item<SPS, 1, 0>(ra, la, oa);
+        if (t + 1 < n) load_item<SPS>(ra, pla, psa, STRIDE);
+        compute_item<SPS, 1, 1>(rb, la, ob);
+        atomicAdd(accp, oa[0] + ob[0]);
+        pla += STRIDE; psa += STRIDE; plb += STRIDE; psb += STRIDE; pp += STRIDE;
+        accp += kWarps * 32;
     }
 }
 
@@ -481,7 +520,7 @@ __device__ __forceinline__ void reduce_and_store(const LinearEntry &E, int nb, i
 #ifndef FB_MINB
 #define FB_MINB 3
 #endif
-template <int SPS0, int SPS1, int BT>
+template <int SPS0, int SPS1, int BT, int NP>
 __global__ void __launch_bounds__(kThreads, (BT == 2) ? 2 : FB_MINB)
 fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
 {
@@ -496,6 +535,7 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
     int *range = tile_cnt + kMaxTiles + 4;        // [0]: first item, [1]: end item of this CTA in the entry
     LinearEntry *Es = (LinearEntry *)(range + 8);  // the current entry, copied once (128 bytes)
     static_assert(sizeof(LinearEntry) == 128, "entry copy below moves 32 words");
+    static_assert(NP == 1 || BT == 1, "two table sets side by side need the 4-byte slots of BT == 1");
     const int tid = threadIdx.x;
     FB_TRACE_AT(0);
 
@@ -538,19 +578,27 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
         if (tid < 32) ((uint32_t *)Es)[tid] = ((const uint32_t *)src)[tid];
         __syncthreads();
         const LinearEntry &E = *Es;
-        const int I0 = E.npairs[0] * E.nrb, I1 = E.npairs[1] * E.nrb;
+        // With NP == 2 region 0 is walked two pairs at a time, their table sets side by side (BT == 1,
+        // every entry with an even number of global pairs): a "work pair" is then a couple of pairs, a
+        // work row block their two items.  Costs per pair are unchanged, only the cut granularity doubles.
+        // (NP is a kernel template parameter: the host picks the two-pair kernel for launches whose
+        // shares span whole couples -- long runs of rows per table build, as in a plan of many layers;
+        // in a small launch it would make every CTA build twice as much.  Deciding it at run time was
+        // measured slower than either variant: both row loops in one kernel cost registers.)
+        const int wp0 = E.npairs[0] / NP;
+        const int I0 = wp0 * E.nrb, I1 = E.npairs[1] * E.nrb;
         if (tid == 0) {
             // Cost line of this entry: every pair costs build_cost + nrb * item_cost of its region.
-            // The CTA owns the items whose start lies in [lo, hi); a cut inside a pair's build part
-            // goes to that pair's first row block.
-            const long long Pc0 = P.build_cost + (long long)E.nrb * w0, Pc1 = P.build_cost + (long long)E.nrb * w1;
-            const long long T0 = (long long)E.npairs[0] * Pc0, T = T0 + (long long)E.npairs[1] * Pc1;
+            // The CTA owns the work row blocks whose start lies in [lo, hi); a cut inside the build
+            // part of a work pair goes to its first row block.
+            const long long Pc0 = NP * (P.build_cost + (long long)E.nrb * w0), Pc1 = P.build_cost + (long long)E.nrb * w1;
+            const long long T0 = (long long)wp0 * Pc0, T = T0 + (long long)E.npairs[1] * Pc1;
             auto first_item = [&](long long pos) -> int {
                 if (pos <= 0) return 0;
                 if (pos >= T) return I0 + I1;
                 const bool reg1 = pos >= T0;
-                const long long rel = reg1 ? pos - T0 : pos, Pc = reg1 ? Pc1 : Pc0, w = reg1 ? w1 : w0;
-                const long long pair = rel / Pc, within = rel - pair * Pc - P.build_cost;
+                const long long rel = reg1 ? pos - T0 : pos, Pc = reg1 ? Pc1 : Pc0, w = reg1 ? w1 : NP * w0;
+                const long long pair = rel / Pc, within = rel - pair * Pc - (reg1 ? 1 : NP) * P.build_cost;
                 long long rb = within <= 0 ? 0 : (within + w - 1) / w;
                 if (rb > E.nrb) rb = E.nrb;
                 return (reg1 ? I0 : 0) + (int)(pair * E.nrb + rb);
@@ -565,39 +613,48 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
         __syncthreads();                           // range[] is rewritten for the next entry
         if (cur >= end) continue;
 
-        // a segment = the CTA's row blocks of one pair
-        auto fetch_for = [&](int item, BuildInput<BT> &in) {
-            const int region = item >= I0;
-            const int pair = (region ? item - I0 : item) / E.nrb;
+        // a segment = the CTA's row blocks of one work pair
+        auto fetch_for = [&](int region, int pair, BuildInput<BT> &in) {
             const uint8_t *desc = E.packed + E.off_coldesc + (size_t)((region ? E.npairs[0] : 0) + pair) * FB_PAIR_DESC_BYTES;
             fetch_build_input<BT>(in, desc, E.x, E.ldx, P.nb, region ? -1 : (2 * pair) / E.Kb * 128,
                                   (2 * pair + 1) / E.Kb * 128, E.N);
         };
-        BuildInput<BT> bin;
         while (cur < end) {
             const int region = cur >= I0;
             const int local = region ? cur - I0 : cur;
-            const int pair = local / E.nrb, rb_lo = local - pair * E.nrb;
+            const int wpair = local / E.nrb, rb_lo = local - wpair * E.nrb;
             const int seg_end = min(end, cur - rb_lo + E.nrb);
             const int rb_hi = rb_lo + (seg_end - cur);
+            const int np = region ? 1 : NP;                 // pairs walked together in this segment
+            const int pair = wpair * np;
             const int ib = region ? ItemBytes<SPS1>::value : ItemBytes<SPS0>::value;
             const uint8_t *items = E.packed + E.off_items[region] + (size_t)pair * E.nrb * ib;
-            prefetch_run_head(items, ib, (region ? SPS1 : SPS0) == 1 ? 1 : kDepth, rb_lo, rb_hi);   // weights start moving now
+            const uint8_t *items_b = items + (size_t)E.nrb * ib;
+            const int pf_d = np == 2 ? 1 : (region ? SPS1 : SPS0) == 1 ? 1 : kDepth;
+            prefetch_run_head(items, ib, pf_d, rb_lo, rb_hi);                 // weights start moving now
+            if (np == 2) prefetch_run_head(items_b, ib, pf_d, rb_lo, rb_hi);
 
             __syncthreads();     // previous segment's lookups are done before the tables are overwritten
-            // (fetching the next pair's inputs here, ahead of the lookups, was measured 15 % slower: the
-            // two extra live registers push the lookup loop over the 80-register budget of 3 CTAs per SM)
-            fetch_for(cur, bin);
+            // (fetching the next pair's inputs ahead of the lookups was measured 15 % slower: the extra
+            // live registers push the lookup loop over the 80-register budget of 3 CTAs per SM)
+            BuildInput<BT> bin, bin_b;
+            fetch_for(region, pair, bin);
+            if (np == 2) fetch_for(region, pair + 1, bin_b);
             build_tables<BT>(bin, abuf);
+            if (np == 2) build_tables<BT>(bin_b, abuf, 128u);
             FB_TRACE_AT(1);
-            if (region == 0) process_rows<SPS0, BT>(items, rb_lo, rb_hi, la, E.acc, E.Mpad);
-            else process_rows<SPS1, BT>(items, rb_lo, rb_hi, la, E.acc, E.Mpad);
+            if (region == 0) {
+                if constexpr (NP == 2) process_rows2<SPS0>(items, items_b, rb_lo, rb_hi, la, E.acc);
+                else process_rows<SPS0, BT>(items, rb_lo, rb_hi, la, E.acc, E.Mpad);
+            } else {
+                process_rows<SPS1, BT>(items, rb_lo, rb_hi, la, E.acc, E.Mpad);
+            }
 
             // how many items this CTA contributed to each tile of rows
             const int t_lo = rb_lo / E.tile_rb, t_hi = (rb_hi - 1) / E.tile_rb;
             for (int t = t_lo + tid; t <= t_hi; t += kThreads) {
                 int a = max(rb_lo, t * E.tile_rb), b = min(rb_hi, (t + 1) * E.tile_rb);
-                tile_cnt[t] += b - a;            // one thread per tile, segments are serial: no race
+                tile_cnt[t] += (b - a) * np;     // one thread per tile, segments are serial: no race
             }
             cur = seg_end;
         }
