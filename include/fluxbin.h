@@ -150,7 +150,9 @@ fluxbin_status_t fluxbin_workspace_init(void *d_workspace, size_t bytes, void *c
  *   d_workspace / ws_bytes   see fluxbin_workspace_size
  *
  * Asynchronous on cuda_stream; performs no allocation and no synchronisation, so calls can be
- * captured into a CUDA graph.  B >= 1 arbitrary (processed in chunks of up to 2 vectors).  Calls
+ * captured into a CUDA graph.  The kernel is launched with programmatic stream serialization: it may
+ * begin (index arithmetic, L2 prefetch of its weights) while the previous kernel on the stream is
+ * draining, and waits on the device before it reads d_x or touches the workspace.  B >= 1 arbitrary (processed in chunks of up to 2 vectors).  Calls
  * sharing a workspace must be ordered on one stream.  Accumulation is fp32 with fp32 atomics
  * across K slices, so results may differ in the last bits from run to run.
  */

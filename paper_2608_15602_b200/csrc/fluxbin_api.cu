@@ -256,13 +256,22 @@ static cudaError_t launch(const fbk::LaunchParams &p, int num_sms, long long ite
     // even pair counts everywhere) and a CTA's share spans several whole couples
     bool couples = false;
     if constexpr (BT == 1) couples = couple_cost > 0 && q.static_cost / grid >= 2 * couple_cost;
+    // launched with programmatic stream serialization: the kernel may start while its predecessor in
+    // the stream drains (it waits inside, before touching activations or workspace)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(fbk::kThreads);
+    cfg.dynamicSmemBytes = fbk::smem_bytes<BT>();
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
     if constexpr (BT == 1) {
-        if (couples) fbk::fluxbin_linear_kernel<S0, S1, BT, 2><<<(int)grid, fbk::kThreads, fbk::smem_bytes<BT>(), s>>>(q);
-        else fbk::fluxbin_linear_kernel<S0, S1, BT, 1><<<(int)grid, fbk::kThreads, fbk::smem_bytes<BT>(), s>>>(q);
-    } else {
-        fbk::fluxbin_linear_kernel<S0, S1, BT, 1><<<(int)grid, fbk::kThreads, fbk::smem_bytes<BT>(), s>>>(q);
+        if (couples) return cudaLaunchKernelEx(&cfg, fbk::fluxbin_linear_kernel<S0, S1, BT, 2>, q);
     }
-    return cudaGetLastError();
+    return cudaLaunchKernelEx(&cfg, fbk::fluxbin_linear_kernel<S0, S1, BT, 1>, q);
 }
 
 // couple_cost: cost of the largest couple of global pairs over the layers of the launch, or 0 when

@@ -539,6 +539,13 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
     const int tid = threadIdx.x;
     FB_TRACE_AT(0);
 
+    // Programmatic dependent launch: let the next kernel in the stream start its own prologue as soon
+    // as SM resources free up; below, this kernel in turn waits for its predecessor only at the point
+    // where it first touches data the predecessor may have written (activations, workspace) -- the
+    // index arithmetic and the first L2 prefetches of the (static) weights run ahead of that.
+    asm volatile("griddepcontrol.launch_dependents;");
+    bool predecessor_done = false;
+
     LaneAddr<BT> la;
     la.init(tid & 31);
 
@@ -634,6 +641,10 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
             prefetch_run_head(items, ib, pf_d, rb_lo, rb_hi);                 // weights start moving now
             if (np == 2) prefetch_run_head(items_b, ib, pf_d, rb_lo, rb_hi);
 
+            if (!predecessor_done) {
+                asm volatile("griddepcontrol.wait;" ::: "memory");
+                predecessor_done = true;
+            }
             __syncthreads();     // previous segment's lookups are done before the tables are overwritten
             // (fetching the next pair's inputs ahead of the lookups was measured 15 % slower: the extra
             // live registers push the lookup loop over the 80-register budget of 3 CTAs per SM)
@@ -663,6 +674,10 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
         FB_TRACE_AT(3);
     }
         if (P.nshares <= (int)gridDim.x) break;    // one share per CTA: nothing to draw
+        if (!predecessor_done) {
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            predecessor_done = true;
+        }
         if (tid == 0) range[2] = (int)gridDim.x + (int)atomicAdd(P.counters, 1u);
         __syncthreads();
         share = range[2];

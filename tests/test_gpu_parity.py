@@ -231,3 +231,33 @@ def test_argument_errors_do_not_launch(fb):
     assert fluxbin.linear_status(w, **{**args, "d_x": x.data_ptr() + 2}) == 6
     assert fluxbin.linear_status(w, **{**args, "d_y": 0}) == 1
     torch.cuda.synchronize()
+
+
+def test_back_to_back_dependent_layers_share_a_workspace(fb):
+    """y1 = L1 x, y2 = L2 y1, y3 = L3 y2 launched back to back on one stream with one workspace: each
+    kernel may start while its predecessor drains (programmatic dependent launch) but must see the
+    predecessor's output and a clean workspace."""
+    dims = [(1024, 2048), (768, 1024), (1536, 768)]          # (M, N) chained: N of the next = M of the previous
+    Ls, lins = [], []
+    for i, (M, N) in enumerate(dims):
+        L = layer_of(300 + i, M, N, 2, 1, 128, N // 20)
+        Ls.append(L)
+        lins.append(fb.FluxBinLinear(L))
+    x0 = synth.make_activations(4, 4, 2, 2048)
+    xt = torch.from_numpy(x0.view(np.float16)).cuda()
+    ws = fb.Workspace(max(l.weight.workspace_size(2) for l in lins))
+    for rep in range(3):
+        h = xt
+        outs = []
+        for lin in lins:
+            h = lin.forward(h, ws)                            # fp16 output feeds the next layer directly
+            outs.append(h)
+        torch.cuda.synchronize()
+        cur = x0
+        for L, got in zip(Ls, outs):
+            want = oracle.linear_direct(L, cur)
+            g = got.cpu().numpy()
+            ulp = np.spacing(np.abs(want).astype(np.float16)).astype(np.float64)
+            rms = np.sqrt(np.mean(want ** 2))
+            assert np.all(np.abs(g.astype(np.float64) - want) <= 1.01 * ulp + 5e-3 * np.maximum(np.abs(want), 1e-2 * rms))
+            cur = g.view(np.uint16)                           # the next layer's oracle input is the GPU's fp16 output
