@@ -261,23 +261,23 @@ template <int SPS> __device__ __forceinline__ void load_item(ItemRegs<SPS> &r, c
     }
 }
 
-// Lane constants of the lookup address.  BT == 1: eight registers holding, byte by byte, the slot
-// offset (lane ^ s) * 4 of each of the 32 steps, so that PRMT can drop it into byte 0 of the address.
+// Lane constant of the lookup address.  BT == 1: one register holding, byte by byte, the slot offsets
+// (lane ^ k) * 4 of steps k = 0..3, so that PRMT can drop one into byte 0 of the address; the offsets
+// of steps 4q + k differ from these by an XOR with 16q in every byte ((lane ^ (4q + k)) * 4 ==
+// ((lane ^ k) * 4) ^ 16q), one LOP per group of four lookups instead of eight live registers.
 template <int BT> struct LaneAddr {
-    uint32_t c[(BT == 1) ? 8 : 1];
+    uint32_t c0;
     __device__ __forceinline__ void init(int lane)
     {
         if constexpr (BT == 1) {
+            uint32_t v = 0;
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                uint32_t v = 0;
-#pragma unroll
-                for (int k = 0; k < 4; ++k) v |= (uint32_t)(((lane ^ (4 * q + k)) * 4) & 0xff) << (8 * k);
-                c[q] = v;
-            }
+            for (int k = 0; k < 4; ++k) v |= (uint32_t)(((lane ^ k) * 4) & 0xff) << (8 * k);
+            c0 = v;
         } else {
-            c[0] = TabCfg<BT>::lane_const((uint32_t)lane);
+            c0 = TabCfg<BT>::lane_const((uint32_t)lane);
         }
+        asm volatile("" : "+r"(c0));      // keep it in its register: recomputing it per item costs more
     }
 };
 
@@ -302,10 +302,10 @@ __device__ __forceinline__ void compute_item(const ItemRegs<SPS> &r, const LaneA
                 const uint32_t k = (uint32_t)(s & 3);
                 uint32_t addr;
                 if constexpr (BT == 1) {
-                    addr = prmt(w[s >> 2], la.c[s >> 2], ((0xCu | k) << 12) | ((0xCu | k) << 8) | (k << 4) | (4u | k));
+                    addr = prmt(w[s >> 2], la.c0 ^ (0x10101010u * (uint32_t)(s >> 2)), ((0xCu | k) << 12) | ((0xCu | k) << 8) | (k << 4) | (4u | k));
                 } else {
                     uint32_t idx = __byte_perm(w[s >> 2], 0u, 0x4404u | (k << 4));
-                    addr = idx | (la.c[0] ^ TabCfg<BT>::lane_const((uint32_t)s));
+                    addr = idx | (la.c0 ^ TabCfg<BT>::lane_const((uint32_t)s));
                 }
                 Vec<BT> e = lds_entry<BT, HALF>(addr);
 #pragma unroll
