@@ -3,8 +3,9 @@
     python -m paper_2608_15602_b200.profile_case --config 4 --linear 4 --copies 3 --reps 5
 
 builds `copies` distinct packed layers of that shape (different seeded layers, so together they
-exceed L2), runs them round-robin `reps` times with plain launches and prints the mean time per
-call from CUDA events, the algorithmic bytes and the resulting GB/s.
+can exceed L2), replays a CUDA graph of one fluxbin_linear call per copy `reps` times and prints
+the mean time per call from CUDA events, the algorithmic bytes and the resulting GB/s.
+--variant/--shape time the paper's deployed formats (2b, 2b-s8, 2b-s16, 4b at g = 128) instead.
 """
 from __future__ import annotations
 
@@ -32,14 +33,26 @@ def main():
     ap.add_argument("--reps", type=int, default=5)
     ap.add_argument("--batch", type=int, default=1)
     ap.add_argument("--g", type=int, default=128)
+    ap.add_argument("--variant", default=None, choices=["2b", "2b-s8", "2b-s16", "4b"],
+                    help="one of the paper's deployed formats at --shape MxN instead of a workload linear: "
+                         "2 or 4 global bases; s8/s16 = exactly 8/16 salient columns per group with 2 extra bases")
+    ap.add_argument("--shape", default="4096x4096", help="MxN for --variant")
     args = ap.parse_args()
     build.build()
     from . import layer as fb_layer
 
     lins = []
     for c in range(args.copies):
-        L = synth.make_config_linear(args.config, c, args.linear, g=args.g)
-        x = synth.make_config_activations(args.config, c, args.linear, args.batch)
+        if args.variant:
+            M, N = (int(t) for t in args.shape.lower().split("x"))
+            Kb = 4 if args.variant == "4b" else 2
+            s_per_group = {"2b": 0, "4b": 0, "2b-s8": 8, "2b-s16": 16}[args.variant]
+            idx = synth.salient_per_group(7, c, N, args.g, s_per_group) if s_per_group else None
+            L = synth.make_linear(7, c, M, N, Kb, 2 if s_per_group else 0, args.g, idx)
+            x = synth.make_activations(7, c, args.batch, N)
+        else:
+            L = synth.make_config_linear(args.config, c, args.linear, g=args.g)
+            x = synth.make_config_activations(args.config, c, args.linear, args.batch)
         lin = fb_layer.FluxBinLinear(L)
         xt = torch.from_numpy(x.view(np.float16)).cuda()
         y = torch.empty((args.batch, L.M), dtype=torch.float16, device="cuda")
@@ -51,13 +64,20 @@ def main():
     for lin, xt, y in lins:                      # one warm-up pass
         lin.forward(xt, ws, out=y)
     torch.cuda.synchronize()
-    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a.record(stream)
-    for _ in range(args.reps):
-        for lin, xt, y in lins:
-            lin.forward(xt, ws, out=y)
-    b.record(stream)
-    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()                # plain launches pay Python's call overhead; replay a graph
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            for lin, xt, y in lins:
+                lin.forward(xt, ws, out=y, stream=side)
+        graph.replay()
+        side.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(side)
+        for _ in range(args.reps):
+            graph.replay()
+        b.record(side)
+        side.synchronize()
     us = a.elapsed_time(b) * 1e3 / (args.reps * len(lins))
     print(json.dumps({"dims_M_N_Kb_Ks_g_nsal": dims, "batch": args.batch, "copies": args.copies, "us_per_call": round(us, 2),
                       "algorithmic_bytes": nbytes, "GBps": round(nbytes / us / 1e3, 1),
