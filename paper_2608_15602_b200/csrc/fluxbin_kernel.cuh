@@ -331,6 +331,20 @@ __device__ __forceinline__ void finish_item(const ItemRegs<SPS> &r, const LaneAd
     for (int b = 0; b < BT; ++b) atomicAdd(accp + (int64_t)b * Mpad, out[b]);
 }
 
+// The first item of this warp's run, loaded ahead of the table build so that its latency hides
+// behind the build (the weights do not depend on the activations).
+template <int SPS>
+__device__ __forceinline__ void preload_first(ItemRegs<SPS> &r, const uint8_t *pair_items, int rb_lo, int rb_hi)
+{
+    constexpr int IB = ItemBytes<SPS>::value;
+    constexpr int SB = (SPS == 16) ? 4 : (SPS == 8) ? 8 : 16;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int first = rb_lo + warp;
+    if (first >= rb_hi) return;
+    const uint8_t *item = pair_items + (int64_t)first * IB;
+    load_item<SPS>(r, item + lane * 16, item + FB_ITEM_BITS_BYTES + lane * SB, 0);
+}
+
 // Row blocks rb_lo + warp, + kWarps, ... of one pair.  kDepth register sets rotate so that the
 // loads of the next kDepth-1 items are in flight while the current one is looked up (enough bytes
 // in flight per SM to cover the L2 latency at full HBM rate).  A trip of the steady loop handles
@@ -338,7 +352,8 @@ __device__ __forceinline__ void finish_item(const ItemRegs<SPS> &r, const LaneAd
 // kPrefetchTrips trips ahead, its share of the kDepth*kWarps items the CTA reads per trip.
 template <int SPS, int BT>
 __device__ __forceinline__ void process_rows(const uint8_t *pair_items, int rb_lo, int rb_hi,
-                                             const LaneAddr<BT> &la, float *acc, int Mpad)
+                                             const LaneAddr<BT> &la, float *acc, int Mpad,
+                                             const ItemRegs<SPS> *pre = nullptr)   // pre: preload_first's result
 {
     constexpr int IB = ItemBytes<SPS>::value;
     constexpr int STRIDE = kWarps * IB;                   // bytes between a warp's consecutive items
@@ -357,8 +372,10 @@ __device__ __forceinline__ void process_rows(const uint8_t *pair_items, int rb_l
 
     ItemRegs<SPS> r[D];
 #pragma unroll
-    for (int d = 0; d < D - 1; ++d)
-        if (d < n) load_item<SPS>(r[d], pl, ps, d * STRIDE);
+    for (int d = 0; d < D - 1; ++d) {
+        if (d == 0 && pre) r[0] = *pre;
+        else if (d < n) load_item<SPS>(r[d], pl, ps, d * STRIDE);
+    }
     // items t .. t+D-1 are looked up while items t+D-1 .. t+2D-2 are loaded (warp-uniform guards)
     for (int t = 0; t < n; t += D) {
         if (lane == 0 && pp + D * IB <= pend) prefetch_l2(pp, D * IB);
@@ -651,12 +668,16 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
             BuildInput<BT> bin, bin_b;
             fetch_for(region, pair, bin);
             if (np == 2) fetch_for(region, pair + 1, bin_b);
+            // region 0, one pair at a time (short runs): first item in flight during the build.  (With two
+            // pairs per row block the runs are long and the extra live registers cost more than they hide.)
+            ItemRegs<SPS0> pre;
+            if (NP == 1 && region == 0) preload_first<SPS0>(pre, items, rb_lo, rb_hi);
             build_tables<BT>(bin, abuf);
             if (np == 2) build_tables<BT>(bin_b, abuf, 128u);
             FB_TRACE_AT(1);
             if (region == 0) {
                 if constexpr (NP == 2) process_rows2<SPS0>(items, items_b, rb_lo, rb_hi, la, E.acc);
-                else process_rows<SPS0, BT>(items, rb_lo, rb_hi, la, E.acc, E.Mpad);
+                else process_rows<SPS0, BT>(items, rb_lo, rb_hi, la, E.acc, E.Mpad, &pre);
             } else {
                 process_rows<SPS1, BT>(items, rb_lo, rb_hi, la, E.acc, E.Mpad);
             }
