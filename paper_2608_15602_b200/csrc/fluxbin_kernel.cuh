@@ -43,6 +43,14 @@ constexpr int kMaxTiles = 1024;
 #define FB_DEPTH 2
 #endif
 constexpr int kDepth = FB_DEPTH;    // register sets (items in flight per warp) in the main loop
+#ifndef FB_DEPTH2
+#define FB_DEPTH2 3
+#endif
+// The two-vector kernel runs 2 CTAs per SM (its tables are twice as large), so a thread may hold 128
+// registers and fewer warps cover the load latency: it keeps more items in flight per warp
+// (measured at batch 2 on a 16-layer stack: depth 2 3.49 TB/s, depth 3 3.56, depth 4 3.38).
+constexpr int kDepth2 = FB_DEPTH2;
+template <int BT> struct DepthFor { static constexpr int value = BT == 2 ? kDepth2 : kDepth; };
 #ifndef FB_PF
 #define FB_PF 1
 #endif
@@ -265,19 +273,41 @@ template <int SPS> __device__ __forceinline__ void load_item(ItemRegs<SPS> &r, c
 // (lane ^ k) * 4 of steps k = 0..3, so that PRMT can drop one into byte 0 of the address; the offsets
 // of steps 4q + k differ from these by an XOR with 16q in every byte ((lane ^ (4q + k)) * 4 ==
 // ((lane ^ k) * 4) ^ 16q), one LOP per group of four lookups instead of eight live registers.
-template <int BT> struct LaneAddr {
+// BT == 2: the slot offsets (lane ^ s) * 8 reach 248, so a byte of them cannot double as the zero
+// fill of the upper address bytes; each register holds the offsets of two steps and two zero bytes,
+// and with 128 registers per thread all sixteen stay resident (no LOP at all).
+template <int BT> struct LaneAddr;
+template <> struct LaneAddr<1> {
     uint32_t c0;
     __device__ __forceinline__ void init(int lane)
     {
-        if constexpr (BT == 1) {
-            uint32_t v = 0;
+        uint32_t v = 0;
 #pragma unroll
-            for (int k = 0; k < 4; ++k) v |= (uint32_t)(((lane ^ k) * 4) & 0xff) << (8 * k);
-            c0 = v;
-        } else {
-            c0 = TabCfg<BT>::lane_const((uint32_t)lane);
-        }
+        for (int k = 0; k < 4; ++k) v |= (uint32_t)(((lane ^ k) * 4) & 0xff) << (8 * k);
+        c0 = v;
         asm volatile("" : "+r"(c0));      // keep it in its register: recomputing it per item costs more
+    }
+    // address of the lookup of step s: byte 1 = table index (byte s%4 of w), byte 0 = slot offset
+    __device__ __forceinline__ uint32_t addr(int s, uint32_t w) const     // s: compile-time after unrolling
+    {
+        const uint32_t k = (uint32_t)s & 3u;
+        return prmt(w, c0 ^ (0x10101010u * (uint32_t)(s >> 2)), ((0xCu | k) << 12) | ((0xCu | k) << 8) | (k << 4) | (4u | k));
+    }
+};
+template <> struct LaneAddr<2> {
+    uint32_t c[16];
+    __device__ __forceinline__ void init(int lane)
+    {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            c[i] = (uint32_t)((lane ^ (2 * i)) * 8) | ((uint32_t)((lane ^ (2 * i + 1)) * 8) << 8);
+            asm volatile("" : "+r"(c[i]));
+        }
+    }
+    __device__ __forceinline__ uint32_t addr(int s, uint32_t w) const
+    {
+        const uint32_t k = (uint32_t)s & 3u, j = (uint32_t)s & 1u;
+        return prmt(w, c[s >> 1], (6u << 12) | (6u << 8) | (k << 4) | (4u | j));
     }
 };
 
@@ -299,14 +329,7 @@ __device__ __forceinline__ void compute_item(const ItemRegs<SPS> &r, const LaneA
 #pragma unroll
             for (int q = 0; q < SPS; ++q) {
                 const int s = j * SPS + q;
-                const uint32_t k = (uint32_t)(s & 3);
-                uint32_t addr;
-                if constexpr (BT == 1) {
-                    addr = prmt(w[s >> 2], la.c0 ^ (0x10101010u * (uint32_t)(s >> 2)), ((0xCu | k) << 12) | ((0xCu | k) << 8) | (k << 4) | (4u | k));
-                } else {
-                    uint32_t idx = __byte_perm(w[s >> 2], 0u, 0x4404u | (k << 4));
-                    addr = idx | (la.c0 ^ TabCfg<BT>::lane_const((uint32_t)s));
-                }
+                const uint32_t addr = la.addr(s, w[s >> 2]);
                 Vec<BT> e = lds_entry<BT, HALF>(addr);
 #pragma unroll
                 for (int b = 0; b < BT; ++b) {
@@ -358,7 +381,7 @@ __device__ __forceinline__ void process_rows(const uint8_t *pair_items, int rb_l
     constexpr int IB = ItemBytes<SPS>::value;
     constexpr int STRIDE = kWarps * IB;                   // bytes between a warp's consecutive items
     constexpr int SB = (SPS == 16) ? 4 : (SPS == 8) ? 8 : 16;   // scale bytes per lane (per plane)
-    constexpr int D = (SPS == 1) ? 1 : kDepth;
+    constexpr int D = (SPS == 1) ? 1 : DepthFor<BT>::value;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int first = rb_lo + warp;
     if (first >= rb_hi) return;
@@ -452,9 +475,28 @@ __device__ __forceinline__ void trace(int slot)
         g_fb_trace[blockIdx.x][slot] = t;
     }
 }
+__device__ __forceinline__ unsigned long long trace_now()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// accumulate the time since t0 into a per-CTA phase total
+__device__ __forceinline__ void trace_add(int slot, unsigned long long t0)
+{
+    if (threadIdx.x == 0 && blockIdx.x < 1024) g_fb_trace[blockIdx.x][slot] += trace_now() - t0;
+}
 #define FB_TRACE_AT(slot) trace(slot)
+#define FB_TRACE_T0(var) unsigned long long var = trace_now()
+#define FB_TRACE_ADD(slot, var) trace_add(slot, var)
+#define FB_TRACE_SET(var) var = trace_now()
+#define FB_TRACE_ZERO() do { if (threadIdx.x == 0 && blockIdx.x < 1024) { g_fb_trace[blockIdx.x][4] = 0; g_fb_trace[blockIdx.x][5] = 0; g_fb_trace[blockIdx.x][6] = 0; g_fb_trace[blockIdx.x][7] = 0; g_fb_trace[blockIdx.x][1] = 0; g_fb_trace[blockIdx.x][2] = 0; } } while (0)
 #else
 #define FB_TRACE_AT(slot)
+#define FB_TRACE_T0(var)
+#define FB_TRACE_ADD(slot, var)
+#define FB_TRACE_SET(var)
+#define FB_TRACE_ZERO()
 #endif
 
 // Stage (iii) for the entry a CTA has just finished contributing to: publish, take a ticket per
@@ -555,6 +597,7 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
     static_assert(NP == 1 || BT == 1, "two table sets side by side need the 4-byte slots of BT == 1");
     const int tid = threadIdx.x;
     FB_TRACE_AT(0);
+    FB_TRACE_ZERO();
 
     // Programmatic dependent launch: let the next kernel in the stream start its own prologue as soon
     // as SM resources free up; below, this kernel in turn waits for its predecessor only at the point
@@ -574,6 +617,7 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
     // quick ones pick up the small shares and the SM stays fully occupied until the end.
     const int G = (int)gridDim.x;
     for (int share = blockIdx.x; share < P.nshares;) {
+    FB_TRACE_T0(t_pro);
     long long lo, hi;
     if (share < G) {
         lo = P.static_cost * (long long)share / G;
@@ -635,7 +679,8 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
         int cur = range[0];
         const int end = range[1];
         __syncthreads();                           // range[] is rewritten for the next entry
-        if (cur >= end) continue;
+        FB_TRACE_ADD(7, t_pro);
+        if (cur >= end) { FB_TRACE_SET(t_pro); continue; }
 
         // a segment = the CTA's row blocks of one work pair
         auto fetch_for = [&](int region, int pair, BuildInput<BT> &in) {
@@ -654,7 +699,7 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
             const int ib = region ? ItemBytes<SPS1>::value : ItemBytes<SPS0>::value;
             const uint8_t *items = E.packed + E.off_items[region] + (size_t)pair * E.nrb * ib;
             const uint8_t *items_b = items + (size_t)E.nrb * ib;
-            const int pf_d = np == 2 ? 1 : (region ? SPS1 : SPS0) == 1 ? 1 : kDepth;
+            const int pf_d = np == 2 ? 1 : (region ? SPS1 : SPS0) == 1 ? 1 : DepthFor<BT>::value;
             prefetch_run_head(items, ib, pf_d, rb_lo, rb_hi);                 // weights start moving now
             if (np == 2) prefetch_run_head(items_b, ib, pf_d, rb_lo, rb_hi);
 
@@ -662,6 +707,7 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
                 asm volatile("griddepcontrol.wait;" ::: "memory");
                 predecessor_done = true;
             }
+            FB_TRACE_T0(t_build);
             __syncthreads();     // previous segment's lookups are done before the tables are overwritten
             // (fetching the next pair's inputs ahead of the lookups was measured 15 % slower: the extra
             // live registers push the lookup loop over the 80-register budget of 3 CTAs per SM)
@@ -674,7 +720,8 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
             if (NP == 1 && region == 0) preload_first<SPS0>(pre, items, rb_lo, rb_hi);
             build_tables<BT>(bin, abuf);
             if (np == 2) build_tables<BT>(bin_b, abuf, 128u);
-            FB_TRACE_AT(1);
+            FB_TRACE_ADD(4, t_build);
+            FB_TRACE_T0(t_rows);
             if (region == 0) {
                 if constexpr (NP == 2) process_rows2<SPS0>(items, items_b, rb_lo, rb_hi, la, E.acc);
                 else process_rows<SPS0, BT>(items, rb_lo, rb_hi, la, E.acc, E.Mpad, &pre);
@@ -682,6 +729,8 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
                 process_rows<SPS1, BT>(items, rb_lo, rb_hi, la, E.acc, E.Mpad);
             }
 
+            FB_TRACE_ADD(5, t_rows);
+            FB_TRACE_T0(t_cnt);
             // how many items this CTA contributed to each tile of rows
             const int t_lo = rb_lo / E.tile_rb, t_hi = (rb_hi - 1) / E.tile_rb;
             for (int t = t_lo + tid; t <= t_hi; t += kThreads) {
@@ -689,11 +738,15 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
                 tile_cnt[t] += (b - a) * np;     // one thread per tile, segments are serial: no race
             }
             cur = seg_end;
+            FB_TRACE_ADD(1, t_cnt);
         }
-        FB_TRACE_AT(2);
+        FB_TRACE_T0(t_red);
         reduce_and_store<BT>(E, P.nb, P.y_fp32, tile_cnt, done_list);
+        FB_TRACE_ADD(6, t_red);
         FB_TRACE_AT(3);
+        FB_TRACE_SET(t_pro);
     }
+        FB_TRACE_T0(t_draw);
         if (P.nshares <= (int)gridDim.x) break;    // one share per CTA: nothing to draw
         if (!predecessor_done) {
             asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -703,6 +756,7 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
         __syncthreads();
         share = range[2];
         __syncthreads();
+        FB_TRACE_ADD(2, t_draw);
     }
     // the last CTA to leave puts the two launch counters back to zero for the next launch
     if (P.nshares > (int)gridDim.x && tid == 0) {
