@@ -152,7 +152,7 @@ fluxbin_status_t fluxbin_workspace_init(void *d_workspace, size_t bytes, void *c
  * Asynchronous on cuda_stream; performs no allocation and no synchronisation, so calls can be
  * captured into a CUDA graph.  The kernel is launched with programmatic stream serialization: it may
  * begin (index arithmetic, L2 prefetch of its weights) while the previous kernel on the stream is
- * draining, and waits on the device before it reads d_x or touches the workspace.  B >= 1 arbitrary (processed in chunks of up to 2 vectors).  Calls
+ * draining, and waits on the device before it reads d_x or touches the workspace.  B >= 1 arbitrary (processed in chunks of up to 4 vectors).  Calls
  * sharing a workspace must be ordered on one stream.  Accumulation is fp32 with fp32 atomics
  * across K slices, so results may differ in the last bits from run to run.
  */
@@ -249,7 +249,7 @@ fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_t *const *w
  */
 fluxbin_status_t fluxbin_plan_run(const fluxbin_plan_t *plan, void *cuda_stream);
 
-/* Kernel launches one fluxbin_plan_run issues (one per chunk of up to 2 batch vectors); -1 on NULL. */
+/* Kernel launches one fluxbin_plan_run issues (one per chunk of up to 4 batch vectors); -1 on NULL. */
 int32_t fluxbin_plan_num_launches(const fluxbin_plan_t *plan);
 
 /* Release the host object (never touches device memory).  NULL is allowed. */

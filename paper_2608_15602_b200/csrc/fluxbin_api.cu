@@ -88,6 +88,7 @@ fluxbin_status_t device_setup(int dev, int *num_sms)
         if (major == 10) {
             FB_CUDA(opt_in_bt<1>());
             FB_CUDA(opt_in_bt<2>());
+            FB_CUDA(opt_in_bt<4>());
             FB_CUDA(cudaFuncSetAttribute(fbk::fluxbin_debug_tables_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)fbk::smem_bytes<1>()));
             FB_CUDA(cudaFuncSetAttribute(fbk::fluxbin_smem_base_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -194,12 +195,16 @@ extern "C" void fluxbin_free(fluxbin_weight_t *w) { delete w; }
 
 extern "C" int32_t fluxbin_num_table_sets(const fluxbin_weight_t *w) { return w ? w->h.npairs[0] + w->h.npairs[1] : -1; }
 
-// Batch vectors per launch: B is processed in chunks of two (the last chunk may hold one).  Measured
-// on B200: two passes with two vectors' table entries side by side (LDS.64, 3 CTAs per SM) beat one
-// pass with four (LDS.128, 128 KB of tables, 1 CTA per SM) by 12 % -- both are shared-memory bound.
-static int chunk_size() { return 2; }
+// Batch vectors per launch: B is processed in chunks of up to four.  A chunk of 1, 2 or 3..4 vectors
+// runs the kernel whose table entries hold 1, 2 or 4 vectors side by side (LDS.32 / .64 / .128): the
+// weights stream once per chunk and one address computation serves the whole entry.
+#ifndef FB_CHUNK
+#define FB_CHUNK 4
+#endif
+static int chunk_size() { return FB_CHUNK; }
 static int num_chunks(int B) { return (B + chunk_size() - 1) / chunk_size(); }
-static int ws_bt(int B) { return B == 1 ? 1 : 2; }
+static int bt_for(int nb) { return nb == 1 ? 1 : nb == 2 ? 2 : 4; }
+static int ws_bt(int B) { return bt_for(B < chunk_size() ? B : chunk_size()); }
 
 extern "C" int32_t fluxbin_num_launches(const fluxbin_weight_t *w, int32_t B)
 {
@@ -234,7 +239,7 @@ static cudaError_t launch(const fbk::LaunchParams &p, int num_sms, long long ite
     if (occ == 0) {
         int o = 0;
         cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, fbk::fluxbin_linear_kernel<S0, S1, BT, 1>,
-                                                                      fbk::kThreads, fbk::smem_bytes<BT>());
+                                                                      fbk::Cfg<BT>::kThreads, fbk::smem_bytes<BT>());
         if (e != cudaSuccess) return e;
         occ = o > 0 ? o : 1;
     }
@@ -260,7 +265,7 @@ static cudaError_t launch(const fbk::LaunchParams &p, int num_sms, long long ite
     // the stream drains (it waits inside, before touching activations or workspace)
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3(fbk::kThreads);
+    cfg.blockDim = dim3(fbk::Cfg<BT>::kThreads);
     cfg.dynamicSmemBytes = fbk::smem_bytes<BT>();
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
@@ -361,7 +366,8 @@ extern "C" fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint
         cudaError_t e;
         const int s1 = w->h.npairs[1] > 0 ? w->h.sps[1] : 1;
         if (nb == 1) e = launch_bt<1>(w->h.sps[0], s1, w->num_sms, p, items, couple_cost_of(w->h), s);
-        else e = launch_bt<2>(w->h.sps[0], s1, w->num_sms, p, items, 0, s);
+        else if (nb == 2) e = launch_bt<2>(w->h.sps[0], s1, w->num_sms, p, items, 0, s);
+        else e = launch_bt<4>(w->h.sps[0], s1, w->num_sms, p, items, 0, s);
         if (e != cudaSuccess) return cuda_fail(e);
     }
     return FLUXBIN_OK;
@@ -497,7 +503,8 @@ extern "C" fluxbin_status_t fluxbin_plan_run(const fluxbin_plan_t *plan, void *c
         p.nb = nb;
         cudaError_t e;
         if (nb == 1) e = launch_bt<1>(plan->sps0, plan->sps1, plan->num_sms, p, plan->items, plan->couple_cost, s);
-        else e = launch_bt<2>(plan->sps0, plan->sps1, plan->num_sms, p, plan->items, 0, s);
+        else if (nb == 2) e = launch_bt<2>(plan->sps0, plan->sps1, plan->num_sms, p, plan->items, 0, s);
+        else e = launch_bt<4>(plan->sps0, plan->sps1, plan->num_sms, p, plan->items, 0, s);
         if (e != cudaSuccess) return cuda_fail(e);
     }
     return FLUXBIN_OK;
@@ -515,7 +522,7 @@ extern "C" fluxbin_status_t fluxbin_debug_tables(const fluxbin_weight_t *w, cons
     if (pair < 0 || pair >= np) return FLUXBIN_ERR_RANGE;
     cudaStream_t s = (cudaStream_t)cuda_stream;
     const uint8_t *desc = (const uint8_t *)w->d_packed + w->h.off_coldesc + (size_t)pair * FB_PAIR_DESC_BYTES;
-    fbk::fluxbin_debug_tables_kernel<<<1, fbk::kThreads, fbk::smem_bytes<1>(), s>>>(desc, d_x, d_tables);
+    fbk::fluxbin_debug_tables_kernel<<<1, fbk::Cfg<1>::kThreads, fbk::smem_bytes<1>(), s>>>(desc, d_x, d_tables);
     FB_CUDA(cudaGetLastError());
     if (h_cols || h_alpha) {
         uint16_t tmp[512];
@@ -533,6 +540,6 @@ extern "C" fluxbin_status_t fluxbin_debug_tables(const fluxbin_weight_t *w, cons
 // Instrumented build only: copy the per-CTA phase timestamps of the last launch to the host.
 extern "C" int fluxbin_debug_trace(unsigned long long *h_out)
 {
-    return (int)cudaMemcpyFromSymbol(h_out, fbk::g_fb_trace, sizeof(unsigned long long) * 1024 * 8);
+    return (int)cudaMemcpyFromSymbol(h_out, fbk::g_fb_trace, sizeof(unsigned long long) * 1024 * 12);
 }
 #endif

@@ -36,8 +36,13 @@
 
 namespace fbk {
 
-constexpr int kThreads = 256;
-constexpr int kWarps = kThreads / 32;
+// Threads per CTA: 8 warps with 1 or 2 batch vectors per launch (3 or 2 CTAs per SM); with 4 vectors the
+// tables fill 128 KB, one CTA owns the SM and runs 16 warps.
+template <int BT> struct Cfg {
+    static constexpr int kThreads = (BT == 4) ? 512 : 256;
+    static constexpr int kWarps = kThreads / 32;
+    static constexpr int kMinBlocks = (BT == 4) ? 1 : (BT == 2) ? 2 : 3;
+};
 constexpr int kMaxTiles = 1024;
 #ifndef FB_DEPTH
 #define FB_DEPTH 2
@@ -50,7 +55,10 @@ constexpr int kDepth = FB_DEPTH;    // register sets (items in flight per warp) 
 // registers and fewer warps cover the load latency: it keeps more items in flight per warp
 // (measured at batch 2 on a 16-layer stack: depth 2 3.49 TB/s, depth 3 3.56, depth 4 3.38).
 constexpr int kDepth2 = FB_DEPTH2;
-template <int BT> struct DepthFor { static constexpr int value = BT == 2 ? kDepth2 : kDepth; };
+#ifndef FB_DEPTH4
+#define FB_DEPTH4 2
+#endif
+template <int BT> struct DepthFor { static constexpr int value = BT == 4 ? FB_DEPTH4 : BT == 2 ? kDepth2 : kDepth; };
 #ifndef FB_PF
 #define FB_PF 1
 #endif
@@ -95,14 +103,14 @@ struct LaunchParams {
 constexpr uint32_t kTabBase = 0x800u;
 
 template <int BT> struct TabCfg {
-    static constexpr int kTableBytes = 65536;
+    static constexpr int kTableBytes = (BT == 4) ? 131072 : 65536;
     // scale-fusion scratch, tile counters (+ count of completed tiles), work range, copy of the current entry
     static constexpr int kSmallBytes = 256 * BT * 4 + (kMaxTiles + 4) * 4 + 32 + 128;
     // offset of slot sigma from the table base at step 0; entry p adds p << 8.
     // lane_const(lane ^ s) == lane_const(lane) ^ lane_const(s)
     __host__ __device__ static constexpr uint32_t lane_const(uint32_t sigma)
     {
-        return BT == 1 ? sigma * 4u : sigma * 8u;
+        return BT == 1 ? sigma * 4u : BT == 2 ? sigma * 8u : ((sigma & 15u) * 16u) | ((sigma >> 4) << 16);
     }
 };
 
@@ -133,6 +141,7 @@ __device__ __forceinline__ uint32_t ldg_stream_u32(const void *p)
 template <int BT> struct Vec;
 template <> struct Vec<1> { float v[1]; };
 template <> struct Vec<2> { float v[2]; };
+template <> struct Vec<4> { float v[4]; };
 
 // HALF selects the table set inside the 256-byte p-rows: slots 0..31 or (BT == 1 only) slots 32..63.
 template <int BT, int HALF> __device__ __forceinline__ Vec<BT> lds_entry(uint32_t addr)
@@ -140,14 +149,17 @@ template <int BT, int HALF> __device__ __forceinline__ Vec<BT> lds_entry(uint32_
     Vec<BT> r;
     // addr is an offset from the table base; base and half ride in the immediate
     if constexpr (BT == 1) asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(r.v[0]) : "r"(addr), "n"(kTabBase + HALF * 128));
-    else asm volatile("ld.shared.v2.f32 {%0,%1}, [%2+%3];" : "=f"(r.v[0]), "=f"(r.v[1]) : "r"(addr), "n"(kTabBase));
+    else if constexpr (BT == 2) asm volatile("ld.shared.v2.f32 {%0,%1}, [%2+%3];" : "=f"(r.v[0]), "=f"(r.v[1]) : "r"(addr), "n"(kTabBase));
+    else asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4+%5];" : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3]) : "r"(addr), "n"(kTabBase));
     return r;
 }
 
-template <int BT> __device__ __forceinline__ void sts_entry(uint32_t addr, const float *v)
+// the NV batch vectors of one entry at table offset addr
+template <int NV> __device__ __forceinline__ void sts_entry(uint32_t addr, const float *v)
 {
-    if constexpr (BT == 1) asm volatile("st.shared.f32 [%0+%2], %1;" ::"r"(addr), "f"(v[0]), "n"(kTabBase) : "memory");
-    else asm volatile("st.shared.v2.f32 [%0+%3], {%1,%2};" ::"r"(addr), "f"(v[0]), "f"(v[1]), "n"(kTabBase) : "memory");
+    if constexpr (NV == 1) asm volatile("st.shared.f32 [%0+%2], %1;" ::"r"(addr), "f"(v[0]), "n"(kTabBase) : "memory");
+    else if constexpr (NV == 2) asm volatile("st.shared.v2.f32 [%0+%3], {%1,%2};" ::"r"(addr), "f"(v[0]), "f"(v[1]), "n"(kTabBase) : "memory");
+    else asm volatile("st.shared.v4.f32 [%0+%5], {%1,%2,%3,%4};" ::"r"(addr), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "n"(kTabBase) : "memory");
 }
 
 // PRMT with the full selector: bit 3 of a nibble replicates the sign bit of the selected byte
@@ -183,6 +195,7 @@ __device__ __forceinline__ void fetch_build_input(BuildInput<BT> &in, const uint
                                                   int64_t ldx, int nb, int col0_a, int col0_b, int ncols)
 {
     const int tid = threadIdx.x;
+    if (Cfg<BT>::kThreads > 256 && tid >= 256) return;      // one thread per table column
     // {u16 column, fp16 alpha} of (slot tid/8, n tid%8).  For a global pair the column is also known
     // from the pair's position, so x and alpha are fetched side by side, not in a chain.
     if (col0_a >= 0) {       // first unit of the pair: slots 0..15, second unit: slots 16..31
@@ -199,44 +212,53 @@ __device__ __forceinline__ void fetch_build_input(BuildInput<BT> &in, const uint
     }
 }
 
+// Scratch index of a_n of table slot `slot`, batch vector b: rows of 32 slots, rotated by 4n so that both
+// the writers (8 n x 4 slots per warp) and the readers (32 slots per warp, one n) touch 32 different banks.
+template <int BT> __device__ __forceinline__ int abuf_index(int slot, int n, int b)
+{
+    return (n * BT + b) * 32 + ((slot + 4 * n) & 31);
+}
+
 template <int BT>
 __device__ __forceinline__ void build_tables(const BuildInput<BT> &in, float *abuf, uint32_t half_off = 0)
 {
     const int tid = threadIdx.x;
-    {
+    if (Cfg<BT>::kThreads == 256 || tid < 256) {
         const float al = h2f(in.e >> 16);
 #pragma unroll
-        for (int b = 0; b < BT; ++b) abuf[tid * BT + b] = in.xv[b] * al;     // exact in fp32: two 11-bit significands
+        for (int b = 0; b < BT; ++b) abuf[abuf_index<BT>(tid >> 3, tid & 7, b)] = in.xv[b] * al;   // exact in fp32: two 11-bit significands
     }
     __syncthreads();
     const int lane = tid & 31, warp = tid >> 5;
-    constexpr int PW = 256 / kWarps;          // table entries per warp: p = warp*PW + ...
-    static_assert(kThreads == 256 && PW % 16 == 0, "the builder maps one thread to one table column");
+    constexpr int PW = 256 / Cfg<BT>::kWarps;          // table entries per warp: p = warp*PW + ...
+    // EB entries at a time: the high index bits fix a base value, the low LB bits are enumerated by
+    // doubling (entry p | 2^n = entry p + 2 a_n), one add per entry.  All BT batch vectors of an entry are
+    // stored with one instruction (with four vectors, blocks of 8 entries keep the registers in bounds).
+    constexpr int LB = (BT == 4) ? 3 : 4, EB = 1 << LB;
+    static_assert(PW % EB == 0, "a warp enumerates whole blocks of entries");
     float a[8][BT];
 #pragma unroll
     for (int n = 0; n < 8; ++n)
 #pragma unroll
-        for (int b = 0; b < BT; ++b) a[n][b] = abuf[(lane * 8 + n) * BT + b];
-    // 16 entries at a time: the high four index bits fix a base value, the low four are enumerated
-    // by doubling (entry p | 2^n = entry p + 2 a_n), one add per entry
+        for (int b = 0; b < BT; ++b) a[n][b] = abuf[abuf_index<BT>(lane, n, b)];
 #pragma unroll 1
-    for (int p0 = warp * PW; p0 < (warp + 1) * PW; p0 += 16) {
-        float v[16][BT];
+    for (int p0 = warp * PW; p0 < (warp + 1) * PW; p0 += EB) {
+        float v[EB][BT];
 #pragma unroll
         for (int b = 0; b < BT; ++b) {
             float base = 0.f;
 #pragma unroll
-            for (int n = 7; n >= 4; --n) base += ((p0 >> n) & 1) ? a[n][b] : -a[n][b];
+            for (int n = 7; n >= LB; --n) base += ((p0 >> n) & 1) ? a[n][b] : -a[n][b];
 #pragma unroll
-            for (int n = 3; n >= 0; --n) base -= a[n][b];
+            for (int n = LB - 1; n >= 0; --n) base -= a[n][b];
             v[0][b] = base;
 #pragma unroll
-            for (int n = 0; n < 4; ++n)
+            for (int n = 0; n < LB; ++n)
 #pragma unroll
                 for (int q = 0; q < (1 << n); ++q) v[q | (1 << n)][b] = v[q][b] + 2.f * a[n][b];
         }
 #pragma unroll
-        for (int q = 0; q < 16; ++q)
+        for (int q = 0; q < EB; ++q)
             sts_entry<BT>(half_off | TabCfg<BT>::lane_const((uint32_t)lane) | ((uint32_t)(p0 + q) << 8), v[q]);
     }
     __syncthreads();
@@ -311,6 +333,26 @@ template <> struct LaneAddr<2> {
     }
 };
 
+// BT == 4: 16-byte entries; slots 0..15 and 16..31 live in two 64 KB halves, so byte 2 of the address
+// carries the half ((lane ^ s) >> 4, the same for steps 2i and 2i + 1) and byte 3 is zero.
+template <> struct LaneAddr<4> {
+    uint32_t c[16];
+    __device__ __forceinline__ void init(int lane)
+    {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const uint32_t s0 = (uint32_t)(lane ^ (2 * i)), s1 = (uint32_t)(lane ^ (2 * i + 1));
+            c[i] = ((s0 & 15u) * 16u) | (((s1 & 15u) * 16u) << 8) | ((s0 >> 4) << 16);
+            asm volatile("" : "+r"(c[i]));
+        }
+    }
+    __device__ __forceinline__ uint32_t addr(int s, uint32_t w) const
+    {
+        const uint32_t k = (uint32_t)s & 3u, j = (uint32_t)s & 1u;
+        return prmt(w, c[s >> 1], (7u << 12) | (6u << 8) | (k << 4) | (4u | j));
+    }
+};
+
 template <int SPS, int BT, int HALF = 0>
 __device__ __forceinline__ void compute_item(const ItemRegs<SPS> &r, const LaneAddr<BT> &la, float (&out)[BT])
 {
@@ -356,7 +398,7 @@ __device__ __forceinline__ void finish_item(const ItemRegs<SPS> &r, const LaneAd
 
 // The first item of this warp's run, loaded ahead of the table build so that its latency hides
 // behind the build (the weights do not depend on the activations).
-template <int SPS>
+template <int SPS, int BT>
 __device__ __forceinline__ void preload_first(ItemRegs<SPS> &r, const uint8_t *pair_items, int rb_lo, int rb_hi)
 {
     constexpr int IB = ItemBytes<SPS>::value;
@@ -379,6 +421,7 @@ __device__ __forceinline__ void process_rows(const uint8_t *pair_items, int rb_l
                                              const ItemRegs<SPS> *pre = nullptr)   // pre: preload_first's result
 {
     constexpr int IB = ItemBytes<SPS>::value;
+    constexpr int kWarps = Cfg<BT>::kWarps;
     constexpr int STRIDE = kWarps * IB;                   // bytes between a warp's consecutive items
     constexpr int SB = (SPS == 16) ? 4 : (SPS == 8) ? 8 : 16;   // scale bytes per lane (per plane)
     constexpr int D = (SPS == 1) ? 1 : DepthFor<BT>::value;
@@ -423,6 +466,7 @@ __device__ __forceinline__ void process_rows2(const uint8_t *items_a, const uint
                                               const LaneAddr<1> &la, float *acc)
 {
     constexpr int IB = ItemBytes<SPS>::value;
+    constexpr int kWarps = Cfg<1>::kWarps;
     constexpr int STRIDE = kWarps * IB;
     constexpr int SB = (SPS == 16) ? 4 : (SPS == 8) ? 8 : 16;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -454,7 +498,7 @@ __device__ __forceinline__ void process_rows2(const uint8_t *items_a, const uint
 
 // First L2 prefetches of a run of row blocks (issued before the tables are built): the first
 // kPrefetchTrips blocks of D*kWarps items, one D-item request per lane.
-__device__ __forceinline__ void prefetch_run_head(const uint8_t *pair_items, int item_bytes, int D, int rb_lo, int rb_hi)
+__device__ __forceinline__ void prefetch_run_head(const uint8_t *pair_items, int item_bytes, int D, int kWarps, int rb_lo, int rb_hi)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (lane < kPrefetchTrips) {
@@ -466,7 +510,7 @@ __device__ __forceinline__ void prefetch_run_head(const uint8_t *pair_items, int
 
 #ifdef FB_TRACE
 // Instrumented build only: per-CTA phase timestamps (globaltimer, ns) for the cycle breakdown.
-__device__ unsigned long long g_fb_trace[1024][8];
+__device__ unsigned long long g_fb_trace[1024][12];
 __device__ __forceinline__ void trace(int slot)
 {
     if (threadIdx.x == 0 && blockIdx.x < 1024) {
@@ -490,7 +534,7 @@ __device__ __forceinline__ void trace_add(int slot, unsigned long long t0)
 #define FB_TRACE_T0(var) unsigned long long var = trace_now()
 #define FB_TRACE_ADD(slot, var) trace_add(slot, var)
 #define FB_TRACE_SET(var) var = trace_now()
-#define FB_TRACE_ZERO() do { if (threadIdx.x == 0 && blockIdx.x < 1024) { g_fb_trace[blockIdx.x][4] = 0; g_fb_trace[blockIdx.x][5] = 0; g_fb_trace[blockIdx.x][6] = 0; g_fb_trace[blockIdx.x][7] = 0; g_fb_trace[blockIdx.x][1] = 0; g_fb_trace[blockIdx.x][2] = 0; } } while (0)
+#define FB_TRACE_ZERO() do { if (threadIdx.x == 0 && blockIdx.x < 1024) { g_fb_trace[blockIdx.x][4] = 0; g_fb_trace[blockIdx.x][5] = 0; g_fb_trace[blockIdx.x][6] = 0; g_fb_trace[blockIdx.x][7] = 0; g_fb_trace[blockIdx.x][1] = 0; g_fb_trace[blockIdx.x][2] = 0; g_fb_trace[blockIdx.x][8] = 0; g_fb_trace[blockIdx.x][9] = 0; g_fb_trace[blockIdx.x][10] = 0; } } while (0)
 #else
 #define FB_TRACE_AT(slot)
 #define FB_TRACE_T0(var)
@@ -505,6 +549,7 @@ template <int BT>
 __device__ __forceinline__ void reduce_and_store(const LinearEntry &E, int nb, int y_fp32, int *tile_cnt, int *done_list)
 {
     const int tid = threadIdx.x;
+    constexpr int kThreads = Cfg<BT>::kThreads;
     __threadfence();
     __syncthreads();
     const int npairs = E.npairs[0] + E.npairs[1];
@@ -580,9 +625,10 @@ __device__ __forceinline__ void reduce_and_store(const LinearEntry &E, int nb, i
 #define FB_MINB 3
 #endif
 template <int SPS0, int SPS1, int BT, int NP>
-__global__ void __launch_bounds__(kThreads, (BT == 2) ? 2 : FB_MINB)
+__global__ void __launch_bounds__(Cfg<BT>::kThreads, (BT == 1) ? FB_MINB : Cfg<BT>::kMinBlocks)
 fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
 {
+    constexpr int kThreads = Cfg<BT>::kThreads, kWarps = Cfg<BT>::kWarps;
     // dynamic shared memory: [kTabBase, +tables) at a fixed window address, small buffers after it
     extern __shared__ __align__(16) uint8_t smem[];
     const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem);
@@ -595,6 +641,7 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
     LinearEntry *Es = (LinearEntry *)(range + 8);  // the current entry, copied once (128 bytes)
     static_assert(sizeof(LinearEntry) == 128, "entry copy below moves 32 words");
     static_assert(NP == 1 || BT == 1, "two table sets side by side need the 4-byte slots of BT == 1");
+    static_assert(BT == 1 || BT == 2 || BT == 4, "batch vectors per launch");
     const int tid = threadIdx.x;
     FB_TRACE_AT(0);
     FB_TRACE_ZERO();
@@ -700,8 +747,8 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
             const uint8_t *items = E.packed + E.off_items[region] + (size_t)pair * E.nrb * ib;
             const uint8_t *items_b = items + (size_t)E.nrb * ib;
             const int pf_d = np == 2 ? 1 : (region ? SPS1 : SPS0) == 1 ? 1 : DepthFor<BT>::value;
-            prefetch_run_head(items, ib, pf_d, rb_lo, rb_hi);                 // weights start moving now
-            if (np == 2) prefetch_run_head(items_b, ib, pf_d, rb_lo, rb_hi);
+            prefetch_run_head(items, ib, pf_d, kWarps, rb_lo, rb_hi);         // weights start moving now
+            if (np == 2) prefetch_run_head(items_b, ib, pf_d, kWarps, rb_lo, rb_hi);
 
             if (!predecessor_done) {
                 asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -709,6 +756,8 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
             }
             FB_TRACE_T0(t_build);
             __syncthreads();     // previous segment's lookups are done before the tables are overwritten
+            FB_TRACE_ADD(8, t_build);
+            FB_TRACE_T0(t_fetch);
             // (fetching the next pair's inputs ahead of the lookups was measured 15 % slower: the extra
             // live registers push the lookup loop over the 80-register budget of 3 CTAs per SM)
             BuildInput<BT> bin, bin_b;
@@ -717,7 +766,8 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
             // region 0, one pair at a time (short runs): first item in flight during the build.  (With two
             // pairs per row block the runs are long and the extra live registers cost more than they hide.)
             ItemRegs<SPS0> pre;
-            if (NP == 1 && region == 0) preload_first<SPS0>(pre, items, rb_lo, rb_hi);
+            if (NP == 1 && region == 0) preload_first<SPS0, BT>(pre, items, rb_lo, rb_hi);
+            FB_TRACE_ADD(9, t_fetch);
             build_tables<BT>(bin, abuf);
             if (np == 2) build_tables<BT>(bin_b, abuf, 128u);
             FB_TRACE_ADD(4, t_build);
@@ -766,9 +816,10 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
 }
 
 // Test hook: build one table set exactly as the kernel does and write it out as [32][256] fp32.
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(Cfg<1>::kThreads, 1)
 fluxbin_debug_tables_kernel(const uint8_t *pair_desc, const uint16_t *x, float *out)
 {
+    constexpr int kThreads = Cfg<1>::kThreads;
     extern __shared__ __align__(16) uint8_t smem[];
     const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem);
     if (smem_base > kTabBase) return;
