@@ -252,6 +252,12 @@ fluxbin_status_t fluxbin_plan_run(const fluxbin_plan_t *plan, void *cuda_stream)
 /* Kernel launches one fluxbin_plan_run issues (one per chunk of up to 4 batch vectors); -1 on NULL. */
 int32_t fluxbin_plan_num_launches(const fluxbin_plan_t *plan);
 
+/* Introspection: how many table sets (pairs of 16-sub-vector units) the plan's kernel keeps resident per row
+ * block -- 2 when every member has an even number of global pairs, the batch is 1 and each CTA's share of the
+ * plan spans several whole couples of pairs (then two pairs' row sums share one reduction, stage (iii)), else 1.
+ * Both variants compute the same sums (Eq. 15) in a different order.  -1 on NULL. */
+int32_t fluxbin_plan_pairs_per_row_block(const fluxbin_plan_t *plan);
+
 /* Release the host object (never touches device memory).  NULL is allowed. */
 void fluxbin_plan_free(fluxbin_plan_t *plan);
 

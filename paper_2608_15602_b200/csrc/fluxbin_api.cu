@@ -232,8 +232,16 @@ extern "C" fluxbin_status_t fluxbin_workspace_init(void *d_workspace, size_t byt
 
 // ---- the layer ------------------------------------------------------------------------------------
 
+// How a launch is cut: grid size, the statically dealt part of the cost line, the number of shares, and
+// whether the two-pairs-per-row-block kernel runs.
+struct LaunchShape {
+    long long grid, static_cost;
+    int nshares;
+    bool couples;
+};
+
 template <int S0, int S1, int BT>
-static cudaError_t launch(const fbk::LaunchParams &p, int num_sms, long long items, long long couple_cost, cudaStream_t s)
+static cudaError_t launch_shape(long long total_cost, int num_sms, long long items, long long couple_cost, LaunchShape *out)
 {
     static int occ = 0;     // resident CTAs per SM of this instantiation (same on every B200)
     if (occ == 0) {
@@ -247,20 +255,33 @@ static cudaError_t launch(const fbk::LaunchParams &p, int num_sms, long long ite
     if (items < grid) grid = items;
     // Launches with enough work deal 90 % of it out statically and cut the rest into three small
     // shares per CTA (each worth >= ~200 items), drawn dynamically; small launches stay static.
-    fbk::LaunchParams q = p;
     constexpr int dyn_pct = 10, dyn_k = 3;
-    const long long rest = p.total_cost * dyn_pct / 100;
+    const long long rest = total_cost * dyn_pct / 100;
     if (dyn_pct > 0 && dyn_k > 0 && rest / (grid * dyn_k) >= 400) {
-        q.static_cost = p.total_cost - rest;
-        q.nshares = (int)(grid * (1 + dyn_k));
+        out->static_cost = total_cost - rest;
+        out->nshares = (int)(grid * (1 + dyn_k));
     } else {
-        q.static_cost = p.total_cost;
-        q.nshares = (int)grid;
+        out->static_cost = total_cost;
+        out->nshares = (int)grid;
     }
+    out->grid = grid;
     // two pairs per row block (half the reduction traffic) when every layer allows it (couple_cost > 0:
     // even pair counts everywhere) and a CTA's share spans several whole couples
-    bool couples = false;
-    if constexpr (BT == 1) couples = couple_cost > 0 && q.static_cost / grid >= 2 * couple_cost;
+    out->couples = BT == 1 && couple_cost > 0 && out->static_cost / grid >= 2 * couple_cost;
+    return cudaSuccess;
+}
+
+template <int S0, int S1, int BT>
+static cudaError_t launch(const fbk::LaunchParams &p, int num_sms, long long items, long long couple_cost, cudaStream_t s)
+{
+    LaunchShape shape;
+    cudaError_t se = launch_shape<S0, S1, BT>(p.total_cost, num_sms, items, couple_cost, &shape);
+    if (se != cudaSuccess) return se;
+    const long long grid = shape.grid;
+    const bool couples = shape.couples;
+    fbk::LaunchParams q = p;
+    q.static_cost = shape.static_cost;
+    q.nshares = shape.nshares;
     // launched with programmatic stream serialization: the kernel may start while its predecessor in
     // the stream drains (it waits inside, before touching activations or workspace)
     cudaLaunchConfig_t cfg = {};
@@ -511,6 +532,20 @@ extern "C" fluxbin_status_t fluxbin_plan_run(const fluxbin_plan_t *plan, void *c
 }
 
 extern "C" int32_t fluxbin_plan_num_launches(const fluxbin_plan_t *plan) { return plan ? plan->nchunks : -1; }
+
+extern "C" int32_t fluxbin_plan_pairs_per_row_block(const fluxbin_plan_t *plan)
+{
+    if (!plan) return -1;
+    if (plan->B != 1) return 1;          // the two-pair kernel exists for single-vector launches only
+    LaunchShape shape;
+    cudaError_t e;
+    if (plan->sps0 == 16 && plan->sps1 == 16) e = launch_shape<16, 16, 1>(plan->total_cost, plan->num_sms, plan->items, plan->couple_cost, &shape);
+    else if (plan->sps0 == 16) e = launch_shape<16, 1, 1>(plan->total_cost, plan->num_sms, plan->items, plan->couple_cost, &shape);
+    else if (plan->sps0 == 8) e = launch_shape<8, 1, 1>(plan->total_cost, plan->num_sms, plan->items, plan->couple_cost, &shape);
+    else e = launch_shape<4, 1, 1>(plan->total_cost, plan->num_sms, plan->items, plan->couple_cost, &shape);
+    if (e != cudaSuccess) return -1;
+    return shape.couples ? 2 : 1;
+}
 
 extern "C" void fluxbin_plan_free(fluxbin_plan_t *plan) { delete plan; }
 

@@ -37,7 +37,8 @@ EXPORTS = ["fluxbin_packed_size", "fluxbin_validate", "fluxbin_pack_host", "flux
            "fluxbin_workspace_size", "fluxbin_workspace_init", "fluxbin_linear", "fluxbin_debug_tables",
            "fluxbin_num_table_sets", "fluxbin_num_launches", "fluxbin_free", "fluxbin_status_string",
            "fluxbin_last_cuda_error", "fluxbin_plan_table_bytes", "fluxbin_plan_workspace_bytes",
-           "fluxbin_plan_create", "fluxbin_plan_run", "fluxbin_plan_num_launches", "fluxbin_plan_free",
+           "fluxbin_plan_create", "fluxbin_plan_run", "fluxbin_plan_num_launches", "fluxbin_plan_pairs_per_row_block",
+           "fluxbin_plan_free",
            "fluxbin_linear_noalloc", "fluxbin_noalloc_capacity"]
 
 _LIB = None
@@ -81,6 +82,7 @@ def _lib():
                                             ctypes.POINTER(vp)]
         lib.fluxbin_plan_run.restype, lib.fluxbin_plan_run.argtypes = ctypes.c_int, [vp, vp]
         lib.fluxbin_plan_num_launches.restype, lib.fluxbin_plan_num_launches.argtypes = i32, [vp]
+        lib.fluxbin_plan_pairs_per_row_block.restype, lib.fluxbin_plan_pairs_per_row_block.argtypes = i32, [vp]
         lib.fluxbin_plan_free.restype, lib.fluxbin_plan_free.argtypes = None, [vp]
         lib.fluxbin_linear_noalloc.restype = ctypes.c_int
         lib.fluxbin_linear_noalloc.argtypes = [vp, vp, i32, i64, vp, i32, i64, vp]
@@ -259,6 +261,9 @@ class Plan:
 
     def num_launches(self) -> int:
         return int(_lib().fluxbin_plan_num_launches(self.handle))
+
+    def pairs_per_row_block(self) -> int:
+        return int(_lib().fluxbin_plan_pairs_per_row_block(self.handle))
 
     def close(self):
         if self.handle:

@@ -87,3 +87,6 @@ class FluxBinPlan:
 
     def num_launches(self) -> int:
         return self.plan.num_launches()
+
+    def pairs_per_row_block(self) -> int:
+        return self.plan.pairs_per_row_block()

@@ -94,6 +94,40 @@ def test_plan_equals_single_calls_on_a_70b_layer(fb):
         check(y.cpu().numpy(), want, f"70B member {lin.M}x{lin.N}")
 
 
+def test_long_plan_runs_the_two_pair_kernel(fb):
+    """A plan whose shares span whole couples of pairs launches the kernel variant that keeps two table sets
+    resident and reduces two pairs' row sums at once (the variant the full-stack benchmark times); a short
+    plan of the same members launches the one-pair variant.  Both must match the oracle on every output."""
+    shapes = [(256, 4096), (250, 4096), (512, 4096), (96, 8192)]
+    members, wants = [], []
+    for i in range(72):
+        M, N = shapes[i % len(shapes)]
+        n_sal = int(round(0.05 * N))
+        L = layer_of(500 + i, M, N, 2, 1, 128, n_sal)
+        x = synth.make_activations(9, i, 1, N)
+        lin = fb.FluxBinLinear(L)
+        members.append((lin, torch.from_numpy(x.view(np.float16)).cuda(),
+                        torch.full((1, M), float("nan"), dtype=torch.float32, device="cuda")))
+        wants.append(oracle.linear_direct(L, x))
+    long_plan = fb.FluxBinPlan(members)
+    assert long_plan.pairs_per_row_block() == 2
+    for _ in range(2):                      # twice: the workspace must come back zeroed
+        for _, _, y in members:
+            y.fill_(float("nan"))
+        long_plan.run()
+        torch.cuda.synchronize()
+        for (lin, _, y), want in zip(members, wants):
+            check(y.cpu().numpy(), want, f"two-pair kernel, member {lin.M}x{lin.N}")
+    short_plan = fb.FluxBinPlan(members[:4])
+    assert short_plan.pairs_per_row_block() == 1
+    for _, _, y in members[:4]:
+        y.fill_(float("nan"))
+    short_plan.run()
+    torch.cuda.synchronize()
+    for (lin, _, y), want in zip(members[:4], wants[:4]):
+        check(y.cpu().numpy(), want, f"one-pair kernel, member {lin.M}x{lin.N}")
+
+
 def test_plan_rejects_mixed_scale_formats_and_bad_buffers(fb):
     from paper_2608_15602_b200 import fluxbin
     a = fb.FluxBinLinear(layer_of(1, 64, 256, 2, 0, 128, 0))
