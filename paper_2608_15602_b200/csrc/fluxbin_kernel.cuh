@@ -171,17 +171,24 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
     return d;
 }
 
+// One 128-byte line into L2, under a predicate (no branch, no reconvergence point in the caller's loop).
+__device__ __forceinline__ void prefetch_line_if(const void *p, bool pred)
+{
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %1, 0;\n\t@q prefetch.global.L2 [%0];\n\t}" ::"l"(p), "r"((uint32_t)pred) : "memory");
+}
+
+// fp32 add into the split-K accumulator (global memory by contract).  Spelled out as a reduction on the
+// global window: through a generic pointer the compiler emits an address-space check with a divergence
+// barrier, a vote and a branch around every atomic.
+__device__ __forceinline__ void red_add_f32(float *p, float v)
+{
+    asm volatile("red.global.add.f32 [%0], %1;" ::"l"(__cvta_generic_to_global(p)), "f"(v) : "memory");
+}
+
 // One bulk request that pulls `bytes` (a multiple of 16) starting at p into L2.
 __device__ __forceinline__ void prefetch_l2(const void *p, uint32_t bytes)
 {
     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
-}
-
-// The same under a predicate (no branch, no reconvergence point in the caller's loop).
-__device__ __forceinline__ void prefetch_l2_if(const void *p, uint32_t bytes, bool pred)
-{
-    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %2, 0;\n\t@q cp.async.bulk.prefetch.L2.global [%0], %1;\n\t}"
-                 ::"l"(p), "r"(bytes), "r"((uint32_t)pred) : "memory");
 }
 
 
@@ -401,7 +408,7 @@ __device__ __forceinline__ void finish_item(const ItemRegs<SPS> &r, const LaneAd
     float out[BT];
     compute_item<SPS, BT>(r, la, out);
 #pragma unroll
-    for (int b = 0; b < BT; ++b) atomicAdd(accp + (int64_t)b * Mpad, out[b]);
+    for (int b = 0; b < BT; ++b) red_add_f32(accp + (int64_t)b * Mpad, out[b]);
 }
 
 // The first item of this warp's run, loaded ahead of the table build so that its latency hides
@@ -484,25 +491,30 @@ __device__ __forceinline__ void process_rows2(const uint8_t *items_a, const uint
     const int64_t o_l = (int64_t)first * IB + lane * 16, o_s = (int64_t)first * IB + FB_ITEM_BITS_BYTES + lane * SB;
     const uint8_t *pla = items_a + o_l, *psa = items_a + o_s;
     const uint8_t *plb = items_b + o_l, *psb = items_b + o_s;
-    // the CTA reads kWarps items of each pair per trip; lanes 0 and 1 of every warp prefetch the
-    // warp's own item of the trip kPrefetchTrips + 1 ahead in the first and the second pair
-    const uint8_t *pp = (lane == 0 ? items_a : items_b) + (int64_t)first * IB + (int64_t)(kPrefetchTrips + 1) * STRIDE;
+    // lanes 0..8 and 9..17 of every warp prefetch, line by line, the warp's own item of the trip
+    // kPrefetchTrips + 1 ahead in the first and the second pair (one ordinary instruction per trip: the bulk
+    // prefetch is a uniform-datapath instruction and costs a lane-by-lane loop when its address is per lane)
+    static_assert(IB % 128 == 0 && IB / 128 <= 16, "an item is at most 16 lines");
+    constexpr int LPI = IB / 128;
+    const uint8_t *pp = (lane < LPI ? items_a : items_b) + (int64_t)first * IB + (int64_t)(kPrefetchTrips + 1) * STRIDE +
+                        (lane < LPI ? lane : lane - LPI) * 128;
     float *accp = acc + first * 32 + lane;
 
     ItemRegs<SPS> ra, rb;
     load_item<SPS>(ra, pla, psa, 0);
     // steady state without a condition in it (the last row block is peeled off below): the loads of the
     // next item are unconditional and the prefetch is one predicated instruction (measured +4 %: the
-    // guarded form cost about 20 extra instructions per item in moves, predicate logic and branches)
-    const int n_pf = lane < 2 ? n - (kPrefetchTrips + 1) : 0;      // trips in which this lane prefetches
+    // guarded form cost about 20 extra instructions per item in moves, predicate logic and branches;
+    // per-line instead of bulk prefetch another +1.5 %)
+    const int n_pf = lane < 2 * LPI ? n - (kPrefetchTrips + 1) : 0;      // trips in which this lane prefetches
     for (int t = 0; t < n - 1; ++t) {
-        prefetch_l2_if(pp, IB, t < n_pf);
+        prefetch_line_if(pp, t < n_pf);
         load_item<SPS>(rb, plb, psb, 0);
         float oa[1], ob[1];
         compute_item<SPS, 1, 0>(ra, la, oa);
         load_item<SPS>(ra, pla, psa, STRIDE);
         compute_item<SPS, 1, 1>(rb, la, ob);
-        atomicAdd(accp, oa[0] + ob[0]);
+        red_add_f32(accp, oa[0] + ob[0]);
         pla += STRIDE; psa += STRIDE; plb += STRIDE; psb += STRIDE; pp += STRIDE;
         accp += kWarps * 32;
     }
@@ -511,7 +523,7 @@ __device__ __forceinline__ void process_rows2(const uint8_t *items_a, const uint
         float oa[1], ob[1];
         compute_item<SPS, 1, 0>(ra, la, oa);
         compute_item<SPS, 1, 1>(rb, la, ob);
-        atomicAdd(accp, oa[0] + ob[0]);
+        red_add_f32(accp, oa[0] + ob[0]);
     }
 }
 
