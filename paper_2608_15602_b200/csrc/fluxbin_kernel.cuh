@@ -306,6 +306,14 @@ template <int SPS> __device__ __forceinline__ void load_item(ItemRegs<SPS> &r, c
     }
 }
 
+// The three parts of an item separately (SPS >= 2), each into the registers its predecessor's lookups have freed.
+template <int SPS> __device__ __forceinline__ void load_scales(ItemRegs<SPS> &r, const uint8_t *ps, int off)
+{
+    if constexpr (SPS == 16) r.sc[0] = ldg_stream_u32(ps + off);
+    else if constexpr (SPS == 8) { uint2 t = ldg_stream_v2(ps + off); r.sc[0] = t.x; r.sc[1] = t.y; }
+    else { uint4 t = ldg_stream_v4(ps + off); r.sc[0] = t.x; r.sc[1] = t.y; r.sc[2] = t.z; r.sc[3] = t.w; }
+}
+
 // Lane constant of the lookup address.  BT == 1: one register holding, byte by byte, the slot offsets
 // (lane ^ k) * 4 of steps k = 0..3, so that PRMT can drop one into byte 0 of the address; the offsets
 // of steps 4q + k differ from these by an XOR with 16q in every byte ((lane ^ (4q + k)) * 4 ==
@@ -399,6 +407,29 @@ __device__ __forceinline__ void compute_item(const ItemRegs<SPS> &r, const LaneA
         float scale = h2f((r.sc[j >> 1] >> ((j & 1) * 16)) & 0xffffu);
 #pragma unroll
         for (int b = 0; b < BT; ++b) out[b] = fmaf(scale, seg[b], out[b]);
+    }
+}
+
+// Half an item (steps 16H .. 16H+15, the weight bytes of one 128-bit load) for one batch vector: adds the
+// scaled segment sums of that half to out.  SPS >= 2.
+template <int SPS, int HALF, int H>
+__device__ __forceinline__ void compute_half(const uint4 &b, const uint32_t *sc, const LaneAddr<1> &la, float &out)
+{
+    static_assert(SPS >= 2 && SPS <= 16, "segments do not straddle the two halves");
+    constexpr int NSEG_H = 16 / SPS;
+    const uint32_t w[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+    for (int jj = 0; jj < NSEG_H; ++jj) {
+        const int j = H * NSEG_H + jj;
+        float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+        for (int q = 0; q < SPS; ++q) {
+            const int s = j * SPS + q;
+            const float e = lds_entry<1, HALF>(la.addr(s, w[(s >> 2) & 3])).v[0];
+            if (q & 1) s1 += e; else s0 += e;
+        }
+        const float scale = h2f((sc[j >> 1] >> ((j & 1) * 16)) & 0xffffu);
+        out = fmaf(scale, s0 + s1, out);
     }
 }
 
@@ -500,30 +531,39 @@ __device__ __forceinline__ void process_rows2(const uint8_t *items_a, const uint
                         (lane < LPI ? lane : lane - LPI) * 128;
     float *accp = acc + first * 32 + lane;
 
+    // Both items of the current row block are in registers (or on their way) at the top of a trip; each
+    // 128-bit half of the next row block's items is requested as soon as the lookups of the half it
+    // replaces are done, so a load has 1.5 item times to arrive instead of one, with no extra registers.
+    // The last row block is peeled off: the steady state has no guards in it, and the prefetch is one
+    // predicated instruction (guards cost about 20 instructions per item in moves, predicates and branches).
     ItemRegs<SPS> ra, rb;
     load_item<SPS>(ra, pla, psa, 0);
-    // steady state without a condition in it (the last row block is peeled off below): the loads of the
-    // next item are unconditional and the prefetch is one predicated instruction (measured +4 %: the
-    // guarded form cost about 20 extra instructions per item in moves, predicate logic and branches;
-    // per-line instead of bulk prefetch another +1.5 %)
+    load_item<SPS>(rb, plb, psb, 0);
     const int n_pf = lane < 2 * LPI ? n - (kPrefetchTrips + 1) : 0;      // trips in which this lane prefetches
     for (int t = 0; t < n - 1; ++t) {
         prefetch_line_if(pp, t < n_pf);
-        load_item<SPS>(rb, plb, psb, 0);
-        float oa[1], ob[1];
-        compute_item<SPS, 1, 0>(ra, la, oa);
-        load_item<SPS>(ra, pla, psa, STRIDE);
-        compute_item<SPS, 1, 1>(rb, la, ob);
-        red_add_f32(accp, oa[0] + ob[0]);
+        float o = 0.f;
+        compute_half<SPS, 0, 0>(ra.b0, ra.sc, la, o);
+        ra.b0 = ldg_stream_v4(pla + STRIDE);
+        compute_half<SPS, 0, 1>(ra.b1, ra.sc, la, o);
+        ra.b1 = ldg_stream_v4(pla + STRIDE + 512);
+        load_scales<SPS>(ra, psa, STRIDE);
+        compute_half<SPS, 1, 0>(rb.b0, rb.sc, la, o);
+        rb.b0 = ldg_stream_v4(plb + STRIDE);
+        compute_half<SPS, 1, 1>(rb.b1, rb.sc, la, o);
+        rb.b1 = ldg_stream_v4(plb + STRIDE + 512);
+        load_scales<SPS>(rb, psb, STRIDE);
+        red_add_f32(accp, o);
         pla += STRIDE; psa += STRIDE; plb += STRIDE; psb += STRIDE; pp += STRIDE;
         accp += kWarps * 32;
     }
     {
-        load_item<SPS>(rb, plb, psb, 0);
-        float oa[1], ob[1];
-        compute_item<SPS, 1, 0>(ra, la, oa);
-        compute_item<SPS, 1, 1>(rb, la, ob);
-        red_add_f32(accp, oa[0] + ob[0]);
+        float o = 0.f;
+        compute_half<SPS, 0, 0>(ra.b0, ra.sc, la, o);
+        compute_half<SPS, 0, 1>(ra.b1, ra.sc, la, o);
+        compute_half<SPS, 1, 0>(rb.b0, rb.sc, la, o);
+        compute_half<SPS, 1, 1>(rb.b1, rb.sc, la, o);
+        red_add_f32(accp, o);
     }
 }
 
