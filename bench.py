@@ -125,6 +125,42 @@ def cpu_oracle_sample(config: int, B: int, max_linears: int = 28):
     return tot_b / tot_t / 1e9, tot_t, tot_b, oracle.num_threads(), f"first {n} linears of the stack (B={B})"
 
 
+def dense_fp16_gemv_context(lins, nl, B):
+    """Context, not a target: a dense fp16 weight of every distinct shape of the workload through cuBLAS
+    (torch.matmul, harness only), rotating over enough copies that the weights come from HBM; returns the
+    time the whole stack would take at those per-shape rates and the per-shape timings."""
+    import torch
+    shapes = {}
+    for _, M, N in lins:
+        shapes[(M, N)] = shapes.get((M, N), 0) + nl
+    per_shape, total_us, total_bytes = {}, 0.0, 0
+    for (M, N), count in shapes.items():
+        copies = max(2, int(600e6 // (2 * M * N)) + 1)               # > 4x L2 of weights in rotation
+        w = [torch.randn(M, N, device="cuda", dtype=torch.float16) for _ in range(copies)]
+        x = torch.randn(N, B, device="cuda", dtype=torch.float16)
+        for i in range(copies):
+            torch.matmul(w[i], x)
+        torch.cuda.synchronize()
+        reps = max(1, 60 // copies)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            for i in range(copies):
+                torch.matmul(w[i], x)
+        b.record()
+        torch.cuda.synchronize()
+        us = a.elapsed_time(b) * 1e3 / (reps * copies)
+        per_shape[f"{M}x{N}"] = {"us": round(us, 2), "GBps": round(2 * M * N / us / 1e3, 1), "count": count}
+        total_us += us * count
+        total_bytes += 2 * M * N * count
+        del w, x
+    torch.cuda.empty_cache()
+    return {"ms_per_step": total_us / 1e3, "dense_weight_bytes_per_step": total_bytes,
+            "GBps_of_dense_bytes": total_bytes / total_us / 1e3, "per_shape": per_shape,
+            "how": "torch.matmul (cuBLAS) on random fp16 weights of the same shapes, plain launches, rotating copies "
+                   "larger than L2; per-shape time x count"}
+
+
 def run_reference(args, rank):
     """--impl reference: the CPU oracle on the host cores, each step a bounded sample."""
     if rank != 0:
@@ -163,6 +199,7 @@ def main():
                          "layer; stack: one plan for the whole stack (valid because the workload gives every "
                          "linear its own input)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-context", action="store_true", help="skip the dense fp16 cuBLAS GEMV context timing")
     ap.add_argument("--ref-linears", type=int, default=7, help="linears per step of --impl reference")
     ap.add_argument("--per-linear", action="store_true", help="also print per-linear timings to stderr")
     args = ap.parse_args()
@@ -199,6 +236,7 @@ def main():
             synth.make_config_activations(args.config, layer, li, B)
 
     linears, xs_host, alg_bytes = [], [], []
+    eff_flops = 0.0
     nthreads = max(1, min(16, (os.cpu_count() or 4) - 1))
     with cf.ThreadPoolExecutor(nthreads) as ex:
         window = []
@@ -216,6 +254,7 @@ def main():
             linears.append(lin)
             xs_host.append(x)
             alg_bytes.append(algorithmic_bytes(L.M, L.N, L.Kb, L.Ks, L.g, L.n_sal, B))
+            eff_flops += 2.0 * L.M * (L.N + L.n_sal) * B
             del L
     setup_s = time.perf_counter() - t_setup
 
@@ -456,6 +495,10 @@ def main():
             "gpu_launches": launches_per_step * args.steps,
             "clocks": clocks, "setup_s": round(setup_s, 1),
         }
+        # the paper's effective-throughput figure: 2 * M * (N + n_sal) * B flops per linear over the measured time
+        line["effective_tflops"] = eff_flops / (ms_per_step * 1e-3) / 1e12
+        if not args.no_context:
+            line["context_dense_fp16_gemv"] = dense_fp16_gemv_context(lins, nl, B)
         if not args.no_cpu_baseline:
             gbps, tsec, nbytes, cores, sample = cpu_oracle_sample(args.config, B)
             line["cpu_baseline"] = {"value": gbps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
