@@ -101,9 +101,15 @@ class ClockSampler:
 
 
 def stack_spec(config: int, layers: int | None):
+    """Linears of one layer (or set) of the workload and how many such layers a step runs.  The single-layer
+    and single-set workloads (configs 0-3) are run as a rotation of independently seeded copies, enough of them
+    that a step streams more than four times the L2 capacity: weights come from HBM, as in decode."""
     lins, nl = synth.config_linears(config)
     if layers is not None:
         nl = layers
+    elif config < 4:
+        set_bytes = sum(M * N for _, M, N in lins) * 2.43 / 8          # about 2.43 bits per weight
+        nl = max(1, int(540e6 // set_bytes) + 1)
     return lins, nl
 
 
@@ -474,7 +480,8 @@ def main():
             "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": f"config {args.config}: Llama-2-70B-shaped decode linear stack" if args.config == 4
-                       else f"config {args.config}", "layers": nl, "linears_per_step": len(linears), "batch": B,
+                       else f"config {args.config}: {nl} independently seeded copies of the layer/set per step",
+                       "layers": nl, "linears_per_step": len(linears), "batch": B,
                        "Kb": 2, "Ks": 0 if args.config == 0 else 1, "salient_frac": 0.0 if args.config == 0 else 0.05,
                        "g": args.g or "N", "packed_bytes_resident": packed_bytes, "algorithmic_bytes_per_step": bytes_per_step,
                        "l2": "inputs larger than L2 (weights streamed once per step)" if packed_bytes > 4e8
