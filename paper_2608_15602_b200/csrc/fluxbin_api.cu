@@ -533,17 +533,23 @@ extern "C" fluxbin_status_t fluxbin_plan_run(const fluxbin_plan_t *plan, void *c
 
 extern "C" int32_t fluxbin_plan_num_launches(const fluxbin_plan_t *plan) { return plan ? plan->nchunks : -1; }
 
+// the launch shape of the single-vector kernel family that reads (sps0, sps1) layers
+static cudaError_t launch_shape_bt1(int s0, int s1, long long total_cost, int num_sms, long long items, long long couple_cost,
+                                    LaunchShape *shape)
+{
+    if (s0 == 16 && s1 == 16) return launch_shape<16, 16, 1>(total_cost, num_sms, items, couple_cost, shape);
+    if (s0 == 16) return launch_shape<16, 1, 1>(total_cost, num_sms, items, couple_cost, shape);
+    if (s0 == 8) return launch_shape<8, 1, 1>(total_cost, num_sms, items, couple_cost, shape);
+    return launch_shape<4, 1, 1>(total_cost, num_sms, items, couple_cost, shape);
+}
+
 extern "C" int32_t fluxbin_plan_pairs_per_row_block(const fluxbin_plan_t *plan)
 {
     if (!plan) return -1;
     if (plan->B != 1) return 1;          // the two-pair kernel exists for single-vector launches only
     LaunchShape shape;
-    cudaError_t e;
-    if (plan->sps0 == 16 && plan->sps1 == 16) e = launch_shape<16, 16, 1>(plan->total_cost, plan->num_sms, plan->items, plan->couple_cost, &shape);
-    else if (plan->sps0 == 16) e = launch_shape<16, 1, 1>(plan->total_cost, plan->num_sms, plan->items, plan->couple_cost, &shape);
-    else if (plan->sps0 == 8) e = launch_shape<8, 1, 1>(plan->total_cost, plan->num_sms, plan->items, plan->couple_cost, &shape);
-    else e = launch_shape<4, 1, 1>(plan->total_cost, plan->num_sms, plan->items, plan->couple_cost, &shape);
-    if (e != cudaSuccess) return -1;
+    if (launch_shape_bt1(plan->sps0, plan->sps1, plan->total_cost, plan->num_sms, plan->items, plan->couple_cost, &shape) != cudaSuccess)
+        return -1;
     return shape.couples ? 2 : 1;
 }
 
