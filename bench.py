@@ -87,17 +87,22 @@ class ClockSampler:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
         self.thread.join(timeout=2)
-        sm, smax, reasons = [], [], set()
+        sm, smax, power, reasons = [], [], [], set()
         for r in self.rows:
             try:
                 sm.append(float(r[0])); smax.append(float(r[1]))
             except (ValueError, IndexError):
                 continue
+            try:
+                power.append(float(r[2]))
+            except (ValueError, IndexError):
+                pass
             for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "reasons": sorted(reasons),
+                "power_w": statistics.median(power) if power else None}
 
 
 def stack_spec(config: int, layers: int | None):
@@ -113,22 +118,33 @@ def stack_spec(config: int, layers: int | None):
     return lins, nl
 
 
-def cpu_oracle_sample(config: int, B: int, max_linears: int = 28):
+def cpu_oracle_sample(config: int, B: int, max_linears: int = 28, g: int = 128, nl: int | None = None, gpu_y=None):
     """Time the oracle as it stands on the first linears of the stack (bounded sample); returns
-    (GB/s of algorithmic bytes, seconds, bytes, cores, description)."""
+    (GB/s of algorithmic bytes, seconds, bytes, cores, description, agreement).  gpu_y(i) -> the fp16 outputs
+    [B][M] the timed GPU run left for linear i: since the oracle's results are at hand anyway, the leg also
+    reports how far the two are apart (same measures as the parity tests)."""
     import oracle
-    lins, nl = synth.config_linears(config)
-    n = min(max_linears, len(lins) * nl)
+    lins, nl_default = synth.config_linears(config)
+    n = min(max_linears, len(lins) * (nl or nl_default))
     tot_b, tot_t = 0, 0.0
+    worst_l2, worst_rel = 0.0, 0.0
     for i in range(n):
         layer, li = divmod(i, len(lins))
-        L = synth.make_config_linear(config, layer, li)
+        L = synth.make_config_linear(config, layer, li, g=(g or lins[li][2]))
         x = synth.make_config_activations(config, layer, li, B)
         t0 = time.perf_counter()
-        oracle.linear_direct(L, x)
+        want = oracle.linear_direct(L, x)
         tot_t += time.perf_counter() - t0
         tot_b += algorithmic_bytes(L.M, L.N, L.Kb, L.Ks, L.g, L.n_sal, B)
-    return tot_b / tot_t / 1e9, tot_t, tot_b, oracle.num_threads(), f"first {n} linears of the stack (B={B})"
+        if gpu_y is not None:
+            got = gpu_y(i).astype(np.float64)
+            for b in range(B):
+                rms = float(np.sqrt(np.mean(want[b] ** 2)))
+                worst_l2 = max(worst_l2, float(np.linalg.norm(got[b] - want[b]) / np.linalg.norm(want[b])))
+                worst_rel = max(worst_rel, float((np.abs(got[b] - want[b]) / np.maximum(np.abs(want[b]), 1e-2 * rms)).max()))
+    agreement = None if gpu_y is None else {"linears": n, "max_rel_l2": worst_l2, "max_rel_err": worst_rel,
+                                            "outputs": "fp16 (adds up to 2^-11 of rounding)"}
+    return tot_b / tot_t / 1e9, tot_t, tot_b, oracle.num_threads(), f"first {n} linears of the stack (B={B})", agreement
 
 
 def dense_fp16_gemv_context(lins, nl, B):
@@ -173,7 +189,7 @@ def run_reference(args, rank):
         return
     vals = []
     for i in range(args.warmup + args.steps):
-        gbps, t, b, cores, sample = cpu_oracle_sample(args.config, args.batch, max_linears=args.ref_linears)
+        gbps, t, b, cores, sample, _ = cpu_oracle_sample(args.config, args.batch, max_linears=args.ref_linears)
         if i >= args.warmup:
             vals.append((gbps, t))
     gbps = statistics.mean(v[0] for v in vals)
@@ -506,10 +522,18 @@ def main():
         line["effective_tflops"] = eff_flops / (ms_per_step * 1e-3) / 1e12
         if not args.no_context:
             line["context_dense_fp16_gemv"] = dense_fp16_gemv_context(lins, nl, B)
+        if clocks.get("power_w"):
+            line["joules_per_step"] = clocks["power_w"] * ms_per_step * 1e-3      # board power x time, context only
         if not args.no_cpu_baseline:
-            gbps, tsec, nbytes, cores, sample = cpu_oracle_sample(args.config, B)
+            y_timed = y_dev.cpu().numpy()                  # outputs of the device-resident steps
+            y_offs = np.cumsum([0] + [B * l.M for l in linears])
+
+            def gpu_y(i):
+                return y_timed[y_offs[i]:y_offs[i + 1]].reshape(B, linears[i].M)
+
+            gbps, tsec, nbytes, cores, sample, agreement = cpu_oracle_sample(args.config, B, g=args.g, nl=nl, gpu_y=gpu_y)
             line["cpu_baseline"] = {"value": gbps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
-                                    "seconds": round(tsec, 2)}
+                                    "seconds": round(tsec, 2), "gpu_vs_oracle_on_sample": agreement}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()
