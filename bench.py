@@ -102,7 +102,9 @@ class ClockSampler:
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
                 "samples": len(sm), "reasons": sorted(reasons),
-                "power_w": statistics.median(power) if power else None}
+                # nvidia-smi's power.draw is a moving average over about a second: the largest sample of a
+                # short timed region is still a lower bound of the power under load
+                "power_w": max(power) if power else None}
 
 
 def stack_spec(config: int, layers: int | None):
@@ -523,7 +525,8 @@ def main():
         if not args.no_context:
             line["context_dense_fp16_gemv"] = dense_fp16_gemv_context(lins, nl, B)
         if clocks.get("power_w"):
-            line["joules_per_step"] = clocks["power_w"] * ms_per_step * 1e-3      # board power x time, context only
+            # board power (largest sample; see ClockSampler) x time: context only, a lower bound for short runs
+            line["joules_per_step_lower_bound"] = clocks["power_w"] * ms_per_step * 1e-3
         if not args.no_cpu_baseline:
             y_timed = y_dev.cpu().numpy()                  # outputs of the device-resident steps
             y_offs = np.cumsum([0] + [B * l.M for l in linears])
