@@ -92,12 +92,13 @@ def test_config1_hybrid_with_outliers(fb, B):
     check(run(fb, L, x), oracle.linear_direct(L, x), f"config 1 B={B}")
 
 
-@pytest.mark.parametrize("g", [128, 4096])
-def test_row_scale_formats(fb, g):
-    """g = 128 (one scale per row and group, the paper's format) and g = N (one per row)."""
+@pytest.mark.parametrize("g,B", [(128, 2), (4096, 2), (32, 1), (64, 1), (64, 4), (256, 1), (256, 3)])
+def test_row_scale_formats(fb, g, B):
+    """g = 128 (one scale per row and group, the paper's format), g = N (one per row) and the group sizes of the
+    paper's ablation (32, 64, 256): 4, 8 or 16 sub-vectors per row-scale segment in the global region."""
     L = synth.make_config_linear(1, 0, 0, g=g)
-    x = synth.make_config_activations(1, 0, 0, 2)
-    check(run(fb, L, x), oracle.linear_direct(L, x), f"g={g}")
+    x = synth.make_config_activations(1, 0, 0, B)
+    check(run(fb, L, x), oracle.linear_direct(L, x), f"g={g} B={B}")
 
 
 def test_paper_structured_salient_pattern(fb):
