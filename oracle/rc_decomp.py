@@ -29,10 +29,13 @@ from __future__ import annotations
 import numpy as np
 
 
-def _scale_update(T, other, B, eps):
+def _scale_update(T, other, B, eps, axis=None):
     """Eq. 5 for one scale vector: T [M][n] target, `other` the fixed scale vector broadcast along the summed
-    axis (shape [1][n] for the row update, [M][1] for the column update), B the signs (+-1)."""
-    axis = 1 if other.shape[0] == 1 else 0
+    axis (shape [1][n] for the row update, which sums over j = axis 1; [M][1] for the column update, which sums
+    over i = axis 0), B the signs (+-1).  `axis` must be given when M = 1 or n = 1 makes the shapes ambiguous."""
+    if axis is None:
+        assert other.shape != (1, 1), "say which form of Eq. 5 is meant"
+        axis = 1 if other.shape[0] == 1 else 0
     v = other * B                                    # (alpha_other . B) per element
     num = (v * T).sum(axis=axis)
     den = (v * v).sum(axis=axis) + eps
@@ -80,7 +83,7 @@ def rc_decomp(X, K, T, eps=1e-8, dtype=np.float64, trace=None):
     for k in range(K):
         B[k] = np.where(R >= 0, 1.0, -1.0)
         ac[k] = 1.0
-        ar[k] = _scale_update(R, ac[k][None, :], B[k], eps)
+        ar[k] = _scale_update(R, ac[k][None, :], B[k], eps, axis=1)
         R = R - (ar[k][:, None] * ac[k][None, :]) * B[k]
     if trace is not None:
         trace.append(("init", loss()))
@@ -88,10 +91,10 @@ def rc_decomp(X, K, T, eps=1e-8, dtype=np.float64, trace=None):
     for it in range(T):
         for k in range(K):
             target = X - reconstruct(np.delete(ar, k, 0), np.delete(ac, k, 0), np.delete(B, k, 0)) if K > 1 else X   # R2
-            ar[k] = _scale_update(target, ac[k][None, :], B[k], eps)
+            ar[k] = _scale_update(target, ac[k][None, :], B[k], eps, axis=1)
             if trace is not None:
                 trace.append((f"row{k}", loss()))
-            ac[k] = _scale_update(target, ar[k][:, None], B[k], eps)
+            ac[k] = _scale_update(target, ar[k][:, None], B[k], eps, axis=0)
             if trace is not None:
                 trace.append((f"col{k}", loss()))
         B = sign_search(X, ar, ac, dtype)

@@ -158,3 +158,15 @@ def test_matrix_form_decomposes_column_groups_independently():
     assert ar.shape == (2, 12, 3) and ac.shape == (2, 96) and B.shape == (2, 12, 96)
     a1, c1, b1 = rc.rc_decomp(W[:, 32:64], 2, 3)
     assert np.array_equal(ar[:, :, 1], a1) and np.array_equal(ac[:, 32:64], c1) and np.array_equal(B[:, :, 32:64], b1)
+
+
+def test_single_row_and_single_column_blocks():
+    """Degenerate shapes: with one row every column has a scale of its own, so one column update of Eq. 5 (the sum
+    over i has a single term) reproduces X exactly; with one column the row update does."""
+    x = rng(80).standard_normal((1, 16))
+    ar, ac, B = rc.rc_decomp(x, 1, 1, eps=0.0)
+    assert np.allclose(rc.reconstruct(ar, ac, B), x, rtol=1e-13)
+    assert np.allclose(ac[0], np.abs(x[0]) / np.abs(x[0]).mean(), rtol=1e-13)       # a_r = mean |x|, a_c = |x| / a_r
+    y = rng(81).standard_normal((9, 1))
+    ar, ac, B = rc.rc_decomp(y, 1, 0, eps=0.0)
+    assert np.allclose(rc.reconstruct(ar, ac, B), y, rtol=1e-13)
