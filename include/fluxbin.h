@@ -261,6 +261,34 @@ int32_t fluxbin_plan_pairs_per_row_block(const fluxbin_plan_t *plan);
 /* Release the host object (never touches device memory).  NULL is allowed. */
 void fluxbin_plan_free(fluxbin_plan_t *plan);
 
+/* ---- the step before packing: row-column binary decomposition (Definition 3.1, Eq. 4-6, Algorithm 3) ----
+ *
+ * RC_Decomp of the paper's sub-routine listing on every column group of g columns of a dense matrix, each
+ * group on its own (the block loop of Algorithm 1 without the Hessian error compensation, which needs
+ * calibration data): greedy residual initialisation of the K bases, then T rounds of { for each base: row
+ * scales by Eq. 5, column scales by Eq. 5 } followed by the joint sign update of Eq. 6 (all 2^K sign tuples per
+ * element).  Readings where the paper is silent: the initial signs are sign(R) with sign(0) = +1, the initial
+ * column scales 1 and the initial row scales Eq. 5 for those; with K >= 2 the target of base k's scale update is
+ * W minus the other bases; ties of Eq. 6 go to the lowest tuple index sum_k [b_k = +1] 2^k.  A salient refinement
+ * (mask) is run by handing over the gathered salient columns of the residual as the matrix.
+ *
+ *   d_W            device, fp32 [M][ldw] row-major, ldw >= N; read only
+ *   M, N, g        rows, columns, columns per group: N % g == 0, g in {32, 64, 128, 256}
+ *   K, T, eps      bases 1..4, alternating rounds >= 0, the stability constant of Eq. 5 (>= 0)
+ *   d_bits         device out, uint32 [K][M][N/32]: bit (j % 32) of word j/32 is 1 <=> B_ij = +1
+ *   d_row_scale    device out, fp16 bit patterns [K][M][N/g]   } the canonical layout of a layer description,
+ *   d_col_scale    device out, fp16 bit patterns [K][N]        } rounded to nearest even
+ *   d_row_scale_f32, d_col_scale_f32   optional device out (NULL to skip): the same scales before rounding
+ *   d_workspace    device scratch of fluxbin_rc_decomp_workspace_size() bytes, 16-byte aligned, any contents
+ * All arithmetic is fp32.  Asynchronous on cuda_stream; allocates nothing; caller owns every buffer.
+ * Errors: NULL / SHAPE / RANGE / UNSUPPORTED (other g) / ALIGNMENT / BUFFER_TOO_SMALL before any launch, CUDA.
+ */
+size_t fluxbin_rc_decomp_workspace_size(int32_t M, int32_t N, int32_t g, int32_t K);   /* 0 on invalid arguments */
+fluxbin_status_t fluxbin_rc_decomp(const float *d_W, int64_t ldw, int32_t M, int32_t N, int32_t g, int32_t K, int32_t T,
+                                   float eps, uint32_t *d_bits, uint16_t *d_row_scale, uint16_t *d_col_scale,
+                                   float *d_row_scale_f32, float *d_col_scale_f32, void *d_workspace, size_t ws_bytes,
+                                   void *cuda_stream);
+
 const char *fluxbin_status_string(fluxbin_status_t s);
 
 /* The cudaError_t of the most recent FLUXBIN_ERR_CUDA on the calling thread (0 if none). */

@@ -22,6 +22,9 @@ static fluxbin_status_t cuda_fail(cudaError_t e)
 
 extern "C" int fluxbin_last_cuda_error(void) { return g_last_cuda_error; }
 
+// the same bookkeeping for the library's other translation units
+fluxbin_status_t fb::record_cuda_error(int cuda_error) { return cuda_fail((cudaError_t)cuda_error); }
+
 extern "C" const char *fluxbin_status_string(fluxbin_status_t s)
 {
     switch (s) {

@@ -18,6 +18,8 @@ struct SalSvec {
 fluxbin_status_t validate_dims(const fluxbin_layer_desc_t *d);
 void salient_svecs(const fluxbin_layer_desc_t *d, int sps1, std::vector<SalSvec> &out);
 fluxbin_status_t check_header(const void *p, size_t bytes, FbHeader &h);
+// remember a CUDA error code for fluxbin_last_cuda_error(), clear the runtime's sticky state, return FLUXBIN_ERR_CUDA
+fluxbin_status_t record_cuda_error(int cuda_error);
 
 } // namespace fb
 

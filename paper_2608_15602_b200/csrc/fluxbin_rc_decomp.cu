@@ -1,0 +1,285 @@
+// Row-column binary decomposition on the GPU (the step before packing): RC_Decomp of the paper's sub-routine
+// listing (Algorithm 3) with the closed-form scale updates of Eq. 5 and the exhaustive sign search of Eq. 6,
+// applied to every column group of g columns of a dense fp32 matrix on its own (the block loop of Algorithm 1
+// without the Hessian compensation, which needs calibration data).  Output is the canonical layout
+// fluxbin_pack takes: sign bits, fp16 row scales per (base, row, group), fp16 column scales per (base, column).
+//
+// All arithmetic is fp32.  The path is a sequence of memory-bound passes over W (no tensor cores: there is no
+// contraction in it); one warp owns one (row, group) at a time, lane l the columns l, l+32, ... of the group, so
+// every global access of a warp is one contiguous 128-byte line and a sign word is one ballot.
+//
+//   init        one pass: greedy residual initialisation, all K bases of a (row, group) in registers
+//   per iteration, per base k:
+//     row pass  target = W - (other bases); a_r(k) by Eq. 5; with the new a_r the numerators of the column form
+//               of Eq. 5, reduced over the 64 rows of a CTA in shared memory, then one atomic per column and CTA
+//     col pass  a_c(k) = numerator / (sum_i a_r^2 + eps)   (B^2 = 1), accumulators re-zeroed
+//   sign pass   per element the tuple minimising |W - sum_k M(k) b_k| over all 2^K tuples, lowest index on ties,
+//               evaluated one base at a time with single roundings (M = a_r * a_c rounded once)
+//   final       scales rounded to fp16 (round to nearest even)
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/fluxbin.h"
+#include "fluxbin_internal.h"
+
+namespace rcd {
+
+constexpr int kWarpsPerCta = 8;
+constexpr int kRowsPerWarp = 8;                       // a CTA covers 64 rows of one column group
+constexpr int kRowsPerCta = kWarpsPerCta * kRowsPerWarp;
+constexpr int kMaxK = 4;
+
+struct Args {
+    const float *W;        // [M][ldw]
+    long long ldw;
+    int M, N, g, NG, K;
+    float eps;
+    uint32_t *bits;        // [K][M][N/32]
+    float *ar;             // [K][M][NG]
+    float *ac;             // [K][N]
+    float *colnum;         // [N]
+    float *colden;         // [NG]
+};
+
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// C = g / 32 columns per lane
+template <int C> __global__ void __launch_bounds__(kWarpsPerCta * 32) init_kernel(Args a)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int G = blockIdx.x, row0 = blockIdx.y * kRowsPerCta + warp * kRowsPerWarp;
+    const int nw = a.N / 32;
+    for (int r = 0; r < kRowsPerWarp; ++r) {
+        const int i = row0 + r;
+        if (i >= a.M) break;
+        float R[C];
+#pragma unroll
+        for (int c = 0; c < C; ++c) R[c] = a.W[(long long)i * a.ldw + G * a.g + c * 32 + lane];
+        for (int k = 0; k < a.K; ++k) {
+            float s = 0.f;
+#pragma unroll
+            for (int c = 0; c < C; ++c) s += fabsf(R[c]);
+            s = warp_sum(s) / ((float)a.g + a.eps);                       // Eq. 5 with a_c = 1
+#pragma unroll
+            for (int c = 0; c < C; ++c) {
+                const bool pos = R[c] >= 0.f;                             // sign(0) = +1
+                const unsigned word = __ballot_sync(0xffffffffu, pos);
+                if (lane == 0) a.bits[((size_t)k * a.M + i) * nw + G * C + c] = word;
+                R[c] = pos ? __fsub_rn(R[c], s) : __fadd_rn(R[c], s);
+            }
+            if (lane == 0) a.ar[((size_t)k * a.M + i) * a.NG + G] = s;
+        }
+    }
+}
+
+__global__ void fill_kernel(float *p, float v, long long n)
+{
+    long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    if (i < n) p[i] = v;
+}
+
+// Row form of Eq. 5 for base k, then the column form's numerators with the new row scale.
+template <int C, int K> __global__ void __launch_bounds__(kWarpsPerCta * 32) row_kernel(Args a, int k)
+{
+    __shared__ float part[kWarpsPerCta][C * 32];
+    __shared__ float den_part[kWarpsPerCta];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int G = blockIdx.x, row0 = blockIdx.y * kRowsPerCta + warp * kRowsPerWarp;
+    const int nw = a.N / 32;
+    float ack[K][C];                     // column scales of every base for this lane's columns
+    float akc[C];                        // those of base k
+#pragma unroll
+    for (int q = 0; q < K; ++q)
+#pragma unroll
+        for (int c = 0; c < C; ++c) {
+            ack[q][c] = a.ac[(size_t)q * a.N + G * a.g + c * 32 + lane];
+            if (q == k) akc[c] = ack[q][c];
+        }
+    float den_c = 0.f;
+#pragma unroll
+    for (int c = 0; c < C; ++c) den_c += akc[c] * akc[c];
+    den_c = warp_sum(den_c) + a.eps;                                      // sum_j (a_c B)^2 + eps, B^2 = 1
+    float colsum[C];
+#pragma unroll
+    for (int c = 0; c < C; ++c) colsum[c] = 0.f;
+    float ar2 = 0.f;
+    for (int r = 0; r < kRowsPerWarp; ++r) {
+        const int i = row0 + r;
+        if (i >= a.M) break;
+        float t[C], bk[C];
+#pragma unroll
+        for (int c = 0; c < C; ++c) t[c] = a.W[(long long)i * a.ldw + G * a.g + c * 32 + lane];
+#pragma unroll
+        for (int q = 0; q < K; ++q) {
+            const float arq = a.ar[((size_t)q * a.M + i) * a.NG + G];
+#pragma unroll
+            for (int c = 0; c < C; ++c) {
+                const unsigned word = a.bits[((size_t)q * a.M + i) * nw + G * C + c];
+                const float b = ((word >> lane) & 1u) ? 1.f : -1.f;
+                if (q == k) bk[c] = b;
+                else t[c] -= arq * ack[q][c] * b;                         // what the other bases leave
+            }
+        }
+        float num = 0.f;
+#pragma unroll
+        for (int c = 0; c < C; ++c) num += akc[c] * bk[c] * t[c];
+        const float arn = warp_sum(num) / den_c;
+        if (lane == 0) a.ar[((size_t)k * a.M + i) * a.NG + G] = arn;
+        ar2 += arn * arn;
+#pragma unroll
+        for (int c = 0; c < C; ++c) colsum[c] += arn * bk[c] * t[c];
+    }
+#pragma unroll
+    for (int c = 0; c < C; ++c) part[warp][c * 32 + lane] = colsum[c];
+    if (lane == 0) den_part[warp] = ar2;
+    __syncthreads();
+    for (int j = threadIdx.x; j < C * 32; j += kWarpsPerCta * 32) {
+        float s = 0.f;
+#pragma unroll
+        for (int w = 0; w < kWarpsPerCta; ++w) s += part[w][j];
+        atomicAdd(a.colnum + G * a.g + j, s);
+    }
+    if (threadIdx.x == 0) {
+        float s = 0.f;
+        for (int w = 0; w < kWarpsPerCta; ++w) s += den_part[w];
+        atomicAdd(a.colden + G, s);
+    }
+}
+
+// Column form of Eq. 5: a_c(k)_j = numerator_j / (sum_i a_r_i^2 + eps); the accumulators go back to zero.
+__global__ void col_kernel(Args a, int k)
+{
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= a.N) return;
+    a.ac[(size_t)k * a.N + j] = a.colnum[j] / (a.colden[j / a.g] + a.eps);
+    a.colnum[j] = 0.f;
+}
+__global__ void zero_kernel(float *p, int n)
+{
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j < n) p[j] = 0.f;
+}
+
+// Eq. 6 for every element.
+template <int C, int K> __global__ void __launch_bounds__(kWarpsPerCta * 32) sign_kernel(Args a)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int G = blockIdx.x, row0 = blockIdx.y * kRowsPerCta + warp * kRowsPerWarp;
+    const int nw = a.N / 32;
+    float ack[K][C];
+#pragma unroll
+    for (int q = 0; q < K; ++q)
+#pragma unroll
+        for (int c = 0; c < C; ++c) ack[q][c] = a.ac[(size_t)q * a.N + G * a.g + c * 32 + lane];
+    for (int r = 0; r < kRowsPerWarp; ++r) {
+        const int i = row0 + r;
+        if (i >= a.M) break;
+        float arq[K];
+#pragma unroll
+        for (int q = 0; q < K; ++q) arq[q] = a.ar[((size_t)q * a.M + i) * a.NG + G];
+#pragma unroll
+        for (int c = 0; c < C; ++c) {
+            const float x = a.W[(long long)i * a.ldw + G * a.g + c * 32 + lane];
+            float mag[K];
+#pragma unroll
+            for (int q = 0; q < K; ++q) mag[q] = __fmul_rn(arq[q], ack[q][c]);        // rounded once
+            int best = 0;
+            float best_e = 0.f;
+#pragma unroll
+            for (int t = 0; t < (1 << K); ++t) {
+                float e = x;
+#pragma unroll
+                for (int q = 0; q < K; ++q) e = ((t >> q) & 1) ? __fsub_rn(e, mag[q]) : __fadd_rn(e, mag[q]);
+                e = fabsf(e);
+                if (t == 0 || e < best_e) { best_e = e; best = t; }                   // lowest index wins ties
+            }
+#pragma unroll
+            for (int q = 0; q < K; ++q) {
+                const unsigned word = __ballot_sync(0xffffffffu, (best >> q) & 1);
+                if (lane == 0) a.bits[((size_t)q * a.M + i) * nw + G * C + c] = word;
+            }
+        }
+    }
+}
+
+__global__ void to_half_kernel(const float *src, uint16_t *dst, long long n)
+{
+    long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    if (i < n) dst[i] = __half_as_ushort(__float2half_rn(src[i]));
+}
+
+template <int C, int K> cudaError_t run(const Args &a, int T, cudaStream_t s)
+{
+    const dim3 grid(a.NG, (a.M + kRowsPerCta - 1) / kRowsPerCta), block(kWarpsPerCta * 32);
+    const long long nac = (long long)a.K * a.N;
+    fill_kernel<<<(unsigned)((nac + 255) / 256), 256, 0, s>>>(a.ac, 1.f, nac);
+    zero_kernel<<<(a.N + 255) / 256, 256, 0, s>>>(a.colnum, a.N);
+    zero_kernel<<<(a.NG + 255) / 256, 256, 0, s>>>(a.colden, a.NG);
+    init_kernel<C><<<grid, block, 0, s>>>(a);
+    for (int it = 0; it < T; ++it) {
+        for (int k = 0; k < a.K; ++k) {
+            row_kernel<C, K><<<grid, block, 0, s>>>(a, k);
+            col_kernel<<<(a.N + 255) / 256, 256, 0, s>>>(a, k);
+            zero_kernel<<<(a.NG + 255) / 256, 256, 0, s>>>(a.colden, a.NG);
+        }
+        sign_kernel<C, K><<<grid, block, 0, s>>>(a);
+    }
+    return cudaGetLastError();
+}
+
+} // namespace rcd
+
+static size_t align256(size_t n) { return (n + 255) / 256 * 256; }
+#define FB_CUDA(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return fb::record_cuda_error((int)e_); } while (0)
+
+extern "C" size_t fluxbin_rc_decomp_workspace_size(int32_t M, int32_t N, int32_t g, int32_t K)
+{
+    if (M < 1 || N < 32 || g < 32 || K < 1 || K > rcd::kMaxK || N % g != 0) return 0;
+    const size_t NG = (size_t)N / g;
+    return align256((size_t)K * M * NG * 4) + align256((size_t)K * N * 4) + align256((size_t)N * 4) + align256(NG * 4);
+}
+
+extern "C" fluxbin_status_t fluxbin_rc_decomp(const float *d_W, int64_t ldw, int32_t M, int32_t N, int32_t g, int32_t K,
+                                              int32_t T, float eps, uint32_t *d_bits, uint16_t *d_row_scale,
+                                              uint16_t *d_col_scale, float *d_row_scale_f32, float *d_col_scale_f32,
+                                              void *d_workspace, size_t ws_bytes, void *cuda_stream)
+{
+    if (!d_W || !d_bits || !d_row_scale || !d_col_scale || !d_workspace) return FLUXBIN_ERR_NULL;
+    if (M < 1 || N < 32 || N % 32 != 0 || g < 32 || g % 32 != 0 || N % g != 0 || ldw < N) return FLUXBIN_ERR_SHAPE;
+    if (K < 1 || K > rcd::kMaxK || T < 0 || !(eps >= 0.f)) return FLUXBIN_ERR_RANGE;
+    if (g != 32 && g != 64 && g != 128 && g != 256) return FLUXBIN_ERR_UNSUPPORTED;
+    if (((uintptr_t)d_workspace & 15) != 0) return FLUXBIN_ERR_ALIGNMENT;
+    if (ws_bytes < fluxbin_rc_decomp_workspace_size(M, N, g, K)) return FLUXBIN_ERR_BUFFER_TOO_SMALL;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    rcd::Args a;
+    a.W = d_W; a.ldw = ldw; a.M = M; a.N = N; a.g = g; a.NG = N / g; a.K = K; a.eps = eps;
+    a.bits = d_bits;
+    uint8_t *ws = (uint8_t *)d_workspace;
+    a.ar = (float *)ws;     ws += align256((size_t)K * M * a.NG * 4);
+    a.ac = (float *)ws;     ws += align256((size_t)K * N * 4);
+    a.colnum = (float *)ws; ws += align256((size_t)N * 4);
+    a.colden = (float *)ws;
+    cudaError_t e = cudaErrorInvalidValue;
+#define RCD_K(CC) (K == 1 ? rcd::run<CC, 1>(a, T, s) : K == 2 ? rcd::run<CC, 2>(a, T, s) : K == 3 ? rcd::run<CC, 3>(a, T, s) : rcd::run<CC, 4>(a, T, s))
+    switch (g / 32) {
+    case 1: e = RCD_K(1); break;
+    case 2: e = RCD_K(2); break;
+    case 4: e = RCD_K(4); break;
+    default: e = RCD_K(8); break;
+    }
+#undef RCD_K
+    if (e != cudaSuccess) return fb::record_cuda_error((int)e);
+    const long long nar = (long long)K * M * a.NG, nac = (long long)K * N;
+    rcd::to_half_kernel<<<(unsigned)((nar + 255) / 256), 256, 0, s>>>(a.ar, d_row_scale, nar);
+    rcd::to_half_kernel<<<(unsigned)((nac + 255) / 256), 256, 0, s>>>(a.ac, d_col_scale, nac);
+    if (d_row_scale_f32) FB_CUDA(cudaMemcpyAsync(d_row_scale_f32, a.ar, (size_t)nar * 4, cudaMemcpyDeviceToDevice, s));
+    if (d_col_scale_f32) FB_CUDA(cudaMemcpyAsync(d_col_scale_f32, a.ac, (size_t)nac * 4, cudaMemcpyDeviceToDevice, s));
+    FB_CUDA(cudaGetLastError());
+    return FLUXBIN_OK;
+}

@@ -39,7 +39,8 @@ EXPORTS = ["fluxbin_packed_size", "fluxbin_validate", "fluxbin_pack_host", "flux
            "fluxbin_last_cuda_error", "fluxbin_plan_table_bytes", "fluxbin_plan_workspace_bytes",
            "fluxbin_plan_create", "fluxbin_plan_run", "fluxbin_plan_num_launches", "fluxbin_plan_pairs_per_row_block",
            "fluxbin_plan_free",
-           "fluxbin_linear_noalloc", "fluxbin_noalloc_capacity"]
+           "fluxbin_linear_noalloc", "fluxbin_noalloc_capacity",
+           "fluxbin_rc_decomp", "fluxbin_rc_decomp_workspace_size"]
 
 _LIB = None
 
@@ -87,6 +88,10 @@ def _lib():
         lib.fluxbin_linear_noalloc.restype = ctypes.c_int
         lib.fluxbin_linear_noalloc.argtypes = [vp, vp, i32, i64, vp, i32, i64, vp]
         lib.fluxbin_noalloc_capacity.restype, lib.fluxbin_noalloc_capacity.argtypes = sz, []
+        lib.fluxbin_rc_decomp_workspace_size.restype = sz
+        lib.fluxbin_rc_decomp_workspace_size.argtypes = [i32, i32, i32, i32]
+        lib.fluxbin_rc_decomp.restype = ctypes.c_int
+        lib.fluxbin_rc_decomp.argtypes = [vp, i64, i32, i32, i32, i32, i32, ctypes.c_float, vp, vp, vp, vp, vp, vp, sz, vp]
         _LIB = lib
     return _LIB
 
@@ -239,6 +244,21 @@ def linear_noalloc(w: Weight, d_x: int, B: int, ldx: int, d_y: int, y_is_fp32: b
 
 def noalloc_capacity() -> int:
     return int(_lib().fluxbin_noalloc_capacity())
+
+
+def rc_decomp_workspace_size(M: int, N: int, g: int, K: int) -> int:
+    return int(_lib().fluxbin_rc_decomp_workspace_size(M, N, g, K))
+
+
+def rc_decomp_status(d_W, ldw, M, N, g, K, T, eps, d_bits, d_row_scale, d_col_scale, d_row_f32, d_col_f32, d_ws, ws_bytes,
+                     stream=0) -> int:
+    """fluxbin_rc_decomp (argument marshalling only; every pointer is a device address or None)."""
+    return int(_lib().fluxbin_rc_decomp(d_W, ldw, M, N, g, K, T, eps, d_bits, d_row_scale, d_col_scale, d_row_f32,
+                                        d_col_f32, d_ws, ws_bytes, stream))
+
+
+def rc_decomp(*args, **kw):
+    _check(rc_decomp_status(*args, **kw), "fluxbin_rc_decomp")
 
 
 def debug_tables(w: Weight, d_x: int, pair: int, d_tables: int, stream: int = 0):

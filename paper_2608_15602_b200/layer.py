@@ -90,3 +90,23 @@ class FluxBinPlan:
 
     def pairs_per_row_block(self) -> int:
         return self.plan.pairs_per_row_block()
+
+
+def rc_decompose(W: torch.Tensor, g: int, K: int, T: int, eps: float = 1e-8, stream=None):
+    """fluxbin_rc_decomp on a CUDA fp32 matrix W [M][N] (last dimension contiguous).  Returns a dict of CUDA tensors:
+    bits uint32-as-int32 [K][M][N/32], row_scale / col_scale fp16 [K][M][N/g] / [K][N] (the canonical layout of a
+    layer description) and their fp32 originals row_scale_f32 / col_scale_f32."""
+    assert W.is_cuda and W.dtype == torch.float32 and W.dim() == 2 and W.stride(1) == 1
+    M, N = W.shape
+    dev = W.device
+    out = {"bits": torch.empty((K, M, N // 32), dtype=torch.int32, device=dev),
+           "row_scale": torch.empty((K, M, N // g), dtype=torch.float16, device=dev),
+           "col_scale": torch.empty((K, N), dtype=torch.float16, device=dev),
+           "row_scale_f32": torch.empty((K, M, N // g), dtype=torch.float32, device=dev),
+           "col_scale_f32": torch.empty((K, N), dtype=torch.float32, device=dev)}
+    ws = Workspace(max(fluxbin.rc_decomp_workspace_size(M, N, g, K), 256), device=dev)
+    fluxbin.rc_decomp(W.data_ptr(), W.stride(0), M, N, g, K, T, eps, out["bits"].data_ptr(), out["row_scale"].data_ptr(),
+                      out["col_scale"].data_ptr(), out["row_scale_f32"].data_ptr(), out["col_scale_f32"].data_ptr(),
+                      ws.tensor.data_ptr(), ws.tensor.numel() * ws.tensor.element_size(), _stream_ptr(stream))
+    out["_workspace"] = ws
+    return out

@@ -183,3 +183,18 @@ def make_config_activations(config: int, layer: int, li: int, B: int) -> np.ndar
     _, _, N = lins[li]
     seed = BASE_SEED + config
     return make_activations(seed, layer * 16 + li, B, N, 0.01 if config == 1 else 0.0)
+
+
+def make_dense_weight(seed: int, matrix_id: int, M: int, N: int, outlier_col_frac: float = 0.0) -> np.ndarray:
+    """A dense fp32 weight matrix for the decomposition step: entries N(0, 0.02^2) times a per-row and a per-column
+    gain |N(1, 0.25^2)| (the anisotropy the row-column scales are meant to capture); a fraction of the columns
+    may be multiplied by 8 (outlier columns).  Random numbers only: none of the method's arithmetic."""
+    w = _rng(seed, matrix_id, "dense_w").standard_normal(size=(M, N), dtype=np.float32)
+    w *= np.float32(0.02)
+    w *= np.abs(_rng(seed, matrix_id, "dense_row_gain").normal(1.0, 0.25, size=(M, 1))).astype(np.float32)
+    w *= np.abs(_rng(seed, matrix_id, "dense_col_gain").normal(1.0, 0.25, size=(1, N))).astype(np.float32)
+    n_out = int(round(outlier_col_frac * N))
+    if n_out > 0:
+        cols = _rng(seed, matrix_id, "dense_outlier_cols").choice(N, size=n_out, replace=False)
+        w[:, cols] *= np.float32(8.0)
+    return np.ascontiguousarray(w)

@@ -1,0 +1,141 @@
+"""GPU parity of the row-column binary decomposition (fluxbin_rc_decomp, through the C-ABI) against the numpy
+oracle of Algorithm 3 / Eq. 5-6.
+
+The scales are fp32 on the GPU and fp64 in the oracle: they agree to a relative tolerance.  The signs are an
+integer decision taken in floating point: both sides take it in fp32 in the same order (the oracle's
+dtype=float32 mode), and where they still differ -- the scales feeding the decision differ in their last bits --
+the element must be a near-tie, i.e. the GPU's choice is as good as the oracle's within rounding (several results
+are correct; what is unique, the achieved error, is compared).
+"""
+import numpy as np
+import pytest
+
+from oracle import rc_decomp as rc
+from paper_2608_15602_b200 import synth
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def fb():
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_2608_15602_b200 import build
+    build.build()
+    from paper_2608_15602_b200 import layer
+    return layer
+
+
+def unpack_bits(bits_i32, N):
+    """[K][M][N/32] words -> [K][M][N] of +-1."""
+    w = bits_i32.view(np.uint32)
+    b = (w[..., None] >> np.arange(32, dtype=np.uint32)) & 1
+    return np.where(b.reshape(w.shape[0], w.shape[1], N) == 1, 1.0, -1.0)
+
+
+def gpu_decomp(fb, W, g, K, T, eps):
+    out = fb.rc_decompose(torch.from_numpy(W).cuda(), g, K, T, eps)
+    torch.cuda.synchronize()
+    ar = out["row_scale_f32"].cpu().numpy().astype(np.float64)
+    ac = out["col_scale_f32"].cpu().numpy().astype(np.float64)
+    B = unpack_bits(out["bits"].cpu().numpy(), W.shape[1])
+    return ar, ac, B, out
+
+
+def recon(ar, ac, B, g):
+    return np.einsum("kmn,kn,kmn->mn", np.repeat(ar, g, axis=2), ac, B)
+
+
+@pytest.mark.parametrize("M,N,g,K,T", [(64, 128, 128, 1, 0), (64, 128, 128, 1, 3), (100, 256, 128, 2, 4), (37, 192, 64, 3, 3),
+                                       (130, 96, 32, 4, 2), (65, 512, 256, 2, 5), (1, 128, 128, 2, 2)])
+def test_matches_the_oracle(fb, M, N, g, K, T):
+    W = synth.make_dense_weight(7, M * 7 + N + K, M, N, outlier_col_frac=0.05)
+    eps = 1e-8
+    ar, ac, B, _ = gpu_decomp(fb, W, g, K, T, eps)
+    want_ar, want_ac, want_B = rc.rc_decomp_matrix(W, g, K, T, eps, dtype=np.float32)
+    loss_gpu = ((W - recon(ar, ac, B, g)) ** 2).sum()
+    loss_ref = ((W - recon(want_ar, want_ac, want_B, g)) ** 2).sum()
+    energy = (W.astype(np.float64) ** 2).sum()
+    assert abs(loss_gpu - loss_ref) <= 1e-4 * loss_ref + 1e-9 * energy, (loss_gpu, loss_ref)
+    mism = (B != want_B).any(axis=0)
+    assert mism.mean() <= 2e-3, f"{mism.sum()} of {mism.size} elements chose other signs"
+    # where the signs agree over a whole (row, group) block and column, the scales are the same numbers
+    assert np.allclose(ar, want_ar, rtol=2e-3, atol=1e-6 * np.abs(want_ar).max())
+    assert np.allclose(ac, want_ac, rtol=2e-3, atol=1e-6)
+    # every differing element is a near-tie under the GPU's own scales: its choice is optimal within rounding
+    Mag = np.repeat(ar, g, axis=2) * ac[:, None, :]
+    for i, j in np.argwhere(mism):
+        errs = []
+        for t in range(1 << K):
+            b = np.array([1.0 if (t >> k) & 1 else -1.0 for k in range(K)])
+            errs.append(abs(W[i, j] - (Mag[:, i, j] * b).sum()))
+        mine = abs(W[i, j] - (Mag[:, i, j] * B[:, i, j]).sum())
+        assert mine <= min(errs) + 1e-5 * (abs(W[i, j]) + np.abs(Mag[:, i, j]).sum())
+
+
+def test_gpu_signs_are_optimal_for_the_gpu_scales(fb):
+    """Eq. 6 on the device, element by element: no tuple beats the chosen one (beyond fp32 rounding)."""
+    M, N, g, K = 96, 256, 128, 3
+    W = synth.make_dense_weight(8, 1, M, N)
+    ar, ac, B, _ = gpu_decomp(fb, W, g, K, 3, 1e-8)
+    Mag = np.repeat(ar, g, axis=2) * ac[:, None, :]
+    chosen = np.abs(W - (Mag * B).sum(axis=0))
+    best = np.full(W.shape, np.inf)
+    for t in range(1 << K):
+        b = np.array([1.0 if (t >> k) & 1 else -1.0 for k in range(K)])[:, None, None]
+        best = np.minimum(best, np.abs(W - (Mag * b).sum(axis=0)))
+    assert (chosen <= best + 1e-6 * (np.abs(W) + np.abs(Mag).sum(axis=0))).all()
+
+
+def test_rank_one_matrix_is_recovered(fb):
+    r = np.random.default_rng(5)
+    M, N = 64, 128
+    a, b = np.abs(r.standard_normal(M)) + 0.1, np.abs(r.standard_normal(N)) + 0.1
+    S = np.where(r.random((M, N)) < 0.5, -1.0, 1.0)
+    W = (np.outer(a, b) * S).astype(np.float32)
+    ar, ac, B, _ = gpu_decomp(fb, W, 128, 1, 2, 0.0)
+    assert np.array_equal(B[0], S)
+    assert np.allclose(recon(ar, ac, B, 128), W, rtol=1e-5, atol=1e-6)
+
+
+def test_output_feeds_the_packer_and_the_linear_layer(fb):
+    """Decompose on the GPU, hand the canonical arrays to fluxbin_pack, run the decode linear layer: the result is
+    the product with the reconstructed matrix (computed from the fp16-rounded scales the layer stores)."""
+    M, N, g, K = 256, 512, 128, 2
+    W = synth.make_dense_weight(9, 2, M, N)
+    _, _, B, out = gpu_decomp(fb, W, g, K, 4, 1e-8)
+    rs = out["row_scale"].cpu().numpy().view(np.uint16)
+    cs = out["col_scale"].cpu().numpy().view(np.uint16)
+    L = synth.Linear(M, N, K, 0, g, 0, out["bits"].cpu().numpy().view(np.uint32), rs, cs, np.zeros(0, np.int32),
+                     np.zeros((0, M, 0), np.uint32), np.zeros((0, M, N // g), np.uint16), np.zeros((0, 0), np.uint16))
+    x = synth.make_activations(9, 3, 2, N)
+    lin = fb.FluxBinLinear(L)
+    y = lin.forward(torch.from_numpy(x.view(np.float16)).cuda(), lin.workspace(2), fp32_out=True)
+    torch.cuda.synchronize()
+    What = recon(rs.view(np.float16).astype(np.float64), cs.view(np.float16).astype(np.float64), B, g)
+    want = x.view(np.float16).astype(np.float64) @ What.T
+    got = y.cpu().numpy().astype(np.float64)
+    assert np.linalg.norm(got - want) / np.linalg.norm(want) <= 1e-3
+    # and the decomposition is a useful approximation of W: two bases leave well under a fifth of its energy
+    assert ((W - What) ** 2).sum() / (W.astype(np.float64) ** 2).sum() < 0.2
+
+
+def test_argument_errors(fb):
+    from paper_2608_15602_b200 import fluxbin
+    W = torch.zeros((32, 128), dtype=torch.float32, device="cuda")
+    bits = torch.zeros((1, 32, 4), dtype=torch.int32, device="cuda")
+    rs = torch.zeros((1, 32, 1), dtype=torch.float16, device="cuda")
+    cs = torch.zeros((1, 128), dtype=torch.float16, device="cuda")
+    ws = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+    args = [W.data_ptr(), 128, 32, 128, 128, 1, 1, 1e-8, bits.data_ptr(), rs.data_ptr(), cs.data_ptr(), None, None,
+            ws.data_ptr(), ws.numel()]
+    assert fluxbin.rc_decomp_status(*args) == 0
+    bad = list(args); bad[0] = None
+    assert fluxbin.rc_decomp_status(*bad) == 1                   # NULL
+    bad = list(args); bad[4] = 96
+    assert fluxbin.rc_decomp_status(*bad) == 2                   # N % g != 0: shape
+    bad = list(args); bad[5] = 5
+    assert fluxbin.rc_decomp_status(*bad) == 3                   # K out of range
+    bad = list(args); bad[14] = 16
+    assert fluxbin.rc_decomp_status(*bad) == 5                   # workspace too small
+    assert fluxbin.rc_decomp_workspace_size(32, 128, 96, 1) == 0
