@@ -139,3 +139,23 @@ def test_argument_errors(fb):
     bad = list(args); bad[14] = 16
     assert fluxbin.rc_decomp_status(*bad) == 5                   # workspace too small
     assert fluxbin.rc_decomp_workspace_size(32, 128, 96, 1) == 0
+
+
+def test_full_size_matrix_on_sampled_groups(fb):
+    """A 4096 x 4096 matrix (the size the timing is quoted on), g = 128, K = 2, T = 4: three column groups checked
+    against the oracle in full; every group's error ratio must lie in the band two bases reach on this input."""
+    M = N = 4096
+    g, K, T = 128, 2, 4
+    W = synth.make_dense_weight(10, 1, M, N, outlier_col_frac=0.05)
+    ar, ac, B, _ = gpu_decomp(fb, W, g, K, T, 1e-8)
+    for G in (0, 13, 31):
+        cols = slice(G * g, (G + 1) * g)
+        want_ar, want_ac, want_B = rc.rc_decomp(W[:, cols], K, T, 1e-8, dtype=np.float32)
+        mism = (B[:, :, cols] != want_B).any(axis=0)
+        assert mism.mean() <= 2e-3
+        assert np.allclose(ar[:, :, G], want_ar, rtol=2e-3, atol=1e-6 * np.abs(want_ar).max())
+        assert np.allclose(ac[:, cols], want_ac, rtol=2e-3, atol=1e-6)
+    err = ((W - recon(ar, ac, B, g)) ** 2).reshape(M, N // g, g).sum(axis=(0, 2))
+    energy = (W.astype(np.float64) ** 2).reshape(M, N // g, g).sum(axis=(0, 2))
+    ratio = err / energy
+    assert (ratio > 0.03).all() and (ratio < 0.15).all(), (ratio.min(), ratio.max())
