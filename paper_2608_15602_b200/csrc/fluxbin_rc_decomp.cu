@@ -39,7 +39,7 @@ struct Args {
     float *ar;             // [K][M][NG]
     float *ac;             // [K][N]
     float *colnum;         // [N]
-    float *colden;         // [NG]
+    float *colden;         // [2][NG], double buffered
 };
 
 __device__ __forceinline__ float warp_sum(float v)
@@ -55,9 +55,9 @@ template <int C> __global__ void __launch_bounds__(kWarpsPerCta * 32) init_kerne
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int G = blockIdx.x, row0 = blockIdx.y * kRowsPerCta + warp * kRowsPerWarp;
     const int nw = a.N / 32;
-    for (int r = 0; r < kRowsPerWarp; ++r) {
+    const int nrows = min(kRowsPerWarp, a.M - row0);
+    for (int r = 0; r < nrows; ++r) {
         const int i = row0 + r;
-        if (i >= a.M) break;
         float R[C];
 #pragma unroll
         for (int c = 0; c < C; ++c) R[c] = a.W[(long long)i * a.ldw + G * a.g + c * 32 + lane];
@@ -85,7 +85,7 @@ __global__ void fill_kernel(float *p, float v, long long n)
 }
 
 // Row form of Eq. 5 for base k, then the column form's numerators with the new row scale.
-template <int C, int K> __global__ void __launch_bounds__(kWarpsPerCta * 32) row_kernel(Args a, int k)
+template <int C, int K> __global__ void __launch_bounds__(kWarpsPerCta * 32) row_kernel(Args a, int k, int parity)
 {
     __shared__ float part[kWarpsPerCta][C * 32];
     __shared__ float den_part[kWarpsPerCta];
@@ -109,9 +109,9 @@ template <int C, int K> __global__ void __launch_bounds__(kWarpsPerCta * 32) row
 #pragma unroll
     for (int c = 0; c < C; ++c) colsum[c] = 0.f;
     float ar2 = 0.f;
-    for (int r = 0; r < kRowsPerWarp; ++r) {
+    const int nrows = min(kRowsPerWarp, a.M - row0);
+    for (int r = 0; r < nrows; ++r) {
         const int i = row0 + r;
-        if (i >= a.M) break;
         float t[C], bk[C];
 #pragma unroll
         for (int c = 0; c < C; ++c) t[c] = a.W[(long long)i * a.ldw + G * a.g + c * 32 + lane];
@@ -148,17 +148,20 @@ template <int C, int K> __global__ void __launch_bounds__(kWarpsPerCta * 32) row
     if (threadIdx.x == 0) {
         float s = 0.f;
         for (int w = 0; w < kWarpsPerCta; ++w) s += den_part[w];
-        atomicAdd(a.colden + G, s);
+        atomicAdd(a.colden + (size_t)(parity & 1) * a.NG + G, s);
     }
 }
 
 // Column form of Eq. 5: a_c(k)_j = numerator_j / (sum_i a_r_i^2 + eps); the accumulators go back to zero.
-__global__ void col_kernel(Args a, int k)
+// (the group denominators are double buffered: this pass reads buffer `parity` and clears the other one, which the
+// next row pass accumulates into -- no thread reads what another clears)
+__global__ void col_kernel(Args a, int k, int parity)
 {
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= a.N) return;
-    a.ac[(size_t)k * a.N + j] = a.colnum[j] / (a.colden[j / a.g] + a.eps);
+    a.ac[(size_t)k * a.N + j] = a.colnum[j] / (a.colden[(size_t)(parity & 1) * a.NG + j / a.g] + a.eps);
     a.colnum[j] = 0.f;
+    if (j < a.NG) a.colden[(size_t)((parity + 1) & 1) * a.NG + j] = 0.f;
 }
 __global__ void zero_kernel(float *p, int n)
 {
@@ -177,9 +180,9 @@ template <int C, int K> __global__ void __launch_bounds__(kWarpsPerCta * 32) sig
     for (int q = 0; q < K; ++q)
 #pragma unroll
         for (int c = 0; c < C; ++c) ack[q][c] = a.ac[(size_t)q * a.N + G * a.g + c * 32 + lane];
-    for (int r = 0; r < kRowsPerWarp; ++r) {
+    const int nrows = min(kRowsPerWarp, a.M - row0);
+    for (int r = 0; r < nrows; ++r) {
         const int i = row0 + r;
-        if (i >= a.M) break;
         float arq[K];
 #pragma unroll
         for (int q = 0; q < K; ++q) arq[q] = a.ar[((size_t)q * a.M + i) * a.NG + G];
@@ -220,13 +223,14 @@ template <int C, int K> cudaError_t run(const Args &a, int T, cudaStream_t s)
     const long long nac = (long long)a.K * a.N;
     fill_kernel<<<(unsigned)((nac + 255) / 256), 256, 0, s>>>(a.ac, 1.f, nac);
     zero_kernel<<<(a.N + 255) / 256, 256, 0, s>>>(a.colnum, a.N);
-    zero_kernel<<<(a.NG + 255) / 256, 256, 0, s>>>(a.colden, a.NG);
+    zero_kernel<<<(2 * a.NG + 255) / 256, 256, 0, s>>>(a.colden, 2 * a.NG);
     init_kernel<C><<<grid, block, 0, s>>>(a);
+    int parity = 0;
     for (int it = 0; it < T; ++it) {
         for (int k = 0; k < a.K; ++k) {
-            row_kernel<C, K><<<grid, block, 0, s>>>(a, k);
-            col_kernel<<<(a.N + 255) / 256, 256, 0, s>>>(a, k);
-            zero_kernel<<<(a.NG + 255) / 256, 256, 0, s>>>(a.colden, a.NG);
+            row_kernel<C, K><<<grid, block, 0, s>>>(a, k, parity);
+            col_kernel<<<(a.N + 255) / 256, 256, 0, s>>>(a, k, parity);
+            parity ^= 1;
         }
         sign_kernel<C, K><<<grid, block, 0, s>>>(a);
     }
@@ -242,7 +246,7 @@ extern "C" size_t fluxbin_rc_decomp_workspace_size(int32_t M, int32_t N, int32_t
 {
     if (M < 1 || N < 32 || g < 32 || K < 1 || K > rcd::kMaxK || N % g != 0) return 0;
     const size_t NG = (size_t)N / g;
-    return align256((size_t)K * M * NG * 4) + align256((size_t)K * N * 4) + align256((size_t)N * 4) + align256(NG * 4);
+    return align256((size_t)K * M * NG * 4) + align256((size_t)K * N * 4) + align256((size_t)N * 4) + align256(2 * NG * 4);
 }
 
 extern "C" fluxbin_status_t fluxbin_rc_decomp(const float *d_W, int64_t ldw, int32_t M, int32_t N, int32_t g, int32_t K,
