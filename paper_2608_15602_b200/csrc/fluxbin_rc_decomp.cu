@@ -49,6 +49,44 @@ __device__ __forceinline__ float warp_sum(float v)
     return v;
 }
 
+// Everything a warp needs from global memory for its kRowsPerWarp rows of one group, requested up front so that
+// all of it is in flight at once (the passes are bound by load latency, not by arithmetic): the W values in
+// registers, the sign words and row scales one or a few per lane, handed out by shuffles.
+template <int C, int K> struct WarpRows {
+    static constexpr int kWords = kRowsPerWarp * K * C;          // sign words [row][base][c]
+    static constexpr int kWordRegs = (kWords + 31) / 32;
+    float w[kRowsPerWarp][C];
+    uint32_t bw[kWordRegs];
+    float arv;                                                   // row scale of (row, base) = lane, lane < 8 * K
+
+    __device__ __forceinline__ void load_w(const Args &a, int G, int row0, int nrows, int lane)
+    {
+#pragma unroll
+        for (int r = 0; r < kRowsPerWarp; ++r)
+#pragma unroll
+            for (int c = 0; c < C; ++c)
+                w[r][c] = r < nrows ? __ldg(a.W + (long long)(row0 + r) * a.ldw + G * a.g + c * 32 + lane) : 0.f;
+    }
+    __device__ __forceinline__ void load_signs_and_scales(const Args &a, int G, int row0, int nrows, int lane)
+    {
+        const int nw = a.N / 32;
+#pragma unroll
+        for (int m = 0; m < kWordRegs; ++m) {
+            const int f = lane + 32 * m, c = f % C, q = (f / C) % K, r = f / (C * K);
+            bw[m] = (f < kWords && r < nrows) ? a.bits[((size_t)q * a.M + row0 + r) * nw + G * C + c] : 0u;
+        }
+        const int q = lane % K, r = lane / K;
+        arv = (lane < kRowsPerWarp * K && r < nrows) ? a.ar[((size_t)q * a.M + row0 + r) * a.NG + G] : 0.f;
+    }
+    // r, q, c are compile-time after unrolling
+    __device__ __forceinline__ uint32_t word(int r, int q, int c) const
+    {
+        const int f = (r * K + q) * C + c;
+        return __shfl_sync(0xffffffffu, bw[f >> 5], f & 31);
+    }
+    __device__ __forceinline__ float ar(int r, int q) const { return __shfl_sync(0xffffffffu, arv, r * K + q); }
+};
+
 // C = g / 32 columns per lane
 template <int C> __global__ void __launch_bounds__(kWarpsPerCta * 32) init_kernel(Args a)
 {
@@ -56,11 +94,14 @@ template <int C> __global__ void __launch_bounds__(kWarpsPerCta * 32) init_kerne
     const int G = blockIdx.x, row0 = blockIdx.y * kRowsPerCta + warp * kRowsPerWarp;
     const int nw = a.N / 32;
     const int nrows = min(kRowsPerWarp, a.M - row0);
-    for (int r = 0; r < nrows; ++r) {
+    WarpRows<C, 1> in;                                                    // (only the W part is used here)
+    in.load_w(a, G, row0, nrows, lane);
+#pragma unroll
+    for (int r = 0; r < kRowsPerWarp; ++r) {
         const int i = row0 + r;
         float R[C];
 #pragma unroll
-        for (int c = 0; c < C; ++c) R[c] = a.W[(long long)i * a.ldw + G * a.g + c * 32 + lane];
+        for (int c = 0; c < C; ++c) R[c] = in.w[r][c];
         for (int k = 0; k < a.K; ++k) {
             float s = 0.f;
 #pragma unroll
@@ -70,10 +111,10 @@ template <int C> __global__ void __launch_bounds__(kWarpsPerCta * 32) init_kerne
             for (int c = 0; c < C; ++c) {
                 const bool pos = R[c] >= 0.f;                             // sign(0) = +1
                 const unsigned word = __ballot_sync(0xffffffffu, pos);
-                if (lane == 0) a.bits[((size_t)k * a.M + i) * nw + G * C + c] = word;
+                if (lane == 0 && r < nrows) a.bits[((size_t)k * a.M + i) * nw + G * C + c] = word;
                 R[c] = pos ? __fsub_rn(R[c], s) : __fadd_rn(R[c], s);
             }
-            if (lane == 0) a.ar[((size_t)k * a.M + i) * a.NG + G] = s;
+            if (lane == 0 && r < nrows) a.ar[((size_t)k * a.M + i) * a.NG + G] = s;
         }
     }
 }
@@ -91,7 +132,6 @@ template <int C, int K> __global__ void __launch_bounds__(kWarpsPerCta * 32) row
     __shared__ float den_part[kWarpsPerCta];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int G = blockIdx.x, row0 = blockIdx.y * kRowsPerCta + warp * kRowsPerWarp;
-    const int nw = a.N / 32;
     float ack[K][C];                     // column scales of every base for this lane's columns
     float akc[C];                        // those of base k
 #pragma unroll
@@ -110,18 +150,20 @@ template <int C, int K> __global__ void __launch_bounds__(kWarpsPerCta * 32) row
     for (int c = 0; c < C; ++c) colsum[c] = 0.f;
     float ar2 = 0.f;
     const int nrows = min(kRowsPerWarp, a.M - row0);
-    for (int r = 0; r < nrows; ++r) {
-        const int i = row0 + r;
+    WarpRows<C, K> in;
+    in.load_w(a, G, row0, nrows, lane);
+    in.load_signs_and_scales(a, G, row0, nrows, lane);
+#pragma unroll
+    for (int r = 0; r < kRowsPerWarp; ++r) {
         float t[C], bk[C];
 #pragma unroll
-        for (int c = 0; c < C; ++c) t[c] = a.W[(long long)i * a.ldw + G * a.g + c * 32 + lane];
+        for (int c = 0; c < C; ++c) t[c] = in.w[r][c];
 #pragma unroll
         for (int q = 0; q < K; ++q) {
-            const float arq = a.ar[((size_t)q * a.M + i) * a.NG + G];
+            const float arq = in.ar(r, q);
 #pragma unroll
             for (int c = 0; c < C; ++c) {
-                const unsigned word = a.bits[((size_t)q * a.M + i) * nw + G * C + c];
-                const float b = ((word >> lane) & 1u) ? 1.f : -1.f;
+                const float b = ((in.word(r, q, c) >> lane) & 1u) ? 1.f : -1.f;
                 if (q == k) bk[c] = b;
                 else t[c] -= arq * ack[q][c] * b;                         // what the other bases leave
             }
@@ -129,8 +171,8 @@ template <int C, int K> __global__ void __launch_bounds__(kWarpsPerCta * 32) row
         float num = 0.f;
 #pragma unroll
         for (int c = 0; c < C; ++c) num += akc[c] * bk[c] * t[c];
-        const float arn = warp_sum(num) / den_c;
-        if (lane == 0) a.ar[((size_t)k * a.M + i) * a.NG + G] = arn;
+        const float arn = r < nrows ? warp_sum(num) / den_c : 0.f;        // (r < nrows is warp-uniform)
+        if (lane == 0 && r < nrows) a.ar[((size_t)k * a.M + row0 + r) * a.NG + G] = arn;
         ar2 += arn * arn;
 #pragma unroll
         for (int c = 0; c < C; ++c) colsum[c] += arn * bk[c] * t[c];
@@ -181,14 +223,20 @@ template <int C, int K> __global__ void __launch_bounds__(kWarpsPerCta * 32) sig
 #pragma unroll
         for (int c = 0; c < C; ++c) ack[q][c] = a.ac[(size_t)q * a.N + G * a.g + c * 32 + lane];
     const int nrows = min(kRowsPerWarp, a.M - row0);
-    for (int r = 0; r < nrows; ++r) {
-        const int i = row0 + r;
+    WarpRows<C, K> in;
+    in.load_w(a, G, row0, nrows, lane);
+    {
+        const int q = lane % K, r = lane / K;
+        in.arv = (lane < kRowsPerWarp * K && r < nrows) ? a.ar[((size_t)q * a.M + row0 + r) * a.NG + G] : 0.f;
+    }
+#pragma unroll
+    for (int r = 0; r < kRowsPerWarp; ++r) {
         float arq[K];
 #pragma unroll
-        for (int q = 0; q < K; ++q) arq[q] = a.ar[((size_t)q * a.M + i) * a.NG + G];
+        for (int q = 0; q < K; ++q) arq[q] = in.ar(r, q);
 #pragma unroll
         for (int c = 0; c < C; ++c) {
-            const float x = a.W[(long long)i * a.ldw + G * a.g + c * 32 + lane];
+            const float x = in.w[r][c];
             float mag[K];
 #pragma unroll
             for (int q = 0; q < K; ++q) mag[q] = __fmul_rn(arq[q], ack[q][c]);        // rounded once
@@ -205,7 +253,7 @@ template <int C, int K> __global__ void __launch_bounds__(kWarpsPerCta * 32) sig
 #pragma unroll
             for (int q = 0; q < K; ++q) {
                 const unsigned word = __ballot_sync(0xffffffffu, (best >> q) & 1);
-                if (lane == 0) a.bits[((size_t)q * a.M + i) * nw + G * C + c] = word;
+                if (lane == 0 && r < nrows) a.bits[((size_t)q * a.M + row0 + r) * nw + G * C + c] = word;
             }
         }
     }
