@@ -569,10 +569,11 @@ __device__ __forceinline__ void process_rows2(const uint8_t *items_a, const uint
 
 // First L2 prefetches of a run of row blocks (issued before the tables are built): the first
 // kPrefetchTrips blocks of D*kWarps items, one D-item request per lane.
-__device__ __forceinline__ void prefetch_run_head(const uint8_t *pair_items, int item_bytes, int D, int kWarps, int rb_lo, int rb_hi)
+__device__ __forceinline__ void prefetch_run_head(const uint8_t *pair_items, int item_bytes, int D, int kWarps, int rb_lo, int rb_hi,
+                                                  int trips = kPrefetchTrips)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (lane < kPrefetchTrips) {
+    if (lane < trips) {
         int rb = rb_lo + lane * D * kWarps + D * warp;
         int cnt = min(D, rb_hi - rb);
         if (cnt > 0) prefetch_l2(pair_items + (int64_t)rb * item_bytes, (uint32_t)(cnt * item_bytes));
@@ -818,8 +819,11 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
             const uint8_t *items = E.packed + E.off_items[region] + (size_t)pair * E.nrb * ib;
             const uint8_t *items_b = items + (size_t)E.nrb * ib;
             const int pf_d = np == 2 ? 1 : (region ? SPS1 : SPS0) == 1 ? 1 : DepthFor<BT>::value;
-            prefetch_run_head(items, ib, pf_d, kWarps, rb_lo, rb_hi);         // weights start moving now
-            if (np == 2) prefetch_run_head(items_b, ib, pf_d, kWarps, rb_lo, rb_hi);
+            // weights start moving now.  The two-pair loop prefetches the trip two ahead, so its head covers
+            // trips 0 and 1 (+2 %); longer heads were measured slower in every launch mode.
+            const int head_trips = np == 2 ? kPrefetchTrips + 1 : kPrefetchTrips;
+            prefetch_run_head(items, ib, pf_d, kWarps, rb_lo, rb_hi, head_trips);
+            if (np == 2) prefetch_run_head(items_b, ib, pf_d, kWarps, rb_lo, rb_hi, head_trips);
 
             if (!predecessor_done) {
                 asm volatile("griddepcontrol.wait;" ::: "memory");
