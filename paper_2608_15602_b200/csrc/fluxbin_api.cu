@@ -235,6 +235,14 @@ extern "C" fluxbin_status_t fluxbin_workspace_init(void *d_workspace, size_t byt
 
 // ---- the layer ------------------------------------------------------------------------------------
 
+// The two-pairs-per-row-block kernel pays two table builds per run of rows but has the better row loop (one
+// reduction per two items, loads requested half an item earlier).  Measured on B200 (batch 1): it wins as soon
+// as a CTA's share is worth about 30 plain items (cost 60) -- +11 % with one launch per 70B linear, +15 % with
+// one per dependency group, +21 % with one per layer -- and loses below that (4096 x 4096 alone, 18 items per
+// CTA: 6.7 -> 7.7 us per call).
+#ifndef FB_NP2_MIN
+#define FB_NP2_MIN 60
+#endif
 // How a launch is cut: grid size, the statically dealt part of the cost line, the number of shares, and
 // whether the two-pairs-per-row-block kernel runs.
 struct LaunchShape {
@@ -268,9 +276,9 @@ static cudaError_t launch_shape(long long total_cost, int num_sms, long long ite
         out->nshares = (int)grid;
     }
     out->grid = grid;
-    // two pairs per row block (half the reduction traffic) when every layer allows it (couple_cost > 0:
-    // even pair counts everywhere) and a CTA's share spans several whole couples
-    out->couples = BT == 1 && couple_cost > 0 && out->static_cost / grid >= 2 * couple_cost;
+    // two pairs per row block when every layer allows it (couple_cost > 0: even pair counts everywhere) and a
+    // CTA's share is large enough to pay for the second table build
+    out->couples = BT == 1 && couple_cost > 0 && out->static_cost / grid >= FB_NP2_MIN;
     return cudaSuccess;
 }
 

@@ -768,10 +768,10 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
         // With NP == 2 region 0 is walked two pairs at a time, their table sets side by side (BT == 1,
         // every entry with an even number of global pairs): a "work pair" is then a couple of pairs, a
         // work row block their two items.  Costs per pair are unchanged, only the cut granularity doubles.
-        // (NP is a kernel template parameter: the host picks the two-pair kernel for launches whose
-        // shares span whole couples -- long runs of rows per table build, as in a plan of many layers;
-        // in a small launch it would make every CTA build twice as much.  Deciding it at run time was
-        // measured slower than either variant: both row loops in one kernel cost registers.)
+        // (NP is a kernel template parameter: the host picks the two-pair kernel unless a CTA's share is
+        // only a handful of items, where building two table sets per run costs more than the better row
+        // loop gains.  Deciding it at run time was measured slower than either variant: both row loops in
+        // one kernel cost registers.)
         const int wp0 = E.npairs[0] / NP;
         const int I0 = wp0 * E.nrb, I1 = E.npairs[1] * E.nrb;
         if (tid == 0) {
