@@ -325,8 +325,9 @@ template <int BT> static cudaError_t launch_bt(int s0, int s1, int num_sms, cons
 
 // Work-split cost model, measured on B200 in units of half a 1152-byte item (about 50 ns per CTA):
 // an item with one row scale per sub-vector (3072 bytes) takes about 2x a plain item; building one
-// table set (two dependent loads, 8K table entries, two barriers) takes about as long as 18 items.
-constexpr int kBuildCost = 36;
+// table set (two dependent loads, 8K table entries, two barriers) takes about as long as 22 items
+// (re-measured against the current row loop: 28 / 36 / 44 / 56 -> 5.61 / 5.80 / 5.85 / 5.83 TB/s on the stack plan).
+constexpr int kBuildCost = 44;
 // The reduction epilogue a CTA runs when it leaves an entry (fence, tickets, read-back of the tiles it
 // completed): a fixed part plus a part that grows with the rows to convert.
 static long long epilogue_cost(const FbHeader &h) { return 80 + h.Mpad / 128; }
