@@ -272,7 +272,7 @@ void fluxbin_plan_free(fluxbin_plan_t *plan);
  * W minus the other bases; ties of Eq. 6 go to the lowest tuple index sum_k [b_k = +1] 2^k.  A salient refinement
  * (mask) is run by handing over the gathered salient columns of the residual as the matrix.
  *
- *   d_W            device, fp32 [M][ldw] row-major, ldw >= N; read only
+ *   d_W            device, fp32 [M][ldw] row-major, ldw >= N, 16-byte aligned with ldw % 4 == 0; read only
  *   M, N, g        rows, columns, columns per group: N % g == 0, g in {32, 64, 128, 256}
  *   K, T, eps      bases 1..4, alternating rounds >= 0, the stability constant of Eq. 5 (>= 0)
  *   d_bits         device out, uint32 [K][M][N/32]: bit (j % 32) of word j/32 is 1 <=> B_ij = +1

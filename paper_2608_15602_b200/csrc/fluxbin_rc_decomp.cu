@@ -5,8 +5,8 @@
 // fluxbin_pack takes: sign bits, fp16 row scales per (base, row, group), fp16 column scales per (base, column).
 //
 // All arithmetic is fp32.  The path is a sequence of memory-bound passes over W (no tensor cores: there is no
-// contraction in it); one warp owns one (row, group) at a time, lane l the columns l, l+32, ... of the group, so
-// every global access of a warp is one contiguous 128-byte line and a sign word is one ballot.
+// contraction in it); one warp owns one (row, group) at a time, lane l the g/32 adjacent columns l*g/32 ... of
+// the group, so a row of a group is one 128-bit load per lane and a lane's signs are adjacent bits of one word.
 //
 //   init        one pass: greedy residual initialisation, all K bases of a (row, group) in registers
 //   per iteration, per base k:
@@ -49,11 +49,35 @@ __device__ __forceinline__ float warp_sum(float v)
     return v;
 }
 
+// Column mapping: lane l owns the C = g / 32 ADJACENT columns l*C .. l*C + C-1 of the group, so its W values are one
+// 128-bit load per row (C = 4), its signs are C adjacent bits of ONE sign word (word (l*C)/32 of the group, bit
+// offset (l*C) % 32) and a sign word is assembled from 32/C neighbouring lanes with an OR over xor-shuffles.
+template <int C> __device__ __forceinline__ void load_cols(float (&dst)[C], const float *p)
+{
+    if constexpr (C == 1) dst[0] = __ldg(p);
+    else if constexpr (C == 2) { const float2 v = __ldg((const float2 *)p); dst[0] = v.x; dst[1] = v.y; }
+    else {
+#pragma unroll
+        for (int c = 0; c < C; c += 4) {
+            const float4 v = __ldg((const float4 *)(p + c));
+            dst[c] = v.x; dst[c + 1] = v.y; dst[c + 2] = v.z; dst[c + 3] = v.w;
+        }
+    }
+}
+
+// OR of `v` over the aligned group of 32/C lanes that share a sign word; every lane of the group gets the word.
+template <int C> __device__ __forceinline__ uint32_t gather_word(uint32_t v)
+{
+#pragma unroll
+    for (int o = 1; o < 32 / C; o <<= 1) v |= __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
 // Everything a warp needs from global memory for its kRowsPerWarp rows of one group, requested up front so that
 // all of it is in flight at once (the passes are bound by load latency, not by arithmetic): the W values in
 // registers, the sign words and row scales one or a few per lane, handed out by shuffles.
 template <int C, int K> struct WarpRows {
-    static constexpr int kWords = kRowsPerWarp * K * C;          // sign words [row][base][c]
+    static constexpr int kWords = kRowsPerWarp * K * C;          // sign words [row][base][word of the group]
     static constexpr int kWordRegs = (kWords + 31) / 32;
     float w[kRowsPerWarp][C];
     uint32_t bw[kWordRegs];
@@ -62,12 +86,20 @@ template <int C, int K> struct WarpRows {
     __device__ __forceinline__ void load_w(const Args &a, int G, int row0, int nrows, int lane)
     {
 #pragma unroll
-        for (int r = 0; r < kRowsPerWarp; ++r)
+        for (int r = 0; r < kRowsPerWarp; ++r) {
+            if (r < nrows) load_cols<C>(w[r], a.W + (long long)(row0 + r) * a.ldw + G * a.g + lane * C);
+            else {
 #pragma unroll
-            for (int c = 0; c < C; ++c)
-                w[r][c] = r < nrows ? __ldg(a.W + (long long)(row0 + r) * a.ldw + G * a.g + c * 32 + lane) : 0.f;
+                for (int c = 0; c < C; ++c) w[r][c] = 0.f;
+            }
+        }
     }
-    __device__ __forceinline__ void load_signs_and_scales(const Args &a, int G, int row0, int nrows, int lane)
+    __device__ __forceinline__ void load_row_scales(const Args &a, int G, int row0, int nrows, int lane)
+    {
+        const int q = lane % K, r = lane / K;
+        arv = (lane < kRowsPerWarp * K && r < nrows) ? a.ar[((size_t)q * a.M + row0 + r) * a.NG + G] : 0.f;
+    }
+    __device__ __forceinline__ void load_signs(const Args &a, int G, int row0, int nrows, int lane)
     {
         const int nw = a.N / 32;
 #pragma unroll
@@ -75,19 +107,21 @@ template <int C, int K> struct WarpRows {
             const int f = lane + 32 * m, c = f % C, q = (f / C) % K, r = f / (C * K);
             bw[m] = (f < kWords && r < nrows) ? a.bits[((size_t)q * a.M + row0 + r) * nw + G * C + c] : 0u;
         }
-        const int q = lane % K, r = lane / K;
-        arv = (lane < kRowsPerWarp * K && r < nrows) ? a.ar[((size_t)q * a.M + row0 + r) * a.NG + G] : 0.f;
     }
-    // r, q, c are compile-time after unrolling
-    __device__ __forceinline__ uint32_t word(int r, int q, int c) const
+    // the C sign bits of this lane's columns for (row r, base q), in the low bits; r, q compile-time after unrolling
+    __device__ __forceinline__ uint32_t signs(int r, int q, int lane) const
     {
-        const int f = (r * K + q) * C + c;
-        return __shfl_sync(0xffffffffu, bw[f >> 5], f & 31);
+        const int f0 = (r * K + q) * C;                          // the group's C words never straddle a register
+        const uint32_t word = __shfl_sync(0xffffffffu, bw[f0 >> 5], (f0 & 31) + (lane * C) / 32);
+        return word >> ((lane * C) & 31);
     }
     __device__ __forceinline__ float ar(int r, int q) const { return __shfl_sync(0xffffffffu, arv, r * K + q); }
 };
 
-// C = g / 32 columns per lane
+// the word index (within the group) this lane's columns live in, and whether this lane stores the gathered word
+template <int C> __device__ __forceinline__ int word_of_lane(int lane) { return (lane * C) / 32; }
+template <int C> __device__ __forceinline__ bool stores_word(int lane) { return (lane % (32 / C)) == 0; }
+
 template <int C> __global__ void __launch_bounds__(kWarpsPerCta * 32) init_kernel(Args a)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -107,13 +141,15 @@ template <int C> __global__ void __launch_bounds__(kWarpsPerCta * 32) init_kerne
 #pragma unroll
             for (int c = 0; c < C; ++c) s += fabsf(R[c]);
             s = warp_sum(s) / ((float)a.g + a.eps);                       // Eq. 5 with a_c = 1
+            uint32_t mine = 0u;
 #pragma unroll
             for (int c = 0; c < C; ++c) {
                 const bool pos = R[c] >= 0.f;                             // sign(0) = +1
-                const unsigned word = __ballot_sync(0xffffffffu, pos);
-                if (lane == 0 && r < nrows) a.bits[((size_t)k * a.M + i) * nw + G * C + c] = word;
+                mine |= (pos ? 1u : 0u) << c;
                 R[c] = pos ? __fsub_rn(R[c], s) : __fadd_rn(R[c], s);
             }
+            const uint32_t word = gather_word<C>(mine << ((lane * C) & 31));
+            if (stores_word<C>(lane) && r < nrows) a.bits[((size_t)k * a.M + i) * nw + G * C + word_of_lane<C>(lane)] = word;
             if (lane == 0 && r < nrows) a.ar[((size_t)k * a.M + i) * a.NG + G] = s;
         }
     }
@@ -132,15 +168,21 @@ template <int C, int K> __global__ void __launch_bounds__(kWarpsPerCta * 32) row
     __shared__ float den_part[kWarpsPerCta];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int G = blockIdx.x, row0 = blockIdx.y * kRowsPerCta + warp * kRowsPerWarp;
+    const int nrows = min(kRowsPerWarp, a.M - row0);
+    WarpRows<C, K> in;
+    in.load_w(a, G, row0, nrows, lane);
+    in.load_signs(a, G, row0, nrows, lane);
+    in.load_row_scales(a, G, row0, nrows, lane);
     float ack[K][C];                     // column scales of every base for this lane's columns
     float akc[C];                        // those of base k
 #pragma unroll
-    for (int q = 0; q < K; ++q)
+    for (int q = 0; q < K; ++q) {
+        load_cols<C>(ack[q], a.ac + (size_t)q * a.N + G * a.g + lane * C);
+        if (q == k) {
 #pragma unroll
-        for (int c = 0; c < C; ++c) {
-            ack[q][c] = a.ac[(size_t)q * a.N + G * a.g + c * 32 + lane];
-            if (q == k) akc[c] = ack[q][c];
+            for (int c = 0; c < C; ++c) akc[c] = ack[q][c];
         }
+    }
     float den_c = 0.f;
 #pragma unroll
     for (int c = 0; c < C; ++c) den_c += akc[c] * akc[c];
@@ -149,36 +191,37 @@ template <int C, int K> __global__ void __launch_bounds__(kWarpsPerCta * 32) row
 #pragma unroll
     for (int c = 0; c < C; ++c) colsum[c] = 0.f;
     float ar2 = 0.f;
-    const int nrows = min(kRowsPerWarp, a.M - row0);
-    WarpRows<C, K> in;
-    in.load_w(a, G, row0, nrows, lane);
-    in.load_signs_and_scales(a, G, row0, nrows, lane);
+    const float inv_den = 1.f / den_c;
 #pragma unroll
     for (int r = 0; r < kRowsPerWarp; ++r) {
-        float t[C], bk[C];
+        // signs enter as a choice between +v and -v (one select, then a fused multiply-add): the passes are
+        // bound by issue slots as much as by memory, so the per-element instruction count matters
+        float t[C];
+        uint32_t sk = 0u;
 #pragma unroll
         for (int c = 0; c < C; ++c) t[c] = in.w[r][c];
 #pragma unroll
         for (int q = 0; q < K; ++q) {
             const float arq = in.ar(r, q);
+            const uint32_t sg = in.signs(r, q, lane);
+            if (q == k) sk = sg;
+            else {
 #pragma unroll
-            for (int c = 0; c < C; ++c) {
-                const float b = ((in.word(r, q, c) >> lane) & 1u) ? 1.f : -1.f;
-                if (q == k) bk[c] = b;
-                else t[c] -= arq * ack[q][c] * b;                         // what the other bases leave
+                for (int c = 0; c < C; ++c)
+                    t[c] = fmaf(((sg >> c) & 1u) ? -arq : arq, ack[q][c], t[c]);          // what the other bases leave
             }
         }
         float num = 0.f;
 #pragma unroll
-        for (int c = 0; c < C; ++c) num += akc[c] * bk[c] * t[c];
-        const float arn = r < nrows ? warp_sum(num) / den_c : 0.f;        // (r < nrows is warp-uniform)
+        for (int c = 0; c < C; ++c) num = fmaf(((sk >> c) & 1u) ? akc[c] : -akc[c], t[c], num);
+        const float arn = r < nrows ? warp_sum(num) * inv_den : 0.f;       // (r < nrows is warp-uniform)
         if (lane == 0 && r < nrows) a.ar[((size_t)k * a.M + row0 + r) * a.NG + G] = arn;
-        ar2 += arn * arn;
+        ar2 = fmaf(arn, arn, ar2);
 #pragma unroll
-        for (int c = 0; c < C; ++c) colsum[c] += arn * bk[c] * t[c];
+        for (int c = 0; c < C; ++c) colsum[c] = fmaf(((sk >> c) & 1u) ? arn : -arn, t[c], colsum[c]);
     }
 #pragma unroll
-    for (int c = 0; c < C; ++c) part[warp][c * 32 + lane] = colsum[c];
+    for (int c = 0; c < C; ++c) part[warp][lane * C + c] = colsum[c];
     if (lane == 0) den_part[warp] = ar2;
     __syncthreads();
     for (int j = threadIdx.x; j < C * 32; j += kWarpsPerCta * 32) {
@@ -217,23 +260,21 @@ template <int C, int K> __global__ void __launch_bounds__(kWarpsPerCta * 32) sig
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int G = blockIdx.x, row0 = blockIdx.y * kRowsPerCta + warp * kRowsPerWarp;
     const int nw = a.N / 32;
-    float ack[K][C];
-#pragma unroll
-    for (int q = 0; q < K; ++q)
-#pragma unroll
-        for (int c = 0; c < C; ++c) ack[q][c] = a.ac[(size_t)q * a.N + G * a.g + c * 32 + lane];
     const int nrows = min(kRowsPerWarp, a.M - row0);
     WarpRows<C, K> in;
     in.load_w(a, G, row0, nrows, lane);
-    {
-        const int q = lane % K, r = lane / K;
-        in.arv = (lane < kRowsPerWarp * K && r < nrows) ? a.ar[((size_t)q * a.M + row0 + r) * a.NG + G] : 0.f;
-    }
+    in.load_row_scales(a, G, row0, nrows, lane);
+    float ack[K][C];
+#pragma unroll
+    for (int q = 0; q < K; ++q) load_cols<C>(ack[q], a.ac + (size_t)q * a.N + G * a.g + lane * C);
 #pragma unroll
     for (int r = 0; r < kRowsPerWarp; ++r) {
         float arq[K];
 #pragma unroll
         for (int q = 0; q < K; ++q) arq[q] = in.ar(r, q);
+        uint32_t mine[K];
+#pragma unroll
+        for (int q = 0; q < K; ++q) mine[q] = 0u;
 #pragma unroll
         for (int c = 0; c < C; ++c) {
             const float x = in.w[r][c];
@@ -251,10 +292,13 @@ template <int C, int K> __global__ void __launch_bounds__(kWarpsPerCta * 32) sig
                 if (t == 0 || e < best_e) { best_e = e; best = t; }                   // lowest index wins ties
             }
 #pragma unroll
-            for (int q = 0; q < K; ++q) {
-                const unsigned word = __ballot_sync(0xffffffffu, (best >> q) & 1);
-                if (lane == 0 && r < nrows) a.bits[((size_t)q * a.M + row0 + r) * nw + G * C + c] = word;
-            }
+            for (int q = 0; q < K; ++q) mine[q] |= (uint32_t)((best >> q) & 1) << c;
+        }
+#pragma unroll
+        for (int q = 0; q < K; ++q) {
+            const uint32_t word = gather_word<C>(mine[q] << ((lane * C) & 31));
+            if (stores_word<C>(lane) && r < nrows)
+                a.bits[((size_t)q * a.M + row0 + r) * nw + G * C + word_of_lane<C>(lane)] = word;
         }
     }
 }
@@ -306,7 +350,7 @@ extern "C" fluxbin_status_t fluxbin_rc_decomp(const float *d_W, int64_t ldw, int
     if (M < 1 || N < 32 || N % 32 != 0 || g < 32 || g % 32 != 0 || N % g != 0 || ldw < N) return FLUXBIN_ERR_SHAPE;
     if (K < 1 || K > rcd::kMaxK || T < 0 || !(eps >= 0.f)) return FLUXBIN_ERR_RANGE;
     if (g != 32 && g != 64 && g != 128 && g != 256) return FLUXBIN_ERR_UNSUPPORTED;
-    if (((uintptr_t)d_workspace & 15) != 0) return FLUXBIN_ERR_ALIGNMENT;
+    if (((uintptr_t)d_workspace & 15) != 0 || ((uintptr_t)d_W & 15) != 0 || (ldw & 3) != 0) return FLUXBIN_ERR_ALIGNMENT;
     if (ws_bytes < fluxbin_rc_decomp_workspace_size(M, N, g, K)) return FLUXBIN_ERR_BUFFER_TOO_SMALL;
     cudaStream_t s = (cudaStream_t)cuda_stream;
     rcd::Args a;
