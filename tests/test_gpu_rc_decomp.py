@@ -138,6 +138,8 @@ def test_argument_errors(fb):
     assert fluxbin.rc_decomp_status(*bad) == 3                   # K out of range
     bad = list(args); bad[14] = 16
     assert fluxbin.rc_decomp_status(*bad) == 5                   # workspace too small
+    bad = list(args); bad[0] = W.data_ptr() + 4
+    assert fluxbin.rc_decomp_status(*bad) == 6                   # W not 16-byte aligned
     assert fluxbin.rc_decomp_workspace_size(32, 128, 96, 1) == 0
 
 
