@@ -845,6 +845,10 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
             FB_TRACE_ADD(9, t_fetch);
             build_tables<BT>(bin, abuf);
             if (np == 2) build_tables<BT>(bin_b, abuf, 128u);
+            // the column tables of the next run's pairs (1 KB each, read once per run: otherwise an HBM miss on the
+            // serial path of the next build) start moving into L2 now (+0.5 to 0.8 % in every launch mode)
+            if (tid < 8 * np && pair + np < E.npairs[region])
+                prefetch_line_if(E.packed + E.off_coldesc + (size_t)((region ? E.npairs[0] : 0) + pair + np) * FB_PAIR_DESC_BYTES + tid * 128, true);
             FB_TRACE_ADD(4, t_build);
             FB_TRACE_T0(t_rows);
             if (region == 0) {
