@@ -110,3 +110,20 @@ def rc_decompose(W: torch.Tensor, g: int, K: int, T: int, eps: float = 1e-8, str
                       ws.tensor.data_ptr(), ws.tensor.numel() * ws.tensor.element_size(), _stream_ptr(stream))
     out["_workspace"] = ws
     return out
+
+
+def quantize_dense(W: torch.Tensor, g: int = 128, K: int = 2, T: int = 10, eps: float = 1e-8) -> "FluxBinLinear":
+    """Dense fp32 CUDA matrix -> packed FluxBin layer with K global bases and no salient refinement: the GPU
+    decomposition (fluxbin_rc_decomp), then the packer.  The canonical arrays pass through host memory because
+    fluxbin_pack takes host pointers."""
+    from . import synth
+    M, N = W.shape
+    out = rc_decompose(W.contiguous(), g, K, T, eps)
+    torch.cuda.synchronize(W.device)
+    L = synth.Linear(M, N, K, 0, g, 0,
+                     np.ascontiguousarray(out["bits"].cpu().numpy().view(np.uint32)),
+                     np.ascontiguousarray(out["row_scale"].cpu().numpy().view(np.uint16)),
+                     np.ascontiguousarray(out["col_scale"].cpu().numpy().view(np.uint16)),
+                     np.zeros(0, np.int32), np.zeros((0, M, 0), np.uint32), np.zeros((0, M, N // g), np.uint16),
+                     np.zeros((0, 0), np.uint16))
+    return FluxBinLinear(L, device=W.device)

@@ -161,3 +161,16 @@ def test_full_size_matrix_on_sampled_groups(fb):
     energy = (W.astype(np.float64) ** 2).reshape(M, N // g, g).sum(axis=(0, 2))
     ratio = err / energy
     assert (ratio > 0.03).all() and (ratio < 0.15).all(), (ratio.min(), ratio.max())
+
+
+def test_quantize_dense_helper(fb):
+    """dense W -> decomposition -> packed layer in one call; the layer multiplies like W up to the quantisation error."""
+    M, N = 512, 1024
+    W = synth.make_dense_weight(12, 1, M, N)
+    lin = fb.quantize_dense(torch.from_numpy(W).cuda(), g=128, K=4, T=6)
+    x = synth.make_activations(12, 2, 1, N)
+    y = lin.forward(torch.from_numpy(x.view(np.float16)).cuda(), lin.workspace(1), fp32_out=True)
+    torch.cuda.synchronize()
+    want = x.view(np.float16).astype(np.float64) @ W.astype(np.float64).T
+    got = y.cpu().numpy().astype(np.float64)
+    assert np.linalg.norm(got - want) / np.linalg.norm(want) < 0.12        # four bases leave < 1 % of W's energy
