@@ -116,3 +116,39 @@ def rc_decomp_matrix(W, g, K, T, eps=1e-8, dtype=np.float64):
         a, c, b = rc_decomp(W[:, G * g:(G + 1) * g], K, T, eps, dtype)
         ar[:, :, G], ac[:, G * g:(G + 1) * g], B[:, :, G * g:(G + 1) * g] = a, c, b
     return ar, ac, B
+
+
+def hybrid_decomp(W, g, Kb, Ks, sal_idx, T, eps=1e-8, dtype=np.float64):
+    """The salient-aware variant (Algorithm 2 without the saliency search and the Hessian compensation, which need
+    calibration data): per column group, step 2 decomposes the whole block with Kb bases, step 3 decomposes the
+    residual restricted to the group's salient columns (given, ascending `sal_idx`) with Ks further bases.  The
+    mask is applied by handing RC_Decomp only the masked-in columns.
+    Returns the global part as rc_decomp_matrix does, plus the salient part in the layer's canonical form:
+    sal_row [Ks][M][N/g] (0 for groups without salient columns), sal_col [Ks][n_sal], sal_B [Ks][M][n_sal]."""
+    W = np.asarray(W, np.float64)
+    M, N = W.shape
+    sal_idx = np.asarray(sal_idx, np.int64)
+    ar, ac, B = rc_decomp_matrix(W, g, Kb, T, eps, dtype)
+    What_g = np.einsum("kmn,kn,kmn->mn", np.repeat(ar, g, axis=2), ac, B)
+    R = W - What_g
+    n_sal = len(sal_idx)
+    sal_row = np.zeros((Ks, M, N // g))
+    sal_col = np.zeros((Ks, n_sal))
+    sal_B = np.ones((Ks, M, n_sal))
+    for G in range(N // g):
+        v = np.nonzero(sal_idx // g == G)[0]                      # virtual columns of this group
+        if len(v) == 0:
+            continue
+        a, c, b = rc_decomp(R[:, sal_idx[v]], Ks, T, eps, dtype)
+        sal_row[:, :, G], sal_col[:, v], sal_B[:, :, v] = a, c, b
+    return ar, ac, B, sal_row, sal_col, sal_B
+
+
+def hybrid_reconstruct(ar, ac, B, sal_row, sal_col, sal_B, sal_idx, g):
+    """The matrix a hybrid decomposition stands for: the global bases plus the salient bases scattered back to
+    their columns (Eq. 9)."""
+    What = np.einsum("kmn,kn,kmn->mn", np.repeat(ar, g, axis=2), ac, B)
+    sal_idx = np.asarray(sal_idx, np.int64)
+    if len(sal_idx):
+        What[:, sal_idx] += np.einsum("kmv,kv,kmv->mv", sal_row[:, :, sal_idx // g], sal_col, sal_B)
+    return What

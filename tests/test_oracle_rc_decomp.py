@@ -170,3 +170,30 @@ def test_single_row_and_single_column_blocks():
     y = rng(81).standard_normal((9, 1))
     ar, ac, B = rc.rc_decomp(y, 1, 0, eps=0.0)
     assert np.allclose(rc.reconstruct(ar, ac, B), y, rtol=1e-13)
+
+
+def test_hybrid_refinement_only_touches_salient_columns_and_never_hurts():
+    """Algorithm 2, steps 2-3: the extra bases approximate the residual on the salient columns, so the other
+    columns keep the global reconstruction and the error on every salient column block does not grow."""
+    r = rng(90)
+    M, N, g = 24, 128, 32
+    W = r.standard_normal((M, N)) * 0.02
+    W[:, [3, 40, 41, 99]] *= 8.0
+    sal_idx = np.array([3, 40, 41, 99, 100])
+    # (a one-column salient block is fitted exactly by its first base; the second base then has a zero residual
+    # and zero scales, and Eq. 5 becomes 0 / (0 + eps): this is what the stability constant is for)
+    ar, ac, B, sr, sc, sB = rc.hybrid_decomp(W, g, 2, 2, sal_idx, 4, eps=1e-12)
+    base = np.einsum("kmn,kn,kmn->mn", np.repeat(ar, g, axis=2), ac, B)
+    full = rc.hybrid_reconstruct(ar, ac, B, sr, sc, sB, sal_idx, g)
+    other = np.setdiff1d(np.arange(N), sal_idx)
+    assert np.array_equal(full[:, other], base[:, other])
+    for G in range(N // g):
+        v = sal_idx[sal_idx // g == G]
+        if len(v):
+            assert ((W[:, v] - full[:, v]) ** 2).sum() <= ((W[:, v] - base[:, v]) ** 2).sum() * (1 + 1e-9)
+    assert np.all(sr[:, :, 2] == 0)                      # group 2 (columns 64..95) has no salient column
+    # with every column salient the refinement is a second RC_Decomp of the whole residual block
+    ar2, ac2, B2, sr2, sc2, sB2 = rc.hybrid_decomp(W[:, :32], 32, 1, 1, np.arange(32), 3, eps=0.0)
+    R = W[:, :32] - np.einsum("kmn,kn,kmn->mn", np.repeat(ar2, 32, axis=2), ac2, B2)
+    a, c, b = rc.rc_decomp(R, 1, 3, eps=0.0)
+    assert np.array_equal(sB2, b) and np.allclose(sr2[:, :, 0], a, rtol=1e-14) and np.allclose(sc2, c, rtol=1e-14)
