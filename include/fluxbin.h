@@ -273,6 +273,9 @@ void fluxbin_plan_free(fluxbin_plan_t *plan);
  * (mask) is run by handing over the gathered salient columns of the residual as the matrix.
  *
  *   d_W            device, fp32 [M][ldw] row-major, ldw >= N, 16-byte aligned with ldw % 4 == 0; read only
+ *   d_col_live     device, fp32 [N], 16-byte aligned, or NULL: 1 for a real column, 0 for a padding column (a block
+ *                  narrower than g -- the salient columns of a group -- is handed over padded with columns whose
+ *                  W entries are 0; their column scales stay 0 and they do not enter Eq. 5).  NULL: all real.
  *   M, N, g        rows, columns, columns per group: N % g == 0, g in {32, 64, 128, 256}
  *   K, T, eps      bases 1..4, alternating rounds >= 0, the stability constant of Eq. 5 (>= 0)
  *   d_bits         device out, uint32 [K][M][N/32]: bit (j % 32) of word j/32 is 1 <=> B_ij = +1
@@ -284,8 +287,8 @@ void fluxbin_plan_free(fluxbin_plan_t *plan);
  * Errors: NULL / SHAPE / RANGE / UNSUPPORTED (other g) / ALIGNMENT / BUFFER_TOO_SMALL before any launch, CUDA.
  */
 size_t fluxbin_rc_decomp_workspace_size(int32_t M, int32_t N, int32_t g, int32_t K);   /* 0 on invalid arguments */
-fluxbin_status_t fluxbin_rc_decomp(const float *d_W, int64_t ldw, int32_t M, int32_t N, int32_t g, int32_t K, int32_t T,
-                                   float eps, uint32_t *d_bits, uint16_t *d_row_scale, uint16_t *d_col_scale,
+fluxbin_status_t fluxbin_rc_decomp(const float *d_W, int64_t ldw, const float *d_col_live, int32_t M, int32_t N, int32_t g,
+                                   int32_t K, int32_t T, float eps, uint32_t *d_bits, uint16_t *d_row_scale, uint16_t *d_col_scale,
                                    float *d_row_scale_f32, float *d_col_scale_f32, void *d_workspace, size_t ws_bytes,
                                    void *cuda_stream);
 
@@ -293,6 +296,20 @@ const char *fluxbin_status_string(fluxbin_status_t s);
 
 /* The cudaError_t of the most recent FLUXBIN_ERR_CUDA on the calling thread (0 if none). */
 int fluxbin_last_cuda_error(void);
+
+/*
+ * The matrix the salient refinement decomposes (Algorithm 2, step 3): R = W - W_g restricted to the salient
+ * columns, W_g the reconstruction from the global decomposition's outputs (fp32 scales and sign bits as
+ * fluxbin_rc_decomp wrote them).  Virtual column v (input column d_sal_idx[v]) is written to column d_pos[v] of
+ * the padded matrix d_P [M][ldp] (fp32, zero elsewhere: the call clears it first) and d_live [ncols_p] gets 1 at
+ * d_pos[v], 0 elsewhere -- the pair of arguments fluxbin_rc_decomp takes for blocks narrower than its group.
+ * All pointers device; M <= 65535; asynchronous on cuda_stream.  Errors: NULL / SHAPE / RANGE / CUDA.
+ */
+fluxbin_status_t fluxbin_rc_salient_residual(const float *d_W, int64_t ldw, int32_t M, int32_t N, int32_t g, int32_t Kb,
+                                             const uint32_t *d_bits, const float *d_row_scale_f32,
+                                             const float *d_col_scale_f32, const int32_t *d_sal_idx, const int32_t *d_pos,
+                                             int32_t n_sal, float *d_P, int64_t ldp, int32_t ncols_p, float *d_live,
+                                             void *cuda_stream);
 
 #ifdef __cplusplus
 }

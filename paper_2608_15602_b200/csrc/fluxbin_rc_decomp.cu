@@ -38,6 +38,7 @@ struct Args {
     uint32_t *bits;        // [K][M][N/32]
     float *ar;             // [K][M][NG]
     float *ac;             // [K][N]
+    const float *live;     // [N] 1 = real column, 0 = padding column (W must be 0 there); nullptr: all real
     float *colnum;         // [N]
     float *colden;         // [2][NG], double buffered
 };
@@ -130,6 +131,16 @@ template <int C> __global__ void __launch_bounds__(kWarpsPerCta * 32) init_kerne
     const int nrows = min(kRowsPerWarp, a.M - row0);
     WarpRows<C, 1> in;                                                    // (only the W part is used here)
     in.load_w(a, G, row0, nrows, lane);
+    // initial column scales: 1 on real columns, 0 on padding columns (which then stay 0 through every update:
+    // their numerators are sums of zeros); Eq. 5 with those scales divides by the number of real columns
+    float lv[C];
+#pragma unroll
+    for (int c = 0; c < C; ++c) lv[c] = 1.f;
+    if (a.live) load_cols<C>(lv, a.live + G * a.g + lane * C);
+    float nlive = 0.f;
+#pragma unroll
+    for (int c = 0; c < C; ++c) nlive += lv[c];
+    const float inv_n = 1.f / (warp_sum(nlive) + a.eps);
 #pragma unroll
     for (int r = 0; r < kRowsPerWarp; ++r) {
         const int i = row0 + r;
@@ -139,14 +150,15 @@ template <int C> __global__ void __launch_bounds__(kWarpsPerCta * 32) init_kerne
         for (int k = 0; k < a.K; ++k) {
             float s = 0.f;
 #pragma unroll
-            for (int c = 0; c < C; ++c) s += fabsf(R[c]);
-            s = warp_sum(s) / ((float)a.g + a.eps);                       // Eq. 5 with a_c = 1
+            for (int c = 0; c < C; ++c) s += fabsf(R[c]) * lv[c];
+            s = warp_sum(s) * inv_n;                                      // Eq. 5 with a_c = 1 on the real columns
             uint32_t mine = 0u;
 #pragma unroll
             for (int c = 0; c < C; ++c) {
                 const bool pos = R[c] >= 0.f;                             // sign(0) = +1
                 mine |= (pos ? 1u : 0u) << c;
-                R[c] = pos ? __fsub_rn(R[c], s) : __fadd_rn(R[c], s);
+                const float step = s * lv[c];
+                R[c] = pos ? __fsub_rn(R[c], step) : __fadd_rn(R[c], step);
             }
             const uint32_t word = gather_word<C>(mine << ((lane * C) & 31));
             if (stores_word<C>(lane) && r < nrows) a.bits[((size_t)k * a.M + i) * nw + G * C + word_of_lane<C>(lane)] = word;
@@ -159,6 +171,13 @@ __global__ void fill_kernel(float *p, float v, long long n)
 {
     long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;
     if (i < n) p[i] = v;
+}
+
+// dst[i] = src[i % n]: the live mask as the initial column scales of every base
+__global__ void tile_kernel(float *dst, const float *src, int n, long long total)
+{
+    long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    if (i < total) dst[i] = src[i % n];
 }
 
 // Row form of Eq. 5 for base k, then the column form's numerators with the new row scale.
@@ -313,7 +332,8 @@ template <int C, int K> cudaError_t run(const Args &a, int T, cudaStream_t s)
 {
     const dim3 grid(a.NG, (a.M + kRowsPerCta - 1) / kRowsPerCta), block(kWarpsPerCta * 32);
     const long long nac = (long long)a.K * a.N;
-    fill_kernel<<<(unsigned)((nac + 255) / 256), 256, 0, s>>>(a.ac, 1.f, nac);
+    if (a.live) tile_kernel<<<(unsigned)((nac + 255) / 256), 256, 0, s>>>(a.ac, a.live, a.N, nac);
+    else fill_kernel<<<(unsigned)((nac + 255) / 256), 256, 0, s>>>(a.ac, 1.f, nac);
     zero_kernel<<<(a.N + 255) / 256, 256, 0, s>>>(a.colnum, a.N);
     zero_kernel<<<(2 * a.NG + 255) / 256, 256, 0, s>>>(a.colden, 2 * a.NG);
     init_kernel<C><<<grid, block, 0, s>>>(a);
@@ -341,7 +361,8 @@ extern "C" size_t fluxbin_rc_decomp_workspace_size(int32_t M, int32_t N, int32_t
     return align256((size_t)K * M * NG * 4) + align256((size_t)K * N * 4) + align256((size_t)N * 4) + align256(2 * NG * 4);
 }
 
-extern "C" fluxbin_status_t fluxbin_rc_decomp(const float *d_W, int64_t ldw, int32_t M, int32_t N, int32_t g, int32_t K,
+extern "C" fluxbin_status_t fluxbin_rc_decomp(const float *d_W, int64_t ldw, const float *d_col_live, int32_t M, int32_t N,
+                                              int32_t g, int32_t K,
                                               int32_t T, float eps, uint32_t *d_bits, uint16_t *d_row_scale,
                                               uint16_t *d_col_scale, float *d_row_scale_f32, float *d_col_scale_f32,
                                               void *d_workspace, size_t ws_bytes, void *cuda_stream)
@@ -350,11 +371,12 @@ extern "C" fluxbin_status_t fluxbin_rc_decomp(const float *d_W, int64_t ldw, int
     if (M < 1 || N < 32 || N % 32 != 0 || g < 32 || g % 32 != 0 || N % g != 0 || ldw < N) return FLUXBIN_ERR_SHAPE;
     if (K < 1 || K > rcd::kMaxK || T < 0 || !(eps >= 0.f)) return FLUXBIN_ERR_RANGE;
     if (g != 32 && g != 64 && g != 128 && g != 256) return FLUXBIN_ERR_UNSUPPORTED;
-    if (((uintptr_t)d_workspace & 15) != 0 || ((uintptr_t)d_W & 15) != 0 || (ldw & 3) != 0) return FLUXBIN_ERR_ALIGNMENT;
+    if (((uintptr_t)d_workspace & 15) != 0 || ((uintptr_t)d_W & 15) != 0 || (ldw & 3) != 0 || ((uintptr_t)d_col_live & 15) != 0)
+        return FLUXBIN_ERR_ALIGNMENT;
     if (ws_bytes < fluxbin_rc_decomp_workspace_size(M, N, g, K)) return FLUXBIN_ERR_BUFFER_TOO_SMALL;
     cudaStream_t s = (cudaStream_t)cuda_stream;
     rcd::Args a;
-    a.W = d_W; a.ldw = ldw; a.M = M; a.N = N; a.g = g; a.NG = N / g; a.K = K; a.eps = eps;
+    a.W = d_W; a.live = d_col_live; a.ldw = ldw; a.M = M; a.N = N; a.g = g; a.NG = N / g; a.K = K; a.eps = eps;
     a.bits = d_bits;
     uint8_t *ws = (uint8_t *)d_workspace;
     a.ar = (float *)ws;     ws += align256((size_t)K * M * a.NG * 4);
@@ -376,6 +398,47 @@ extern "C" fluxbin_status_t fluxbin_rc_decomp(const float *d_W, int64_t ldw, int
     rcd::to_half_kernel<<<(unsigned)((nac + 255) / 256), 256, 0, s>>>(a.ac, d_col_scale, nac);
     if (d_row_scale_f32) FB_CUDA(cudaMemcpyAsync(d_row_scale_f32, a.ar, (size_t)nar * 4, cudaMemcpyDeviceToDevice, s));
     if (d_col_scale_f32) FB_CUDA(cudaMemcpyAsync(d_col_scale_f32, a.ac, (size_t)nac * 4, cudaMemcpyDeviceToDevice, s));
+    FB_CUDA(cudaGetLastError());
+    return FLUXBIN_OK;
+}
+
+
+// ---- the residual the salient refinement decomposes (Algorithm 2, step 3: R = W - W_g on the salient columns) ----
+namespace rcd {
+__global__ void salient_residual_kernel(const float *W, long long ldw, int M, int N, int g, int Kb, const uint32_t *bits,
+                                        const float *ar, const float *ac, const int *sal_idx, const int *pos, int n_sal,
+                                        float *P, long long ldp, float *live)
+{
+    const int v = blockIdx.x * blockDim.x + threadIdx.x, i = blockIdx.y;
+    if (v >= n_sal) return;
+    const int j = sal_idx[v], NG = N / g, nw = N / 32;
+    float r = W[(long long)i * ldw + j];
+    for (int k = 0; k < Kb; ++k) {
+        const float m = __fmul_rn(ar[((size_t)k * M + i) * NG + j / g], ac[(size_t)k * N + j]);
+        const bool plus = (bits[((size_t)k * M + i) * nw + j / 32] >> (j & 31)) & 1u;
+        r = plus ? __fsub_rn(r, m) : __fadd_rn(r, m);
+    }
+    P[(long long)i * ldp + pos[v]] = r;
+    if (i == 0) live[pos[v]] = 1.f;
+}
+} // namespace rcd
+
+extern "C" fluxbin_status_t fluxbin_rc_salient_residual(const float *d_W, int64_t ldw, int32_t M, int32_t N, int32_t g, int32_t Kb,
+                                                        const uint32_t *d_bits, const float *d_row_scale_f32,
+                                                        const float *d_col_scale_f32, const int32_t *d_sal_idx,
+                                                        const int32_t *d_pos, int32_t n_sal, float *d_P, int64_t ldp,
+                                                        int32_t ncols_p, float *d_live, void *cuda_stream)
+{
+    if (!d_W || !d_bits || !d_row_scale_f32 || !d_col_scale_f32 || !d_sal_idx || !d_pos || !d_P || !d_live) return FLUXBIN_ERR_NULL;
+    if (M < 1 || N < 32 || N % 32 != 0 || g < 32 || N % g != 0 || ldw < N || n_sal < 1 || ncols_p < 1 || ldp < ncols_p)
+        return FLUXBIN_ERR_SHAPE;
+    if (Kb < 1 || Kb > rcd::kMaxK || M > 65535) return FLUXBIN_ERR_RANGE;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    FB_CUDA(cudaMemset2DAsync(d_P, (size_t)ldp * 4, 0, (size_t)ncols_p * 4, M, s));
+    FB_CUDA(cudaMemsetAsync(d_live, 0, (size_t)ncols_p * 4, s));
+    const dim3 grid((n_sal + 127) / 128, M);
+    rcd::salient_residual_kernel<<<grid, 128, 0, s>>>(d_W, ldw, M, N, g, Kb, d_bits, d_row_scale_f32, d_col_scale_f32, d_sal_idx,
+                                                       d_pos, n_sal, d_P, ldp, d_live);
     FB_CUDA(cudaGetLastError());
     return FLUXBIN_OK;
 }

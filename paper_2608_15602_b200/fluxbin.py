@@ -40,7 +40,7 @@ EXPORTS = ["fluxbin_packed_size", "fluxbin_validate", "fluxbin_pack_host", "flux
            "fluxbin_plan_create", "fluxbin_plan_run", "fluxbin_plan_num_launches", "fluxbin_plan_pairs_per_row_block",
            "fluxbin_plan_free",
            "fluxbin_linear_noalloc", "fluxbin_noalloc_capacity",
-           "fluxbin_rc_decomp", "fluxbin_rc_decomp_workspace_size"]
+           "fluxbin_rc_decomp", "fluxbin_rc_decomp_workspace_size", "fluxbin_rc_salient_residual"]
 
 _LIB = None
 
@@ -91,7 +91,9 @@ def _lib():
         lib.fluxbin_rc_decomp_workspace_size.restype = sz
         lib.fluxbin_rc_decomp_workspace_size.argtypes = [i32, i32, i32, i32]
         lib.fluxbin_rc_decomp.restype = ctypes.c_int
-        lib.fluxbin_rc_decomp.argtypes = [vp, i64, i32, i32, i32, i32, i32, ctypes.c_float, vp, vp, vp, vp, vp, vp, sz, vp]
+        lib.fluxbin_rc_decomp.argtypes = [vp, i64, vp, i32, i32, i32, i32, i32, ctypes.c_float, vp, vp, vp, vp, vp, vp, sz, vp]
+        lib.fluxbin_rc_salient_residual.restype = ctypes.c_int
+        lib.fluxbin_rc_salient_residual.argtypes = [vp, i64, i32, i32, i32, i32, vp, vp, vp, vp, vp, i32, vp, i64, i32, vp, vp]
         _LIB = lib
     return _LIB
 
@@ -251,10 +253,16 @@ def rc_decomp_workspace_size(M: int, N: int, g: int, K: int) -> int:
 
 
 def rc_decomp_status(d_W, ldw, M, N, g, K, T, eps, d_bits, d_row_scale, d_col_scale, d_row_f32, d_col_f32, d_ws, ws_bytes,
-                     stream=0) -> int:
+                     stream=0, d_col_live=None) -> int:
     """fluxbin_rc_decomp (argument marshalling only; every pointer is a device address or None)."""
-    return int(_lib().fluxbin_rc_decomp(d_W, ldw, M, N, g, K, T, eps, d_bits, d_row_scale, d_col_scale, d_row_f32,
-                                        d_col_f32, d_ws, ws_bytes, stream))
+    return int(_lib().fluxbin_rc_decomp(d_W, ldw, d_col_live, M, N, g, K, T, eps, d_bits, d_row_scale, d_col_scale,
+                                        d_row_f32, d_col_f32, d_ws, ws_bytes, stream))
+
+
+def rc_salient_residual(d_W, ldw, M, N, g, Kb, d_bits, d_row_f32, d_col_f32, d_sal_idx, d_pos, n_sal, d_P, ldp, ncols_p,
+                        d_live, stream=0):
+    _check(int(_lib().fluxbin_rc_salient_residual(d_W, ldw, M, N, g, Kb, d_bits, d_row_f32, d_col_f32, d_sal_idx, d_pos,
+                                                  n_sal, d_P, ldp, ncols_p, d_live, stream)), "fluxbin_rc_salient_residual")
 
 
 def rc_decomp(*args, **kw):

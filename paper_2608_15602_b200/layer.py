@@ -92,7 +92,7 @@ class FluxBinPlan:
         return self.plan.pairs_per_row_block()
 
 
-def rc_decompose(W: torch.Tensor, g: int, K: int, T: int, eps: float = 1e-8, stream=None):
+def rc_decompose(W: torch.Tensor, g: int, K: int, T: int, eps: float = 1e-8, stream=None, col_live: torch.Tensor | None = None):
     """fluxbin_rc_decomp on a CUDA fp32 matrix W [M][N] (last dimension contiguous).  Returns a dict of CUDA tensors:
     bits uint32-as-int32 [K][M][N/32], row_scale / col_scale fp16 [K][M][N/g] / [K][N] (the canonical layout of a
     layer description) and their fp32 originals row_scale_f32 / col_scale_f32."""
@@ -107,23 +107,90 @@ def rc_decompose(W: torch.Tensor, g: int, K: int, T: int, eps: float = 1e-8, str
     ws = Workspace(max(fluxbin.rc_decomp_workspace_size(M, N, g, K), 256), device=dev)
     fluxbin.rc_decomp(W.data_ptr(), W.stride(0), M, N, g, K, T, eps, out["bits"].data_ptr(), out["row_scale"].data_ptr(),
                       out["col_scale"].data_ptr(), out["row_scale_f32"].data_ptr(), out["col_scale_f32"].data_ptr(),
-                      ws.tensor.data_ptr(), ws.tensor.numel() * ws.tensor.element_size(), _stream_ptr(stream))
+                      ws.tensor.data_ptr(), ws.tensor.numel() * ws.tensor.element_size(), _stream_ptr(stream),
+                      d_col_live=None if col_live is None else col_live.data_ptr())
     out["_workspace"] = ws
     return out
 
 
-def quantize_dense(W: torch.Tensor, g: int = 128, K: int = 2, T: int = 10, eps: float = 1e-8) -> "FluxBinLinear":
-    """Dense fp32 CUDA matrix -> packed FluxBin layer with K global bases and no salient refinement: the GPU
-    decomposition (fluxbin_rc_decomp), then the packer.  The canonical arrays pass through host memory because
-    fluxbin_pack takes host pointers."""
+def _pad_width(s_max: int) -> int:
+    for w in (32, 64, 128, 256):
+        if s_max <= w:
+            return w
+    raise ValueError("more than 256 salient columns in one row-scale group")
+
+
+def hybrid_decompose(W: torch.Tensor, g: int, Kb: int, Ks: int, sal_idx, T: int, eps: float = 1e-8):
+    """Global bases plus a refinement on given salient columns (Algorithm 2 without the saliency search and the
+    Hessian compensation): fluxbin_rc_decomp on W, then on the residual of every group's salient columns, each
+    group's block padded with zero columns to a common width (the padding marked in the live mask).  Only data
+    movement happens here (gathers, scatters, bit packing of the result); both decompositions run in the library.
+    Returns a dict of CUDA tensors in the canonical layout of a layer description."""
+    assert W.is_cuda and W.dtype == torch.float32
+    W = W.contiguous()
+    M, N = W.shape
+    dev = W.device
+    out = rc_decompose(W, g, Kb, T, eps)
+    sal_idx = torch.as_tensor(np.asarray(sal_idx, np.int64), device=dev)
+    n_sal = int(sal_idx.numel())
+    res = {"bits": out["bits"], "row_scale": out["row_scale"], "col_scale": out["col_scale"],
+           "row_scale_f32": out["row_scale_f32"], "col_scale_f32": out["col_scale_f32"], "sal_idx": sal_idx}
+    if Ks == 0 or n_sal == 0:
+        return res
+    # one padded block per group that has salient columns (index arithmetic for the layout only)
+    grp = sal_idx // g
+    groups, counts = torch.unique_consecutive(grp, return_counts=True)
+    width = _pad_width(int(counts.max()))
+    first = torch.cumsum(counts, 0) - counts
+    slot = torch.repeat_interleave(torch.arange(len(groups), device=dev), counts)            # block of each virtual column
+    pos = slot * width + (torch.arange(n_sal, device=dev) - first[slot])                     # its column in the padded matrix
+    ncols_p = len(groups) * width
+    P = torch.empty((M, ncols_p), dtype=torch.float32, device=dev)
+    live = torch.empty(ncols_p, dtype=torch.float32, device=dev)
+    idx32, pos32 = sal_idx.to(torch.int32), pos.to(torch.int32)
+    # the residual of the global part on the salient columns, written into the padded layout by the library
+    fluxbin.rc_salient_residual(W.data_ptr(), W.stride(0), M, N, g, Kb, out["bits"].data_ptr(), out["row_scale_f32"].data_ptr(),
+                                out["col_scale_f32"].data_ptr(), idx32.data_ptr(), pos32.data_ptr(), n_sal, P.data_ptr(),
+                                P.stride(0), ncols_p, live.data_ptr(), _stream_ptr())
+    so = rc_decompose(P, width, Ks, T, eps, col_live=live)
+    # back to the canonical salient arrays
+    nws = (n_sal + 31) // 32
+    sw = so["bits"][:, :, pos // 32]
+    sbit = ((sw >> (pos % 32).to(torch.int32)) & 1).to(torch.int64)                           # [Ks][M][n_sal]
+    v = torch.arange(n_sal, device=dev)
+    packed = torch.zeros((Ks, M, nws), dtype=torch.int64, device=dev)
+    packed.scatter_add_(2, (v // 32).expand(Ks, M, n_sal), sbit << (v % 32))
+    res["sal_bits"] = (packed & 0xFFFFFFFF).to(torch.int64)
+    sal_row = torch.zeros((Ks, M, N // g), dtype=torch.float32, device=dev)
+    sal_row[:, :, groups] = so["row_scale_f32"]
+    res["sal_row_scale_f32"] = sal_row
+    res["sal_col_scale_f32"] = so["col_scale_f32"][:, pos]
+    res["sal_row_scale"] = sal_row.to(torch.float16)
+    res["sal_col_scale"] = res["sal_col_scale_f32"].to(torch.float16)
+    res["sal_signs"] = sbit
+    return res
+
+
+def quantize_dense(W: torch.Tensor, g: int = 128, K: int = 2, T: int = 10, eps: float = 1e-8, sal_idx=None,
+                   Ks: int = 0) -> "FluxBinLinear":
+    """Dense fp32 CUDA matrix -> packed FluxBin layer: K global bases and, if `sal_idx` (ascending column indices)
+    and Ks > 0 are given, Ks further bases on those columns.  The decompositions run on the GPU
+    (fluxbin_rc_decomp); the canonical arrays pass through host memory because fluxbin_pack takes host pointers."""
     from . import synth
     M, N = W.shape
-    out = rc_decompose(W.contiguous(), g, K, T, eps)
+    r = hybrid_decompose(W, g, K, Ks if sal_idx is not None else 0, [] if sal_idx is None else sal_idx, T, eps)
     torch.cuda.synchronize(W.device)
-    L = synth.Linear(M, N, K, 0, g, 0,
-                     np.ascontiguousarray(out["bits"].cpu().numpy().view(np.uint32)),
-                     np.ascontiguousarray(out["row_scale"].cpu().numpy().view(np.uint16)),
-                     np.ascontiguousarray(out["col_scale"].cpu().numpy().view(np.uint16)),
-                     np.zeros(0, np.int32), np.zeros((0, M, 0), np.uint32), np.zeros((0, M, N // g), np.uint16),
-                     np.zeros((0, 0), np.uint16))
+    u16 = lambda t: np.ascontiguousarray(t.cpu().numpy().view(np.uint16))
+    if "sal_bits" in r:
+        n_sal = int(r["sal_idx"].numel())
+        L = synth.Linear(M, N, K, Ks, g, n_sal,
+                         np.ascontiguousarray(r["bits"].cpu().numpy().view(np.uint32)), u16(r["row_scale"]), u16(r["col_scale"]),
+                         r["sal_idx"].cpu().numpy().astype(np.int32),
+                         np.ascontiguousarray(r["sal_bits"].cpu().numpy().astype(np.uint32)),
+                         u16(r["sal_row_scale"]), u16(r["sal_col_scale"]))
+    else:
+        L = synth.Linear(M, N, K, 0, g, 0,
+                         np.ascontiguousarray(r["bits"].cpu().numpy().view(np.uint32)), u16(r["row_scale"]), u16(r["col_scale"]),
+                         np.zeros(0, np.int32), np.zeros((0, M, 0), np.uint32), np.zeros((0, M, N // g), np.uint16),
+                         np.zeros((0, 0), np.uint16))
     return FluxBinLinear(L, device=W.device)

@@ -174,3 +174,49 @@ def test_quantize_dense_helper(fb):
     want = x.view(np.float16).astype(np.float64) @ W.astype(np.float64).T
     got = y.cpu().numpy().astype(np.float64)
     assert np.linalg.norm(got - want) / np.linalg.norm(want) < 0.12        # four bases leave < 1 % of W's energy
+
+
+def test_hybrid_decomposition_matches_the_oracle(fb):
+    """Global bases + refinement on given salient columns (Algorithm 2, steps 2-3) on the GPU against the oracle."""
+    M, N, g, Kb, Ks, T = 96, 512, 128, 2, 2, 4
+    W = synth.make_dense_weight(13, 1, M, N, outlier_col_frac=0.05)
+    sal_idx = synth.salient_per_group(13, 2, N, g, 8)
+    r = fb.hybrid_decompose(torch.from_numpy(W).cuda(), g, Kb, Ks, sal_idx, T, 1e-8)
+    torch.cuda.synchronize()
+    want = rc.hybrid_decomp(W, g, Kb, Ks, sal_idx, T, 1e-8, dtype=np.float32)
+    B = unpack_bits(r["bits"].cpu().numpy(), N)
+    sB = r["sal_signs"].cpu().numpy().astype(np.float64) * 2 - 1
+    got = rc.hybrid_reconstruct(r["row_scale_f32"].cpu().numpy().astype(np.float64), r["col_scale_f32"].cpu().numpy().astype(np.float64), B,
+                                r["sal_row_scale_f32"].cpu().numpy().astype(np.float64),
+                                r["sal_col_scale_f32"].cpu().numpy().astype(np.float64), sB, sal_idx, g)
+    ref = rc.hybrid_reconstruct(*want, sal_idx, g)
+    loss_gpu, loss_ref = ((W - got) ** 2).sum(), ((W - ref) ** 2).sum()
+    assert abs(loss_gpu - loss_ref) <= 1e-3 * loss_ref
+    assert ((sB != want[5]).any(axis=0)).mean() <= 5e-3
+    assert np.allclose(r["sal_col_scale_f32"].cpu().numpy(), want[4], rtol=5e-3, atol=1e-5)
+    assert np.allclose(r["sal_row_scale_f32"].cpu().numpy(), want[3], rtol=5e-3, atol=1e-5 * np.abs(want[3]).max())
+    # the refinement helps: the error on the salient columns drops
+    base = np.einsum("kmn,kn,kmn->mn", np.repeat(r["row_scale_f32"].cpu().numpy().astype(np.float64), g, axis=2),
+                     r["col_scale_f32"].cpu().numpy().astype(np.float64), B)
+    assert ((W[:, sal_idx] - got[:, sal_idx]) ** 2).sum() < 0.5 * ((W[:, sal_idx] - base[:, sal_idx]) ** 2).sum()
+
+
+def test_quantize_dense_hybrid_layer_runs_through_the_linear_path(fb):
+    M, N, g = 256, 1024, 128
+    W = synth.make_dense_weight(14, 1, M, N, outlier_col_frac=0.05)
+    sal_idx = synth.salient_random(14, 2, N, 0.05)                  # uneven counts per group, some groups empty
+    Wt = torch.from_numpy(W).cuda()
+    lin2 = fb.quantize_dense(Wt, g=g, K=2, T=6)
+    linh = fb.quantize_dense(Wt, g=g, K=2, T=6, sal_idx=sal_idx, Ks=2)
+    x = synth.make_activations(14, 3, 2, N)
+    xt = torch.from_numpy(x.view(np.float16)).cuda()
+    want = x.view(np.float16).astype(np.float64) @ W.astype(np.float64).T
+    err = []
+    for lin in (lin2, linh):
+        y = lin.forward(xt, lin.workspace(2), fp32_out=True)
+        torch.cuda.synchronize()
+        err.append(np.linalg.norm(y.cpu().numpy().astype(np.float64) - want) / np.linalg.norm(want))
+    assert err[1] < err[0] < 0.4            # the salient bases reduce the output error
+    # and the packed hybrid layer round-trips to the arrays the decomposition produced
+    got = linh.unpack()
+    assert got.n_sal == len(sal_idx) and np.array_equal(got.sal_idx, sal_idx)
