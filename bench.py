@@ -485,7 +485,7 @@ def main():
         peak = float(peaks["hbm_gbs"])
         achieved = bytes_per_step / (ms_per_step * 1e-3) / 1e9     # one GPU's kernels
         traffic = None
-        tpath = os.path.join(ROOT, "profiles", "dram_traffic.json")
+        tpath = os.path.join(ROOT, "profiles", "dram_traffic.txt")
         if os.path.exists(tpath):
             with open(tpath) as f:
                 tj = json.load(f)
