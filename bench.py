@@ -215,6 +215,8 @@ def main():
     ap.add_argument("--config", type=int, default=4, help="workload: 4 = Llama-2-70B-shaped stack")
     ap.add_argument("--layers", type=int, default=None, help="override the number of layers (profiling only)")
     ap.add_argument("--batch", type=int, default=1)
+    ap.add_argument("--fp16-tables", action="store_true",
+                    help="batched launches keep their lookup tables in fp16 (fluxbin_set_table_format); no effect at batch 1")
     ap.add_argument("--g", type=int, default=128, help="columns per row-scale group; 0 = one scale per row (g = N)")
     ap.add_argument("--no-graph", action="store_true", help="plain launches instead of a CUDA graph replay")
     ap.add_argument("--launch", default="stack", choices=["linear", "group", "layer", "stack"],
@@ -274,7 +276,7 @@ def main():
             j = next(it, None)
             if j is not None:
                 window.append(ex.submit(gen, j))
-            lin = fb_layer.FluxBinLinear(L)
+            lin = fb_layer.FluxBinLinear(L, fp16_tables=args.fp16_tables)
             linears.append(lin)
             xs_host.append(x)
             alg_bytes.append(algorithmic_bytes(L.M, L.N, L.Kb, L.Ks, L.g, L.n_sal, B))
@@ -500,6 +502,7 @@ def main():
             "config": {"workload": f"config {args.config}: Llama-2-70B-shaped decode linear stack" if args.config == 4
                        else f"config {args.config}: {nl} independently seeded copies of the layer/set per step",
                        "layers": nl, "linears_per_step": len(linears), "batch": B,
+                       "table_entries": "fp16" if (args.fp16_tables and B > 1) else "fp32",
                        "Kb": 2, "Ks": 0 if args.config == 0 else 1, "salient_frac": 0.0 if args.config == 0 else 0.05,
                        "g": args.g or "N", "packed_bytes_resident": packed_bytes, "algorithmic_bytes_per_step": bytes_per_step,
                        "l2": "inputs larger than L2 (weights streamed once per step)" if packed_bytes > 4e8

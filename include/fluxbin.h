@@ -130,8 +130,35 @@ fluxbin_status_t fluxbin_unpack(const fluxbin_weight_t *w, fluxbin_layer_desc_t 
 fluxbin_status_t fluxbin_weight_dims(const fluxbin_weight_t *w, fluxbin_layer_desc_t *out);
 
 /*
+ * Precision of the lookup-table entries (Eq. 14) of batched launches (B >= 2) that read this layer.
+ *
+ *   FLUXBIN_TABLES_FP32 (default)  entries are fp32, the size the paper's shared-memory model counts
+ *                                  (2^mu entries of 4 bytes per sub-vector and batch index); B runs in chunks
+ *                                  of up to 4 vectors.
+ *   FLUXBIN_TABLES_FP16            entries are the fp32 partial sums rounded once to fp16 (to nearest even),
+ *                                  two batch vectors per 32-bit word: half the shared-memory bytes per lookup,
+ *                                  which is what bounds the batched path; B runs in chunks of up to 8 vectors.
+ *                                  Every sum is still accumulated in fp32.  Each lookup then carries a relative
+ *                                  rounding error of at most 2^-11, so an output differs from the fp32-table
+ *                                  result by about 2^-11 / sqrt(3) of the root-sum-square of its looked-up
+ *                                  terms -- an error relative to the magnitude of the terms, not of the (possibly
+ *                                  cancelling) sum.  Entries beyond the fp16 range (|sum of 8 fused activations|
+ *                                  > 65504) become infinite and tiny ones lose bits below 6e-8: meant for
+ *                                  normalised activations.
+ *
+ * A single vector (B == 1, or a trailing chunk of one) always uses fp32 entries.  The setting is read by
+ * fluxbin_workspace_size, fluxbin_num_launches, fluxbin_linear and fluxbin_plan_create (all members of a plan
+ * must agree, else FLUXBIN_ERR_UNSUPPORTED); change it only between those calls, and size workspaces after
+ * it.  Returns FLUXBIN_ERR_RANGE for an unknown format.  fluxbin_get_table_format: the setting, -1 on NULL.
+ */
+#define FLUXBIN_TABLES_FP32 0
+#define FLUXBIN_TABLES_FP16 1
+fluxbin_status_t fluxbin_set_table_format(fluxbin_weight_t *w, int32_t format);
+int32_t fluxbin_get_table_format(const fluxbin_weight_t *w);
+
+/*
  * DEVICE workspace bytes fluxbin_linear needs for batch size B with this layer: fp32 split-K
- * accumulators for up to 2 batch rows at a time plus one arrival counter per tile of output
+ * accumulators for one chunk of batch rows at a time plus one arrival counter per tile of output
  * rows (stage (iii) "reduction" of Sec. 3.2).  The workspace must be zeroed once with
  * fluxbin_workspace_init before its first use; every call leaves it zeroed again, so one
  * workspace of the maximum size can serve any sequence of stream-ordered calls.
@@ -152,7 +179,7 @@ fluxbin_status_t fluxbin_workspace_init(void *d_workspace, size_t bytes, void *c
  * Asynchronous on cuda_stream; performs no allocation and no synchronisation, so calls can be
  * captured into a CUDA graph.  The kernel is launched with programmatic stream serialization: it may
  * begin (index arithmetic, L2 prefetch of its weights) while the previous kernel on the stream is
- * draining, and waits on the device before it reads d_x or touches the workspace.  B >= 1 arbitrary (processed in chunks of up to 4 vectors).  Calls
+ * draining, and waits on the device before it reads d_x or touches the workspace.  B >= 1 arbitrary (processed in chunks of up to 4 vectors, 8 with fp16 table entries).  Calls
  * sharing a workspace must be ordered on one stream.  Accumulation is fp32 with fp32 atomics
  * across K slices, so results may differ in the last bits from run to run.
  */
@@ -231,7 +258,7 @@ void fluxbin_free(fluxbin_weight_t *w);
  */
 typedef struct fluxbin_plan fluxbin_plan_t;
 
-size_t fluxbin_plan_table_bytes(int32_t n, int32_t B);
+size_t fluxbin_plan_table_bytes(int32_t n, int32_t B);     /* enough for either table format */
 
 size_t fluxbin_plan_workspace_bytes(int32_t n, const fluxbin_weight_t *const *w, int32_t B);
 
@@ -249,7 +276,7 @@ fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_t *const *w
  */
 fluxbin_status_t fluxbin_plan_run(const fluxbin_plan_t *plan, void *cuda_stream);
 
-/* Kernel launches one fluxbin_plan_run issues (one per chunk of up to 4 batch vectors); -1 on NULL. */
+/* Kernel launches one fluxbin_plan_run issues (one per chunk of up to 4 batch vectors, 8 with fp16 table entries); -1 on NULL. */
 int32_t fluxbin_plan_num_launches(const fluxbin_plan_t *plan);
 
 /* Introspection: how many table sets (pairs of 16-sub-vector units) the plan's kernel keeps resident per row

@@ -92,6 +92,9 @@ fluxbin_status_t device_setup(int dev, int *num_sms)
             FB_CUDA(opt_in_bt<1>());
             FB_CUDA(opt_in_bt<2>());
             FB_CUDA(opt_in_bt<4>());
+            FB_CUDA(opt_in_bt<16 + 2>());
+            FB_CUDA(opt_in_bt<16 + 4>());
+            FB_CUDA(opt_in_bt<16 + 8>());
             FB_CUDA(cudaFuncSetAttribute(fbk::fluxbin_debug_tables_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)fbk::smem_bytes<1>()));
             FB_CUDA(cudaFuncSetAttribute(fbk::fluxbin_smem_base_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -129,6 +132,7 @@ fluxbin_status_t make_handle(const FbHeader &h, void *d_packed, size_t d_bytes, 
     w->tile_rb = 16;
     if ((h.nrb + w->tile_rb - 1) / w->tile_rb > fbk::kMaxTiles) w->tile_rb = (h.nrb + fbk::kMaxTiles - 1) / fbk::kMaxTiles;
     w->ntiles = (h.nrb + w->tile_rb - 1) / w->tile_rb;
+    w->table_format = FLUXBIN_TABLES_FP32;
     *out = w;
     return FLUXBIN_OK;
 }
@@ -198,21 +202,30 @@ extern "C" void fluxbin_free(fluxbin_weight_t *w) { delete w; }
 
 extern "C" int32_t fluxbin_num_table_sets(const fluxbin_weight_t *w) { return w ? w->h.npairs[0] + w->h.npairs[1] : -1; }
 
-// Batch vectors per launch: B is processed in chunks of up to four.  A chunk of 1, 2 or 3..4 vectors
-// runs the kernel whose table entries hold 1, 2 or 4 vectors side by side (LDS.32 / .64 / .128): the
-// weights stream once per chunk and one address computation serves the whole entry.
-#ifndef FB_CHUNK
-#define FB_CHUNK 4
-#endif
-static int chunk_size() { return FB_CHUNK; }
-static int num_chunks(int B) { return (B + chunk_size() - 1) / chunk_size(); }
-static int bt_for(int nb) { return nb == 1 ? 1 : nb == 2 ? 2 : 4; }
-static int ws_bt(int B) { return bt_for(B < chunk_size() ? B : chunk_size()); }
+extern "C" fluxbin_status_t fluxbin_set_table_format(fluxbin_weight_t *w, int32_t format)
+{
+    if (!w) return FLUXBIN_ERR_NULL;
+    if (format != FLUXBIN_TABLES_FP32 && format != FLUXBIN_TABLES_FP16) return FLUXBIN_ERR_RANGE;
+    w->table_format = format;
+    return FLUXBIN_OK;
+}
+
+extern "C" int32_t fluxbin_get_table_format(const fluxbin_weight_t *w) { return w ? w->table_format : -1; }
+
+// Batch vectors per launch: B is processed in chunks of up to four (fp32 table entries) or eight (fp16
+// entries).  A chunk runs the kernel whose table entries hold its vectors side by side in 4, 8 or 16 bytes
+// (LDS.32 / .64 / .128): the weights stream once per chunk and one address computation serves the whole
+// entry.  A single vector always uses fp32 entries (nothing to share a word with).
+static int chunk_size(int fmt) { return fmt == FLUXBIN_TABLES_FP16 ? 8 : 4; }
+static int num_chunks(int B, int fmt) { return (B + chunk_size(fmt) - 1) / chunk_size(fmt); }
+static int nvec_for(int nb) { return nb == 1 ? 1 : nb == 2 ? 2 : nb <= 4 ? 4 : 8; }
+static int mode_for(int nb, int fmt) { return (fmt == FLUXBIN_TABLES_FP16 && nb >= 2) ? 16 + nvec_for(nb) : nvec_for(nb); }
+static int ws_bt(int B, int fmt) { return nvec_for(B < chunk_size(fmt) ? B : chunk_size(fmt)); }   // accumulator rows per layer
 
 extern "C" int32_t fluxbin_num_launches(const fluxbin_weight_t *w, int32_t B)
 {
     if (!w || B < 1) return -1;
-    return num_chunks(B);
+    return num_chunks(B, w->table_format);
 }
 
 // ---- workspace ----------------------------------------------------------------------------------
@@ -222,7 +235,7 @@ static size_t acc_bytes(const fluxbin_weight_t *w, int bt) { return ((size_t)bt 
 extern "C" size_t fluxbin_workspace_size(const fluxbin_weight_t *w, int32_t B)
 {
     if (!w || B < 1) return 0;
-    int bt = ws_bt(B);
+    int bt = ws_bt(B, w->table_format);
     return acc_bytes(w, bt) + ((size_t)w->ntiles * 4 + 255) / 256 * 256 + 256;    // + the launch counters
 }
 
@@ -322,6 +335,22 @@ template <int BT> static cudaError_t launch_bt(int s0, int s1, int num_sms, cons
     return launch<4, 1, BT>(p, num_sms, items, couple_cost, s);
 }
 
+// mode: 1, 2, 4 vectors with fp32 tables, 16 + (2, 4, 8) vectors with fp16 tables; the two-pair kernel exists
+// for mode 1 only (couple_cost is ignored elsewhere)
+static cudaError_t launch_mode(int mode, int s0, int s1, int num_sms, const fbk::LaunchParams &p, long long items,
+                               long long couple_cost, cudaStream_t s)
+{
+    switch (mode) {
+    case 1: return launch_bt<1>(s0, s1, num_sms, p, items, couple_cost, s);
+    case 2: return launch_bt<2>(s0, s1, num_sms, p, items, 0, s);
+    case 4: return launch_bt<4>(s0, s1, num_sms, p, items, 0, s);
+    case 16 + 2: return launch_bt<16 + 2>(s0, s1, num_sms, p, items, 0, s);
+    case 16 + 4: return launch_bt<16 + 4>(s0, s1, num_sms, p, items, 0, s);
+    case 16 + 8: return launch_bt<16 + 8>(s0, s1, num_sms, p, items, 0, s);
+    }
+    return cudaErrorInvalidValue;
+}
+
 
 // Work-split cost model, measured on B200 in units of half a 1152-byte item (about 50 ns per CTA):
 // an item with one row scale per sub-vector (3072 bytes) takes about 2x a plain item; building one
@@ -384,23 +413,21 @@ extern "C" fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint
     item_costs(w->h.sps[0], sps1_eff, p.item_cost);
     p.build_cost = kBuildCost;
     p.total_cost = entry_cost(w->h, sps1_eff);
-    const int bt_ws = ws_bt(B);
+    const int fmt = w->table_format;
+    const int bt_ws = ws_bt(B, fmt);
     float *acc = (float *)d_workspace;
     unsigned *tickets = (unsigned *)((uint8_t *)d_workspace + acc_bytes(w, bt_ws));
     p.counters = (unsigned *)((uint8_t *)d_workspace + acc_bytes(w, bt_ws) + ((size_t)w->ntiles * 4 + 255) / 256 * 256);
     const long long items = (long long)(w->h.npairs[0] + w->h.npairs[1]) * w->h.nrb;
 
     const size_t ysz = y_is_fp32 ? 4 : 2;
-    const int CH = chunk_size();
+    const int CH = chunk_size(fmt);
     for (int b0 = 0; b0 < B; b0 += CH) {
         const int nb = (B - b0 < CH) ? B - b0 : CH;
         fill_entry(p.single, w, d_x + (int64_t)b0 * ldx, ldx, (uint8_t *)d_y + (size_t)b0 * ldy * ysz, ldy, acc, tickets, 0);
         p.nb = nb;
-        cudaError_t e;
         const int s1 = w->h.npairs[1] > 0 ? w->h.sps[1] : 1;
-        if (nb == 1) e = launch_bt<1>(w->h.sps[0], s1, w->num_sms, p, items, couple_cost_of(w->h), s);
-        else if (nb == 2) e = launch_bt<2>(w->h.sps[0], s1, w->num_sms, p, items, 0, s);
-        else e = launch_bt<4>(w->h.sps[0], s1, w->num_sms, p, items, 0, s);
+        cudaError_t e = launch_mode(mode_for(nb, fmt), w->h.sps[0], s1, w->num_sms, p, items, couple_cost_of(w->h), s);
         if (e != cudaSuccess) return cuda_fail(e);
     }
     return FLUXBIN_OK;
@@ -409,7 +436,7 @@ extern "C" fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint
 // ---- plans: many layers in one persistent launch -------------------------------------------------
 
 struct fluxbin_plan {
-    int n, B, y_fp32, nchunks;
+    int n, B, y_fp32, nchunks, table_format;
     int sps0, sps1, num_sms;
     long long total_cost, items, couple_cost;
     int item_cost[2];
@@ -425,13 +452,14 @@ static size_t entry_ws_bytes(const fluxbin_weight_t *w, int bt)
 extern "C" size_t fluxbin_plan_table_bytes(int32_t n, int32_t B)
 {
     if (n < 1 || B < 1) return 0;
-    return (size_t)n * sizeof(fbk::LinearEntry) * (size_t)num_chunks(B);
+    return (size_t)n * sizeof(fbk::LinearEntry) * (size_t)num_chunks(B, FLUXBIN_TABLES_FP32);   // the format with more chunks
 }
 
 extern "C" size_t fluxbin_plan_workspace_bytes(int32_t n, const fluxbin_weight_t *const *w, int32_t B)
 {
     if (n < 1 || B < 1 || !w) return 0;
-    const int bt = ws_bt(B);
+    if (!w[0]) return 0;
+    const int bt = ws_bt(B, w[0]->table_format);
     size_t total = 0;
     for (int i = 0; i < n; ++i) {
         if (!w[i]) return 0;
@@ -460,6 +488,7 @@ extern "C" fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_
         if (ldx[i] < w[i]->h.N || ldy[i] < w[i]->h.M) return FLUXBIN_ERR_RANGE;
         if ((((uintptr_t)d_x[i]) & 15) || (((uintptr_t)d_y[i]) & 15)) return FLUXBIN_ERR_ALIGNMENT;
         if (w[i]->h.sps[0] != w[0]->h.sps[0]) return FLUXBIN_ERR_UNSUPPORTED;
+        if (w[i]->table_format != w[0]->table_format) return FLUXBIN_ERR_UNSUPPORTED;
         if (w[i]->h.npairs[1] > 0) {          // the salient format only matters where there is a salient region
             if (w[i]->h.sps[1] == 16 && w[i]->h.sps[0] != 16) return FLUXBIN_ERR_FORMAT;
             if (sps1 != 0 && w[i]->h.sps[1] != sps1) return FLUXBIN_ERR_UNSUPPORTED;
@@ -469,7 +498,8 @@ extern "C" fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_
     if (sps1 == 0) sps1 = 1;
     if (ws_bytes < fluxbin_plan_workspace_bytes(n, w, B)) return FLUXBIN_ERR_BUFFER_TOO_SMALL;
 
-    const int nchunks = num_chunks(B), bt = ws_bt(B), CH = chunk_size();
+    const int fmt = w[0]->table_format;
+    const int nchunks = num_chunks(B, fmt), bt = ws_bt(B, fmt), CH = chunk_size(fmt);
     const size_t ysz = y_is_fp32 ? 4 : 2;
     fbk::LinearEntry *host = (fbk::LinearEntry *)std::malloc(sizeof(fbk::LinearEntry) * (size_t)n * nchunks);
     if (!host) return FLUXBIN_ERR_UNSUPPORTED;
@@ -496,7 +526,7 @@ extern "C" fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_
 
     fluxbin_plan *p = new (std::nothrow) fluxbin_plan;
     if (!p) return FLUXBIN_ERR_UNSUPPORTED;
-    p->n = n; p->B = B; p->y_fp32 = y_is_fp32 != 0; p->nchunks = nchunks;
+    p->n = n; p->B = B; p->y_fp32 = y_is_fp32 != 0; p->nchunks = nchunks; p->table_format = fmt;
     p->sps0 = w[0]->h.sps[0]; p->sps1 = sps1; p->num_sms = w[0]->num_sms;
     p->total_cost = cost; p->items = items;
     p->couple_cost = 0;
@@ -530,14 +560,12 @@ extern "C" fluxbin_status_t fluxbin_plan_run(const fluxbin_plan_t *plan, void *c
     p.total_cost = plan->total_cost;
     p.counters = plan->d_counters;
     for (int c = 0; c < plan->nchunks; ++c) {
-        const int CH = chunk_size();
+        const int CH = chunk_size(plan->table_format);
         const int nb = (plan->B - CH * c < CH) ? plan->B - CH * c : CH;
         p.table = plan->d_table + (size_t)c * plan->n;
         p.nb = nb;
-        cudaError_t e;
-        if (nb == 1) e = launch_bt<1>(plan->sps0, plan->sps1, plan->num_sms, p, plan->items, plan->couple_cost, s);
-        else if (nb == 2) e = launch_bt<2>(plan->sps0, plan->sps1, plan->num_sms, p, plan->items, 0, s);
-        else e = launch_bt<4>(plan->sps0, plan->sps1, plan->num_sms, p, plan->items, 0, s);
+        cudaError_t e = launch_mode(mode_for(nb, plan->table_format), plan->sps0, plan->sps1, plan->num_sms, p, plan->items,
+                                    plan->couple_cost, s);
         if (e != cudaSuccess) return cuda_fail(e);
     }
     return FLUXBIN_OK;

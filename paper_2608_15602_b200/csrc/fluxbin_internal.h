@@ -32,6 +32,7 @@ struct fluxbin_weight {
     int num_sms;
     int tile_rb;  // row blocks (of 32 rows) per arrival-counter tile
     int ntiles;
+    int table_format;   // FLUXBIN_TABLES_FP32 / _FP16: how batched launches (B >= 2) hold their table entries
 };
 
 #endif

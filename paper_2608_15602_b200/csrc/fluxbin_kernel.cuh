@@ -36,12 +36,20 @@
 
 namespace fbk {
 
-// Threads per CTA: 8 warps with 1 or 2 batch vectors per launch (3 or 2 CTAs per SM); with 4 vectors the
+// The template parameter BT of everything below is a launch MODE: 1, 2 or 4 = that many batch vectors per
+// launch with fp32 table entries (the precision the paper's shared-memory model states); 16 + n (n = 2, 4, 8)
+// = n batch vectors with fp16 table entries, two vectors per 32-bit word -- half the shared-memory bytes per
+// lookup, which is what bounds the batched path.  Sums still accumulate in fp32.
+__host__ __device__ constexpr int nvec(int BT) { return BT & 15; }               // batch vectors per launch
+__host__ __device__ constexpr bool half_tables(int BT) { return BT >= 16; }
+__host__ __device__ constexpr int geom(int BT) { return half_tables(BT) ? nvec(BT) / 2 : BT; }   // 32-bit words per table entry
+
+// Threads per CTA: 8 warps with 4- or 8-byte entries (3 or 2 CTAs per SM); with 16-byte entries the
 // tables fill 128 KB, one CTA owns the SM and runs 16 warps.
 template <int BT> struct Cfg {
-    static constexpr int kThreads = (BT == 4) ? 512 : 256;
+    static constexpr int kThreads = (geom(BT) == 4) ? 512 : 256;
     static constexpr int kWarps = kThreads / 32;
-    static constexpr int kMinBlocks = (BT == 4) ? 1 : (BT == 2) ? 2 : 3;
+    static constexpr int kMinBlocks = (geom(BT) == 4) ? 1 : (geom(BT) == 2) ? 2 : 3;
 };
 constexpr int kMaxTiles = 1024;
 #ifndef FB_DEPTH
@@ -58,7 +66,7 @@ constexpr int kDepth2 = FB_DEPTH2;
 #ifndef FB_DEPTH4
 #define FB_DEPTH4 2
 #endif
-template <int BT> struct DepthFor { static constexpr int value = BT == 4 ? FB_DEPTH4 : BT == 2 ? kDepth2 : kDepth; };
+template <int BT> struct DepthFor { static constexpr int value = geom(BT) == 4 ? FB_DEPTH4 : geom(BT) == 2 ? kDepth2 : kDepth; };
 #ifndef FB_PF
 #define FB_PF 1
 #endif
@@ -103,14 +111,14 @@ struct LaunchParams {
 constexpr uint32_t kTabBase = 0x800u;
 
 template <int BT> struct TabCfg {
-    static constexpr int kTableBytes = (BT == 4) ? 131072 : 65536;
+    static constexpr int kTableBytes = (geom(BT) == 4) ? 131072 : 65536;
     // scale-fusion scratch, tile counters (+ count of completed tiles), work range, copy of the current entry
-    static constexpr int kSmallBytes = 256 * BT * 4 + (kMaxTiles + 4) * 4 + 32 + 128;
+    static constexpr int kSmallBytes = 256 * nvec(BT) * 4 + (kMaxTiles + 4) * 4 + 32 + 128;
     // offset of slot sigma from the table base at step 0; entry p adds p << 8.
     // lane_const(lane ^ s) == lane_const(lane) ^ lane_const(s)
     __host__ __device__ static constexpr uint32_t lane_const(uint32_t sigma)
     {
-        return BT == 1 ? sigma * 4u : BT == 2 ? sigma * 8u : ((sigma & 15u) * 16u) | ((sigma >> 4) << 16);
+        return geom(BT) == 1 ? sigma * 4u : geom(BT) == 2 ? sigma * 8u : ((sigma & 15u) * 16u) | ((sigma >> 4) << 16);
     }
 };
 
@@ -138,10 +146,7 @@ __device__ __forceinline__ uint32_t ldg_stream_u32(const void *p)
     return v;
 }
 
-template <int BT> struct Vec;
-template <> struct Vec<1> { float v[1]; };
-template <> struct Vec<2> { float v[2]; };
-template <> struct Vec<4> { float v[4]; };
+template <int BT> struct Vec { float v[nvec(BT)]; };
 
 // HALF selects the table set inside the 256-byte p-rows: slots 0..31 or (BT == 1 only) slots 32..63.
 template <int BT, int HALF> __device__ __forceinline__ Vec<BT> lds_entry(uint32_t addr)
@@ -152,6 +157,31 @@ template <int BT, int HALF> __device__ __forceinline__ Vec<BT> lds_entry(uint32_
     else if constexpr (BT == 2) asm volatile("ld.shared.v2.f32 {%0,%1}, [%2+%3];" : "=f"(r.v[0]), "=f"(r.v[1]) : "r"(addr), "n"(kTabBase));
     else asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4+%5];" : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3]) : "r"(addr), "n"(kTabBase));
     return r;
+}
+
+// fp16 tables: the geom(BT) words of one entry, two batch vectors per word (vector 2i in the low half of word i)
+template <int BT, int HALF> __device__ __forceinline__ void lds_entry_h(uint32_t addr, uint32_t (&w)[geom(BT)])
+{
+    if constexpr (geom(BT) == 1) asm volatile("ld.shared.b32 %0, [%1+%2];" : "=r"(w[0]) : "r"(addr), "n"(kTabBase + HALF * 128));
+    else if constexpr (geom(BT) == 2) asm volatile("ld.shared.v2.b32 {%0,%1}, [%2+%3];" : "=r"(w[0]), "=r"(w[1]) : "r"(addr), "n"(kTabBase));
+    else asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4+%5];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(addr), "n"(kTabBase));
+}
+
+// lo += low half of h2, hi += high half of h2: fp16 addends, fp32 sums (one instruction each on sm_100)
+__device__ __forceinline__ void add_h2(float &lo, float &hi, uint32_t h2)
+{
+    asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %2;\n\tadd.rn.f32.f16 %0, l, %0;\n\tadd.rn.f32.f16 %1, h, %1;\n\t}"
+        : "+f"(lo), "+f"(hi) : "r"(h2));
+}
+
+// NV fp32 values rounded to fp16 (to nearest even) and stored as NV/2 words at byte `off` of the entry at addr
+template <int NV> __device__ __forceinline__ void sts_entry_h(uint32_t addr, const float *v)
+{
+    uint32_t w[NV / 2];
+#pragma unroll
+    for (int i = 0; i < NV / 2; ++i) asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(w[i]) : "f"(v[2 * i + 1]), "f"(v[2 * i]));
+    if constexpr (NV == 2) asm volatile("st.shared.b32 [%0+%2], %1;" ::"r"(addr), "r"(w[0]), "n"(kTabBase) : "memory");
+    else asm volatile("st.shared.v2.b32 [%0+%3], {%1,%2};" ::"r"(addr), "r"(w[0]), "r"(w[1]), "n"(kTabBase) : "memory");
 }
 
 // the NV batch vectors of one entry at table offset addr
@@ -201,7 +231,7 @@ __device__ __forceinline__ void prefetch_l2(const void *p, uint32_t bytes)
 // The two values a thread contributes to a table set: x of its column (per batch vector) and the
 // fused column scale.
 template <int BT> struct BuildInput {
-    float xv[BT];
+    float xv[nvec(BT)];
     uint32_t e;        // {u16 column, fp16 alpha}
 };
 
@@ -217,13 +247,13 @@ __device__ __forceinline__ void fetch_build_input(BuildInput<BT> &in, const uint
         const uint32_t col = (uint32_t)(tid < 128 ? col0_a : col0_b) + (uint32_t)(tid & 127);
         const bool live = col < (uint32_t)ncols;          // padded columns carry alpha = 0
 #pragma unroll
-        for (int b = 0; b < BT; ++b) in.xv[b] = (b < nb && live) ? h2f(__ldg(x + (int64_t)b * ldx + col)) : 0.f;
+        for (int b = 0; b < nvec(BT); ++b) in.xv[b] = (b < nb && live) ? h2f(__ldg(x + (int64_t)b * ldx + col)) : 0.f;
         in.e = __ldg((const uint32_t *)pair_desc + tid);
     } else {
         in.e = __ldg((const uint32_t *)pair_desc + tid);
         const uint32_t col = in.e & 0xffffu;
 #pragma unroll
-        for (int b = 0; b < BT; ++b) in.xv[b] = (b < nb) ? h2f(__ldg(x + (int64_t)b * ldx + col)) : 0.f;
+        for (int b = 0; b < nvec(BT); ++b) in.xv[b] = (b < nb) ? h2f(__ldg(x + (int64_t)b * ldx + col)) : 0.f;
     }
 }
 
@@ -231,50 +261,59 @@ __device__ __forceinline__ void fetch_build_input(BuildInput<BT> &in, const uint
 // the writers (8 n x 4 slots per warp) and the readers (32 slots per warp, one n) touch 32 different banks.
 template <int BT> __device__ __forceinline__ int abuf_index(int slot, int n, int b)
 {
-    return (n * BT + b) * 32 + ((slot + 4 * n) & 31);
+    return (n * nvec(BT) + b) * 32 + ((slot + 4 * n) & 31);
 }
 
 template <int BT>
 __device__ __forceinline__ void build_tables(const BuildInput<BT> &in, float *abuf, uint32_t half_off = 0)
 {
     const int tid = threadIdx.x;
+    constexpr int NV = nvec(BT);
     if (Cfg<BT>::kThreads == 256 || tid < 256) {
         const float al = h2f(in.e >> 16);
 #pragma unroll
-        for (int b = 0; b < BT; ++b) abuf[abuf_index<BT>(tid >> 3, tid & 7, b)] = in.xv[b] * al;   // exact in fp32: two 11-bit significands
+        for (int b = 0; b < NV; ++b) abuf[abuf_index<BT>(tid >> 3, tid & 7, b)] = in.xv[b] * al;   // exact in fp32: two 11-bit significands
     }
     __syncthreads();
     const int lane = tid & 31, warp = tid >> 5;
     constexpr int PW = 256 / Cfg<BT>::kWarps;          // table entries per warp: p = warp*PW + ...
     // EB entries at a time: the high index bits fix a base value, the low LB bits are enumerated by
-    // doubling (entry p | 2^n = entry p + 2 a_n), one add per entry.  All BT batch vectors of an entry are
-    // stored with one instruction (with four vectors, blocks of 8 entries keep the registers in bounds).
-    constexpr int LB = (BT == 4) ? 3 : 4, EB = 1 << LB;
+    // doubling (entry p | 2^n = entry p + 2 a_n), one add per entry.  Up to four batch vectors of an entry are
+    // stored with one instruction (with four, blocks of 8 entries keep the registers in bounds); eight vectors
+    // (fp16 entries) take two passes of four, each filling its half of the 16-byte entries.
+    constexpr int PV = NV < 4 ? NV : 4;                // vectors per pass
+    constexpr int LB = (PV == 4) ? 3 : 4, EB = 1 << LB;
     static_assert(PW % EB == 0, "a warp enumerates whole blocks of entries");
-    float a[8][BT];
-#pragma unroll
-    for (int n = 0; n < 8; ++n)
-#pragma unroll
-        for (int b = 0; b < BT; ++b) a[n][b] = abuf[abuf_index<BT>(lane, n, b)];
 #pragma unroll 1
-    for (int p0 = warp * PW; p0 < (warp + 1) * PW; p0 += EB) {
-        float v[EB][BT];
+    for (int b0 = 0; b0 < NV; b0 += PV) {
+        float a[8][PV];
 #pragma unroll
-        for (int b = 0; b < BT; ++b) {
-            float base = 0.f;
+        for (int n = 0; n < 8; ++n)
 #pragma unroll
-            for (int n = 7; n >= LB; --n) base += ((p0 >> n) & 1) ? a[n][b] : -a[n][b];
+            for (int b = 0; b < PV; ++b) a[n][b] = abuf[abuf_index<BT>(lane, n, b0 + b)];
+#pragma unroll 1
+        for (int p0 = warp * PW; p0 < (warp + 1) * PW; p0 += EB) {
+            float v[EB][PV];
 #pragma unroll
-            for (int n = LB - 1; n >= 0; --n) base -= a[n][b];
-            v[0][b] = base;
+            for (int b = 0; b < PV; ++b) {
+                float base = 0.f;
 #pragma unroll
-            for (int n = 0; n < LB; ++n)
+                for (int n = 7; n >= LB; --n) base += ((p0 >> n) & 1) ? a[n][b] : -a[n][b];
 #pragma unroll
-                for (int q = 0; q < (1 << n); ++q) v[q | (1 << n)][b] = v[q][b] + 2.f * a[n][b];
+                for (int n = LB - 1; n >= 0; --n) base -= a[n][b];
+                v[0][b] = base;
+#pragma unroll
+                for (int n = 0; n < LB; ++n)
+#pragma unroll
+                    for (int q = 0; q < (1 << n); ++q) v[q | (1 << n)][b] = v[q][b] + 2.f * a[n][b];
+            }
+#pragma unroll
+            for (int q = 0; q < EB; ++q) {
+                const uint32_t addr = half_off | TabCfg<BT>::lane_const((uint32_t)lane) | ((uint32_t)(p0 + q) << 8);
+                if constexpr (half_tables(BT)) sts_entry_h<PV>(addr + 2u * (uint32_t)b0, v[q]);    // rounded once, from the fp32 sum
+                else sts_entry<PV>(addr, v[q]);
+            }
         }
-#pragma unroll
-        for (int q = 0; q < EB; ++q)
-            sts_entry<BT>(half_off | TabCfg<BT>::lane_const((uint32_t)lane) | ((uint32_t)(p0 + q) << 8), v[q]);
     }
     __syncthreads();
 }
@@ -376,37 +415,52 @@ template <> struct LaneAddr<4> {
     }
 };
 
+// the table geometry of the fp16 modes is that of the fp32 mode with the same entry size
+template <> struct LaneAddr<16 + 2> : LaneAddr<1> {};
+template <> struct LaneAddr<16 + 4> : LaneAddr<2> {};
+template <> struct LaneAddr<16 + 8> : LaneAddr<4> {};
+
 template <int SPS, int BT, int HALF = 0>
-__device__ __forceinline__ void compute_item(const ItemRegs<SPS> &r, const LaneAddr<BT> &la, float (&out)[BT])
+__device__ __forceinline__ void compute_item(const ItemRegs<SPS> &r, const LaneAddr<BT> &la, float (&out)[nvec(BT)])
 {
     constexpr int NSEG = 32 / SPS;
+    constexpr int NV = nvec(BT);
     const uint32_t w[8] = {r.b0.x, r.b0.y, r.b0.z, r.b0.w, r.b1.x, r.b1.y, r.b1.z, r.b1.w};
 #pragma unroll
-    for (int b = 0; b < BT; ++b) out[b] = 0.f;
+    for (int b = 0; b < NV; ++b) out[b] = 0.f;
 #pragma unroll
     for (int j = 0; j < NSEG; ++j) {
-        float seg[BT];
+        float seg[NV];
         {
             // (a packed add.f32x2 for two lookups was measured 2 % slower: the pairing costs a MOV per lookup)
-            float s0[BT], s1[BT];
+            float s0[NV], s1[NV];
 #pragma unroll
-            for (int b = 0; b < BT; ++b) { s0[b] = 0.f; s1[b] = 0.f; }
+            for (int b = 0; b < NV; ++b) { s0[b] = 0.f; s1[b] = 0.f; }
 #pragma unroll
             for (int q = 0; q < SPS; ++q) {
                 const int s = j * SPS + q;
                 const uint32_t addr = la.addr(s, w[s >> 2]);
-                Vec<BT> e = lds_entry<BT, HALF>(addr);
+                if constexpr (half_tables(BT)) {
+                    uint32_t e[geom(BT)];
+                    lds_entry_h<BT, HALF>(addr, e);
 #pragma unroll
-                for (int b = 0; b < BT; ++b) {
-                    if (q & 1) s1[b] += e.v[b]; else s0[b] += e.v[b];
+                    for (int i = 0; i < geom(BT); ++i) {
+                        if (q & 1) add_h2(s1[2 * i], s1[2 * i + 1], e[i]); else add_h2(s0[2 * i], s0[2 * i + 1], e[i]);
+                    }
+                } else {
+                    Vec<BT> e = lds_entry<BT, HALF>(addr);
+#pragma unroll
+                    for (int b = 0; b < NV; ++b) {
+                        if (q & 1) s1[b] += e.v[b]; else s0[b] += e.v[b];
+                    }
                 }
             }
 #pragma unroll
-            for (int b = 0; b < BT; ++b) seg[b] = s0[b] + s1[b];
+            for (int b = 0; b < NV; ++b) seg[b] = s0[b] + s1[b];
         }
         float scale = h2f((r.sc[j >> 1] >> ((j & 1) * 16)) & 0xffffu);
 #pragma unroll
-        for (int b = 0; b < BT; ++b) out[b] = fmaf(scale, seg[b], out[b]);
+        for (int b = 0; b < NV; ++b) out[b] = fmaf(scale, seg[b], out[b]);
     }
 }
 
@@ -436,10 +490,10 @@ __device__ __forceinline__ void compute_half(const uint4 &b, const uint32_t *sc,
 template <int SPS, int BT>
 __device__ __forceinline__ void finish_item(const ItemRegs<SPS> &r, const LaneAddr<BT> &la, float *accp, int Mpad)
 {
-    float out[BT];
+    float out[nvec(BT)];
     compute_item<SPS, BT>(r, la, out);
 #pragma unroll
-    for (int b = 0; b < BT; ++b) red_add_f32(accp + (int64_t)b * Mpad, out[b]);
+    for (int b = 0; b < nvec(BT); ++b) red_add_f32(accp + (int64_t)b * Mpad, out[b]);
 }
 
 // The first item of this warp's run, loaded ahead of the table build so that its latency hides
@@ -655,7 +709,8 @@ __device__ __forceinline__ void reduce_and_store(const LinearEntry &E, int nb, i
         // all rows of all completed tiles in one flat loop of 4-row groups, four 128-bit loads in
         // flight per thread (the accumulators live in L2; one round trip serves ~8K rows per CTA)
         const int gpt = E.tile_rb * 8;                 // 4-row groups per tile
-        const int total = ndone * gpt * BT;
+        constexpr int NV = nvec(BT);
+        const int total = ndone * gpt * NV;
         constexpr int U = 4;
         for (int base = tid; base < total; base += U * kThreads) {
             float4 v[U];
@@ -666,7 +721,7 @@ __device__ __forceinline__ void reduce_and_store(const LinearEntry &E, int nb, i
                 int idx = base + u * kThreads;
                 a[u] = nullptr;
                 if (idx < total) {
-                    int li = idx / (gpt * BT), rem = idx - li * (gpt * BT);
+                    int li = idx / (gpt * NV), rem = idx - li * (gpt * NV);
                     bb[u] = rem / gpt;
                     row[u] = (done_list[li] * gpt + (rem - bb[u] * gpt)) * 4;
                     if (row[u] < E.Mpad) a[u] = E.acc + (int64_t)bb[u] * E.Mpad + row[u];
@@ -697,7 +752,7 @@ __device__ __forceinline__ void reduce_and_store(const LinearEntry &E, int nb, i
 #define FB_MINB 3
 #endif
 template <int SPS0, int SPS1, int BT, int NP>
-__global__ void __launch_bounds__(Cfg<BT>::kThreads, (BT == 1) ? FB_MINB : Cfg<BT>::kMinBlocks)
+__global__ void __launch_bounds__(Cfg<BT>::kThreads, (geom(BT) == 1) ? FB_MINB : Cfg<BT>::kMinBlocks)
 fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
 {
     constexpr int kThreads = Cfg<BT>::kThreads, kWarps = Cfg<BT>::kWarps;
@@ -707,13 +762,13 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
     if (smem_base > kTabBase) return;                                    // the host probes this first
     uint8_t *small = smem + (kTabBase - smem_base) + TabCfg<BT>::kTableBytes;
     float *abuf = (float *)small;
-    int *tile_cnt = (int *)(abuf + 256 * BT);
+    int *tile_cnt = (int *)(abuf + 256 * nvec(BT));
     int *done_list = tile_cnt;                     // compacted in place over the counters
     int *range = tile_cnt + kMaxTiles + 4;        // [0]: first item, [1]: end item of this CTA in the entry
     LinearEntry *Es = (LinearEntry *)(range + 8);  // the current entry, copied once (128 bytes)
     static_assert(sizeof(LinearEntry) == 128, "entry copy below moves 32 words");
     static_assert(NP == 1 || BT == 1, "two table sets side by side need the 4-byte slots of BT == 1");
-    static_assert(BT == 1 || BT == 2 || BT == 4, "batch vectors per launch");
+    static_assert(BT == 1 || BT == 2 || BT == 4 || BT == 16 + 2 || BT == 16 + 4 || BT == 16 + 8, "launch mode");
     const int tid = threadIdx.x;
     FB_TRACE_AT(0);
     FB_TRACE_ZERO();

@@ -39,7 +39,7 @@ EXPORTS = ["fluxbin_packed_size", "fluxbin_validate", "fluxbin_pack_host", "flux
            "fluxbin_last_cuda_error", "fluxbin_plan_table_bytes", "fluxbin_plan_workspace_bytes",
            "fluxbin_plan_create", "fluxbin_plan_run", "fluxbin_plan_num_launches", "fluxbin_plan_pairs_per_row_block",
            "fluxbin_plan_free",
-           "fluxbin_linear_noalloc", "fluxbin_noalloc_capacity",
+           "fluxbin_linear_noalloc", "fluxbin_noalloc_capacity", "fluxbin_set_table_format", "fluxbin_get_table_format",
            "fluxbin_rc_decomp", "fluxbin_rc_decomp_workspace_size", "fluxbin_rc_salient_residual"]
 
 _LIB = None
@@ -71,6 +71,8 @@ def _lib():
         lib.fluxbin_debug_tables.argtypes = [vp, vp, i32, vp, vp, vp, vp]
         lib.fluxbin_num_table_sets.restype, lib.fluxbin_num_table_sets.argtypes = i32, [vp]
         lib.fluxbin_num_launches.restype, lib.fluxbin_num_launches.argtypes = i32, [vp, i32]
+        lib.fluxbin_set_table_format.restype, lib.fluxbin_set_table_format.argtypes = ctypes.c_int, [vp, i32]
+        lib.fluxbin_get_table_format.restype, lib.fluxbin_get_table_format.argtypes = i32, [vp]
         lib.fluxbin_free.restype, lib.fluxbin_free.argtypes = None, [vp]
         lib.fluxbin_status_string.restype, lib.fluxbin_status_string.argtypes = ctypes.c_char_p, [ctypes.c_int]
         lib.fluxbin_last_cuda_error.restype, lib.fluxbin_last_cuda_error.argtypes = ctypes.c_int, []
@@ -166,6 +168,9 @@ def unpack_host(buf: np.ndarray):
     return out
 
 
+TABLES_FP32, TABLES_FP16 = 0, 1
+
+
 class Weight:
     """A packed layer resident in device memory (the caller's buffer) plus its handle."""
 
@@ -193,6 +198,13 @@ class Weight:
 
     def num_launches(self, B: int) -> int:
         return int(_lib().fluxbin_num_launches(self.handle, B))
+
+    def set_table_format(self, fmt: int) -> None:
+        """TABLES_FP32 (default) or TABLES_FP16 entries for batched launches; size workspaces afterwards."""
+        _check(_lib().fluxbin_set_table_format(self.handle, fmt), "fluxbin_set_table_format")
+
+    def table_format(self) -> int:
+        return int(_lib().fluxbin_get_table_format(self.handle))
 
 
 def pack(L, d_packed: int, d_bytes: int, stream: int = 0, buffer=None) -> Weight:

@@ -32,6 +32,7 @@ def main():
     ap.add_argument("--copies", type=int, default=3)
     ap.add_argument("--reps", type=int, default=5)
     ap.add_argument("--batch", type=int, default=1)
+    ap.add_argument("--fp16-tables", action="store_true", help="fp16 lookup-table entries for batched launches")
     ap.add_argument("--g", type=int, default=128)
     ap.add_argument("--variant", default=None, choices=["2b", "2b-s8", "2b-s16", "4b"],
                     help="one of the paper's deployed formats at --shape MxN instead of a workload linear: "
@@ -53,7 +54,7 @@ def main():
         else:
             L = synth.make_config_linear(args.config, c, args.linear, g=args.g)
             x = synth.make_config_activations(args.config, c, args.linear, args.batch)
-        lin = fb_layer.FluxBinLinear(L)
+        lin = fb_layer.FluxBinLinear(L, fp16_tables=args.fp16_tables)
         xt = torch.from_numpy(x.view(np.float16)).cuda()
         y = torch.empty((args.batch, L.M), dtype=torch.float16, device="cuda")
         lins.append((lin, xt, y))

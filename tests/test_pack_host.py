@@ -121,6 +121,8 @@ def test_validation_statuses():
     assert lib.fluxbin_packed_dims(corrupt.ctypes.data, corrupt.size, ctypes.byref(fluxbin.LayerDesc())) == 9
     assert lib.fluxbin_linear(None, None, 1, 0, None, 0, 0, None, 0, None) == 1
     assert lib.fluxbin_workspace_size(None, 1) == 0
+    assert lib.fluxbin_set_table_format(None, 1) == 1 and lib.fluxbin_get_table_format(None) == -1
+    assert lib.fluxbin_num_launches(None, 4) == -1
 
 
 def test_packed_bytes_track_the_storage_model():
