@@ -280,8 +280,9 @@ fluxbin_status_t fluxbin_plan_run(const fluxbin_plan_t *plan, void *cuda_stream)
 int32_t fluxbin_plan_num_launches(const fluxbin_plan_t *plan);
 
 /* Introspection: how many table sets (pairs of 16-sub-vector units) the plan's kernel keeps resident per row
- * block -- 2 when every member has an even number of global pairs, the batch is 1 and each CTA's share of the
- * plan is worth at least about 30 items (then two pairs' row sums share one reduction, stage (iii)), else 1.
+ * block -- 2 when every member has an even number of global pairs, the table entries are 4 bytes (batch 1, or
+ * batch 2 with fp16 entries) and each CTA's share of the plan is worth at least about 30 items (then two pairs'
+ * row sums share one reduction, stage (iii)), else 1.
  * Both variants compute the same sums (Eq. 15) in a different order.  -1 on NULL. */
 int32_t fluxbin_plan_pairs_per_row_block(const fluxbin_plan_t *plan);
 

@@ -62,7 +62,7 @@ template <int S0, int S1, int BT> cudaError_t opt_in()
     cudaError_t e = cudaFuncSetAttribute(fbk::fluxbin_linear_kernel<S0, S1, BT, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)fbk::smem_bytes<BT>());
     if (e != cudaSuccess) return e;
-    if constexpr (BT == 1)
+    if constexpr (fbk::geom(BT) == 1)
         e = cudaFuncSetAttribute(fbk::fluxbin_linear_kernel<S0, S1, BT, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)fbk::smem_bytes<BT>());
     return e;
@@ -291,7 +291,7 @@ static cudaError_t launch_shape(long long total_cost, int num_sms, long long ite
     out->grid = grid;
     // two pairs per row block when every layer allows it (couple_cost > 0: even pair counts everywhere) and a
     // CTA's share is large enough to pay for the second table build
-    out->couples = BT == 1 && couple_cost > 0 && out->static_cost / grid >= FB_NP2_MIN;
+    out->couples = fbk::geom(BT) == 1 && couple_cost > 0 && out->static_cost / grid >= FB_NP2_MIN;
     return cudaSuccess;
 }
 
@@ -318,7 +318,7 @@ static cudaError_t launch(const fbk::LaunchParams &p, int num_sms, long long ite
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if constexpr (BT == 1) {
+    if constexpr (fbk::geom(BT) == 1) {
         if (couples) return cudaLaunchKernelEx(&cfg, fbk::fluxbin_linear_kernel<S0, S1, BT, 2>, q);
     }
     return cudaLaunchKernelEx(&cfg, fbk::fluxbin_linear_kernel<S0, S1, BT, 1>, q);
@@ -336,7 +336,7 @@ template <int BT> static cudaError_t launch_bt(int s0, int s1, int num_sms, cons
 }
 
 // mode: 1, 2, 4 vectors with fp32 tables, 16 + (2, 4, 8) vectors with fp16 tables; the two-pair kernel exists
-// for mode 1 only (couple_cost is ignored elsewhere)
+// for the modes with 4-byte table entries (1 and 16 + 2; couple_cost is ignored elsewhere)
 static cudaError_t launch_mode(int mode, int s0, int s1, int num_sms, const fbk::LaunchParams &p, long long items,
                                long long couple_cost, cudaStream_t s)
 {
@@ -344,7 +344,7 @@ static cudaError_t launch_mode(int mode, int s0, int s1, int num_sms, const fbk:
     case 1: return launch_bt<1>(s0, s1, num_sms, p, items, couple_cost, s);
     case 2: return launch_bt<2>(s0, s1, num_sms, p, items, 0, s);
     case 4: return launch_bt<4>(s0, s1, num_sms, p, items, 0, s);
-    case 16 + 2: return launch_bt<16 + 2>(s0, s1, num_sms, p, items, 0, s);
+    case 16 + 2: return launch_bt<16 + 2>(s0, s1, num_sms, p, items, couple_cost, s);
     case 16 + 4: return launch_bt<16 + 4>(s0, s1, num_sms, p, items, 0, s);
     case 16 + 8: return launch_bt<16 + 8>(s0, s1, num_sms, p, items, 0, s);
     }
@@ -573,23 +573,31 @@ extern "C" fluxbin_status_t fluxbin_plan_run(const fluxbin_plan_t *plan, void *c
 
 extern "C" int32_t fluxbin_plan_num_launches(const fluxbin_plan_t *plan) { return plan ? plan->nchunks : -1; }
 
-// the launch shape of the single-vector kernel family that reads (sps0, sps1) layers
-static cudaError_t launch_shape_bt1(int s0, int s1, long long total_cost, int num_sms, long long items, long long couple_cost,
-                                    LaunchShape *shape)
+// the launch shape of a kernel family with 4-byte table entries that reads (sps0, sps1) layers
+template <int BT>
+static cudaError_t launch_shape_geom1(int s0, int s1, long long total_cost, int num_sms, long long items, long long couple_cost,
+                                      LaunchShape *shape)
 {
-    if (s0 == 16 && s1 == 16) return launch_shape<16, 16, 1>(total_cost, num_sms, items, couple_cost, shape);
-    if (s0 == 16) return launch_shape<16, 1, 1>(total_cost, num_sms, items, couple_cost, shape);
-    if (s0 == 8) return launch_shape<8, 1, 1>(total_cost, num_sms, items, couple_cost, shape);
-    return launch_shape<4, 1, 1>(total_cost, num_sms, items, couple_cost, shape);
+    if (s0 == 16 && s1 == 16) return launch_shape<16, 16, BT>(total_cost, num_sms, items, couple_cost, shape);
+    if (s0 == 16) return launch_shape<16, 1, BT>(total_cost, num_sms, items, couple_cost, shape);
+    if (s0 == 8) return launch_shape<8, 1, BT>(total_cost, num_sms, items, couple_cost, shape);
+    return launch_shape<4, 1, BT>(total_cost, num_sms, items, couple_cost, shape);
 }
 
 extern "C" int32_t fluxbin_plan_pairs_per_row_block(const fluxbin_plan_t *plan)
 {
     if (!plan) return -1;
-    if (plan->B != 1) return 1;          // the two-pair kernel exists for single-vector launches only
+    // the two-pair kernel exists for 4-byte table entries only: one vector, or two with fp16 entries
+    const int mode = mode_for(plan->B, plan->table_format);
     LaunchShape shape;
-    if (launch_shape_bt1(plan->sps0, plan->sps1, plan->total_cost, plan->num_sms, plan->items, plan->couple_cost, &shape) != cudaSuccess)
-        return -1;
+    cudaError_t e;
+    if (mode == 1)
+        e = launch_shape_geom1<1>(plan->sps0, plan->sps1, plan->total_cost, plan->num_sms, plan->items, plan->couple_cost, &shape);
+    else if (mode == 16 + 2 && plan->B == 2)
+        e = launch_shape_geom1<16 + 2>(plan->sps0, plan->sps1, plan->total_cost, plan->num_sms, plan->items, plan->couple_cost, &shape);
+    else
+        return 1;
+    if (e != cudaSuccess) return -1;
     return shape.couples ? 2 : 1;
 }
 

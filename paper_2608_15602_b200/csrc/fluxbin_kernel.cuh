@@ -31,6 +31,7 @@
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <type_traits>
 
 #include "fluxbin_layout.h"
 
@@ -420,6 +421,9 @@ template <> struct LaneAddr<16 + 2> : LaneAddr<1> {};
 template <> struct LaneAddr<16 + 4> : LaneAddr<2> {};
 template <> struct LaneAddr<16 + 8> : LaneAddr<4> {};
 
+#ifndef FB_SPLIT_NV
+#define FB_SPLIT_NV 4
+#endif
 template <int SPS, int BT, int HALF = 0>
 __device__ __forceinline__ void compute_item(const ItemRegs<SPS> &r, const LaneAddr<BT> &la, float (&out)[nvec(BT)])
 {
@@ -445,7 +449,8 @@ __device__ __forceinline__ void compute_item(const ItemRegs<SPS> &r, const LaneA
                     lds_entry_h<BT, HALF>(addr, e);
 #pragma unroll
                     for (int i = 0; i < geom(BT); ++i) {
-                        if (q & 1) add_h2(s1[2 * i], s1[2 * i + 1], e[i]); else add_h2(s0[2 * i], s0[2 * i + 1], e[i]);
+                        // (with four or more vectors the adds of one lookup already space out each sum's chain)
+                        if ((q & 1) && NV < FB_SPLIT_NV) add_h2(s1[2 * i], s1[2 * i + 1], e[i]); else add_h2(s0[2 * i], s0[2 * i + 1], e[i]);
                     }
                 } else {
                     Vec<BT> e = lds_entry<BT, HALF>(addr);
@@ -456,7 +461,7 @@ __device__ __forceinline__ void compute_item(const ItemRegs<SPS> &r, const LaneA
                 }
             }
 #pragma unroll
-            for (int b = 0; b < NV; ++b) seg[b] = s0[b] + s1[b];
+            for (int b = 0; b < NV; ++b) seg[b] = (half_tables(BT) && NV >= FB_SPLIT_NV) ? s0[b] : s0[b] + s1[b];
         }
         float scale = h2f((r.sc[j >> 1] >> ((j & 1) * 16)) & 0xffffu);
 #pragma unroll
@@ -484,6 +489,30 @@ __device__ __forceinline__ void compute_half(const uint4 &b, const uint32_t *sc,
         }
         const float scale = h2f((sc[j >> 1] >> ((j & 1) * 16)) & 0xffffu);
         out = fmaf(scale, s0 + s1, out);
+    }
+}
+
+// The same for two batch vectors with fp16 table entries (one 32-bit word per lookup holds both).
+template <int SPS, int HALF, int H>
+__device__ __forceinline__ void compute_half_h2(const uint4 &b, const uint32_t *sc, const LaneAddr<1> &la, float &out0, float &out1)
+{
+    static_assert(SPS >= 2 && SPS <= 16, "segments do not straddle the two halves");
+    constexpr int NSEG_H = 16 / SPS;
+    const uint32_t w[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+    for (int jj = 0; jj < NSEG_H; ++jj) {
+        const int j = H * NSEG_H + jj;
+        float s0 = 0.f, s1 = 0.f, t0 = 0.f, t1 = 0.f;
+#pragma unroll
+        for (int q = 0; q < SPS; ++q) {
+            const int s = j * SPS + q;
+            uint32_t e[1];
+            lds_entry_h<16 + 2, HALF>(la.addr(s, w[(s >> 2) & 3]), e);
+            if (q & 1) add_h2(s1, t1, e[0]); else add_h2(s0, t0, e[0]);
+        }
+        const float scale = h2f((sc[j >> 1] >> ((j & 1) * 16)) & 0xffffu);
+        out0 = fmaf(scale, s0 + s1, out0);
+        out1 = fmaf(scale, t0 + t1, out1);
     }
 }
 
@@ -561,10 +590,19 @@ __device__ __forceinline__ void process_rows(const uint8_t *pair_items, int rb_l
 // for every row block the lane looks up the item of the first pair, then the item of the second
 // (items_b = the second pair's items), adds the two row sums and issues ONE reduction -- half the
 // atomic traffic and half the per-item bookkeeping.  One item is always in flight ahead.
-template <int SPS>
+// BT: 1 (one vector, fp32 entries) or 16 + 2 (two vectors, fp16 entries: the same 4-byte slots).
+template <int SPS, int BT>
 __device__ __forceinline__ void process_rows2(const uint8_t *items_a, const uint8_t *items_b, int rb_lo, int rb_hi,
-                                              const LaneAddr<1> &la, float *acc)
+                                              const LaneAddr<1> &la, float *acc, int Mpad)
 {
+    static_assert(geom(BT) == 1, "two table sets side by side need 4-byte entries");
+    // lookups of one 128-bit half of an item, added to the row sums of the batch vectors
+    auto half = [&](auto set, auto h, const uint4 &b, const uint32_t *sc, float &o0, float &o1) {
+        if constexpr (BT == 1) compute_half<SPS, decltype(set)::value, decltype(h)::value>(b, sc, la, o0);
+        else compute_half_h2<SPS, decltype(set)::value, decltype(h)::value>(b, sc, la, o0, o1);
+    };
+    using I0 = std::integral_constant<int, 0>;
+    using I1 = std::integral_constant<int, 1>;
     constexpr int IB = ItemBytes<SPS>::value;
     constexpr int kWarps = Cfg<1>::kWarps;
     constexpr int STRIDE = kWarps * IB;
@@ -596,28 +634,30 @@ __device__ __forceinline__ void process_rows2(const uint8_t *items_a, const uint
     const int n_pf = lane < 2 * LPI ? n - (kPrefetchTrips + 1) : 0;      // trips in which this lane prefetches
     for (int t = 0; t < n - 1; ++t) {
         prefetch_line_if(pp, t < n_pf);
-        float o = 0.f;
-        compute_half<SPS, 0, 0>(ra.b0, ra.sc, la, o);
+        float o = 0.f, o1 = 0.f;
+        half(I0{}, I0{}, ra.b0, ra.sc, o, o1);
         ra.b0 = ldg_stream_v4(pla + STRIDE);
-        compute_half<SPS, 0, 1>(ra.b1, ra.sc, la, o);
+        half(I0{}, I1{}, ra.b1, ra.sc, o, o1);
         ra.b1 = ldg_stream_v4(pla + STRIDE + 512);
         load_scales<SPS>(ra, psa, STRIDE);
-        compute_half<SPS, 1, 0>(rb.b0, rb.sc, la, o);
+        half(I1{}, I0{}, rb.b0, rb.sc, o, o1);
         rb.b0 = ldg_stream_v4(plb + STRIDE);
-        compute_half<SPS, 1, 1>(rb.b1, rb.sc, la, o);
+        half(I1{}, I1{}, rb.b1, rb.sc, o, o1);
         rb.b1 = ldg_stream_v4(plb + STRIDE + 512);
         load_scales<SPS>(rb, psb, STRIDE);
         red_add_f32(accp, o);
+        if constexpr (BT != 1) red_add_f32(accp + Mpad, o1);
         pla += STRIDE; psa += STRIDE; plb += STRIDE; psb += STRIDE; pp += STRIDE;
         accp += kWarps * 32;
     }
     {
-        float o = 0.f;
-        compute_half<SPS, 0, 0>(ra.b0, ra.sc, la, o);
-        compute_half<SPS, 0, 1>(ra.b1, ra.sc, la, o);
-        compute_half<SPS, 1, 0>(rb.b0, rb.sc, la, o);
-        compute_half<SPS, 1, 1>(rb.b1, rb.sc, la, o);
+        float o = 0.f, o1 = 0.f;
+        half(I0{}, I0{}, ra.b0, ra.sc, o, o1);
+        half(I0{}, I1{}, ra.b1, ra.sc, o, o1);
+        half(I1{}, I0{}, rb.b0, rb.sc, o, o1);
+        half(I1{}, I1{}, rb.b1, rb.sc, o, o1);
         red_add_f32(accp, o);
+        if constexpr (BT != 1) red_add_f32(accp + Mpad, o1);
     }
 }
 
@@ -767,7 +807,7 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
     int *range = tile_cnt + kMaxTiles + 4;        // [0]: first item, [1]: end item of this CTA in the entry
     LinearEntry *Es = (LinearEntry *)(range + 8);  // the current entry, copied once (128 bytes)
     static_assert(sizeof(LinearEntry) == 128, "entry copy below moves 32 words");
-    static_assert(NP == 1 || BT == 1, "two table sets side by side need the 4-byte slots of BT == 1");
+    static_assert(NP == 1 || geom(BT) == 1, "two table sets side by side need 4-byte table entries");
     static_assert(BT == 1 || BT == 2 || BT == 4 || BT == 16 + 2 || BT == 16 + 4 || BT == 16 + 8, "launch mode");
     const int tid = threadIdx.x;
     FB_TRACE_AT(0);
@@ -907,7 +947,7 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
             FB_TRACE_ADD(4, t_build);
             FB_TRACE_T0(t_rows);
             if (region == 0) {
-                if constexpr (NP == 2) process_rows2<SPS0>(items, items_b, rb_lo, rb_hi, la, E.acc);
+                if constexpr (NP == 2) process_rows2<SPS0, BT>(items, items_b, rb_lo, rb_hi, la, E.acc, E.Mpad);
                 else process_rows<SPS0, BT>(items, rb_lo, rb_hi, la, E.acc, E.Mpad, &pre);
             } else {
                 process_rows<SPS1, BT>(items, rb_lo, rb_hi, la, E.acc, E.Mpad);

@@ -177,6 +177,38 @@ def test_plan_with_fp16_tables(fb):
                 check_fp16_tables(y.cpu().numpy(), want, L, x, f"plan B={B} member M={lin.M} rep {rep}")
 
 
+def test_long_plan_of_two_vectors_runs_the_two_pair_kernel(fb):
+    """Two vectors with fp16 entries share the 4-byte table slots of the single-vector kernel, so a plan with
+    enough work per CTA runs the variant that keeps two table sets resident (g = 128 and g = 64 formats)."""
+    for g, shapes in ((128, [(256, 4096), (250, 4096), (512, 4096), (96, 8192)]), (64, [(300, 2048), (512, 4096)])):
+        members, cases = [], []
+        for i in range(72):
+            M, N = shapes[i % len(shapes)]
+            L = layer_of(700 + i, M, N, 2, 1, g, int(round(0.05 * N)))
+            x = synth.make_activations(19, i, 2, N)
+            lin = fb.FluxBinLinear(L, fp16_tables=True)
+            members.append((lin, torch.from_numpy(x.view(np.float16)).cuda(),
+                            torch.full((2, M), float("nan"), dtype=torch.float32, device="cuda")))
+            cases.append((L, x, oracle.linear_direct(L, x)))
+        plan = fb.FluxBinPlan(members)
+        assert plan.pairs_per_row_block() == 2 and plan.num_launches() == 1
+        for rep in range(2):                      # twice: the workspace must come back zeroed
+            for _, _, y in members:
+                y.fill_(float("nan"))
+            plan.run()
+            torch.cuda.synchronize()
+            for (lin, _, y), (L, x, want) in zip(members, cases):
+                check_fp16_tables(y.cpu().numpy(), want, L, x, f"two-pair kernel g={g}, member {lin.M}x{lin.N} rep {rep}", strict=True)
+        short = fb.FluxBinPlan(members[:4])
+        assert short.pairs_per_row_block() == 1
+        for _, _, y in members[:4]:
+            y.fill_(float("nan"))
+        short.run()
+        torch.cuda.synchronize()
+        for (lin, _, y), (L, x, want) in zip(members[:4], cases[:4]):
+            check_fp16_tables(y.cpu().numpy(), want, L, x, f"one-pair kernel g={g}, member {lin.M}x{lin.N}", strict=True)
+
+
 def test_plan_rejects_mixed_table_formats(fb):
     from paper_2608_15602_b200 import fluxbin
     L = layer_of(5, 64, 256, 2, 0, 128, 0)
