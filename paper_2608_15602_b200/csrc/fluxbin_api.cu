@@ -357,6 +357,16 @@ static cudaError_t launch_mode(int mode, int s0, int s1, int num_sms, const fbk:
 // table set (two dependent loads, 8K table entries, two barriers) takes about as long as 22 items
 // (re-measured against the current row loop: 28 / 36 / 44 / 56 -> 5.61 / 5.80 / 5.85 / 5.83 TB/s on the stack plan).
 constexpr int kBuildCost = 44;
+// With four or eight vectors in fp16 table entries an item takes about half the time it takes with fp32 entries,
+// a build (more vectors per entry, conversions) does not: measured 44 / 66 / 88 / 132 -> 3.29 / 3.47 / 3.51 / 3.46
+// TB/s at batch 4 and 1.73 / 1.81 / 1.81 / 1.81 at batch 8.  (With fp32 entries, batch 2 and 4: no effect.)
+#ifndef FB_BCH
+#define FB_BCH 88
+#endif
+static int build_cost_for(int mode)
+{
+    return (mode == 16 + 4 || mode == 16 + 8) ? FB_BCH : kBuildCost;    // two vectors in fp16 entries: 36 / 44 / 56 / 66 all within 1 %
+}
 // The reduction epilogue a CTA runs when it leaves an entry (fence, tickets, read-back of the tiles it
 // completed): a fixed part plus a part that grows with the rows to convert.
 static long long epilogue_cost(const FbHeader &h) { return 80 + h.Mpad / 128; }
@@ -373,12 +383,12 @@ static void item_costs(int sps0, int sps1, int cost[2])
     cost[1] = (sps1 == sps0) ? 2 : 4;
 }
 
-static long long entry_cost(const FbHeader &h, int sps1)
+static long long entry_cost(const FbHeader &h, int sps1, int build_cost)
 {
     int c[2];
     item_costs(h.sps[0], sps1, c);
-    return (long long)h.npairs[0] * (kBuildCost + (long long)h.nrb * c[0]) +
-           (long long)h.npairs[1] * (kBuildCost + (long long)h.nrb * c[1]) + epilogue_cost(h);
+    return (long long)h.npairs[0] * (build_cost + (long long)h.nrb * c[0]) +
+           (long long)h.npairs[1] * (build_cost + (long long)h.nrb * c[1]) + epilogue_cost(h);
 }
 
 static void fill_entry(fbk::LinearEntry &E, const fluxbin_weight_t *w, const uint16_t *x, int64_t ldx, void *y, int64_t ldy,
@@ -411,8 +421,6 @@ extern "C" fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint
     p.y_fp32 = y_is_fp32 != 0;
     const int sps1_eff = w->h.npairs[1] > 0 ? w->h.sps[1] : 1;
     item_costs(w->h.sps[0], sps1_eff, p.item_cost);
-    p.build_cost = kBuildCost;
-    p.total_cost = entry_cost(w->h, sps1_eff);
     const int fmt = w->table_format;
     const int bt_ws = ws_bt(B, fmt);
     float *acc = (float *)d_workspace;
@@ -427,6 +435,8 @@ extern "C" fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint
         fill_entry(p.single, w, d_x + (int64_t)b0 * ldx, ldx, (uint8_t *)d_y + (size_t)b0 * ldy * ysz, ldy, acc, tickets, 0);
         p.nb = nb;
         const int s1 = w->h.npairs[1] > 0 ? w->h.sps[1] : 1;
+        p.build_cost = build_cost_for(mode_for(nb, fmt));
+        p.total_cost = entry_cost(w->h, sps1_eff, p.build_cost);
         cudaError_t e = launch_mode(mode_for(nb, fmt), w->h.sps[0], s1, w->num_sms, p, items, couple_cost_of(w->h), s);
         if (e != cudaSuccess) return cuda_fail(e);
     }
@@ -438,7 +448,8 @@ extern "C" fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint
 struct fluxbin_plan {
     int n, B, y_fp32, nchunks, table_format;
     int sps0, sps1, num_sms;
-    long long total_cost, items, couple_cost;
+    long long total_cost[2], items, couple_cost;     // [0]: every chunk but the last, [1]: the last chunk
+    int build_cost[2];
     int item_cost[2];
     const fbk::LinearEntry *d_table;     // [nchunks][n]
     unsigned *d_counters;
@@ -503,9 +514,12 @@ extern "C" fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_
     const size_t ysz = y_is_fp32 ? 4 : 2;
     fbk::LinearEntry *host = (fbk::LinearEntry *)std::malloc(sizeof(fbk::LinearEntry) * (size_t)n * nchunks);
     if (!host) return FLUXBIN_ERR_UNSUPPORTED;
-    long long cost = 0, items = 0;
+    long long cost = 0, items = 0, cost_first = 0;
+    int bc = kBuildCost, bc_first = kBuildCost;
     for (int c = 0; c < nchunks; ++c) {
         uint8_t *ws = (uint8_t *)d_workspace;
+        if (c == 1) { cost_first = cost; bc_first = bc; }
+        bc = build_cost_for(mode_for(B - c * CH < CH ? B - c * CH : CH, fmt));
         cost = 0;
         items = 0;
         for (int i = 0; i < n; ++i) {
@@ -513,7 +527,7 @@ extern "C" fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_
             unsigned *tickets = (unsigned *)(ws + acc_bytes(w[i], bt));
             fill_entry(host[(size_t)c * n + i], w[i], d_x[i] + (int64_t)c * CH * ldx[i], ldx[i],
                        (uint8_t *)d_y[i] + (size_t)c * CH * ldy[i] * ysz, ldy[i], acc, tickets, cost);
-            cost += entry_cost(w[i]->h, sps1);
+            cost += entry_cost(w[i]->h, sps1, bc);
             items += (long long)(w[i]->h.npairs[0] + w[i]->h.npairs[1]) * w[i]->h.nrb;
             ws += entry_ws_bytes(w[i], bt);
         }
@@ -528,7 +542,8 @@ extern "C" fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_
     if (!p) return FLUXBIN_ERR_UNSUPPORTED;
     p->n = n; p->B = B; p->y_fp32 = y_is_fp32 != 0; p->nchunks = nchunks; p->table_format = fmt;
     p->sps0 = w[0]->h.sps[0]; p->sps1 = sps1; p->num_sms = w[0]->num_sms;
-    p->total_cost = cost; p->items = items;
+    p->total_cost[0] = nchunks > 1 ? cost_first : cost; p->total_cost[1] = cost; p->items = items;
+    p->build_cost[0] = nchunks > 1 ? bc_first : bc; p->build_cost[1] = bc;
     p->couple_cost = 0;
     {
         bool all_even = true;
@@ -556,14 +571,14 @@ extern "C" fluxbin_status_t fluxbin_plan_run(const fluxbin_plan_t *plan, void *c
     p.y_fp32 = plan->y_fp32;
     p.item_cost[0] = plan->item_cost[0];
     p.item_cost[1] = plan->item_cost[1];
-    p.build_cost = kBuildCost;
-    p.total_cost = plan->total_cost;
     p.counters = plan->d_counters;
     for (int c = 0; c < plan->nchunks; ++c) {
         const int CH = chunk_size(plan->table_format);
         const int nb = (plan->B - CH * c < CH) ? plan->B - CH * c : CH;
         p.table = plan->d_table + (size_t)c * plan->n;
         p.nb = nb;
+        p.build_cost = plan->build_cost[c == plan->nchunks - 1];
+        p.total_cost = plan->total_cost[c == plan->nchunks - 1];
         cudaError_t e = launch_mode(mode_for(nb, plan->table_format), plan->sps0, plan->sps1, plan->num_sms, p, plan->items,
                                     plan->couple_cost, s);
         if (e != cudaSuccess) return cuda_fail(e);
@@ -592,9 +607,9 @@ extern "C" int32_t fluxbin_plan_pairs_per_row_block(const fluxbin_plan_t *plan)
     LaunchShape shape;
     cudaError_t e;
     if (mode == 1)
-        e = launch_shape_geom1<1>(plan->sps0, plan->sps1, plan->total_cost, plan->num_sms, plan->items, plan->couple_cost, &shape);
+        e = launch_shape_geom1<1>(plan->sps0, plan->sps1, plan->total_cost[1], plan->num_sms, plan->items, plan->couple_cost, &shape);
     else if (mode == 16 + 2 && plan->B == 2)
-        e = launch_shape_geom1<16 + 2>(plan->sps0, plan->sps1, plan->total_cost, plan->num_sms, plan->items, plan->couple_cost, &shape);
+        e = launch_shape_geom1<16 + 2>(plan->sps0, plan->sps1, plan->total_cost[1], plan->num_sms, plan->items, plan->couple_cost, &shape);
     else
         return 1;
     if (e != cudaSuccess) return -1;
