@@ -263,6 +263,7 @@ def main():
 
     linears, xs_host, alg_bytes = [], [], []
     eff_flops = 0.0
+    lookups = 0
     nthreads = max(1, min(16, (os.cpu_count() or 4) - 1))
     with cf.ThreadPoolExecutor(nthreads) as ex:
         window = []
@@ -281,6 +282,7 @@ def main():
             xs_host.append(x)
             alg_bytes.append(algorithmic_bytes(L.M, L.N, L.Kb, L.Ks, L.g, L.n_sal, B))
             eff_flops += 2.0 * L.M * (L.N + L.n_sal) * B
+            lookups += L.Kb * L.M * (L.N // 8) + L.Ks * L.M * ((L.n_sal + 7) // 8)      # one per weight byte
             del L
     setup_s = time.perf_counter() - t_setup
 
@@ -528,6 +530,21 @@ def main():
         }
         # the paper's effective-throughput figure: 2 * M * (N + n_sal) * B flops per linear over the measured time
         line["effective_tflops"] = eff_flops / (ms_per_step * 1e-3) / 1e12
+        if B > 1:
+            # Batched launches are bound by shared-memory bandwidth, not HBM: every weight byte costs one table
+            # lookup per chunk of vectors, an entry of 4 bytes (fp32) or 2 bytes (fp16) per vector of the chunk.
+            fp16 = bool(args.fp16_tables)
+            ch = 8 if fp16 else 4
+            nvec = lambda nb: 1 if nb == 1 else 2 if nb == 2 else 4 if nb <= 4 else 8
+            chunks = [min(ch, B - c) for c in range(0, B, ch)]
+            entry_bytes = sum((2 if (fp16 and nb >= 2) else 4) * nvec(nb) for nb in chunks)
+            mhz = clocks.get("sm_mhz") or clocks.get("sm_max_mhz") or 1965.0
+            sms = torch.cuda.get_device_properties(0).multi_processor_count
+            smem_peak = sms * 128 * mhz * 1e6 / 1e9                     # GB/s at 128 B/clk/SM
+            smem_achieved = lookups * entry_bytes / (ms_per_step * 1e-3) / 1e9
+            line["lookup_ceiling"] = {"bound": "smem", "achieved": smem_achieved, "peak": smem_peak, "unit": "GB/s",
+                                      "frac": smem_achieved / smem_peak, "entry_bytes_per_weight_byte": entry_bytes,
+                                      "peak_source": f"{sms} SMs x 128 B/clk at the median SM clock under load ({mhz} MHz)"}
         if not args.no_context:
             line["context_dense_fp16_gemv"] = dense_fp16_gemv_context(lins, nl, B)
         if clocks.get("power_w"):

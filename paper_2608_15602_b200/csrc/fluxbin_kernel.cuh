@@ -277,23 +277,27 @@ __device__ __forceinline__ void build_tables(const BuildInput<BT> &in, float *ab
     }
     __syncthreads();
     const int lane = tid & 31, warp = tid >> 5;
-    constexpr int PW = 256 / Cfg<BT>::kWarps;          // table entries per warp: p = warp*PW + ...
     // EB entries at a time: the high index bits fix a base value, the low LB bits are enumerated by
     // doubling (entry p | 2^n = entry p + 2 a_n), one add per entry.  Up to four batch vectors of an entry are
-    // stored with one instruction (with four, blocks of 8 entries keep the registers in bounds); eight vectors
-    // (fp16 entries) take two passes of four, each filling its half of the 16-byte entries.
-    constexpr int PV = NV < 4 ? NV : 4;                // vectors per pass
+    // stored with one instruction (with four, blocks of 8 entries keep the registers in bounds).  With eight
+    // vectors (fp16 entries) half of the warps fill vectors 0..3 and half vectors 4..7 of all entries -- and
+    // within a warp lanes 8..15 and 24..31 take the other group than lanes 0..7 and 16..23, so that the 8-byte
+    // stores of a warp, 16 bytes apart, cover all 32 banks (two wavefronts per 256 bytes instead of four).
+    constexpr int PV = NV < 4 ? NV : 4;                // vectors per thread
+    constexpr int NG = NV / PV;                        // groups of vectors (1 or 2)
+    constexpr int PW = 256 / (Cfg<BT>::kWarps / NG);   // table entries per warp: p = (warp % (kWarps/NG))*PW + ...
     constexpr int LB = (PV == 4) ? 3 : 4, EB = 1 << LB;
     static_assert(PW % EB == 0, "a warp enumerates whole blocks of entries");
-#pragma unroll 1
-    for (int b0 = 0; b0 < NV; b0 += PV) {
+    {
+        const int wl = NG == 1 ? warp : warp % (Cfg<BT>::kWarps / NG);
+        const int b0 = NG == 1 ? 0 : PV * ((warp / (Cfg<BT>::kWarps / NG)) ^ ((lane >> 3) & 1));
         float a[8][PV];
 #pragma unroll
         for (int n = 0; n < 8; ++n)
 #pragma unroll
             for (int b = 0; b < PV; ++b) a[n][b] = abuf[abuf_index<BT>(lane, n, b0 + b)];
 #pragma unroll 1
-        for (int p0 = warp * PW; p0 < (warp + 1) * PW; p0 += EB) {
+        for (int p0 = wl * PW; p0 < (wl + 1) * PW; p0 += EB) {
             float v[EB][PV];
 #pragma unroll
             for (int b = 0; b < PV; ++b) {
