@@ -15,17 +15,18 @@
 //
 // Weight stream: every item is one contiguous block of memory.  A lane pulls its 32 weight bytes
 // and its row scales straight into registers with 128-bit loads (staging them in shared memory
-// would add traffic to the port the lookups saturate); one lane per warp runs a bulk L2 prefetch
-// a few items ahead so those loads find their lines in L2.
+// would add traffic to the port the lookups saturate); L2 prefetches a trip or two ahead make
+// those loads find their lines in L2.
 //
-// Shared-memory table layout: entry p of table slot sigma lives at  kTabBase + p*256 + sigma*4*BT
-// (BT = 1 or 2 batch vectors per launch, their entries side by side).  A lane at step s reads slot
-// lane ^ s, so the 32 lanes of a warp
+// Shared-memory table layout: entry p of table slot sigma lives at  kTabBase + p*256 + sigma*E for
+// entries of E = 4 or 8 bytes (the batch vectors of a launch side by side: 1 or 2 in fp32, 2 or 4 in
+// fp16); 16-byte entries (4 vectors in fp32, 8 in fp16) put slots 16..31 into a second 64 KB half.
+// A lane at step s reads slot lane ^ s, so the 32 lanes of a warp
 // always hit 32 different slots: every lookup is bank-conflict free by construction, and the
 // packer has stored each lane's weight bytes in exactly that order, so the byte of step s sits at
-// a compile-time position.  For BT = 1 the whole address is formed by ONE byte-permute (table
+// a compile-time position.  In every mode the whole address is formed by ONE byte-permute (table
 // index into byte 1, the lane's pre-packed slot offset into byte 0) and the table base rides in
-// the load's immediate: 3 instructions per lookup (PRMT, LDS, FADD).
+// the load's immediate: 3 instructions per lookup and vector at batch 1 (PRMT, LDS, FADD).
 #pragma once
 
 #include <cuda_fp16.h>
@@ -149,7 +150,7 @@ __device__ __forceinline__ uint32_t ldg_stream_u32(const void *p)
 
 template <int BT> struct Vec { float v[nvec(BT)]; };
 
-// HALF selects the table set inside the 256-byte p-rows: slots 0..31 or (BT == 1 only) slots 32..63.
+// HALF selects the table set inside the 256-byte p-rows: slots 0..31 or (4-byte entries only) slots 32..63.
 template <int BT, int HALF> __device__ __forceinline__ Vec<BT> lds_entry(uint32_t addr)
 {
     Vec<BT> r;
@@ -590,7 +591,7 @@ __device__ __forceinline__ void process_rows(const uint8_t *pair_items, int rb_l
     }
 }
 
-// The same for TWO pairs whose table sets are resident together (slots 0..31 and 32..63, BT == 1):
+// The same for TWO pairs whose table sets are resident together (slots 0..31 and 32..63, 4-byte entries):
 // for every row block the lane looks up the item of the first pair, then the item of the second
 // (items_b = the second pair's items), adds the two row sums and issues ONE reduction -- half the
 // atomic traffic and half the per-item bookkeeping.  One item is always in flight ahead.
@@ -864,7 +865,7 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
         if (tid < 32) ((uint32_t *)Es)[tid] = ((const uint32_t *)src)[tid];
         __syncthreads();
         const LinearEntry &E = *Es;
-        // With NP == 2 region 0 is walked two pairs at a time, their table sets side by side (BT == 1,
+        // With NP == 2 region 0 is walked two pairs at a time, their table sets side by side (4-byte entries,
         // every entry with an even number of global pairs): a "work pair" is then a couple of pairs, a
         // work row block their two items.  Costs per pair are unchanged, only the cut granularity doubles.
         // (NP is a kernel template parameter: the host picks the two-pair kernel unless a CTA's share is
