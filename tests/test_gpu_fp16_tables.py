@@ -219,3 +219,32 @@ def test_plan_rejects_mixed_table_formats(fb):
         fb.FluxBinPlan([(a, x, ya), (b, x, yb)])
     with pytest.raises(fluxbin.FluxBinError):
         a.weight.set_table_format(7)
+
+
+@pytest.mark.parametrize("case", range(16))
+def test_random_single_calls(fb, case):
+    """Seeded random shapes, group sizes, base counts, salient maps (none, random, every column, one group only),
+    batch sizes 2..20 and activation outliers."""
+    from test_gpu_random import random_layer
+    r = np.random.default_rng(260815602 + 3000 + case)
+    L = random_layer(r, 9000 + case)
+    B = int(r.integers(2, 21))
+    x = synth.make_activations(9000 + case, 3, B, L.N, outlier_frac=float(r.choice([0.0, 0.02])))
+    check_fp16_tables(run(fb, L, x), oracle.linear_direct(L, x), L, x,
+                      f"case {case}: M={L.M} N={L.N} g={L.g} Kb={L.Kb} Ks={L.Ks} n_sal={L.n_sal} B={B}")
+
+
+def test_entries_beyond_the_fp16_range_saturate(fb):
+    """The documented limit of the mode: a table entry is a sum of 8 fused activations rounded to fp16, so with
+    activations of 6e4 and column scales near 1 the entries overflow to infinity and the outputs are not finite;
+    the fp32 entries of the default mode hold the same sums."""
+    L = layer_of(77, 64, 256, 2, 0, 128, 0)
+    L.col_scale[:] = np.float16(1.0).view(np.uint16)
+    x = np.full((2, 256), np.float16(6.0e4).view(np.uint16), np.uint16)
+    xt = torch.from_numpy(x.view(np.float16)).cuda()
+    lin32, lin16 = fb.FluxBinLinear(L), fb.FluxBinLinear(L, fp16_tables=True)
+    y32 = lin32.forward(xt, lin32.workspace(2), fp32_out=True).cpu().numpy()
+    y16 = lin16.forward(xt, lin16.workspace(2), fp32_out=True).cpu().numpy()
+    want = oracle.linear_direct(L, x)
+    assert np.isfinite(y32).all() and np.allclose(y32, want, rtol=1e-4, atol=1e-4 * np.abs(want).max())
+    assert not np.isfinite(y16).all()
