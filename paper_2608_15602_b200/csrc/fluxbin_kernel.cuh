@@ -429,6 +429,8 @@ template <> struct LaneAddr<16 + 8> : LaneAddr<4> {};
 #ifndef FB_SPLIT_NV
 #define FB_SPLIT_NV 4
 #endif
+// Two alternating partial sums per vector shorten the dependency chain of a segment's adds; with four or more
+// vectors the adds of one lookup already space out each vector's chain (+1-5 % without the split there).
 template <int SPS, int BT, int HALF = 0>
 __device__ __forceinline__ void compute_item(const ItemRegs<SPS> &r, const LaneAddr<BT> &la, float (&out)[nvec(BT)])
 {
@@ -454,19 +456,18 @@ __device__ __forceinline__ void compute_item(const ItemRegs<SPS> &r, const LaneA
                     lds_entry_h<BT, HALF>(addr, e);
 #pragma unroll
                     for (int i = 0; i < geom(BT); ++i) {
-                        // (with four or more vectors the adds of one lookup already space out each sum's chain)
                         if ((q & 1) && NV < FB_SPLIT_NV) add_h2(s1[2 * i], s1[2 * i + 1], e[i]); else add_h2(s0[2 * i], s0[2 * i + 1], e[i]);
                     }
                 } else {
                     Vec<BT> e = lds_entry<BT, HALF>(addr);
 #pragma unroll
                     for (int b = 0; b < NV; ++b) {
-                        if (q & 1) s1[b] += e.v[b]; else s0[b] += e.v[b];
+                        if ((q & 1) && NV < FB_SPLIT_NV) s1[b] += e.v[b]; else s0[b] += e.v[b];
                     }
                 }
             }
 #pragma unroll
-            for (int b = 0; b < NV; ++b) seg[b] = (half_tables(BT) && NV >= FB_SPLIT_NV) ? s0[b] : s0[b] + s1[b];
+            for (int b = 0; b < NV; ++b) seg[b] = (NV >= FB_SPLIT_NV) ? s0[b] : s0[b] + s1[b];
         }
         float scale = h2f((r.sc[j >> 1] >> ((j & 1) * 16)) & 0xffffu);
 #pragma unroll
