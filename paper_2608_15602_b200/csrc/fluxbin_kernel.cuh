@@ -908,6 +908,12 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
             fetch_build_input<BT>(in, desc, E.x, E.ldx, P.nb, region ? -1 : (2 * pair) / E.Kb * 128,
                                   (2 * pair + 1) / E.Kb * 128, E.N);
         };
+        // With 16-byte entries one CTA owns the SM, so nothing covers the load latency of a build's inputs: the
+        // inputs of the CTA's next pair are requested before the rows of the current one (+2 % at batch 8 with
+        // fp16 entries; with two or three CTAs per SM the others cover it and the extra registers only cost).
+        constexpr bool kNextInputsEarly = geom(BT) == 4;
+        BuildInput<BT> bin_next;
+        bool have_next = false;
         while (cur < end) {
             const int region = cur >= I0;
             const int local = region ? cur - I0 : cur;
@@ -937,8 +943,12 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
             // (fetching the next pair's inputs ahead of the lookups was measured 15 % slower: the extra
             // live registers push the lookup loop over the 80-register budget of 3 CTAs per SM)
             BuildInput<BT> bin, bin_b;
-            fetch_for(region, pair, bin);
-            if (np == 2) fetch_for(region, pair + 1, bin_b);
+            if constexpr (kNextInputsEarly) {
+                if (have_next) bin = bin_next; else fetch_for(region, pair, bin);
+            } else {
+                fetch_for(region, pair, bin);
+                if (np == 2) fetch_for(region, pair + 1, bin_b);
+            }
             // region 0, one pair at a time (short runs): first item in flight during the build.  (With two
             // pairs per row block the runs are long and the extra live registers cost more than they hide.)
             ItemRegs<SPS0> pre;
@@ -950,6 +960,11 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
             // serial path of the next build) start moving into L2 now (+0.5 to 0.8 % in every launch mode)
             if (tid < 8 * np && pair + np < E.npairs[region])
                 prefetch_line_if(E.packed + E.off_coldesc + (size_t)((region ? E.npairs[0] : 0) + pair + np) * FB_PAIR_DESC_BYTES + tid * 128, true);
+            if constexpr (kNextInputsEarly) {
+                // the CTA's next segment is the next pair of this entry's global region: its inputs start moving now
+                have_next = seg_end < end && seg_end < I0;
+                if (have_next) fetch_for(0, pair + 1, bin_next);
+            }
             FB_TRACE_ADD(4, t_build);
             FB_TRACE_T0(t_rows);
             if (region == 0) {
