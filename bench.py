@@ -536,7 +536,13 @@ def main():
             fp16 = bool(args.fp16_tables)
             ch = 8 if fp16 else 4
             nvec = lambda nb: 1 if nb == 1 else 2 if nb == 2 else 4 if nb <= 4 else 8
-            chunks = [min(ch, B - c) for c in range(0, B, ch)]
+            chunks = [ch] * (B // ch)
+            rest = B % ch
+            if rest:                                                      # the library's rule for the last chunk
+                big = packed_bytes >= (128 << 20)
+                first = 2 if (big and not fp16 and rest == 3) else 4 if (big and fp16 and rest in (5, 6)) else rest
+                chunks += [first] + ([rest - first] if first < rest else [])
+            assert len(chunks) == launches_per_step or args.launch != "stack"
             entry_bytes = sum((2 if (fp16 and nb >= 2) else 4) * nvec(nb) for nb in chunks)
             mhz = clocks.get("sm_mhz") or clocks.get("sm_max_mhz") or 1965.0
             sms = torch.cuda.get_device_properties(0).multi_processor_count

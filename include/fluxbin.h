@@ -179,7 +179,7 @@ fluxbin_status_t fluxbin_workspace_init(void *d_workspace, size_t bytes, void *c
  * Asynchronous on cuda_stream; performs no allocation and no synchronisation, so calls can be
  * captured into a CUDA graph.  The kernel is launched with programmatic stream serialization: it may
  * begin (index arithmetic, L2 prefetch of its weights) while the previous kernel on the stream is
- * draining, and waits on the device before it reads d_x or touches the workspace.  B >= 1 arbitrary (processed in chunks of up to 4 vectors, 8 with fp16 table entries).  Calls
+ * draining, and waits on the device before it reads d_x or touches the workspace.  B >= 1 arbitrary (processed in chunks of up to 4 vectors, 8 with fp16 table entries; a last chunk that would carry dead vectors in its table entries -- 3 vectors with fp32 entries, 5 or 6 with fp16 entries -- is cut into two launches when the layer, or the plan, holds at least 128 MiB of packed weights).  Calls
  * sharing a workspace must be ordered on one stream.  Accumulation is fp32 with fp32 atomics
  * across K slices, so results may differ in the last bits from run to run.
  */
@@ -231,7 +231,8 @@ fluxbin_status_t fluxbin_debug_tables(const fluxbin_weight_t *w, const uint16_t 
 /* Number of table sets (global + salient) of a layer; -1 on NULL. */
 int32_t fluxbin_num_table_sets(const fluxbin_weight_t *w);
 
-/* Kernel launches fluxbin_linear issues for this layer and batch size (for launch accounting). */
+/* Kernel launches fluxbin_linear issues for this layer and batch size (for launch accounting): one per chunk of
+ * batch vectors, see fluxbin_linear. */
 int32_t fluxbin_num_launches(const fluxbin_weight_t *w, int32_t B);
 
 /* Release the host object (never touches device memory).  NULL is allowed. */
@@ -276,13 +277,13 @@ fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_t *const *w
  */
 fluxbin_status_t fluxbin_plan_run(const fluxbin_plan_t *plan, void *cuda_stream);
 
-/* Kernel launches one fluxbin_plan_run issues (one per chunk of up to 4 batch vectors, 8 with fp16 table entries); -1 on NULL. */
+/* Kernel launches one fluxbin_plan_run issues (one per chunk of batch vectors, see fluxbin_linear); -1 on NULL. */
 int32_t fluxbin_plan_num_launches(const fluxbin_plan_t *plan);
 
-/* Introspection: how many table sets (pairs of 16-sub-vector units) the plan's kernel keeps resident per row
- * block -- 2 when every member has an even number of global pairs, the table entries are 4 bytes (batch 1, or
- * batch 2 with fp16 entries) and each CTA's share of the plan is worth at least about 30 items (then two pairs'
- * row sums share one reduction, stage (iii)), else 1.
+/* Introspection: how many table sets (pairs of 16-sub-vector units) the kernel of the plan's first launch keeps
+ * resident per row block -- 2 when every member has an even number of global pairs, the table entries are 4 bytes
+ * (batch 1, or batch 2 with fp16 entries) and each CTA's share of the plan is worth at least about 30 items (then
+ * two pairs' row sums share one reduction, stage (iii)), else 1.
  * Both variants compute the same sums (Eq. 15) in a different order.  -1 on NULL. */
 int32_t fluxbin_plan_pairs_per_row_block(const fluxbin_plan_t *plan);
 

@@ -217,15 +217,52 @@ extern "C" int32_t fluxbin_get_table_format(const fluxbin_weight_t *w) { return 
 // (LDS.32 / .64 / .128): the weights stream once per chunk and one address computation serves the whole
 // entry.  A single vector always uses fp32 entries (nothing to share a word with).
 static int chunk_size(int fmt) { return fmt == FLUXBIN_TABLES_FP16 ? 8 : 4; }
-static int num_chunks(int B, int fmt) { return (B + chunk_size(fmt) - 1) / chunk_size(fmt); }
 static int nvec_for(int nb) { return nb == 1 ? 1 : nb == 2 ? 2 : nb <= 4 ? 4 : 8; }
 static int mode_for(int nb, int fmt) { return (fmt == FLUXBIN_TABLES_FP16 && nb >= 2) ? 16 + nvec_for(nb) : nvec_for(nb); }
 static int ws_bt(int B, int fmt) { return nvec_for(B < chunk_size(fmt) ? B : chunk_size(fmt)); }   // accumulator rows per layer
 
+// The chunks of a batch of B vectors, largest first: full chunks, then the rest.  A rest that would run with
+// dead vectors in its entries (3 with fp32 entries; 5 or 6 with fp16 entries) is cut once more (2 + 1, 4 + 1,
+// 4 + 2) when the launch streams enough weight bytes for the second pass to cost less than the dead vectors do
+// (measured on a 16-layer 70B-shaped stack: 12 %, 16 % and 11 % faster; an extra launch costs a few microseconds,
+// about what 32 MB of weights take).
+constexpr long long kSplitRestBytes = 128ll << 20;
+struct Chunks {
+    int n = 0;
+    int nb[4] = {0, 0, 0, 0};       // sizes of the chunks after the full ones
+    int full = 0;                   // number of full chunks (of chunk_size vectors)
+    int rest_n = 0;
+};
+static Chunks chunks_of(int B, int fmt, long long weight_bytes)
+{
+    Chunks c;
+    const int CH = chunk_size(fmt);
+    c.full = B / CH;
+    const int r = B % CH;
+    const bool big = weight_bytes >= kSplitRestBytes;
+    if (r > 0) {
+        int first = r;
+        if (big && fmt != FLUXBIN_TABLES_FP16 && r == 3) first = 2;
+        if (big && fmt == FLUXBIN_TABLES_FP16 && (r == 5 || r == 6)) first = 4;
+        c.nb[c.rest_n++] = first;
+        if (first < r) c.nb[c.rest_n++] = r - first;
+    }
+    c.n = c.full + c.rest_n;
+    return c;
+}
+// size and first vector of chunk i
+static int chunk_nb(const Chunks &c, int fmt, int i) { return i < c.full ? chunk_size(fmt) : c.nb[i - c.full]; }
+static int chunk_begin(const Chunks &c, int fmt, int i)
+{
+    int b = (i < c.full ? i : c.full) * chunk_size(fmt);
+    for (int j = c.full; j < i; ++j) b += c.nb[j - c.full];
+    return b;
+}
+
 extern "C" int32_t fluxbin_num_launches(const fluxbin_weight_t *w, int32_t B)
 {
     if (!w || B < 1) return -1;
-    return num_chunks(B, w->table_format);
+    return chunks_of(B, w->table_format, (long long)w->h.total_bytes).n;
 }
 
 // ---- workspace ----------------------------------------------------------------------------------
@@ -429,9 +466,9 @@ extern "C" fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint
     const long long items = (long long)(w->h.npairs[0] + w->h.npairs[1]) * w->h.nrb;
 
     const size_t ysz = y_is_fp32 ? 4 : 2;
-    const int CH = chunk_size(fmt);
-    for (int b0 = 0; b0 < B; b0 += CH) {
-        const int nb = (B - b0 < CH) ? B - b0 : CH;
+    const Chunks ch = chunks_of(B, fmt, (long long)w->h.total_bytes);
+    for (int c = 0; c < ch.n; ++c) {
+        const int nb = chunk_nb(ch, fmt, c), b0 = chunk_begin(ch, fmt, c);
         fill_entry(p.single, w, d_x + (int64_t)b0 * ldx, ldx, (uint8_t *)d_y + (size_t)b0 * ldy * ysz, ldy, acc, tickets, 0);
         p.nb = nb;
         const int s1 = w->h.npairs[1] > 0 ? w->h.sps[1] : 1;
@@ -448,8 +485,9 @@ extern "C" fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint
 struct fluxbin_plan {
     int n, B, y_fp32, nchunks, table_format;
     int sps0, sps1, num_sms;
-    long long total_cost[2], items, couple_cost;     // [0]: every chunk but the last, [1]: the last chunk
-    int build_cost[2];
+    long long items, couple_cost;
+    std::vector<int> chunk_nb, chunk_build_cost;     // per chunk: vectors, build cost of its kernel's cost model
+    std::vector<long long> chunk_total_cost;
     int item_cost[2];
     const fbk::LinearEntry *d_table;     // [nchunks][n]
     unsigned *d_counters;
@@ -463,7 +501,9 @@ static size_t entry_ws_bytes(const fluxbin_weight_t *w, int bt)
 extern "C" size_t fluxbin_plan_table_bytes(int32_t n, int32_t B)
 {
     if (n < 1 || B < 1) return 0;
-    return (size_t)n * sizeof(fbk::LinearEntry) * (size_t)num_chunks(B, FLUXBIN_TABLES_FP32);   // the format with more chunks
+    // an upper bound over the table formats and the cut of the rest
+    const int most = chunks_of(B, FLUXBIN_TABLES_FP32, kSplitRestBytes).n;
+    return (size_t)n * sizeof(fbk::LinearEntry) * (size_t)most;
 }
 
 extern "C" size_t fluxbin_plan_workspace_bytes(int32_t n, const fluxbin_weight_t *const *w, int32_t B)
@@ -510,40 +550,44 @@ extern "C" fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_
     if (ws_bytes < fluxbin_plan_workspace_bytes(n, w, B)) return FLUXBIN_ERR_BUFFER_TOO_SMALL;
 
     const int fmt = w[0]->table_format;
-    const int nchunks = num_chunks(B, fmt), bt = ws_bt(B, fmt), CH = chunk_size(fmt);
+    long long weight_bytes = 0;
+    for (int i = 0; i < n; ++i) weight_bytes += (long long)w[i]->h.total_bytes;
+    const Chunks ch = chunks_of(B, fmt, weight_bytes);
+    const int nchunks = ch.n, bt = ws_bt(B, fmt);
     const size_t ysz = y_is_fp32 ? 4 : 2;
     fbk::LinearEntry *host = (fbk::LinearEntry *)std::malloc(sizeof(fbk::LinearEntry) * (size_t)n * nchunks);
     if (!host) return FLUXBIN_ERR_UNSUPPORTED;
-    long long cost = 0, items = 0, cost_first = 0;
-    int bc = kBuildCost, bc_first = kBuildCost;
+    fluxbin_plan *p = new (std::nothrow) fluxbin_plan;
+    if (!p) { std::free(host); return FLUXBIN_ERR_UNSUPPORTED; }
+    long long items = 0;
     for (int c = 0; c < nchunks; ++c) {
         uint8_t *ws = (uint8_t *)d_workspace;
-        if (c == 1) { cost_first = cost; bc_first = bc; }
-        bc = build_cost_for(mode_for(B - c * CH < CH ? B - c * CH : CH, fmt));
-        cost = 0;
+        const int nb = chunk_nb(ch, fmt, c), b0 = chunk_begin(ch, fmt, c);
+        const int bc = build_cost_for(mode_for(nb, fmt));
+        long long cost = 0;
         items = 0;
         for (int i = 0; i < n; ++i) {
             float *acc = (float *)ws;
             unsigned *tickets = (unsigned *)(ws + acc_bytes(w[i], bt));
-            fill_entry(host[(size_t)c * n + i], w[i], d_x[i] + (int64_t)c * CH * ldx[i], ldx[i],
-                       (uint8_t *)d_y[i] + (size_t)c * CH * ldy[i] * ysz, ldy[i], acc, tickets, cost);
+            fill_entry(host[(size_t)c * n + i], w[i], d_x[i] + (int64_t)b0 * ldx[i], ldx[i],
+                       (uint8_t *)d_y[i] + (size_t)b0 * ldy[i] * ysz, ldy[i], acc, tickets, cost);
             cost += entry_cost(w[i]->h, sps1, bc);
             items += (long long)(w[i]->h.npairs[0] + w[i]->h.npairs[1]) * w[i]->h.nrb;
             ws += entry_ws_bytes(w[i], bt);
         }
+        p->chunk_nb.push_back(nb);
+        p->chunk_build_cost.push_back(bc);
+        p->chunk_total_cost.push_back(cost);
     }
     cudaStream_t s = (cudaStream_t)cuda_stream;
     cudaError_t e = cudaMemcpyAsync(d_table, host, sizeof(fbk::LinearEntry) * (size_t)n * nchunks, cudaMemcpyHostToDevice, s);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     std::free(host);
-    if (e != cudaSuccess) return cuda_fail(e);
+    if (e != cudaSuccess) { delete p; return cuda_fail(e); }
 
-    fluxbin_plan *p = new (std::nothrow) fluxbin_plan;
-    if (!p) return FLUXBIN_ERR_UNSUPPORTED;
     p->n = n; p->B = B; p->y_fp32 = y_is_fp32 != 0; p->nchunks = nchunks; p->table_format = fmt;
     p->sps0 = w[0]->h.sps[0]; p->sps1 = sps1; p->num_sms = w[0]->num_sms;
-    p->total_cost[0] = nchunks > 1 ? cost_first : cost; p->total_cost[1] = cost; p->items = items;
-    p->build_cost[0] = nchunks > 1 ? bc_first : bc; p->build_cost[1] = bc;
+    p->items = items;
     p->couple_cost = 0;
     {
         bool all_even = true;
@@ -573,12 +617,11 @@ extern "C" fluxbin_status_t fluxbin_plan_run(const fluxbin_plan_t *plan, void *c
     p.item_cost[1] = plan->item_cost[1];
     p.counters = plan->d_counters;
     for (int c = 0; c < plan->nchunks; ++c) {
-        const int CH = chunk_size(plan->table_format);
-        const int nb = (plan->B - CH * c < CH) ? plan->B - CH * c : CH;
+        const int nb = plan->chunk_nb[c];
         p.table = plan->d_table + (size_t)c * plan->n;
         p.nb = nb;
-        p.build_cost = plan->build_cost[c == plan->nchunks - 1];
-        p.total_cost = plan->total_cost[c == plan->nchunks - 1];
+        p.build_cost = plan->chunk_build_cost[c];
+        p.total_cost = plan->chunk_total_cost[c];
         cudaError_t e = launch_mode(mode_for(nb, plan->table_format), plan->sps0, plan->sps1, plan->num_sms, p, plan->items,
                                     plan->couple_cost, s);
         if (e != cudaSuccess) return cuda_fail(e);
@@ -603,13 +646,13 @@ extern "C" int32_t fluxbin_plan_pairs_per_row_block(const fluxbin_plan_t *plan)
 {
     if (!plan) return -1;
     // the two-pair kernel exists for 4-byte table entries only: one vector, or two with fp16 entries
-    const int mode = mode_for(plan->B, plan->table_format);
+    const int mode = mode_for(plan->chunk_nb[0], plan->table_format);       // the plan's first launch
     LaunchShape shape;
     cudaError_t e;
     if (mode == 1)
-        e = launch_shape_geom1<1>(plan->sps0, plan->sps1, plan->total_cost[1], plan->num_sms, plan->items, plan->couple_cost, &shape);
-    else if (mode == 16 + 2 && plan->B == 2)
-        e = launch_shape_geom1<16 + 2>(plan->sps0, plan->sps1, plan->total_cost[1], plan->num_sms, plan->items, plan->couple_cost, &shape);
+        e = launch_shape_geom1<1>(plan->sps0, plan->sps1, plan->chunk_total_cost[0], plan->num_sms, plan->items, plan->couple_cost, &shape);
+    else if (mode == 16 + 2)
+        e = launch_shape_geom1<16 + 2>(plan->sps0, plan->sps1, plan->chunk_total_cost[0], plan->num_sms, plan->items, plan->couple_cost, &shape);
     else
         return 1;
     if (e != cudaSuccess) return -1;

@@ -147,3 +147,40 @@ def test_plan_rejects_mixed_scale_formats_and_bad_buffers(fb):
     st, h = fluxbin.plan_create_status([a.weight, a.weight], *args, table.data_ptr(), 1024, ws.data_ptr(), 1 << 16)
     assert st == 0
     fluxbin.library().fluxbin_plan_free(h)
+
+
+@pytest.mark.parametrize("B,fp16,launches", [(3, False, 2), (7, False, 3), (5, True, 2), (6, True, 2), (13, True, 3), (7, True, 1)])
+def test_large_plans_cut_a_rest_with_dead_vectors_once_more(fb, B, fp16, launches):
+    """A plan that streams at least 128 MiB of packed weights runs a rest of 3 vectors (fp32 entries) as 2 + 1 and a
+    rest of 5 or 6 vectors (fp16 entries) as 4 + 1 / 4 + 2; every batch row must still come out right."""
+    from test_gpu_fp16_tables import check_fp16_tables
+    members, cases, nbytes = [], [], 0
+    for i in range(4):
+        L = synth.make_config_linear(4, 1, 4)                    # 28672 x 8192: 65 MB packed each
+        x = synth.make_activations(23, i, B, L.N)
+        lin = fb.FluxBinLinear(L, fp16_tables=fp16)
+        nbytes += lin.packed_bytes
+        members.append((lin, torch.from_numpy(x.view(np.float16)).cuda(),
+                        torch.full((B, L.M), float("nan"), dtype=torch.float32, device="cuda")))
+        if i == 0:
+            cases.append((L, x, oracle.linear_direct(L, x)))
+    assert nbytes >= 128 << 20
+    plan = fb.FluxBinPlan(members)
+    assert plan.num_launches() == launches
+    assert members[0][0].weight.num_launches(B) == ((B + 7) // 8 if fp16 else (B + 3) // 4), "one layer alone stays below the threshold"
+    for rep in range(2):
+        for _, _, y in members:
+            y.fill_(float("nan"))
+        plan.run()
+        torch.cuda.synchronize()
+        assert int(plan.ws.tensor.count_nonzero()) == 0, "workspace must be left zeroed"
+        for _, _, y in members:
+            assert bool(torch.isfinite(y).all()), "every batch row of every member is written"
+        L, x, want = cases[0]
+        got = members[0][2].cpu().numpy()
+        if fp16:
+            check_fp16_tables(got, want, L, x, f"B={B} rep {rep}", strict=True)
+        else:
+            check(got, want, f"B={B} rep {rep}")
+        # the four members hold the same layer: same weights, different activations -> rows must differ between members
+        assert not torch.equal(members[0][2], members[1][2])
