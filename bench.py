@@ -1,20 +1,31 @@
 #!/usr/bin/env python
 """Benchmark of the FluxBin decode linear stack on B200 (one JSON line on stdout).
 
-Workload (N=1): the Llama-2-70B-shaped stack of decode linears -- 80 layers x {q, k, v, o, gate,
+Headline workload (N=1): the Llama-2-70B-shaped stack of decode linears -- 80 layers x {q, k, v, o, gate,
 up, down}, 2 global bases + 1 extra base on a seeded random 5 % of the input columns, g = 128,
 batch 1, fp16 activations, every linear with its own input, all 560 packed layers resident in HBM
 at once (about 21 GB, far larger than L2, so every step streams the weights from HBM).  A "step" is
 one forward token.  --launch says how its 560 linears are launched (replayed from a CUDA graph):
   stack   one fluxbin_plan launch for the whole step (default; the workload gives every linear its own
-          input, so all 560 are independent and the persistent kernel streams them back to back)
+          input, so all 560 are independent and the persistent kernel streams them back to back: the
+          throughput of the kernel, an upper bound for a decoder)
   layer   one plan per layer (80 launches)
-  group   one plan per set of linears a decoder could run together: {q,k,v} {o} {gate,up} {down} (320)
+  group   one plan per set of linears a decoder could run together: {q,k,v} {o} {gate,up} {down} (320):
+          the finest launch structure a real decoder allows; reported in the same line as `group_mode`
   linear  one fluxbin_linear call per linear (560)
 
 value = algorithmic bytes moved per second over all GPUs (GB/s); us_per_layer and us_per_linear
 carry the latency side of the metric.  With --gpus N the N ranks run independent replicas (the
 path has no exchange step): weak scaling, no collective on the data path.
+
+Beside the headline the line carries (rank 0, one GPU; --sections picks them):
+  group_mode  the same stack with one launch per dependency group
+  sustained   the headline launch replayed for at least two seconds under the clock sampler
+  configs     the smaller workloads (one layer, hybrid layer, 7B set, 13B set) in linear / group / stack mode
+              as rotations of copies larger than L2, and the batched cases of the workloads
+  variants    the paper's deployed formats at the shapes of its per-operator latency table, one chained call each
+  rc_decomp   the decomposition step (Algorithm 3) on dense matrices
+  cpu_baseline, context_dense_fp16_gemv
 
 --impl reference times the CPU oracle (oracle/) on a bounded sample of the same workload.
 """
@@ -39,6 +50,8 @@ from paper_2608_15602_b200 import synth  # noqa: E402
 
 METRIC = "decode_linear_stack_effective_hbm_gbps_batch1"
 UNIT = "GB/s"
+L2_BYTES = 126e6
+ALL_SECTIONS = ["group_mode", "sustained", "configs", "variants", "rc_decomp", "context", "cpu_baseline"]
 
 
 def algorithmic_bytes(M, N, Kb, Ks, g, n_sal, B):
@@ -59,7 +72,7 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """nvidia-smi clocks and throttle reasons sampled every 50 ms while the timed region runs."""
+    """nvidia-smi clocks and throttle reasons sampled every 20 ms while a timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
@@ -72,23 +85,33 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "50", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+                                          "-lms", "20", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except OSError:
             self.proc = None
+        return self
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([t.strip() for t in line.split(",")])
+            self.rows.append((time.perf_counter(), [t.strip() for t in line.split(",")]))
 
-    def stop(self):
+    def wait_for_samples(self, n: int, timeout: float = 3.0):
+        """Block until the sampler has delivered n rows (nvidia-smi takes a while to print its first one)."""
+        t0 = time.perf_counter()
+        while self.proc is not None and len(self.rows) < n and time.perf_counter() - t0 < timeout:
+            time.sleep(0.01)
+
+    def stop(self, since: float | None = None):
+        """Summary of the rows sampled after perf_counter() time `since` (all rows if None)."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
         self.thread.join(timeout=2)
         sm, smax, power, reasons = [], [], [], set()
-        for r in self.rows:
+        for ts, r in self.rows:
+            if since is not None and ts < since:
+                continue
             try:
                 sm.append(float(r[0])); smax.append(float(r[1]))
             except (ValueError, IndexError):
@@ -101,24 +124,211 @@ class ClockSampler:
                 if v.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
-                "samples": len(sm), "reasons": sorted(reasons),
+                "sm_mhz_min": min(sm) if sm else None, "samples": len(sm), "reasons": sorted(reasons),
                 # nvidia-smi's power.draw is a moving average over about a second: the largest sample of a
                 # short timed region is still a lower bound of the power under load
                 "power_w": max(power) if power else None}
 
 
-def stack_spec(config: int, layers: int | None):
-    """Linears of one layer (or set) of the workload and how many such layers a step runs.  The single-layer
-    and single-set workloads (configs 0-3) are run as a rotation of independently seeded copies, enough of them
-    that a step streams more than four times the L2 capacity: weights come from HBM, as in decode."""
-    lins, nl = synth.config_linears(config)
-    if layers is not None:
-        nl = layers
-    elif config < 4:
-        set_bytes = sum(M * N for _, M, N in lins) * 2.43 / 8          # about 2.43 bits per weight
-        nl = max(1, int(540e6 // set_bytes) + 1)
-    return lins, nl
+# ---------------------------------------------------------------------------------------------------------
+# resident workloads
+# ---------------------------------------------------------------------------------------------------------
 
+def rotation_copies(set_bytes: float) -> int:
+    """Copies of a layer / set in rotation so that a step streams more than four times the L2 capacity."""
+    return max(1, int(4.3 * L2_BYTES // set_bytes) + 1)
+
+
+class Stack:
+    """Packed linears resident on the device plus activation / output arenas for one batch size.
+
+    members: list of (FluxBinLinear, canonical dims, x fp16 bits [B][N]); `names` the linears of one layer / set in
+    order, `nl` how many such layers the members hold (member index = layer * len(names) + linear)."""
+
+    def __init__(self, members, names, nl, B, fp16_tables=False):
+        import torch
+        from paper_2608_15602_b200 import fluxbin, layer as fb_layer
+        self.names, self.nl, self.B, self.fp16 = names, nl, B, bool(fp16_tables and B > 1)
+        self.linears = [m[0] for m in members]
+        self.dims = [m[1] for m in members]
+        self._fmt_before = [l.weight.table_format() for l in self.linears]
+        for l in self.linears:                      # workspaces and plans are sized after the format is set
+            l.weight.set_table_format(fluxbin.TABLES_FP16 if self.fp16 else fluxbin.TABLES_FP32)
+        self.alg_bytes = [algorithmic_bytes(*d, B) for d in self.dims]
+        self.eff_flops = sum(2.0 * d[0] * (d[1] + d[5]) * B for d in self.dims)
+        self.lookups = sum(d[2] * d[0] * (d[1] // 8) + d[3] * d[0] * ((d[5] + 7) // 8) for d in self.dims)   # one per weight byte
+        self.packed_bytes = sum(l.packed_bytes for l in self.linears)
+        n_in = sum(l.N for l in self.linears) * B
+        n_out = sum(l.M for l in self.linears) * B
+        self.x_host = torch.empty(n_in, dtype=torch.float16).pin_memory()
+        self.y_host = torch.empty(n_out, dtype=torch.float16).pin_memory()
+        off = 0
+        for l, m in zip(self.linears, members):
+            self.x_host[off:off + B * l.N] = torch.from_numpy(m[2].view(np.float16).reshape(-1))
+            off += B * l.N
+        self.x_dev = torch.empty(n_in, dtype=torch.float16, device="cuda")
+        self.y_dev = torch.empty(n_out, dtype=torch.float16, device="cuda")
+        self.x_dev.copy_(self.x_host)
+        self.ws = fb_layer.Workspace(max(l.weight.workspace_size(B) for l in self.linears))
+        self.views = self.make_views(self.x_dev, self.y_dev)
+
+    def make_views(self, x_dev, y_dev):
+        views, ox, oy, B = [], 0, 0, self.B
+        for l in self.linears:
+            views.append((l, x_dev[ox:ox + B * l.N].view(B, l.N), y_dev[oy:oy + B * l.M].view(B, l.M)))
+            ox += B * l.N
+            oy += B * l.M
+        return views
+
+    def restore_formats(self):
+        for l, f in zip(self.linears, self._fmt_before):
+            l.weight.set_table_format(f)
+
+    def groups(self, launch):
+        """Member indices per launch; None = one fluxbin_linear call per member."""
+        nlin, names = len(self.names), self.names
+        if launch == "linear":
+            return None
+        if launch == "group":
+            dep_sets = [["q", "k", "v"], ["o"], ["gate", "up"], ["down"]] if "gate" in names else [[n] for n in names]
+            return [[layer * nlin + names.index(n) for n in ds] for layer in range(self.nl) for ds in dep_sets]
+        if launch == "layer":
+            return [[layer * nlin + li for li in range(nlin)] for layer in range(self.nl)]
+        return [list(range(len(self.linears)))]
+
+    def runner(self, launch, stream, views=None, graph=True):
+        return Runner(self, launch, stream, views if views is not None else self.views, graph)
+
+
+class Runner:
+    """One step of a stack in a launch mode: plans (or plain calls) captured into a CUDA graph."""
+
+    def __init__(self, stack, launch, stream, views, graph=True):
+        import torch
+        from paper_2608_15602_b200 import layer as fb_layer
+        self.stack, self.launch, self.stream, self.views = stack, launch, stream, views
+        groups = stack.groups(launch)
+        self.plans = None if groups is None else [fb_layer.FluxBinPlan([views[i] for i in g]) for g in groups]
+        if self.plans is not None:
+            self.launches_per_step = sum(p.num_launches() for p in self.plans)
+        else:
+            self.launches_per_step = sum(l.weight.num_launches(stack.B) for l in stack.linears)
+        self.graph = None
+        with torch.cuda.stream(stream):
+            self.issue()                                   # first call per device does the one-time set-up
+            stream.synchronize()
+            if graph:
+                self.graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(self.graph, stream=stream):
+                    self.issue()
+
+    def issue(self):
+        if self.plans is not None:
+            for p in self.plans:
+                p.run(stream=self.stream)
+        else:
+            for l, xv, yv in self.views:
+                l.forward(xv, self.stack.ws, out=yv, stream=self.stream)
+
+    def step(self):
+        if self.graph is not None:
+            self.graph.replay()
+        else:
+            self.issue()
+
+    def time(self, steps, warmup, barrier=None):
+        """(total ms, per-step ms) of `steps` steps after `warmup` untimed ones, CUDA events on the launch stream."""
+        import torch
+        with torch.cuda.stream(self.stream):
+            for _ in range(warmup):
+                self.step()
+            (barrier or torch.cuda.synchronize)()
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+            ev[0].record(self.stream)
+            for i in range(steps):
+                self.step()
+                ev[i + 1].record(self.stream)
+            (barrier or torch.cuda.synchronize)()
+        return ev[0].elapsed_time(ev[-1]), [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
+
+
+def generate_members(jobs, make, fp16_tables=False):
+    """(FluxBinLinear, dims, x) per job; generation runs in a thread pool ahead of packing and upload."""
+    from paper_2608_15602_b200 import layer as fb_layer
+    members = []
+    nthreads = max(1, min(16, (os.cpu_count() or 4) - 1))
+    with cf.ThreadPoolExecutor(nthreads) as ex:
+        window, it = [], iter(jobs)
+        for _ in range(2 * nthreads):
+            j = next(it, None)
+            if j is not None:
+                window.append(ex.submit(make, j))
+        while window:
+            L, x = window.pop(0).result()
+            j = next(it, None)
+            if j is not None:
+                window.append(ex.submit(make, j))
+            lin = fb_layer.FluxBinLinear(L, fp16_tables=fp16_tables)
+            members.append((lin, (L.M, L.N, L.Kb, L.Ks, L.g, L.n_sal), x))
+            del L
+    return members
+
+
+def build_config_stack(config, nl, B, g=128, fp16_tables=False):
+    """Workload `config` with nl independently seeded layers / sets (config 4: the layers of the stack)."""
+    lins, _ = synth.config_linears(config)
+    jobs = [(layer, li) for layer in range(nl) for li in range(len(lins))]
+
+    def make(job):
+        layer, li = job
+        return synth.make_config_linear(config, layer, li, g=(g or lins[li][2])), synth.make_config_activations(config, layer, li, B)
+
+    return Stack(generate_members(jobs, make, fp16_tables), [n for n, _, _ in lins], nl, B, fp16_tables)
+
+
+def build_rotation(make_layers, names, B, fp16_tables=False):
+    """A rotation of copies of one set of layers, enough of them that a step streams more than four times L2.
+    The set is generated and packed once; the copies are device-side clones at their own addresses (what the
+    memory system sees is the same as with independently seeded copies: every copy is read once per step)."""
+    from paper_2608_15602_b200 import layer as fb_layer
+    base = []
+    for L, x in make_layers():
+        lin = fb_layer.FluxBinLinear(L, fp16_tables=fp16_tables)
+        base.append((lin, (L.M, L.N, L.Kb, L.Ks, L.g, L.n_sal), x))
+    set_bytes = sum(m[0].packed_bytes for m in base)
+    copies = rotation_copies(set_bytes)
+    members = list(base)
+    for _ in range(copies - 1):
+        members += [(m[0].clone(), m[1], m[2]) for m in base]
+    return Stack(members, names, copies, B, fp16_tables)
+
+
+def lookup_ceiling(stack, ms_per_step, launches_per_step, mhz, launch="stack"):
+    """Batched launches are bound by shared-memory bandwidth, not HBM: every weight byte costs one table lookup
+    per chunk of vectors, an entry of 4 bytes (fp32) or 2 bytes (fp16) per vector of the chunk."""
+    import torch
+    B, fp16 = stack.B, stack.fp16
+    ch = 8 if fp16 else 4
+    nvec = lambda nb: 1 if nb == 1 else 2 if nb == 2 else 4 if nb <= 4 else 8
+    chunks = [ch] * (B // ch)
+    rest = B % ch
+    if rest:                                                      # the library's rule for the last chunk
+        big = stack.packed_bytes >= (128 << 20)
+        first = 2 if (big and not fp16 and rest == 3) else 4 if (big and fp16 and rest in (5, 6)) else rest
+        chunks += [first] + ([rest - first] if first < rest else [])
+    assert len(chunks) == launches_per_step or launch != "stack"
+    entry_bytes = sum((2 if (fp16 and nb >= 2) else 4) * nvec(nb) for nb in chunks)
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    smem_peak = sms * 128 * mhz * 1e6 / 1e9                     # GB/s at 128 B/clk/SM
+    smem_achieved = stack.lookups * entry_bytes / (ms_per_step * 1e-3) / 1e9
+    return {"bound": "smem", "achieved": smem_achieved, "peak": smem_peak, "unit": "GB/s",
+            "frac": smem_achieved / smem_peak, "entry_bytes_per_weight_byte": entry_bytes,
+            "peak_source": f"{sms} SMs x 128 B/clk at {mhz} MHz"}
+
+
+# ---------------------------------------------------------------------------------------------------------
+# baselines and context
+# ---------------------------------------------------------------------------------------------------------
 
 def cpu_oracle_sample(config: int, B: int, max_linears: int = 28, g: int = 128, nl: int | None = None, gpu_y=None):
     """Time the oracle as it stands on the first linears of the stack (bounded sample); returns
@@ -206,6 +416,167 @@ def run_reference(args, rank):
     print(json.dumps(line), flush=True)
 
 
+# ---------------------------------------------------------------------------------------------------------
+# the sections beside the headline
+# ---------------------------------------------------------------------------------------------------------
+
+def summarize(stack, runner, total_ms, step_ms, steps, peak, per="linear"):
+    nbytes = sum(stack.alg_bytes)
+    ms = total_ms / steps
+    n_lin = len(stack.linears)
+    gbps = nbytes / (ms * 1e-3) / 1e9
+    out = {"launch": runner.launch, "launches_per_step": runner.launches_per_step, "batch": stack.B,
+           "table_entries": "fp16" if stack.fp16 else "fp32", "GBps": round(gbps, 1), "frac_of_measured_peak": round(gbps / peak, 4),
+           "frac_of_8TBps": round(gbps / 8000.0, 4), "us_per_linear": round(ms * 1e3 / n_lin, 3),
+           "us_per_set": round(ms * 1e3 / stack.nl, 3), "ms_per_step": round(ms, 4),
+           "step_ms_min": round(min(step_ms), 4), "copies_or_layers": stack.nl,
+           "packed_MB_streamed_per_step": round(stack.packed_bytes / 1e6, 1)}
+    if stack.B > 1:
+        lc = lookup_ceiling(stack, ms, runner.launches_per_step, 1965.0, runner.launch)
+        out["lookup_ceiling_frac_at_1965MHz"] = round(lc["frac"], 4)
+    return out
+
+
+def section_configs(main_stack, stream, peak, steps=20, warmup=3):
+    """Configs 0-3 at batch 1 in every launch mode, and the batched cases of the workloads."""
+    import torch
+    rows = []
+
+    def timed(stack, launch):
+        r = stack.runner(launch, stream)
+        total, step_ms = r.time(steps, warmup)
+        row = summarize(stack, r, total, step_ms, steps, peak)
+        del r
+        return row
+
+    for config in (0, 1, 2, 3):
+        lins, _ = synth.config_linears(config)
+        names = [n for n, _, _ in lins]
+
+        def make_layers(config=config, lins=lins, B=1):
+            return [(synth.make_config_linear(config, 0, li), synth.make_config_activations(config, 0, li, B))
+                    for li in range(len(lins))]
+
+        st = build_rotation(make_layers, names, 1)
+        for launch in (("linear", "stack") if config < 2 else ("linear", "group", "stack")):
+            row = timed(st, launch)
+            row["workload"] = f"config {config}"
+            rows.append(row)
+        del st
+        torch.cuda.empty_cache()
+        batches = {1: (4, 16), 3: (8,)}.get(config, ())
+        for B in batches:
+            for fp16 in (False, True):
+                st = build_rotation(lambda: make_layers(B=B), names, B, fp16_tables=fp16)
+                row = timed(st, "stack")
+                row["workload"] = f"config {config}"
+                rows.append(row)
+                if config == 3:
+                    row = timed(st, "group")
+                    row["workload"] = f"config {config}"
+                    rows.append(row)
+                st.restore_formats()
+                del st
+                torch.cuda.empty_cache()
+    # config 4 (the first 16 layers of the resident stack) at batch 4 and 16
+    nlin = len(main_stack.names)
+    nl16 = min(16, main_stack.nl)
+    for B in (4, 16):
+        for fp16 in (False, True):
+            members = []
+            for i in range(nl16 * nlin):
+                layer, li = divmod(i, nlin)
+                members.append((main_stack.linears[i], main_stack.dims[i], synth.make_config_activations(4, layer, li, B)))
+            st = Stack(members, main_stack.names, nl16, B, fp16_tables=fp16)
+            for launch in ("stack", "group"):
+                row = timed(st, launch)
+                row["workload"] = f"config 4, first {nl16} layers"
+                rows.append(row)
+            st.restore_formats()
+            del st
+            torch.cuda.empty_cache()
+    return {"rows": rows, "how": f"CUDA-graph replay, {warmup} warm-up + {steps} timed steps each, CUDA events; configs 0-3: a step "
+            "runs a rotation of device-resident copies of the layer / set at distinct addresses, more than four times L2 "
+            "in total, so the weights stream from HBM; linear = one fluxbin_linear call per linear (chained on one stream), "
+            "group = one plan per dependency group ({q,k,v} {o} {gate,up} {down}), stack = one plan for all copies "
+            "(throughput); frac_of_measured_peak is against the measured copy rate"}
+
+
+def section_variants(stream, peak, steps=10, warmup=3):
+    """The paper's deployed formats (2b, 2b-s8, 2b-s16, 4b at g = 128) at the shapes of its per-operator latency
+    table: one chained fluxbin_linear call per copy, copies rotating through more than L2."""
+    import torch
+    rows = []
+    for (M, N) in ((4096, 4096), (5120, 5120), (4096, 11008), (5120, 13824)):
+        for variant in ("2b", "2b-s8", "2b-s16", "4b"):
+            Kb = 4 if variant == "4b" else 2
+            s = {"2b": 0, "4b": 0, "2b-s8": 8, "2b-s16": 16}[variant]
+
+            def make_layers(M=M, N=N, Kb=Kb, s=s):
+                idx = synth.salient_per_group(7, 0, N, 128, s) if s else None
+                return [(synth.make_linear(7, 0, M, N, Kb, 2 if s else 0, 128, idx), synth.make_activations(7, 0, 1, N))]
+
+            st = build_rotation(make_layers, ["lin"], 1)
+            for launch in ("linear", "stack"):
+                r = st.runner(launch, stream)
+                total, step_ms = r.time(steps, warmup)
+                row = summarize(st, r, total, step_ms, steps, peak)
+                rows.append({"format": f"{variant}-g128", "shape": f"{M}x{N}", "launch": launch, "us_per_call": row["us_per_linear"],
+                             "GBps": row["GBps"], "frac_of_measured_peak": row["frac_of_measured_peak"],
+                             "effective_tflops": round(st.eff_flops / (total / steps * 1e-3) / 1e12, 2), "copies": st.nl})
+                del r
+            del st
+            torch.cuda.empty_cache()
+    return {"rows": rows, "how": "batch 1; linear = dependent calls chained on one stream (the per-operator latency the paper's "
+            "table reports, its kernels on A100: 41-252 us), stack = the same copies as one plan (throughput); effective_tflops = "
+            "2 M (N + n_sal) / t as in the paper"}
+
+
+def section_rc_decomp(shapes=((4096, 4096), (8192, 8192)), K=2, T=10, g=128):
+    """fluxbin_rc_decomp (Algorithm 3) on seeded dense matrices: ms per call and the rate at which W is streamed."""
+    import torch
+    from paper_2608_15602_b200 import fluxbin
+    rows = []
+    for (M, N) in shapes:
+        copies = max(1, int(3 * L2_BYTES // (4 * M * N))) + 1           # W rotates through more than L2
+        Ws = [torch.from_numpy(synth.make_dense_weight(11, c, M, N, 0.05)).cuda() for c in range(copies)]
+        out = {"bits": torch.empty((K, M, N // 32), dtype=torch.int32, device="cuda"),
+               "row_scale": torch.empty((K, M, N // g), dtype=torch.float16, device="cuda"),
+               "col_scale": torch.empty((K, N), dtype=torch.float16, device="cuda"),
+               "row_scale_f32": torch.empty((K, M, N // g), dtype=torch.float32, device="cuda"),
+               "col_scale_f32": torch.empty((K, N), dtype=torch.float32, device="cuda")}
+        ws = torch.empty(fluxbin.rc_decomp_workspace_size(M, N, g, K), dtype=torch.uint8, device="cuda")
+        stream = int(torch.cuda.current_stream().cuda_stream)
+
+        def call(W):
+            fluxbin.rc_decomp(W.data_ptr(), W.stride(0), M, N, g, K, T, 1e-8, out["bits"].data_ptr(),
+                              out["row_scale"].data_ptr(), out["col_scale"].data_ptr(), out["row_scale_f32"].data_ptr(),
+                              out["col_scale_f32"].data_ptr(), ws.data_ptr(), ws.numel(), stream)
+
+        for W in Ws:
+            call(W)
+        torch.cuda.synchronize()
+        reps = 3
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            for W in Ws:
+                call(W)
+        b.record()
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / (reps * copies)
+        passes = 1 + T * (K + 1)                     # initialisation + per round: one row pass per base, one sign pass
+        rows.append({"shape": f"{M}x{N}", "g": g, "K": K, "T": T, "ms_per_call": round(ms, 4), "passes_over_W": passes,
+                     "us_per_pass": round(ms * 1e3 / passes, 2), "GBps_of_W": round(4.0 * M * N * passes / (ms * 1e-3) / 1e9, 1),
+                     "copies": copies})
+        del Ws, out, ws
+        torch.cuda.empty_cache()
+    return {"rows": rows, "how": "CUDA events around whole calls, matrices rotating through more than L2; every pass reads the "
+            "fp32 matrix once (4 M N algorithmic bytes)"}
+
+
+# ---------------------------------------------------------------------------------------------------------
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -224,10 +595,13 @@ def main():
                          "depend on nothing inside the set ({q,k,v}, {o}, {gate,up}, {down}); layer: one plan per "
                          "layer; stack: one plan for the whole stack (valid because the workload gives every "
                          "linear its own input)")
+    ap.add_argument("--sections", default=None,
+                    help="comma-separated extra sections of the line (default: all at the default workload on one GPU, "
+                         f"none otherwise): {','.join(ALL_SECTIONS)}; 'none' for the headline alone")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-context", action="store_true", help="skip the dense fp16 cuBLAS GEMV context timing")
     ap.add_argument("--ref-linears", type=int, default=7, help="linears per step of --impl reference")
-    ap.add_argument("--per-linear", action="store_true", help="also print per-linear timings to stderr")
+    ap.add_argument("--rc-shape", default=None, help="MxN: run only the rc_decomp section on this shape (profiling)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -242,7 +616,7 @@ def main():
     import torch.distributed as dist
     from paper_2608_15602_b200 import build as fb_build
     fb_build.build()
-    from paper_2608_15602_b200 import fluxbin, layer as fb_layer
+    from paper_2608_15602_b200 import dist_util
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
@@ -250,166 +624,73 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
+    default_workload = (args.config == 4 and args.layers is None and args.batch == 1 and args.g == 128 and args.launch == "stack")
+    if args.sections is None:
+        sections = list(ALL_SECTIONS) if (default_workload and world == 1) else ["context", "cpu_baseline"]
+    else:
+        sections = [] if args.sections == "none" else [s for s in args.sections.split(",") if s]
+        unknown = [s for s in sections if s not in ALL_SECTIONS]
+        if unknown:
+            raise SystemExit(f"unknown sections {unknown}")
+    if args.no_cpu_baseline and "cpu_baseline" in sections:
+        sections.remove("cpu_baseline")
+    if args.no_context and "context" in sections:
+        sections.remove("context")
+    if rank != 0 or world > 1:
+        sections = [s for s in sections if s in ("context", "cpu_baseline")] if rank == 0 else []
+
+    if args.rc_shape:
+        M, N = (int(t) for t in args.rc_shape.lower().split("x"))
+        print(json.dumps({"rc_decomp": section_rc_decomp(shapes=((M, N),))}), flush=True)
+        return
+
     B = args.batch
-    lins, nl = stack_spec(args.config, args.layers)
-    jobs = [(layer, li) for layer in range(nl) for li in range(len(lins))]
+    lins, nl_default = synth.config_linears(args.config)
+    if args.layers is not None:
+        nl = args.layers
+    elif args.config < 4:
+        set_bytes = sum(M * N for _, M, N in lins) * 2.43 / 8          # about 2.43 bits per weight
+        nl = rotation_copies(set_bytes)
+    else:
+        nl = nl_default
 
     # ---- build the resident stack: generate (threads) -> pack on the host -> upload ----------------
     t_setup = time.perf_counter()
-    def gen(job):
-        layer, li = job
-        return job, synth.make_config_linear(args.config, layer, li, g=(args.g or lins[li][2])), \
-            synth.make_config_activations(args.config, layer, li, B)
-
-    linears, xs_host, alg_bytes = [], [], []
-    eff_flops = 0.0
-    lookups = 0
-    nthreads = max(1, min(16, (os.cpu_count() or 4) - 1))
-    with cf.ThreadPoolExecutor(nthreads) as ex:
-        window = []
-        it = iter(jobs)
-        for _ in range(2 * nthreads):
-            j = next(it, None)
-            if j is not None:
-                window.append(ex.submit(gen, j))
-        while window:
-            job, L, x = window.pop(0).result()
-            j = next(it, None)
-            if j is not None:
-                window.append(ex.submit(gen, j))
-            lin = fb_layer.FluxBinLinear(L, fp16_tables=args.fp16_tables)
-            linears.append(lin)
-            xs_host.append(x)
-            alg_bytes.append(algorithmic_bytes(L.M, L.N, L.Kb, L.Ks, L.g, L.n_sal, B))
-            eff_flops += 2.0 * L.M * (L.N + L.n_sal) * B
-            lookups += L.Kb * L.M * (L.N // 8) + L.Ks * L.M * ((L.n_sal + 7) // 8)      # one per weight byte
-            del L
+    stack = build_config_stack(args.config, nl, B, g=args.g, fp16_tables=args.fp16_tables)
     setup_s = time.perf_counter() - t_setup
-
-    # activations / outputs: one arena each (device) + pinned host mirrors for the end-to-end leg
-    n_in = sum(l.N for l in linears) * B
-    n_out = sum(l.M for l in linears) * B
-    x_host = torch.empty(n_in, dtype=torch.float16).pin_memory()
-    y_host = torch.empty(n_out, dtype=torch.float16).pin_memory()
-    off = 0
-    for l, x in zip(linears, xs_host):
-        x_host[off:off + B * l.N] = torch.from_numpy(x.view(np.float16).reshape(-1))
-        off += B * l.N
-    x_dev = torch.empty(n_in, dtype=torch.float16, device="cuda")
-    y_dev = torch.empty(n_out, dtype=torch.float16, device="cuda")
-    x_dev.copy_(x_host)
-    ws = fb_layer.Workspace(max(l.weight.workspace_size(B) for l in linears))
-    views = []
-    ox = oy = 0
-    for l in linears:
-        views.append((l, x_dev[ox:ox + B * l.N].view(B, l.N), y_dev[oy:oy + B * l.M].view(B, l.M)))
-        ox += B * l.N
-        oy += B * l.M
-    packed_bytes = sum(l.packed_bytes for l in linears)
     stream = torch.cuda.Stream()
-
-    # how the linears of a step are grouped into launches
-    nlin = len(lins)
-    names = [n for n, _, _ in lins]
-    if args.launch == "linear":
-        groups = None
-    elif args.launch == "group":
-        dep_sets = [["q", "k", "v"], ["o"], ["gate", "up"], ["down"]] if "gate" in names else [[n] for n in names]
-        groups = [[layer * nlin + names.index(n) for n in ds] for layer in range(nl) for ds in dep_sets]
-    elif args.launch == "layer":
-        groups = [[layer * nlin + li for li in range(nlin)] for layer in range(nl)]
-    else:
-        groups = [list(range(len(linears)))]
-    plans = None
-    if groups is not None:
-        plans = [fb_layer.FluxBinPlan([views[i] for i in g]) for g in groups]
-        launches_per_step = sum(p.num_launches() for p in plans)
-    else:
-        launches_per_step = sum(l.weight.num_launches(B) for l in linears)
-
-    def issue_all():
-        if plans is not None:
-            for p in plans:
-                p.run(stream=stream)
-        else:
-            for l, xv, yv in views:
-                l.forward(xv, ws, out=yv, stream=stream)
-
-    graph = None
-    with torch.cuda.stream(stream):
-        issue_all()                                   # first call per device does the one-time set-up
-        stream.synchronize()
-        if not args.no_graph:
-            graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graph, stream=stream):
-                issue_all()
-
-    def step():
-        if graph is not None:
-            graph.replay()
-        else:
-            issue_all()
+    runner = stack.runner(args.launch, stream, graph=not args.no_graph)
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- device-resident timing --------------------------------------------------------------------
-    with torch.cuda.stream(stream):
-        for _ in range(max(3, args.warmup)):
-            step()
-        barrier()
-        sampler = ClockSampler(local_rank)
-        sampler.start()
-        ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
-        ev[0].record(stream)
-        for i in range(args.steps):
-            step()
-            ev[i + 1].record(stream)
-        barrier()
-        clocks = sampler.stop()
-    step_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
-    total_ms = ev[0].elapsed_time(ev[-1])
+    # ---- device-resident timing (the sampler runs from before the warm-up: a short timed region alone
+    #      would see one or two samples) ----------------------------------------------------------------
+    sampler = ClockSampler(local_rank).start()
+    sampler.wait_for_samples(1)
+    t_load = time.perf_counter()
+    total_ms, step_ms = runner.time(args.steps, max(3, args.warmup), barrier)
+    clocks = sampler.stop(since=t_load)
+    clocks["window"] = "warm-up steps + timed steps"
 
     # ---- end to end: pinned host x -> device, the stack, y -> pinned host, every step ---------------
     # Two sets of device activation/output buffers alternate, so the copies of one step overlap the kernels
     # of its neighbours (copy-in, compute and copy-out each on a stream of their own, ordered by events);
     # every step still moves its own inputs and outputs inside the timed region.
-    x_dev2, y_dev2 = torch.empty_like(x_dev), torch.empty_like(y_dev)
-    views2 = []
-    ox = oy = 0
-    for l in linears:
-        views2.append((l, x_dev2[ox:ox + B * l.N].view(B, l.N), y_dev2[oy:oy + B * l.M].view(B, l.M)))
-        ox += B * l.N
-        oy += B * l.M
-    plans2 = [fb_layer.FluxBinPlan([views2[i] for i in g]) for g in groups] if groups is not None else None
-
-    def issue_all2():
-        if plans2 is not None:
-            for p in plans2:
-                p.run(stream=stream)
-        else:
-            for l, xv, yv in views2:
-                l.forward(xv, ws, out=yv, stream=stream)
-
-    graph2 = None
-    with torch.cuda.stream(stream):
-        issue_all2()
-        stream.synchronize()
-        if not args.no_graph:
-            graph2 = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graph2, stream=stream):
-                issue_all2()
-    bufs = [(x_dev, y_dev, graph, issue_all), (x_dev2, y_dev2, graph2, issue_all2)]
+    x_dev2, y_dev2 = torch.empty_like(stack.x_dev), torch.empty_like(stack.y_dev)
+    runner2 = stack.runner(args.launch, stream, views=stack.make_views(x_dev2, y_dev2), graph=not args.no_graph)
+    bufs = [(stack.x_dev, stack.y_dev, runner), (x_dev2, y_dev2, runner2)]
     s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    x_host, y_host = stack.x_host, stack.y_host
 
     def e2e_steps(n):
         comp_done = [None, None]
         out_done = [None, None]
         for i in range(n):
             k = i & 1
-            xd, yd, g, issue = bufs[k]
+            xd, yd, r = bufs[k]
             if comp_done[k] is not None:
                 s_in.wait_event(comp_done[k])          # the kernels of step i-2 have read this x buffer
             with torch.cuda.stream(s_in):
@@ -420,10 +701,7 @@ def main():
             if out_done[k] is not None:
                 stream.wait_event(out_done[k])         # step i-2's results have left this y buffer
             with torch.cuda.stream(stream):
-                if g is not None:
-                    g.replay()
-                else:
-                    issue()
+                r.step()
                 comp_done[k] = torch.cuda.Event()
                 comp_done[k].record(stream)
             s_out.wait_event(comp_done[k])
@@ -446,40 +724,19 @@ def main():
     barrier()
     e2e_ms = e0.elapsed_time(e1)
     # the results that reached the host are those of the device-resident steps (same inputs), from either buffer set
-    y_ref = y_dev.float().cpu()
+    y_ref = stack.y_dev.float().cpu()
     y_got = y_host.float()
     y2_got = y_dev2.float().cpu()
     scale = float(y_ref.abs().max())
     e2e_max_diff = max(float((y_got - y_ref).abs().max()), float((y2_got - y_ref).abs().max())) / max(scale, 1e-30)
     if not (e2e_max_diff < 5e-3 and bool(torch.isfinite(y_got).all()) and scale > 0):
         raise RuntimeError(f"end-to-end outputs differ from the device-resident run: {e2e_max_diff}")
-
-    # ---- optional per-linear timing (plain launches, rotating over the layers so L2 stays cold) -----
-    per_linear = None
-    if args.per_linear and rank == 0:
-        per_linear = {}
-        nlin = len(lins)
-        with torch.cuda.stream(stream):
-            for li, (name, M, N) in enumerate(lins):
-                idxs = [layer * nlin + li for layer in range(nl)]
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                reps = 3
-                for r in range(reps + 1):
-                    if r == 1:
-                        a.record(stream)
-                    for i in idxs:
-                        l, xv, yv = views[i]
-                        l.forward(xv, ws, out=yv, stream=stream)
-                b.record(stream)
-                stream.synchronize()
-                us = a.elapsed_time(b) * 1e3 / (reps * len(idxs))
-                per_linear[f"{name}_{M}x{N}"] = {"us": round(us, 2), "GBps": round(alg_bytes[li] / us / 1e3, 1)}
-        print(json.dumps({"per_linear_plain_launches": per_linear}), file=sys.stderr)
+    y_timed = stack.y_dev.cpu().numpy()                  # outputs of the device-resident steps
+    del runner2, x_dev2, y_dev2, bufs
 
     # ---- max over ranks, aggregate ------------------------------------------------------------------
-    from paper_2608_15602_b200 import dist_util
     total_ms, e2e_ms = dist_util.max_over_ranks([total_ms, e2e_ms], device="cuda")
-    bytes_per_step = sum(alg_bytes)
+    bytes_per_step = sum(stack.alg_bytes)
     ms_per_step = total_ms / args.steps
     value = dist_util.replica_throughput(bytes_per_step, ms_per_step, world)
     e2e_value = dist_util.replica_throughput(bytes_per_step, e2e_ms / args.steps, world)
@@ -488,6 +745,7 @@ def main():
         peaks, peak_kind = measured_peaks()
         peak = float(peaks["hbm_gbs"])
         achieved = bytes_per_step / (ms_per_step * 1e-3) / 1e9     # one GPU's kernels
+        launches_per_step = runner.launches_per_step
         traffic = None
         tpath = os.path.join(ROOT, "profiles", "dram_traffic.txt")
         if os.path.exists(tpath):
@@ -503,16 +761,18 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": f"config {args.config}: Llama-2-70B-shaped decode linear stack" if args.config == 4
                        else f"config {args.config}: {nl} independently seeded copies of the layer/set per step",
-                       "layers": nl, "linears_per_step": len(linears), "batch": B,
-                       "table_entries": "fp16" if (args.fp16_tables and B > 1) else "fp32",
+                       "layers": nl, "linears_per_step": len(stack.linears), "batch": B,
+                       "table_entries": "fp16" if stack.fp16 else "fp32",
                        "Kb": 2, "Ks": 0 if args.config == 0 else 1, "salient_frac": 0.0 if args.config == 0 else 0.05,
-                       "g": args.g or "N", "packed_bytes_resident": packed_bytes, "algorithmic_bytes_per_step": bytes_per_step,
-                       "l2": "inputs larger than L2 (weights streamed once per step)" if packed_bytes > 4e8
+                       "g": args.g or "N", "packed_bytes_resident": stack.packed_bytes, "algorithmic_bytes_per_step": bytes_per_step,
+                       "l2": "inputs larger than L2 (weights streamed once per step)" if stack.packed_bytes > 4e8
                        else "working set fits L2: L2-warm number",
-                       "launch": ("cuda graph replay" if graph is not None else "plain launches") + f", {args.launch}: "
-                       f"{launches_per_step} kernel launches per step",
+                       "launch": ("cuda graph replay" if runner.graph is not None else "plain launches") + f", {args.launch}: "
+                       f"{launches_per_step} kernel launches per step"
+                       + (" (all linears independent: the throughput of the kernel; see group_mode for the launch "
+                          "structure a decoder allows)" if args.launch == "stack" else ""),
                        "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
-            "us_per_layer": ms_per_step * 1e3 / nl, "us_per_linear": ms_per_step * 1e3 / len(linears),
+            "us_per_layer": ms_per_step * 1e3 / nl, "us_per_linear": ms_per_step * 1e3 / len(stack.linears),
             "frac_of_8TBps": achieved / 8000.0,
             "step_ms_min_median_max": [min(step_ms), statistics.median(step_ms), max(step_ms)],
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
@@ -529,43 +789,65 @@ def main():
             "clocks": clocks, "setup_s": round(setup_s, 1),
         }
         # the paper's effective-throughput figure: 2 * M * (N + n_sal) * B flops per linear over the measured time
-        line["effective_tflops"] = eff_flops / (ms_per_step * 1e-3) / 1e12
+        line["effective_tflops"] = stack.eff_flops / (ms_per_step * 1e-3) / 1e12
         if B > 1:
-            # Batched launches are bound by shared-memory bandwidth, not HBM: every weight byte costs one table
-            # lookup per chunk of vectors, an entry of 4 bytes (fp32) or 2 bytes (fp16) per vector of the chunk.
-            fp16 = bool(args.fp16_tables)
-            ch = 8 if fp16 else 4
-            nvec = lambda nb: 1 if nb == 1 else 2 if nb == 2 else 4 if nb <= 4 else 8
-            chunks = [ch] * (B // ch)
-            rest = B % ch
-            if rest:                                                      # the library's rule for the last chunk
-                big = packed_bytes >= (128 << 20)
-                first = 2 if (big and not fp16 and rest == 3) else 4 if (big and fp16 and rest in (5, 6)) else rest
-                chunks += [first] + ([rest - first] if first < rest else [])
-            assert len(chunks) == launches_per_step or args.launch != "stack"
-            entry_bytes = sum((2 if (fp16 and nb >= 2) else 4) * nvec(nb) for nb in chunks)
             mhz = clocks.get("sm_mhz") or clocks.get("sm_max_mhz") or 1965.0
-            sms = torch.cuda.get_device_properties(0).multi_processor_count
-            smem_peak = sms * 128 * mhz * 1e6 / 1e9                     # GB/s at 128 B/clk/SM
-            smem_achieved = lookups * entry_bytes / (ms_per_step * 1e-3) / 1e9
-            line["lookup_ceiling"] = {"bound": "smem", "achieved": smem_achieved, "peak": smem_peak, "unit": "GB/s",
-                                      "frac": smem_achieved / smem_peak, "entry_bytes_per_weight_byte": entry_bytes,
-                                      "peak_source": f"{sms} SMs x 128 B/clk at the median SM clock under load ({mhz} MHz)"}
-        if not args.no_context:
-            line["context_dense_fp16_gemv"] = dense_fp16_gemv_context(lins, nl, B)
+            line["lookup_ceiling"] = lookup_ceiling(stack, ms_per_step, launches_per_step, mhz, args.launch)
         if clocks.get("power_w"):
             # board power (largest sample; see ClockSampler) x time: context only, a lower bound for short runs
             line["joules_per_step_lower_bound"] = clocks["power_w"] * ms_per_step * 1e-3
-        if not args.no_cpu_baseline:
-            y_timed = y_dev.cpu().numpy()                  # outputs of the device-resident steps
-            y_offs = np.cumsum([0] + [B * l.M for l in linears])
+
+        t_sections = time.perf_counter()
+        if "sustained" in sections:
+            # the headline launch replayed for at least two seconds: the rate the power cap allows
+            n_sus = max(args.steps, int(2200.0 / ms_per_step) + 1)
+            s2 = ClockSampler(local_rank).start()
+            s2.wait_for_samples(1)
+            t0 = time.perf_counter()
+            tot, sms_ = runner.time(n_sus, 3)
+            c2 = s2.stop(since=t0 + 0.5)                 # clocks once the run has settled
+            tail = sms_[len(sms_) // 2:]
+            ach = bytes_per_step / (statistics.mean(tail) * 1e-3) / 1e9
+            line["roofline"]["sustained"] = {
+                "steps": n_sus, "seconds": round(tot / 1e3, 2), "achieved": bytes_per_step / (tot / n_sus * 1e-3) / 1e9,
+                "achieved_second_half": ach, "frac_second_half": ach / peak, "frac_of_8TBps_second_half": ach / 8000.0,
+                "ms_per_step_second_half": statistics.mean(tail), "sm_mhz_median": c2.get("sm_mhz"), "sm_mhz_min": c2.get("sm_mhz_min"),
+                "power_w_max": c2.get("power_w"), "reasons": c2.get("reasons"), "clock_samples": c2.get("samples"),
+                "ms_times_ghz": statistics.mean(tail) * (c2.get("sm_mhz") or 0) / 1e3,
+                "note": "same launch as the headline replayed back to back; after about half a second the board sits at its "
+                        "power cap (sw_power_cap) and the SM clock settles below its maximum"}
+        if "group_mode" in sections and args.launch != "group" and "gate" in stack.names:
+            rg = stack.runner("group", stream)
+            sg = ClockSampler(local_rank).start()
+            sg.wait_for_samples(1)
+            t0 = time.perf_counter()
+            tot, sms_ = rg.time(args.steps, max(3, args.warmup))
+            cg = sg.stop(since=t0)
+            ach = bytes_per_step / (tot / args.steps * 1e-3) / 1e9
+            line["group_mode"] = {"launches_per_step": rg.launches_per_step, "ms_per_step": tot / args.steps, "value": ach, "unit": UNIT,
+                                  "frac": ach / peak, "frac_of_8TBps": ach / 8000.0, "us_per_launch": tot / args.steps * 1e3 / rg.launches_per_step,
+                                  "step_ms_min_median_max": [min(sms_), statistics.median(sms_), max(sms_)], "sm_mhz_median": cg.get("sm_mhz"),
+                                  "what": "the same resident stack, one plan per dependency group ({q,k,v} {o} {gate,up} {down}), chained on "
+                                          "one stream with programmatic dependent launch, CUDA-graph replay: the launch structure of a real decoder"}
+            del rg
+        if "configs" in sections:
+            line["configs"] = section_configs(stack, stream, peak)
+        if "variants" in sections:
+            line["variants"] = section_variants(stream, peak)
+        if "rc_decomp" in sections:
+            line["rc_decomp"] = section_rc_decomp()
+        if "context" in sections:
+            line["context_dense_fp16_gemv"] = dense_fp16_gemv_context(lins, nl, B)
+        if "cpu_baseline" in sections:
+            y_offs = np.cumsum([0] + [B * l.M for l in stack.linears])
 
             def gpu_y(i):
-                return y_timed[y_offs[i]:y_offs[i + 1]].reshape(B, linears[i].M)
+                return y_timed[y_offs[i]:y_offs[i + 1]].reshape(B, stack.linears[i].M)
 
             gbps, tsec, nbytes, cores, sample, agreement = cpu_oracle_sample(args.config, B, g=args.g, nl=nl, gpu_y=gpu_y)
             line["cpu_baseline"] = {"value": gbps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
                                     "seconds": round(tsec, 2), "gpu_vs_oracle_on_sample": agreement}
+        line["sections_s"] = round(time.perf_counter() - t_sections, 1)
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()

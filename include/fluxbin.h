@@ -129,6 +129,11 @@ fluxbin_status_t fluxbin_unpack(const fluxbin_weight_t *w, fluxbin_layer_desc_t 
 /* Dimensions of a handle (pointers of `out` untouched). */
 fluxbin_status_t fluxbin_weight_dims(const fluxbin_weight_t *w, fluxbin_layer_desc_t *out);
 
+/* CUDA device ordinal that was current when the handle was made, i.e. the device that holds d_packed; -1 on
+ * NULL.  fluxbin_linear, fluxbin_linear_noalloc and fluxbin_plan_create / fluxbin_plan_run must be called with
+ * that device current and return FLUXBIN_ERR_UNSUPPORTED otherwise (nothing is launched). */
+int32_t fluxbin_weight_device(const fluxbin_weight_t *w);
+
 /*
  * Precision of the lookup-table entries (Eq. 14) of batched launches (B >= 2) that read this layer.
  *
@@ -202,8 +207,10 @@ fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint16_t *d_x, 
  * every GPU that loads the library holds it until the process exits).  The call allocates nothing --
  * no cudaMalloc, no cudaFree, no allocating library routine.
  *
- *   - Layers whose fluxbin_workspace_size(w, B) exceeds the capacity (more than about 130,000 output
- *     rows at batch >= 2, 260,000 at batch 1) are rejected with FLUXBIN_ERR_BUFFER_TOO_SMALL.
+ *   - The rule: fluxbin_workspace_size(w, B) <= fluxbin_noalloc_capacity(), else FLUXBIN_ERR_BUFFER_TOO_SMALL.
+ *     The workspace holds 4 bytes per output row (rounded up to 32 rows) for each accumulator row of a chunk of
+ *     batch vectors, so 1 MiB takes about 260,000 output rows at B = 1, 130,000 at B = 2, 65,000 at B >= 3 with
+ *     fp32 table entries (B = 3, 4 with fp16 entries) and 32,000 at B >= 5 with fp16 table entries.
  *   - The first call on each device looks up the device address of the array (with that device
  *     current) and keeps it; make that first call before any stream capture begins.  The current
  *     device must be the one that holds the layer, else FLUXBIN_ERR_UNSUPPORTED.
@@ -227,6 +234,22 @@ size_t fluxbin_noalloc_capacity(void);
  */
 fluxbin_status_t fluxbin_debug_tables(const fluxbin_weight_t *w, const uint16_t *d_x, int32_t pair,
                                       float *d_tables, int32_t *h_cols, uint16_t *h_alpha, void *cuda_stream);
+
+/*
+ * Test hook for the work split (host only, uses no GPU): the bounds of the shares into which a launch of n packed
+ * layers is cut.  The kernel walks the work items of a launch -- (pair or couple of pairs, block of 32 rows),
+ * pair-major, layer after layer; the host cuts that list into `grid` shares of equal cost, one per CTA, plus
+ * `nshares - grid` small ones drawn dynamically from the last (100 - static_percent) % of the cost.
+ *
+ *   h_headers            HOST array of n pointers, each to the first 256 bytes of a packed layer
+ *   mode                 launch mode: 1, 2, 4 vectors with fp32 table entries, 16 + (2, 4, 8) with fp16 entries
+ *   pairs_per_row_block  1 or 2 (2 needs an even number of global pairs in every layer)
+ *   out_cuts             HOST int32 [nshares + 1][2]: {layer, work item} where share s begins; the last is {n, 0}
+ *   out_work_items       HOST int32 [n] or NULL: work items of each layer
+ */
+fluxbin_status_t fluxbin_debug_cut_shares(int32_t n, const void *const *h_headers, int32_t mode, int32_t pairs_per_row_block,
+                                          int32_t grid, int32_t nshares, int32_t static_percent, int32_t *out_cuts,
+                                          int32_t *out_work_items);
 
 /* Number of table sets (global + salient) of a layer; -1 on NULL. */
 int32_t fluxbin_num_table_sets(const fluxbin_weight_t *w);

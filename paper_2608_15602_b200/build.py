@@ -35,7 +35,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     os.makedirs(LIB_DIR, exist_ok=True)
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     tmp = LIB_PATH + f".tmp{os.getpid()}"
-    extra = os.environ.get("FLUXBIN_NVCC_EXTRA", "").split()       # e.g. -DFB_TRACE for the instrumented build
+    extra = ["-DFB_TRACE"] if os.environ.get("FLUXBIN_TRACE") == "1" else []    # the instrumented build (per-CTA phase timestamps)
     cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + _sources()
     subprocess.check_call(cmd)
     os.replace(tmp, LIB_PATH)

@@ -5,10 +5,14 @@
 
 #include <cstdlib>
 #include <cstring>
+#include <atomic>
 #include <mutex>
+#include <vector>
 #include <new>
 
 using namespace fb;
+
+static_assert(fb::kMaxSingleShares == fbk::kMaxSingleShares, "one-layer launches: host and kernel agree on the parameter array");
 
 static thread_local int g_last_cuda_error = 0;
 
@@ -53,29 +57,8 @@ struct DeviceInfo {
     bool ok = false;
     int num_sms = 0;
 };
-constexpr int kMaxDevices = 64;
 DeviceInfo g_dev[kMaxDevices];
 std::mutex g_dev_mutex;
-
-template <int S0, int S1, int BT> cudaError_t opt_in()
-{
-    cudaError_t e = cudaFuncSetAttribute(fbk::fluxbin_linear_kernel<S0, S1, BT, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)fbk::smem_bytes<BT>());
-    if (e != cudaSuccess) return e;
-    if constexpr (fbk::geom(BT) == 1)
-        e = cudaFuncSetAttribute(fbk::fluxbin_linear_kernel<S0, S1, BT, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)fbk::smem_bytes<BT>());
-    return e;
-}
-template <int BT> cudaError_t opt_in_bt()
-{
-    cudaError_t e;
-    if ((e = opt_in<16, 16, BT>()) != cudaSuccess) return e;
-    if ((e = opt_in<16, 1, BT>()) != cudaSuccess) return e;
-    if ((e = opt_in<8, 1, BT>()) != cudaSuccess) return e;
-    if ((e = opt_in<4, 1, BT>()) != cudaSuccess) return e;
-    return cudaSuccess;
-}
 
 fluxbin_status_t device_setup(int dev, int *num_sms)
 {
@@ -89,12 +72,8 @@ fluxbin_status_t device_setup(int dev, int *num_sms)
         d.num_sms = sms;
         d.ok = false;
         if (major == 10) {
-            FB_CUDA(opt_in_bt<1>());
-            FB_CUDA(opt_in_bt<2>());
-            FB_CUDA(opt_in_bt<4>());
-            FB_CUDA(opt_in_bt<16 + 2>());
-            FB_CUDA(opt_in_bt<16 + 4>());
-            FB_CUDA(opt_in_bt<16 + 8>());
+            fluxbin_status_t st = fb::opt_in_all_kernels();
+            if (st != FLUXBIN_OK) return st;
             FB_CUDA(cudaFuncSetAttribute(fbk::fluxbin_debug_tables_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)fbk::smem_bytes<1>()));
             FB_CUDA(cudaFuncSetAttribute(fbk::fluxbin_smem_base_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -133,6 +112,7 @@ fluxbin_status_t make_handle(const FbHeader &h, void *d_packed, size_t d_bytes, 
     if ((h.nrb + w->tile_rb - 1) / w->tile_rb > fbk::kMaxTiles) w->tile_rb = (h.nrb + fbk::kMaxTiles - 1) / fbk::kMaxTiles;
     w->ntiles = (h.nrb + w->tile_rb - 1) / w->tile_rb;
     w->table_format = FLUXBIN_TABLES_FP32;
+    for (auto &slot : w->single) slot.store(nullptr);
     *out = w;
     return FLUXBIN_OK;
 }
@@ -198,7 +178,14 @@ extern "C" fluxbin_status_t fluxbin_weight_dims(const fluxbin_weight_t *w, fluxb
     return FLUXBIN_OK;
 }
 
-extern "C" void fluxbin_free(fluxbin_weight_t *w) { delete w; }
+extern "C" void fluxbin_free(fluxbin_weight_t *w)
+{
+    if (!w) return;
+    for (auto &slot : w->single) delete slot.load();
+    delete w;
+}
+
+extern "C" int32_t fluxbin_weight_device(const fluxbin_weight_t *w) { return w ? w->device : -1; }
 
 extern "C" int32_t fluxbin_num_table_sets(const fluxbin_weight_t *w) { return w ? w->h.npairs[0] + w->h.npairs[1] : -1; }
 
@@ -285,109 +272,61 @@ extern "C" fluxbin_status_t fluxbin_workspace_init(void *d_workspace, size_t byt
 
 // ---- the layer ------------------------------------------------------------------------------------
 
-// The two-pairs-per-row-block kernel pays two table builds per run of rows but has the better row loop (one
-// reduction per two items, loads requested half an item earlier).  Measured on B200 (batch 1): it wins as soon
-// as a CTA's share is worth about 30 plain items (cost 60) -- +11 % with one launch per 70B linear, +15 % with
-// one per dependency group, +21 % with one per layer -- and loses below that (4096 x 4096 alone, 18 items per
-// CTA: 6.7 -> 7.7 us per call).
-#ifndef FB_NP2_MIN
-#define FB_NP2_MIN 60
-#endif
-// How a launch is cut: grid size, the statically dealt part of the cost line, the number of shares, and
-// whether the two-pairs-per-row-block kernel runs.
-struct LaunchShape {
-    long long grid, static_cost;
-    int nshares;
-    bool couples;
-};
-
-template <int S0, int S1, int BT>
-static cudaError_t launch_shape(long long total_cost, int num_sms, long long items, long long couple_cost, LaunchShape *out)
+// The kernel instantiation for a launch mode (1, 2, 4 vectors with fp32 tables, 16 + (2, 4, 8) with fp16 tables),
+// a row-scale format class (sub-vectors per scale segment of the global / salient region) and the number of
+// pairs walked per row block (2 exists for the modes with 4-byte table entries: 1 and 16 + 2).
+template <int S0, int S1, int BT> static const void *kernel_of(int np)
 {
-    static int occ = 0;     // resident CTAs per SM of this instantiation (same on every B200)
-    if (occ == 0) {
-        int o = 0;
-        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, fbk::fluxbin_linear_kernel<S0, S1, BT, 1>,
-                                                                      fbk::Cfg<BT>::kThreads, fbk::smem_bytes<BT>());
-        if (e != cudaSuccess) return e;
-        occ = o > 0 ? o : 1;
-    }
-    long long grid = (long long)num_sms * occ;
-    if (items < grid) grid = items;
-    // Launches with enough work deal 90 % of it out statically and cut the rest into three small
-    // shares per CTA (each worth >= ~200 items), drawn dynamically; small launches stay static.
-    constexpr int dyn_pct = 10, dyn_k = 3;
-    const long long rest = total_cost * dyn_pct / 100;
-    if (dyn_pct > 0 && dyn_k > 0 && rest / (grid * dyn_k) >= 400) {
-        out->static_cost = total_cost - rest;
-        out->nshares = (int)(grid * (1 + dyn_k));
-    } else {
-        out->static_cost = total_cost;
-        out->nshares = (int)grid;
-    }
-    out->grid = grid;
-    // two pairs per row block when every layer allows it (couple_cost > 0: even pair counts everywhere) and a
-    // CTA's share is large enough to pay for the second table build
-    out->couples = fbk::geom(BT) == 1 && couple_cost > 0 && out->static_cost / grid >= FB_NP2_MIN;
-    return cudaSuccess;
-}
-
-template <int S0, int S1, int BT>
-static cudaError_t launch(const fbk::LaunchParams &p, int num_sms, long long items, long long couple_cost, cudaStream_t s)
-{
-    LaunchShape shape;
-    cudaError_t se = launch_shape<S0, S1, BT>(p.total_cost, num_sms, items, couple_cost, &shape);
-    if (se != cudaSuccess) return se;
-    const long long grid = shape.grid;
-    const bool couples = shape.couples;
-    fbk::LaunchParams q = p;
-    q.static_cost = shape.static_cost;
-    q.nshares = shape.nshares;
-    // launched with programmatic stream serialization: the kernel may start while its predecessor in
-    // the stream drains (it waits inside, before touching activations or workspace)
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3(fbk::Cfg<BT>::kThreads);
-    cfg.dynamicSmemBytes = fbk::smem_bytes<BT>();
-    cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
     if constexpr (fbk::geom(BT) == 1) {
-        if (couples) return cudaLaunchKernelEx(&cfg, fbk::fluxbin_linear_kernel<S0, S1, BT, 2>, q);
+        if (np == 2) return (const void *)fbk::fluxbin_linear_kernel<S0, S1, BT, 2>;
     }
-    return cudaLaunchKernelEx(&cfg, fbk::fluxbin_linear_kernel<S0, S1, BT, 1>, q);
+    return (const void *)fbk::fluxbin_linear_kernel<S0, S1, BT, 1>;
 }
-
-// couple_cost: cost of the largest couple of global pairs over the layers of the launch, or 0 when
-// some layer has an odd number of global pairs (then the one-pair kernel runs).
-template <int BT> static cudaError_t launch_bt(int s0, int s1, int num_sms, const fbk::LaunchParams &p, long long items,
-                                               long long couple_cost, cudaStream_t s)
+template <int BT> static const void *kernel_of_bt(int s0, int s1, int np)
 {
-    if (s0 == 16 && s1 == 16) return launch<16, 16, BT>(p, num_sms, items, couple_cost, s);
-    if (s0 == 16) return launch<16, 1, BT>(p, num_sms, items, couple_cost, s);
-    if (s0 == 8) return launch<8, 1, BT>(p, num_sms, items, couple_cost, s);
-    return launch<4, 1, BT>(p, num_sms, items, couple_cost, s);
+    if (s0 == 16 && s1 == 16) return kernel_of<16, 16, BT>(np);
+    if (s0 == 16) return kernel_of<16, 1, BT>(np);
+    if (s0 == 8) return kernel_of<8, 1, BT>(np);
+    return kernel_of<4, 1, BT>(np);
 }
-
-// mode: 1, 2, 4 vectors with fp32 tables, 16 + (2, 4, 8) vectors with fp16 tables; the two-pair kernel exists
-// for the modes with 4-byte table entries (1 and 16 + 2; couple_cost is ignored elsewhere)
-static cudaError_t launch_mode(int mode, int s0, int s1, int num_sms, const fbk::LaunchParams &p, long long items,
-                               long long couple_cost, cudaStream_t s)
+static const void *kernel_for(int mode, int s0, int s1, int np)
 {
     switch (mode) {
-    case 1: return launch_bt<1>(s0, s1, num_sms, p, items, couple_cost, s);
-    case 2: return launch_bt<2>(s0, s1, num_sms, p, items, 0, s);
-    case 4: return launch_bt<4>(s0, s1, num_sms, p, items, 0, s);
-    case 16 + 2: return launch_bt<16 + 2>(s0, s1, num_sms, p, items, couple_cost, s);
-    case 16 + 4: return launch_bt<16 + 4>(s0, s1, num_sms, p, items, 0, s);
-    case 16 + 8: return launch_bt<16 + 8>(s0, s1, num_sms, p, items, 0, s);
+    case 1: return kernel_of_bt<1>(s0, s1, np);
+    case 2: return kernel_of_bt<2>(s0, s1, np);
+    case 4: return kernel_of_bt<4>(s0, s1, np);
+    case 16 + 2: return kernel_of_bt<16 + 2>(s0, s1, np);
+    case 16 + 4: return kernel_of_bt<16 + 4>(s0, s1, np);
+    case 16 + 8: return kernel_of_bt<16 + 8>(s0, s1, np);
     }
-    return cudaErrorInvalidValue;
+    return nullptr;
+}
+static int mode_index(int mode) { return mode == 1 ? 0 : mode == 2 ? 1 : mode == 4 ? 2 : mode == 16 + 2 ? 3 : mode == 16 + 4 ? 4 : 5; }
+static int class_index(int s0, int s1) { return (s0 == 16 && s1 == 16) ? 0 : s0 == 16 ? 1 : s0 == 8 ? 2 : 3; }
+static int threads_for(int mode) { return fbk::geom(mode) == 4 ? 512 : 256; }
+static size_t smem_for(int mode)      // the scratch beside the tables grows with the vectors of the mode
+{
+    switch (mode) {
+    case 1: return fbk::smem_bytes<1>();
+    case 2: return fbk::smem_bytes<2>();
+    case 4: return fbk::smem_bytes<4>();
+    case 16 + 2: return fbk::smem_bytes<16 + 2>();
+    case 16 + 4: return fbk::smem_bytes<16 + 4>();
+    case 16 + 8: return fbk::smem_bytes<16 + 8>();
+    }
+    return 0;
 }
 
+fluxbin_status_t fb::opt_in_all_kernels()
+{
+    static const int modes[6] = {1, 2, 4, 16 + 2, 16 + 4, 16 + 8};
+    static const int cls[4][2] = {{16, 16}, {16, 1}, {8, 1}, {4, 1}};
+    for (int m : modes)
+        for (auto &c : cls)
+            for (int np = 1; np <= (fbk::geom(m) == 1 ? 2 : 1); ++np)
+                FB_CUDA(cudaFuncSetAttribute(kernel_for(m, c[0], c[1], np), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_for(m)));
+    return FLUXBIN_OK;
+}
 
 // Work-split cost model, measured on B200 in units of half a 1152-byte item (about 50 ns per CTA):
 // an item with one row scale per sub-vector (3072 bytes) takes about 2x a plain item; building one
@@ -397,12 +336,10 @@ constexpr int kBuildCost = 44;
 // With four or eight vectors in fp16 table entries an item takes about half the time it takes with fp32 entries,
 // a build (more vectors per entry, conversions) does not: measured 44 / 66 / 88 / 132 -> 3.29 / 3.47 / 3.51 / 3.46
 // TB/s at batch 4 and 1.73 / 1.81 / 1.81 / 1.81 at batch 8.  (With fp32 entries, batch 2 and 4: no effect.)
-#ifndef FB_BCH
-#define FB_BCH 88
-#endif
+constexpr int kBuildCostHalfWide = 88;
 static int build_cost_for(int mode)
 {
-    return (mode == 16 + 4 || mode == 16 + 8) ? FB_BCH : kBuildCost;    // two vectors in fp16 entries: 36 / 44 / 56 / 66 all within 1 %
+    return (mode == 16 + 4 || mode == 16 + 8) ? kBuildCostHalfWide : kBuildCost;    // two vectors in fp16 entries: 36 / 44 / 56 / 66 all within 1 %
 }
 // The reduction epilogue a CTA runs when it leaves an entry (fence, tickets, read-back of the tiles it
 // completed): a fixed part plus a part that grows with the rows to convert.
@@ -420,24 +357,250 @@ static void item_costs(int sps0, int sps1, int cost[2])
     cost[1] = (sps1 == sps0) ? 2 : 4;
 }
 
+// an item of the last salient pair costs in proportion to its steps when that pair is stored narrow
+static int last_salient_item_cost(const FbHeader &h, int cost1)
+{
+    const int c = (h.sps[1] == 1) ? cost1 * h.sal_last_w / 32 : cost1;
+    return c > 0 ? c : 1;
+}
+
 static long long entry_cost(const FbHeader &h, int sps1, int build_cost)
 {
     int c[2];
     item_costs(h.sps[0], sps1, c);
-    return (long long)h.npairs[0] * (build_cost + (long long)h.nrb * c[0]) +
-           (long long)h.npairs[1] * (build_cost + (long long)h.nrb * c[1]) + epilogue_cost(h);
+    long long cost = (long long)h.npairs[0] * (build_cost + (long long)h.nrb * c[0]) + epilogue_cost(h);
+    if (h.npairs[1] > 0)
+        cost += (long long)(h.npairs[1] - 1) * (build_cost + (long long)h.nrb * c[1]) +
+                (build_cost + (long long)h.nrb * last_salient_item_cost(h, c[1]));
+    return cost;
+}
+
+// The two-pairs-per-row-block kernel pays two table builds per run of rows but has the better row loop (one
+// reduction per two items, loads requested half an item earlier).  Measured on B200 (batch 1): it wins as soon
+// as a CTA's share is worth about 30 plain items (cost 60) -- +11 % with one launch per 70B linear, +15 % with
+// one per dependency group, +21 % with one per layer -- and loses below that (4096 x 4096 alone, 18 items per
+// CTA: 6.7 -> 7.7 us per call).
+constexpr long long kCoupleMinShare = 60;
+
+// How a launch is cut: grid size, the statically dealt part of the cost line, the number of shares, and
+// how many pairs the kernel walks per row block (2: the two-pairs-per-row-block kernel).
+struct LaunchShape {
+    int grid, nshares, np;
+    long long static_cost;
+};
+
+static cudaError_t launch_shape(int dev, int mode, int s0, int s1, long long total_cost, int num_sms, long long items,
+                                long long couple_cost, bool allow_dynamic, LaunchShape *out)
+{
+    // resident CTAs per SM of an instantiation, per device (0 = not asked yet; racing threads store the same value)
+    static std::atomic<int> occ_of[kMaxDevices][6][4];
+    std::atomic<int> &slot = occ_of[dev][mode_index(mode)][class_index(s0, s1)];
+    int occ = slot.load(std::memory_order_relaxed);
+    if (occ == 0) {
+        int o = 0;
+        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, kernel_for(mode, s0, s1, 1), threads_for(mode), smem_for(mode));
+        if (e != cudaSuccess) return e;
+        occ = o > 0 ? o : 1;
+        slot.store(occ, std::memory_order_relaxed);
+    }
+    long long grid = (long long)num_sms * occ;
+    {   // EXPERIMENT
+        static const int small_per_sm = getenv("FBX_SMALL_PER_SM") ? atoi(getenv("FBX_SMALL_PER_SM")) : 0;
+        static const long long small_thresh = getenv("FBX_SMALL_THRESH") ? atoll(getenv("FBX_SMALL_THRESH")) : 0;
+        if (small_per_sm > 0 && total_cost / grid < small_thresh && small_per_sm < occ) grid = (long long)num_sms * small_per_sm;
+    }
+    if (items < grid) grid = items;
+    if (grid > kMaxGrid) grid = kMaxGrid;
+    if (!allow_dynamic && grid > fbk::kMaxSingleShares) grid = fbk::kMaxSingleShares;
+    // Launches with enough work deal 90 % of it out statically and cut the rest into three small
+    // shares per CTA (each worth >= ~200 items), drawn dynamically; small launches stay static.
+    static const int dyn_pct = getenv("FBX_DYN_PCT") ? atoi(getenv("FBX_DYN_PCT")) : 10;      // EXPERIMENT
+    static const int dyn_k = getenv("FBX_DYN_K") ? atoi(getenv("FBX_DYN_K")) : 3;
+    static const int dyn_min = getenv("FBX_DYN_MIN") ? atoi(getenv("FBX_DYN_MIN")) : 400;
+    const long long rest = total_cost * dyn_pct / 100;
+    if (allow_dynamic && dyn_pct > 0 && rest / (grid * dyn_k) >= dyn_min) {
+        out->static_cost = total_cost - rest;
+        out->nshares = (int)(grid * (1 + dyn_k));
+    } else {
+        out->static_cost = total_cost;
+        out->nshares = (int)grid;
+    }
+    out->grid = (int)grid;
+    // two pairs per row block when every layer allows it (couple_cost > 0: even pair counts everywhere) and a
+    // CTA's share is large enough to pay for the second table build
+    out->np = (fbk::geom(mode) == 1 && couple_cost > 0 && out->static_cost / grid >= kCoupleMinShare) ? 2 : 1;
+    return cudaSuccess;
+}
+
+// ---- cutting the cost line (host) --------------------------------------------------------------------
+// Every pair of an entry costs build_cost + nrb * item_cost of its region, the entry ends with its epilogue
+// cost; the entries of a launch lie one after the other.  Share s owns the work items whose start lies in its
+// piece [lo, hi) of the line; a cut inside the build part of a work pair goes to its first row block.
+
+struct CutModel {
+    int np, build_cost, item_cost[2];
+};
+
+// first work item of header h at or after position pos of its own cost line (0 .. all items)
+static int first_item_at(const FbHeader &h, const CutModel &m, long long pos)
+{
+    const int np = m.np;
+    const long long w0 = m.item_cost[0], w1 = m.item_cost[1];
+    const int wp0 = h.npairs[0] / np;
+    const int I0 = wp0 * h.nrb, I1 = h.npairs[1] * h.nrb;
+    const long long w1l = last_salient_item_cost(h, m.item_cost[1]);
+    const long long Pc0 = np * (m.build_cost + (long long)h.nrb * w0), Pc1 = m.build_cost + (long long)h.nrb * w1;
+    const long long Pc1l = m.build_cost + (long long)h.nrb * w1l;
+    const long long T0 = (long long)wp0 * Pc0, T1 = h.npairs[1] > 0 ? (long long)(h.npairs[1] - 1) * Pc1 : 0;
+    const long long T = T0 + (h.npairs[1] > 0 ? T1 + Pc1l : 0);
+    if (pos <= 0) return 0;
+    if (pos >= T) return I0 + I1;
+    const bool reg1 = pos >= T0;
+    const bool last1 = reg1 && pos - T0 >= T1;          // inside the last salient pair (its items may be cheaper)
+    const long long rel = reg1 ? pos - T0 : pos, Pc = reg1 ? Pc1 : Pc0, w = last1 ? w1l : reg1 ? w1 : np * w0;
+    const long long pair = last1 ? h.npairs[1] - 1 : rel / Pc;
+    const long long within = rel - (last1 ? T1 : pair * Pc) - (reg1 ? 1 : np) * m.build_cost;
+    long long rb = within <= 0 ? 0 : (within + w - 1) / w;
+    if (rb > h.nrb) rb = h.nrb;
+    return (reg1 ? I0 : 0) + (int)(pair * h.nrb + rb);
+}
+
+static int work_items_of(const FbHeader &h, int np) { return (h.npairs[0] / np + h.npairs[1]) * h.nrb; }
+
+// cuts[s] for s = 0 .. nshares: where share s begins ({n, 0} = the end of the launch).  cost_begin[e] = summed
+// cost of the entries before e, cost_begin[n] = the total.
+static void cut_launch(const FbHeader *const *hs, const long long *cost_begin, int n, const CutModel &m,
+                       const LaunchShape &shape, fbk::ShareCut *cuts)
+{
+    const long long total = cost_begin[n], rest = total - shape.static_cost;
+    const int G = shape.grid, nj = shape.nshares - G;
+    int e = 0;
+    for (int s = 0; s <= shape.nshares; ++s) {
+        long long lo;
+        if (s <= G) lo = shape.static_cost * (long long)s / G;
+        else lo = shape.static_cost + rest * (long long)(s - G) / nj;
+        if (s == shape.nshares) lo = total;
+        while (e + 1 < n && cost_begin[e + 1] <= lo) ++e;     // last entry that begins at or before lo
+        int item = first_item_at(*hs[e], m, lo - cost_begin[e]);
+        int ce = e;
+        if (item >= work_items_of(*hs[e], m.np)) { ce = e + 1; item = 0; }
+        cuts[s].entry = ce;
+        cuts[s].item = item;
+    }
+    cuts[shape.nshares].entry = n;
+    cuts[shape.nshares].item = 0;
+}
+
+// Test hook (host only, no GPU): the share bounds of a launch of n packed layers, given their 256-byte headers.
+extern "C" fluxbin_status_t fluxbin_debug_cut_shares(int32_t n, const void *const *h_headers, int32_t mode, int32_t pairs_per_row_block,
+                                                     int32_t grid, int32_t nshares, int32_t static_percent, int32_t *out_cuts,
+                                                     int32_t *out_work_items)
+{
+    if (!h_headers || !out_cuts) return FLUXBIN_ERR_NULL;
+    if (n < 1 || grid < 1 || nshares < grid || static_percent < 1 || static_percent > 100 || (nshares > grid && static_percent == 100))
+        return FLUXBIN_ERR_RANGE;
+    if (!kernel_for(mode, 16, 1, 1) || pairs_per_row_block < 1 || pairs_per_row_block > 2) return FLUXBIN_ERR_RANGE;
+    std::vector<FbHeader> H((size_t)n);
+    std::vector<const FbHeader *> hs((size_t)n);
+    int sps1 = 0;
+    for (int i = 0; i < n; ++i) {
+        fluxbin_status_t st = check_header(h_headers[i], FB_HEADER_BYTES, H[(size_t)i]);
+        if (st != FLUXBIN_OK) return st;
+        hs[(size_t)i] = &H[(size_t)i];
+        if (H[(size_t)i].npairs[1] > 0) sps1 = H[(size_t)i].sps[1];
+        if (pairs_per_row_block == 2 && (H[(size_t)i].npairs[0] & 1)) return FLUXBIN_ERR_UNSUPPORTED;
+    }
+    if (sps1 == 0) sps1 = 1;
+    CutModel m;
+    m.np = pairs_per_row_block;
+    m.build_cost = build_cost_for(mode);
+    item_costs(H[0].sps[0], sps1, m.item_cost);
+    std::vector<long long> cost_begin((size_t)n + 1);
+    long long cost = 0;
+    for (int i = 0; i < n; ++i) {
+        cost_begin[(size_t)i] = cost;
+        cost += entry_cost(H[(size_t)i], sps1, m.build_cost);
+        if (out_work_items) out_work_items[i] = work_items_of(H[(size_t)i], m.np);
+    }
+    cost_begin[(size_t)n] = cost;
+    LaunchShape shape;
+    shape.grid = grid; shape.nshares = nshares; shape.np = m.np;
+    shape.static_cost = nshares > grid ? cost * static_percent / 100 : cost;
+    std::vector<fbk::ShareCut> cuts((size_t)nshares + 1);
+    cut_launch(hs.data(), cost_begin.data(), n, m, shape, cuts.data());
+    for (int s = 0; s <= nshares; ++s) { out_cuts[2 * s] = cuts[(size_t)s].entry; out_cuts[2 * s + 1] = cuts[(size_t)s].item; }
+    return FLUXBIN_OK;
+}
+
+static cudaError_t launch_kernel(int mode, int s0, int s1, const LaunchShape &shape, const fbk::LaunchParams &p, cudaStream_t s)
+{
+    // launched with programmatic stream serialization: the kernel may start while its predecessor in
+    // the stream drains (it waits inside, before touching activations or workspace)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)shape.grid);
+    cfg.blockDim = dim3((unsigned)threads_for(mode));
+    cfg.dynamicSmemBytes = smem_for(mode);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+#ifdef FB_TRACE
+    static std::atomic<int> launches{0};
+    const_cast<fbk::LaunchParams &>(p).trace_slot = launches.fetch_add(1) & 7;
+#endif
+    {   // EXPERIMENT
+        static const int head = getenv("FBX_HEAD") ? atoi(getenv("FBX_HEAD")) : 0;
+        const_cast<fbk::LaunchParams &>(p).head_bytes = head;
+        static const int early = getenv("FBX_EARLY") ? atoi(getenv("FBX_EARLY")) : 0;
+        const_cast<fbk::LaunchParams &>(p).early_items = early;
+    }
+    void *args[1] = {(void *)&p};
+    return cudaLaunchKernelExC(&cfg, kernel_for(mode, s0, s1, shape.np), args);
 }
 
 static void fill_entry(fbk::LinearEntry &E, const fluxbin_weight_t *w, const uint16_t *x, int64_t ldx, void *y, int64_t ldy,
-                       float *acc, unsigned *tickets, long long cost_begin)
+                       float *acc, unsigned *tickets)
 {
     E.packed = (const uint8_t *)w->d_packed;
     E.x = x; E.y = y; E.acc = acc; E.tickets = tickets;
-    E.ldx = ldx; E.ldy = ldy; E.cost_begin = cost_begin;
+    E.ldx = ldx; E.ldy = ldy; E.reserved0 = 0;
     E.off_coldesc = w->h.off_coldesc; E.off_items[0] = w->h.off_items[0]; E.off_items[1] = w->h.off_items[1];
     E.M = w->h.M; E.N = w->h.N; E.Kb = w->h.Kb; E.Mpad = w->h.Mpad; E.nrb = w->h.nrb;
     E.npairs[0] = w->h.npairs[0]; E.npairs[1] = w->h.npairs[1];
-    E.tile_rb = w->tile_rb; E.ntiles = w->ntiles; E.reserved = 0;
+    E.tile_rb = w->tile_rb; E.ntiles = w->ntiles; E.sal_last_w = w->h.sal_last_w;
+}
+
+// The launch shape and the share bounds of a one-layer launch in a given mode depend on the layer alone: they are
+// worked out on first use and kept with the handle.
+static const SingleLaunch *single_launch_of(const fluxbin_weight_t *w, int mode, cudaError_t *err)
+{
+    std::atomic<SingleLaunch *> &slot = w->single[mode_index(mode)];
+    SingleLaunch *sl = slot.load(std::memory_order_acquire);
+    if (sl) return sl;
+    const int s0 = w->h.sps[0], s1 = w->h.npairs[1] > 0 ? w->h.sps[1] : 1;
+    CutModel m;
+    m.build_cost = build_cost_for(mode);
+    item_costs(s0, s1, m.item_cost);
+    const long long total = entry_cost(w->h, s1, m.build_cost);
+    const long long items = (long long)(w->h.npairs[0] + w->h.npairs[1]) * w->h.nrb;
+    LaunchShape shape;
+    *err = launch_shape(w->device, mode, s0, s1, total, w->num_sms, items, couple_cost_of(w->h), false, &shape);
+    if (*err != cudaSuccess) return nullptr;
+    m.np = shape.np;
+    sl = new (std::nothrow) SingleLaunch;
+    if (!sl) { *err = cudaErrorMemoryAllocation; return nullptr; }
+    sl->grid = shape.grid; sl->np = shape.np;
+    std::vector<fbk::ShareCut> cuts((size_t)shape.nshares + 1);
+    const FbHeader *hs[1] = {&w->h};
+    const long long cb[2] = {0, total};
+    cut_launch(hs, cb, 1, m, shape, cuts.data());
+    const int all = work_items_of(w->h, m.np);
+    for (int s = 0; s <= shape.nshares; ++s) sl->cut[s] = cuts[s].entry >= 1 ? all : cuts[s].item;
+    SingleLaunch *expected = nullptr;
+    if (!slot.compare_exchange_strong(expected, sl, std::memory_order_acq_rel)) { delete sl; sl = expected; }
+    return sl;
 }
 
 extern "C" fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint16_t *d_x, int32_t B, int64_t ldx,
@@ -450,31 +613,38 @@ extern "C" fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint
     if (ws_bytes < fluxbin_workspace_size(w, B)) return FLUXBIN_ERR_BUFFER_TOO_SMALL;
     // a 16-segment salient region only exists with a single scale group, where sps[0] is 16 too
     if (w->h.npairs[1] > 0 && w->h.sps[1] == 16 && w->h.sps[0] != 16) return FLUXBIN_ERR_FORMAT;
+    int dev = -1;
+    FB_CUDA(cudaGetDevice(&dev));
+    if (dev != w->device) return FLUXBIN_ERR_UNSUPPORTED;      // the layer lives on another device than the current one
     cudaStream_t s = (cudaStream_t)cuda_stream;
 
     fbk::LaunchParams p;
     p.table = nullptr;
+    p.cuts = nullptr;
     p.n = 1;
     p.y_fp32 = y_is_fp32 != 0;
-    const int sps1_eff = w->h.npairs[1] > 0 ? w->h.sps[1] : 1;
-    item_costs(w->h.sps[0], sps1_eff, p.item_cost);
     const int fmt = w->table_format;
     const int bt_ws = ws_bt(B, fmt);
     float *acc = (float *)d_workspace;
     unsigned *tickets = (unsigned *)((uint8_t *)d_workspace + acc_bytes(w, bt_ws));
     p.counters = (unsigned *)((uint8_t *)d_workspace + acc_bytes(w, bt_ws) + ((size_t)w->ntiles * 4 + 255) / 256 * 256);
-    const long long items = (long long)(w->h.npairs[0] + w->h.npairs[1]) * w->h.nrb;
+    const int s0 = w->h.sps[0], s1 = w->h.npairs[1] > 0 ? w->h.sps[1] : 1;
 
     const size_t ysz = y_is_fp32 ? 4 : 2;
     const Chunks ch = chunks_of(B, fmt, (long long)w->h.total_bytes);
     for (int c = 0; c < ch.n; ++c) {
         const int nb = chunk_nb(ch, fmt, c), b0 = chunk_begin(ch, fmt, c);
-        fill_entry(p.single, w, d_x + (int64_t)b0 * ldx, ldx, (uint8_t *)d_y + (size_t)b0 * ldy * ysz, ldy, acc, tickets, 0);
+        const int mode = mode_for(nb, fmt);
+        cudaError_t e = cudaSuccess;
+        const SingleLaunch *sl = single_launch_of(w, mode, &e);
+        if (!sl) return cuda_fail(e);
+        fill_entry(p.single, w, d_x + (int64_t)b0 * ldx, ldx, (uint8_t *)d_y + (size_t)b0 * ldy * ysz, ldy, acc, tickets);
         p.nb = nb;
-        const int s1 = w->h.npairs[1] > 0 ? w->h.sps[1] : 1;
-        p.build_cost = build_cost_for(mode_for(nb, fmt));
-        p.total_cost = entry_cost(w->h, sps1_eff, p.build_cost);
-        cudaError_t e = launch_mode(mode_for(nb, fmt), w->h.sps[0], s1, w->num_sms, p, items, couple_cost_of(w->h), s);
+        p.nshares = sl->grid;
+        std::memcpy(p.single_cut, sl->cut, sizeof(int) * ((size_t)sl->grid + 1));
+        LaunchShape shape;
+        shape.grid = sl->grid; shape.nshares = sl->grid; shape.np = sl->np; shape.static_cost = 0;
+        e = launch_kernel(mode, s0, s1, shape, p, s);
         if (e != cudaSuccess) return cuda_fail(e);
     }
     return FLUXBIN_OK;
@@ -482,14 +652,17 @@ extern "C" fluxbin_status_t fluxbin_linear(const fluxbin_weight_t *w, const uint
 
 // ---- plans: many layers in one persistent launch -------------------------------------------------
 
+struct PlanChunk {
+    int nb, mode;
+    LaunchShape shape;
+    const fbk::LinearEntry *d_entries;
+    const fbk::ShareCut *d_cuts;
+};
+
 struct fluxbin_plan {
-    int n, B, y_fp32, nchunks, table_format;
-    int sps0, sps1, num_sms;
-    long long items, couple_cost;
-    std::vector<int> chunk_nb, chunk_build_cost;     // per chunk: vectors, build cost of its kernel's cost model
-    std::vector<long long> chunk_total_cost;
-    int item_cost[2];
-    const fbk::LinearEntry *d_table;     // [nchunks][n]
+    int n, B, y_fp32, table_format, device;
+    int sps0, sps1;
+    std::vector<PlanChunk> chunks;
     unsigned *d_counters;
 };
 
@@ -498,12 +671,18 @@ static size_t entry_ws_bytes(const fluxbin_weight_t *w, int bt)
     return acc_bytes(w, bt) + ((size_t)w->ntiles * 4 + 255) / 256 * 256;
 }
 
+// device table of one chunk: the entries, then the share cuts (at most 4 shares per CTA of the largest grid)
+static size_t chunk_table_bytes(int n)
+{
+    return ((size_t)n * sizeof(fbk::LinearEntry) + ((size_t)4 * kMaxGrid + 1) * sizeof(fbk::ShareCut) + 255) / 256 * 256;
+}
+
 extern "C" size_t fluxbin_plan_table_bytes(int32_t n, int32_t B)
 {
     if (n < 1 || B < 1) return 0;
     // an upper bound over the table formats and the cut of the rest
     const int most = chunks_of(B, FLUXBIN_TABLES_FP32, kSplitRestBytes).n;
-    return (size_t)n * sizeof(fbk::LinearEntry) * (size_t)most;
+    return chunk_table_bytes(n) * (size_t)most;
 }
 
 extern "C" size_t fluxbin_plan_workspace_bytes(int32_t n, const fluxbin_weight_t *const *w, int32_t B)
@@ -538,6 +717,7 @@ extern "C" fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_
         if (!w[i] || !d_x[i] || !d_y[i]) return FLUXBIN_ERR_NULL;
         if (ldx[i] < w[i]->h.N || ldy[i] < w[i]->h.M) return FLUXBIN_ERR_RANGE;
         if ((((uintptr_t)d_x[i]) & 15) || (((uintptr_t)d_y[i]) & 15)) return FLUXBIN_ERR_ALIGNMENT;
+        if (w[i]->device != w[0]->device) return FLUXBIN_ERR_UNSUPPORTED;      // all members on one device
         if (w[i]->h.sps[0] != w[0]->h.sps[0]) return FLUXBIN_ERR_UNSUPPORTED;
         if (w[i]->table_format != w[0]->table_format) return FLUXBIN_ERR_UNSUPPORTED;
         if (w[i]->h.npairs[1] > 0) {          // the salient format only matters where there is a salient region
@@ -548,58 +728,68 @@ extern "C" fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_
     }
     if (sps1 == 0) sps1 = 1;
     if (ws_bytes < fluxbin_plan_workspace_bytes(n, w, B)) return FLUXBIN_ERR_BUFFER_TOO_SMALL;
+    int dev = -1;
+    FB_CUDA(cudaGetDevice(&dev));
+    if (dev != w[0]->device) return FLUXBIN_ERR_UNSUPPORTED;       // create (and run) the plan with the layers' device current
 
-    const int fmt = w[0]->table_format;
-    long long weight_bytes = 0;
-    for (int i = 0; i < n; ++i) weight_bytes += (long long)w[i]->h.total_bytes;
+    const int fmt = w[0]->table_format, sps0 = w[0]->h.sps[0];
+    long long weight_bytes = 0, items = 0, couple_cost = 0;
+    bool all_even = true;
+    std::vector<const FbHeader *> hs((size_t)n);
+    for (int i = 0; i < n; ++i) {
+        weight_bytes += (long long)w[i]->h.total_bytes;
+        items += (long long)(w[i]->h.npairs[0] + w[i]->h.npairs[1]) * w[i]->h.nrb;
+        const long long c = couple_cost_of(w[i]->h);
+        if (c == 0) all_even = false;
+        if (c > couple_cost) couple_cost = c;
+        hs[(size_t)i] = &w[i]->h;
+    }
+    if (!all_even) couple_cost = 0;
     const Chunks ch = chunks_of(B, fmt, weight_bytes);
     const int nchunks = ch.n, bt = ws_bt(B, fmt);
     const size_t ysz = y_is_fp32 ? 4 : 2;
-    fbk::LinearEntry *host = (fbk::LinearEntry *)std::malloc(sizeof(fbk::LinearEntry) * (size_t)n * nchunks);
-    if (!host) return FLUXBIN_ERR_UNSUPPORTED;
+    const size_t ctb = chunk_table_bytes(n);
+    std::vector<uint8_t> host(ctb * (size_t)nchunks, 0);
     fluxbin_plan *p = new (std::nothrow) fluxbin_plan;
-    if (!p) { std::free(host); return FLUXBIN_ERR_UNSUPPORTED; }
-    long long items = 0;
+    if (!p) return FLUXBIN_ERR_UNSUPPORTED;
+    std::vector<long long> cost_begin((size_t)n + 1);
     for (int c = 0; c < nchunks; ++c) {
         uint8_t *ws = (uint8_t *)d_workspace;
-        const int nb = chunk_nb(ch, fmt, c), b0 = chunk_begin(ch, fmt, c);
-        const int bc = build_cost_for(mode_for(nb, fmt));
+        PlanChunk pc;
+        pc.nb = chunk_nb(ch, fmt, c);
+        pc.mode = mode_for(pc.nb, fmt);
+        const int b0 = chunk_begin(ch, fmt, c);
+        CutModel m;
+        m.build_cost = build_cost_for(pc.mode);
+        item_costs(sps0, sps1, m.item_cost);
+        fbk::LinearEntry *entries = (fbk::LinearEntry *)(host.data() + ctb * (size_t)c);
         long long cost = 0;
-        items = 0;
         for (int i = 0; i < n; ++i) {
             float *acc = (float *)ws;
             unsigned *tickets = (unsigned *)(ws + acc_bytes(w[i], bt));
-            fill_entry(host[(size_t)c * n + i], w[i], d_x[i] + (int64_t)b0 * ldx[i], ldx[i],
-                       (uint8_t *)d_y[i] + (size_t)b0 * ldy[i] * ysz, ldy[i], acc, tickets, cost);
-            cost += entry_cost(w[i]->h, sps1, bc);
-            items += (long long)(w[i]->h.npairs[0] + w[i]->h.npairs[1]) * w[i]->h.nrb;
+            fill_entry(entries[i], w[i], d_x[i] + (int64_t)b0 * ldx[i], ldx[i], (uint8_t *)d_y[i] + (size_t)b0 * ldy[i] * ysz,
+                       ldy[i], acc, tickets);
+            cost_begin[(size_t)i] = cost;
+            cost += entry_cost(w[i]->h, sps1, m.build_cost);
             ws += entry_ws_bytes(w[i], bt);
         }
-        p->chunk_nb.push_back(nb);
-        p->chunk_build_cost.push_back(bc);
-        p->chunk_total_cost.push_back(cost);
+        cost_begin[(size_t)n] = cost;
+        cudaError_t e = launch_shape(dev, pc.mode, sps0, sps1, cost, w[0]->num_sms, items, couple_cost, true, &pc.shape);
+        if (e != cudaSuccess) { delete p; return cuda_fail(e); }
+        m.np = pc.shape.np;
+        fbk::ShareCut *cuts = (fbk::ShareCut *)(entries + n);
+        cut_launch(hs.data(), cost_begin.data(), n, m, pc.shape, cuts);
+        pc.d_entries = (const fbk::LinearEntry *)((uint8_t *)d_table + ctb * (size_t)c);
+        pc.d_cuts = (const fbk::ShareCut *)(pc.d_entries + n);
+        p->chunks.push_back(pc);
     }
     cudaStream_t s = (cudaStream_t)cuda_stream;
-    cudaError_t e = cudaMemcpyAsync(d_table, host, sizeof(fbk::LinearEntry) * (size_t)n * nchunks, cudaMemcpyHostToDevice, s);
+    cudaError_t e = cudaMemcpyAsync(d_table, host.data(), host.size(), cudaMemcpyHostToDevice, s);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
-    std::free(host);
     if (e != cudaSuccess) { delete p; return cuda_fail(e); }
 
-    p->n = n; p->B = B; p->y_fp32 = y_is_fp32 != 0; p->nchunks = nchunks; p->table_format = fmt;
-    p->sps0 = w[0]->h.sps[0]; p->sps1 = sps1; p->num_sms = w[0]->num_sms;
-    p->items = items;
-    p->couple_cost = 0;
-    {
-        bool all_even = true;
-        for (int i = 0; i < n; ++i) {
-            long long c = couple_cost_of(w[i]->h);
-            if (c == 0) all_even = false;
-            if (c > p->couple_cost) p->couple_cost = c;
-        }
-        if (!all_even) p->couple_cost = 0;
-    }
-    item_costs(p->sps0, sps1, p->item_cost);
-    p->d_table = (const fbk::LinearEntry *)d_table;
+    p->n = n; p->B = B; p->y_fp32 = y_is_fp32 != 0; p->table_format = fmt; p->device = dev;
+    p->sps0 = sps0; p->sps1 = sps1;
     p->d_counters = (unsigned *)((uint8_t *)d_workspace + fluxbin_plan_workspace_bytes(n, w, B) - 256);
     *out = p;
     return FLUXBIN_OK;
@@ -608,55 +798,32 @@ extern "C" fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_
 extern "C" fluxbin_status_t fluxbin_plan_run(const fluxbin_plan_t *plan, void *cuda_stream)
 {
     if (!plan) return FLUXBIN_ERR_NULL;
+    int dev = -1;
+    FB_CUDA(cudaGetDevice(&dev));
+    if (dev != plan->device) return FLUXBIN_ERR_UNSUPPORTED;      // the plan's layers live on another device
     cudaStream_t s = (cudaStream_t)cuda_stream;
     fbk::LaunchParams p;
     std::memset(&p.single, 0, sizeof(p.single));
     p.n = plan->n;
     p.y_fp32 = plan->y_fp32;
-    p.item_cost[0] = plan->item_cost[0];
-    p.item_cost[1] = plan->item_cost[1];
     p.counters = plan->d_counters;
-    for (int c = 0; c < plan->nchunks; ++c) {
-        const int nb = plan->chunk_nb[c];
-        p.table = plan->d_table + (size_t)c * plan->n;
-        p.nb = nb;
-        p.build_cost = plan->chunk_build_cost[c];
-        p.total_cost = plan->chunk_total_cost[c];
-        cudaError_t e = launch_mode(mode_for(nb, plan->table_format), plan->sps0, plan->sps1, plan->num_sms, p, plan->items,
-                                    plan->couple_cost, s);
+    for (const PlanChunk &pc : plan->chunks) {
+        p.table = pc.d_entries;
+        p.cuts = pc.d_cuts;
+        p.nb = pc.nb;
+        p.nshares = pc.shape.nshares;
+        cudaError_t e = launch_kernel(pc.mode, plan->sps0, plan->sps1, pc.shape, p, s);
         if (e != cudaSuccess) return cuda_fail(e);
     }
     return FLUXBIN_OK;
 }
 
-extern "C" int32_t fluxbin_plan_num_launches(const fluxbin_plan_t *plan) { return plan ? plan->nchunks : -1; }
-
-// the launch shape of a kernel family with 4-byte table entries that reads (sps0, sps1) layers
-template <int BT>
-static cudaError_t launch_shape_geom1(int s0, int s1, long long total_cost, int num_sms, long long items, long long couple_cost,
-                                      LaunchShape *shape)
-{
-    if (s0 == 16 && s1 == 16) return launch_shape<16, 16, BT>(total_cost, num_sms, items, couple_cost, shape);
-    if (s0 == 16) return launch_shape<16, 1, BT>(total_cost, num_sms, items, couple_cost, shape);
-    if (s0 == 8) return launch_shape<8, 1, BT>(total_cost, num_sms, items, couple_cost, shape);
-    return launch_shape<4, 1, BT>(total_cost, num_sms, items, couple_cost, shape);
-}
+extern "C" int32_t fluxbin_plan_num_launches(const fluxbin_plan_t *plan) { return plan ? (int32_t)plan->chunks.size() : -1; }
 
 extern "C" int32_t fluxbin_plan_pairs_per_row_block(const fluxbin_plan_t *plan)
 {
-    if (!plan) return -1;
-    // the two-pair kernel exists for 4-byte table entries only: one vector, or two with fp16 entries
-    const int mode = mode_for(plan->chunk_nb[0], plan->table_format);       // the plan's first launch
-    LaunchShape shape;
-    cudaError_t e;
-    if (mode == 1)
-        e = launch_shape_geom1<1>(plan->sps0, plan->sps1, plan->chunk_total_cost[0], plan->num_sms, plan->items, plan->couple_cost, &shape);
-    else if (mode == 16 + 2)
-        e = launch_shape_geom1<16 + 2>(plan->sps0, plan->sps1, plan->chunk_total_cost[0], plan->num_sms, plan->items, plan->couple_cost, &shape);
-    else
-        return 1;
-    if (e != cudaSuccess) return -1;
-    return shape.couples ? 2 : 1;
+    if (!plan || plan->chunks.empty()) return -1;
+    return plan->chunks[0].shape.np;       // the plan's first launch
 }
 
 extern "C" void fluxbin_plan_free(fluxbin_plan_t *plan) { delete plan; }
@@ -687,6 +854,6 @@ extern "C" fluxbin_status_t fluxbin_debug_tables(const fluxbin_weight_t *w, cons
 // Instrumented build only: copy the per-CTA phase timestamps of the last launch to the host.
 extern "C" int fluxbin_debug_trace(unsigned long long *h_out)
 {
-    return (int)cudaMemcpyFromSymbol(h_out, fbk::g_fb_trace, sizeof(unsigned long long) * 1024 * 12);
+    return (int)cudaMemcpyFromSymbol(h_out, fbk::g_fb_trace, sizeof(unsigned long long) * 8 * 1024 * 12);
 }
 #endif

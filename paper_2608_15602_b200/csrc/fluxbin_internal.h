@@ -5,6 +5,7 @@
 #include "../../include/fluxbin.h"
 #include "fluxbin_layout.h"
 
+#include <atomic>
 #include <vector>
 
 namespace fb {
@@ -18,8 +19,20 @@ struct SalSvec {
 fluxbin_status_t validate_dims(const fluxbin_layer_desc_t *d);
 void salient_svecs(const fluxbin_layer_desc_t *d, int sps1, std::vector<SalSvec> &out);
 fluxbin_status_t check_header(const void *p, size_t bytes, FbHeader &h);
+// shared-memory opt-in of every instantiation of the layer kernel on the current device
+fluxbin_status_t opt_in_all_kernels();
 // remember a CUDA error code for fluxbin_last_cuda_error(), clear the runtime's sticky state, return FLUXBIN_ERR_CUDA
 fluxbin_status_t record_cuda_error(int cuda_error);
+
+constexpr int kMaxDevices = 64;
+constexpr int kMaxGrid = 1024;             // CTAs per launch (a B200 runs 444 at most)
+constexpr int kMaxSingleShares = 512;      // CTAs of a one-layer launch: its share bounds travel in the kernel parameters
+
+// Launch shape and share bounds of a one-layer launch in one launch mode (see cut_launch in fluxbin_api.cu).
+struct SingleLaunch {
+    int grid, np;
+    int cut[kMaxSingleShares + 1];
+};
 
 } // namespace fb
 
@@ -33,6 +46,7 @@ struct fluxbin_weight {
     int tile_rb;  // row blocks (of 32 rows) per arrival-counter tile
     int ntiles;
     int table_format;   // FLUXBIN_TABLES_FP32 / _FP16: how batched launches (B >= 2) hold their table entries
+    mutable std::atomic<fb::SingleLaunch *> single[6];   // per launch mode, made on first use, owned by the handle
 };
 
 #endif

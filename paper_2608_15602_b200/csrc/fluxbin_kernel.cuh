@@ -54,28 +54,17 @@ template <int BT> struct Cfg {
     static constexpr int kMinBlocks = (geom(BT) == 4) ? 1 : (geom(BT) == 2) ? 2 : 3;
 };
 constexpr int kMaxTiles = 1024;
-#ifndef FB_DEPTH
-#define FB_DEPTH 2
-#endif
-constexpr int kDepth = FB_DEPTH;    // register sets (items in flight per warp) in the main loop
-#ifndef FB_DEPTH2
-#define FB_DEPTH2 3
-#endif
+constexpr int kDepth = 2;    // register sets (items in flight per warp) in the main loop
 // The two-vector kernel runs 2 CTAs per SM (its tables are twice as large), so a thread may hold 128
 // registers and fewer warps cover the load latency: it keeps more items in flight per warp
 // (measured at batch 2 on a 16-layer stack: depth 2 3.49 TB/s, depth 3 3.56, depth 4 3.38).
-constexpr int kDepth2 = FB_DEPTH2;
-#ifndef FB_DEPTH4
-#define FB_DEPTH4 2
-#endif
-template <int BT> struct DepthFor { static constexpr int value = geom(BT) == 4 ? FB_DEPTH4 : geom(BT) == 2 ? kDepth2 : kDepth; };
-#ifndef FB_PF
-#define FB_PF 1
-#endif
+constexpr int kDepth2 = 3;
+constexpr int kDepth4 = 2;   // 16-byte entries: one CTA of 16 warps per SM
+template <int BT> struct DepthFor { static constexpr int value = geom(BT) == 4 ? kDepth4 : geom(BT) == 2 ? kDepth2 : kDepth; };
 // L2 prefetch distance in loop trips (one trip = kDepth items per warp).  Measured: 1 trip 5.40 TB/s,
 // 2 trips 5.26, 3 trips 4.21, 8 trips 3.58 in a stripped copy of the loop -- far prefetches compete with
 // the demand loads instead of helping them.
-constexpr int kPrefetchTrips = FB_PF;
+constexpr int kPrefetchTrips = 1;
 
 // One layer of a launch.
 struct LinearEntry {
@@ -85,26 +74,38 @@ struct LinearEntry {
     float *acc;              // [BT][Mpad] split-K accumulators, zero on entry and on exit
     unsigned *tickets;       // [ntiles] arrival counters, zero on entry and on exit
     long long ldx, ldy;
-    long long cost_begin;    // summed cost of the entries before this one
+    long long reserved0;
     unsigned long long off_coldesc, off_items[2];
     int M, N, Kb, Mpad, nrb;
     int npairs[2];
     int tile_rb, ntiles;
-    int reserved;
+    int sal_last_w;          // table slots of the last salient pair (32; 16 or 8: stored narrow)
 };
+
+// Where a share of a launch begins: layer `entry`, work item `item` of it (a work item is one row block of one
+// work pair -- NP pairs of the global region walked together, or one salient pair -- numbered pair-major:
+// global region first).  The host cuts the cost line of the launch once and hands every share its bounds.
+struct ShareCut {
+    int entry, item;
+};
+
+constexpr int kMaxSingleShares = 512;      // shares (= CTAs) of a launch whose cuts travel in the parameters
 
 struct LaunchParams {
     const LinearEntry *table;   // device table of n entries; nullptr: the single entry below
+    const ShareCut *cuts;       // device [nshares + 1] with a table; nullptr: single_cut below
     LinearEntry single;
-    long long total_cost;
     int n;
     int nb;                     // live batch rows (<= BT)
     int y_fp32;
-    int item_cost[2];           // relative time of one item of each region (work split)
-    int build_cost;             // relative time of building one table set
-    long long static_cost;      // part of the cost line dealt out as one share per CTA
-    int nshares;                // grid size + number of small shares drawn dynamically from the rest
+    int nshares;                // grid size + number of small shares drawn dynamically after it
     unsigned *counters;         // [2] share counter and exit counter, zero on entry and on exit
+#ifdef FB_TRACE
+    int trace_slot;             // instrumented build: which of the eight trace buffers this launch writes
+#endif
+    int head_bytes;             // EXPERIMENT: bytes of the first segment prefetched into L2 before the wait
+    int early_items;            // EXPERIMENT: two-pair kernel requests its first items before the wait
+    int single_cut[kMaxSingleShares + 1];    // first work item of share s of the single entry; [nshares] = all items
 };
 
 // The tables start at this shared-window address.  It is a compile-time constant so that it can
@@ -114,8 +115,10 @@ constexpr uint32_t kTabBase = 0x800u;
 
 template <int BT> struct TabCfg {
     static constexpr int kTableBytes = (geom(BT) == 4) ? 131072 : 65536;
-    // scale-fusion scratch, tile counters (+ count of completed tiles), work range, copy of the current entry
-    static constexpr int kSmallBytes = 256 * nvec(BT) * 4 + (kMaxTiles + 4) * 4 + 32 + 128;
+    // scale-fusion scratch (for two table sets when two fit side by side: 4-byte entries), tile counters
+    // (+ count of completed tiles), work range, copy of the current entry
+    static constexpr int kScratchFloats = 256 * nvec(BT) * (geom(BT) == 1 ? 2 : 1);
+    static constexpr int kSmallBytes = kScratchFloats * 4 + (kMaxTiles + 4) * 4 + 32 + 128;
     // offset of slot sigma from the table base at step 0; entry p adds p << 8.
     // lane_const(lane ^ s) == lane_const(lane) ^ lane_const(s)
     __host__ __device__ static constexpr uint32_t lane_const(uint32_t sigma)
@@ -124,7 +127,9 @@ template <int BT> struct TabCfg {
     }
 };
 
-template <int SPS> struct ItemBytes { static constexpr int value = FB_ITEM_BITS_BYTES + 64 * (32 / SPS); };
+// W = steps (table slots) per item: 32, or 16 / 8 for the narrow last pair of a salient region
+template <int SPS, int W = 32> struct ItemBytes { static constexpr int value = 32 * W + 64 * (W / SPS); };
+static_assert(ItemBytes<16>::value == FB_ITEM_BITS_BYTES + 64 * 2, "full items: 1024 bytes of weight bits");
 
 __device__ __forceinline__ float h2f(uint32_t bits16) { return __half2float(__ushort_as_half((unsigned short)bits16)); }
 
@@ -237,26 +242,42 @@ template <int BT> struct BuildInput {
     uint32_t e;        // {u16 column, fp16 alpha}
 };
 
+// The static half of a table set's inputs: {u16 column, fp16 alpha} of (slot tid/8, n tid%8) from the pair's
+// column table.  It belongs to the packed layer, so it may be requested before the launch's predecessor is done.
 template <int BT>
-__device__ __forceinline__ void fetch_build_input(BuildInput<BT> &in, const uint8_t *pair_desc, const uint16_t *x,
-                                                  int64_t ldx, int nb, int col0_a, int col0_b, int ncols)
+__device__ __forceinline__ void fetch_build_desc(BuildInput<BT> &in, const uint8_t *pair_desc)
 {
     const int tid = threadIdx.x;
     if (Cfg<BT>::kThreads > 256 && tid >= 256) return;      // one thread per table column
-    // {u16 column, fp16 alpha} of (slot tid/8, n tid%8).  For a global pair the column is also known
-    // from the pair's position, so x and alpha are fetched side by side, not in a chain.
+    in.e = __ldg((const uint32_t *)pair_desc + tid);
+}
+
+// The activations of the thread's column.  For a global pair the column is known from the pair's position, so
+// this load does not wait for the column table; for a salient pair it is the column the table names.
+template <int BT>
+__device__ __forceinline__ void fetch_build_x(BuildInput<BT> &in, const uint16_t *x, int64_t ldx, int nb, int col0_a, int col0_b,
+                                              int ncols)
+{
+    const int tid = threadIdx.x;
+    if (Cfg<BT>::kThreads > 256 && tid >= 256) return;
     if (col0_a >= 0) {       // first unit of the pair: slots 0..15, second unit: slots 16..31
         const uint32_t col = (uint32_t)(tid < 128 ? col0_a : col0_b) + (uint32_t)(tid & 127);
         const bool live = col < (uint32_t)ncols;          // padded columns carry alpha = 0
 #pragma unroll
         for (int b = 0; b < nvec(BT); ++b) in.xv[b] = (b < nb && live) ? h2f(__ldg(x + (int64_t)b * ldx + col)) : 0.f;
-        in.e = __ldg((const uint32_t *)pair_desc + tid);
     } else {
-        in.e = __ldg((const uint32_t *)pair_desc + tid);
         const uint32_t col = in.e & 0xffffu;
 #pragma unroll
         for (int b = 0; b < nvec(BT); ++b) in.xv[b] = (b < nb) ? h2f(__ldg(x + (int64_t)b * ldx + col)) : 0.f;
     }
+}
+
+template <int BT>
+__device__ __forceinline__ void fetch_build_input(BuildInput<BT> &in, const uint8_t *pair_desc, const uint16_t *x,
+                                                  int64_t ldx, int nb, int col0_a, int col0_b, int ncols)
+{
+    fetch_build_desc<BT>(in, pair_desc);
+    fetch_build_x<BT>(in, x, ldx, nb, col0_a, col0_b, ncols);
 }
 
 // Scratch index of a_n of table slot `slot`, batch vector b: rows of 32 slots, rotated by 4n so that both
@@ -266,8 +287,9 @@ template <int BT> __device__ __forceinline__ int abuf_index(int slot, int n, int
     return (n * nvec(BT) + b) * 32 + ((slot + 4 * n) & 31);
 }
 
+// Scale fusion (Eq. 11): a_n = x * alpha of the thread's table column into the scratch.
 template <int BT>
-__device__ __forceinline__ void build_tables(const BuildInput<BT> &in, float *abuf, uint32_t half_off = 0)
+__device__ __forceinline__ void stage_build_input(const BuildInput<BT> &in, float *abuf)
 {
     const int tid = threadIdx.x;
     constexpr int NV = nvec(BT);
@@ -276,7 +298,15 @@ __device__ __forceinline__ void build_tables(const BuildInput<BT> &in, float *ab
 #pragma unroll
         for (int b = 0; b < NV; ++b) abuf[abuf_index<BT>(tid >> 3, tid & 7, b)] = in.xv[b] * al;   // exact in fp32: two 11-bit significands
     }
-    __syncthreads();
+}
+
+// All 256 entries of the 32 tables of one table set from the staged a_n (Eq. 14); the caller puts a barrier
+// between staging and this, and one after it.
+template <int BT>
+__device__ __forceinline__ void enumerate_tables(const float *abuf, uint32_t half_off)
+{
+    const int tid = threadIdx.x;
+    constexpr int NV = nvec(BT);
     const int lane = tid & 31, warp = tid >> 5;
     // EB entries at a time: the high index bits fix a base value, the low LB bits are enumerated by
     // doubling (entry p | 2^n = entry p + 2 a_n), one add per entry.  Up to four batch vectors of an entry are
@@ -289,38 +319,58 @@ __device__ __forceinline__ void build_tables(const BuildInput<BT> &in, float *ab
     constexpr int PW = 256 / (Cfg<BT>::kWarps / NG);   // table entries per warp: p = (warp % (kWarps/NG))*PW + ...
     constexpr int LB = (PV == 4) ? 3 : 4, EB = 1 << LB;
     static_assert(PW % EB == 0, "a warp enumerates whole blocks of entries");
-    {
-        const int wl = NG == 1 ? warp : warp % (Cfg<BT>::kWarps / NG);
-        const int b0 = NG == 1 ? 0 : PV * ((warp / (Cfg<BT>::kWarps / NG)) ^ ((lane >> 3) & 1));
-        float a[8][PV];
+    const int wl = NG == 1 ? warp : warp % (Cfg<BT>::kWarps / NG);
+    const int b0 = NG == 1 ? 0 : PV * ((warp / (Cfg<BT>::kWarps / NG)) ^ ((lane >> 3) & 1));
+    float a[8][PV];
 #pragma unroll
-        for (int n = 0; n < 8; ++n)
+    for (int n = 0; n < 8; ++n)
 #pragma unroll
-            for (int b = 0; b < PV; ++b) a[n][b] = abuf[abuf_index<BT>(lane, n, b0 + b)];
+        for (int b = 0; b < PV; ++b) a[n][b] = abuf[abuf_index<BT>(lane, n, b0 + b)];
 #pragma unroll 1
-        for (int p0 = wl * PW; p0 < (wl + 1) * PW; p0 += EB) {
-            float v[EB][PV];
+    for (int p0 = wl * PW; p0 < (wl + 1) * PW; p0 += EB) {
+        float v[EB][PV];
 #pragma unroll
-            for (int b = 0; b < PV; ++b) {
-                float base = 0.f;
+        for (int b = 0; b < PV; ++b) {
+            float base = 0.f;
 #pragma unroll
-                for (int n = 7; n >= LB; --n) base += ((p0 >> n) & 1) ? a[n][b] : -a[n][b];
+            for (int n = 7; n >= LB; --n) base += ((p0 >> n) & 1) ? a[n][b] : -a[n][b];
 #pragma unroll
-                for (int n = LB - 1; n >= 0; --n) base -= a[n][b];
-                v[0][b] = base;
+            for (int n = LB - 1; n >= 0; --n) base -= a[n][b];
+            v[0][b] = base;
 #pragma unroll
-                for (int n = 0; n < LB; ++n)
+            for (int n = 0; n < LB; ++n)
 #pragma unroll
-                    for (int q = 0; q < (1 << n); ++q) v[q | (1 << n)][b] = v[q][b] + 2.f * a[n][b];
-            }
+                for (int q = 0; q < (1 << n); ++q) v[q | (1 << n)][b] = v[q][b] + 2.f * a[n][b];
+        }
 #pragma unroll
-            for (int q = 0; q < EB; ++q) {
-                const uint32_t addr = half_off | TabCfg<BT>::lane_const((uint32_t)lane) | ((uint32_t)(p0 + q) << 8);
-                if constexpr (half_tables(BT)) sts_entry_h<PV>(addr + 2u * (uint32_t)b0, v[q]);    // rounded once, from the fp32 sum
-                else sts_entry<PV>(addr, v[q]);
-            }
+        for (int q = 0; q < EB; ++q) {
+            const uint32_t addr = half_off | TabCfg<BT>::lane_const((uint32_t)lane) | ((uint32_t)(p0 + q) << 8);
+            if constexpr (half_tables(BT)) sts_entry_h<PV>(addr + 2u * (uint32_t)b0, v[q]);    // rounded once, from the fp32 sum
+            else sts_entry<PV>(addr, v[q]);
         }
     }
+}
+
+// One table set; ends with the tables visible to the whole CTA.
+template <int BT>
+__device__ __forceinline__ void build_tables(const BuildInput<BT> &in, float *abuf, uint32_t half_off = 0)
+{
+    stage_build_input<BT>(in, abuf);
+    __syncthreads();
+    enumerate_tables<BT>(abuf, half_off);
+    __syncthreads();
+}
+
+// Two table sets side by side (4-byte entries: slots 0..31 and 32..63 of the 256-byte rows) behind one pair of barriers.
+template <int BT>
+__device__ __forceinline__ void build_tables2(const BuildInput<BT> &in_a, const BuildInput<BT> &in_b, float *abuf)
+{
+    static_assert(geom(BT) == 1, "two table sets side by side need 4-byte entries");
+    stage_build_input<BT>(in_a, abuf);
+    stage_build_input<BT>(in_b, abuf + 256 * nvec(BT));
+    __syncthreads();
+    enumerate_tables<BT>(abuf, 0u);
+    enumerate_tables<BT>(abuf + 256 * nvec(BT), 128u);
     __syncthreads();
 }
 
@@ -328,23 +378,25 @@ __device__ __forceinline__ void build_tables(const BuildInput<BT> &in, float *ab
 // Stage (ii)+(iii) for one run of row blocks of one pair.
 // SPS = sub-vectors per row-scale segment (16: one scale per unit and row; 1: one per sub-vector).
 // ---------------------------------------------------------------------------------------------
-template <int SPS> struct ItemRegs {
+template <int SPS, int W = 32> struct ItemRegs {
+    static constexpr int kSc = (W / SPS + 1) / 2;     // 32-bit words of row scales per lane
     uint4 b0, b1;                         // weight bytes of steps 0..15 / 16..31
-    uint32_t sc[(SPS == 16) ? 1 : (SPS == 8) ? 2 : (SPS == 4) ? 4 : 16];
+    uint32_t sc[kSc];
 };
 
-// pl = item + lane*16 (weight bytes), ps = item + 1024 + lane*(scale bytes per lane, at most 16);
-// `off` is a compile-time byte offset added to both (the stride to a later item).
-template <int SPS> __device__ __forceinline__ void load_item(ItemRegs<SPS> &r, const uint8_t *pl, const uint8_t *ps, int off)
+// pl = item + lane * min(W, 16) (weight bytes), ps = item + 32 * W + lane * (scale bytes per lane and plane, at
+// most 16); `off` is a compile-time byte offset added to both (the stride to a later item).
+template <int SPS, int W = 32> __device__ __forceinline__ void load_item(ItemRegs<SPS, W> &r, const uint8_t *pl, const uint8_t *ps, int off)
 {
-    r.b0 = ldg_stream_v4(pl + off);
-    r.b1 = ldg_stream_v4(pl + off + 512);
-    if constexpr (SPS == 16) r.sc[0] = ldg_stream_u32(ps + off);
-    else if constexpr (SPS == 8) { uint2 t = ldg_stream_v2(ps + off); r.sc[0] = t.x; r.sc[1] = t.y; }
-    else if constexpr (SPS == 4) { uint4 t = ldg_stream_v4(ps + off); r.sc[0] = t.x; r.sc[1] = t.y; r.sc[2] = t.z; r.sc[3] = t.w; }
+    constexpr int kSc = ItemRegs<SPS, W>::kSc;
+    if constexpr (W == 8) { const uint2 t = ldg_stream_v2(pl + off); r.b0.x = t.x; r.b0.y = t.y; }
+    else r.b0 = ldg_stream_v4(pl + off);
+    if constexpr (W == 32) r.b1 = ldg_stream_v4(pl + off + 512);
+    if constexpr (kSc == 1) r.sc[0] = ldg_stream_u32(ps + off);
+    else if constexpr (kSc == 2) { uint2 t = ldg_stream_v2(ps + off); r.sc[0] = t.x; r.sc[1] = t.y; }
     else {
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
+        for (int q = 0; q < kSc / 4; ++q) {               // planes of 8 halves per lane
             uint4 t = ldg_stream_v4(ps + off + q * 512);
             r.sc[4 * q] = t.x; r.sc[4 * q + 1] = t.y; r.sc[4 * q + 2] = t.z; r.sc[4 * q + 3] = t.w;
         }
@@ -426,15 +478,13 @@ template <> struct LaneAddr<16 + 2> : LaneAddr<1> {};
 template <> struct LaneAddr<16 + 4> : LaneAddr<2> {};
 template <> struct LaneAddr<16 + 8> : LaneAddr<4> {};
 
-#ifndef FB_SPLIT_NV
-#define FB_SPLIT_NV 4
-#endif
 // Two alternating partial sums per vector shorten the dependency chain of a segment's adds; with four or more
 // vectors the adds of one lookup already space out each vector's chain (+1-5 % without the split there).
-template <int SPS, int BT, int HALF = 0>
-__device__ __forceinline__ void compute_item(const ItemRegs<SPS> &r, const LaneAddr<BT> &la, float (&out)[nvec(BT)])
+constexpr int kSplitBelowVectors = 4;
+template <int SPS, int BT, int HALF = 0, int W = 32>
+__device__ __forceinline__ void compute_item(const ItemRegs<SPS, W> &r, const LaneAddr<BT> &la, float (&out)[nvec(BT)])
 {
-    constexpr int NSEG = 32 / SPS;
+    constexpr int NSEG = W / SPS;
     constexpr int NV = nvec(BT);
     const uint32_t w[8] = {r.b0.x, r.b0.y, r.b0.z, r.b0.w, r.b1.x, r.b1.y, r.b1.z, r.b1.w};
 #pragma unroll
@@ -456,18 +506,18 @@ __device__ __forceinline__ void compute_item(const ItemRegs<SPS> &r, const LaneA
                     lds_entry_h<BT, HALF>(addr, e);
 #pragma unroll
                     for (int i = 0; i < geom(BT); ++i) {
-                        if ((q & 1) && NV < FB_SPLIT_NV) add_h2(s1[2 * i], s1[2 * i + 1], e[i]); else add_h2(s0[2 * i], s0[2 * i + 1], e[i]);
+                        if ((q & 1) && NV < kSplitBelowVectors) add_h2(s1[2 * i], s1[2 * i + 1], e[i]); else add_h2(s0[2 * i], s0[2 * i + 1], e[i]);
                     }
                 } else {
                     Vec<BT> e = lds_entry<BT, HALF>(addr);
 #pragma unroll
                     for (int b = 0; b < NV; ++b) {
-                        if ((q & 1) && NV < FB_SPLIT_NV) s1[b] += e.v[b]; else s0[b] += e.v[b];
+                        if ((q & 1) && NV < kSplitBelowVectors) s1[b] += e.v[b]; else s0[b] += e.v[b];
                     }
                 }
             }
 #pragma unroll
-            for (int b = 0; b < NV; ++b) seg[b] = (NV >= FB_SPLIT_NV) ? s0[b] : s0[b] + s1[b];
+            for (int b = 0; b < NV; ++b) seg[b] = (NV >= kSplitBelowVectors) ? s0[b] : s0[b] + s1[b];
         }
         float scale = h2f((r.sc[j >> 1] >> ((j & 1) * 16)) & 0xffffu);
 #pragma unroll
@@ -522,11 +572,11 @@ __device__ __forceinline__ void compute_half_h2(const uint4 &b, const uint32_t *
     }
 }
 
-template <int SPS, int BT>
-__device__ __forceinline__ void finish_item(const ItemRegs<SPS> &r, const LaneAddr<BT> &la, float *accp, int Mpad)
+template <int SPS, int BT, int W = 32>
+__device__ __forceinline__ void finish_item(const ItemRegs<SPS, W> &r, const LaneAddr<BT> &la, float *accp, int Mpad)
 {
     float out[nvec(BT)];
-    compute_item<SPS, BT>(r, la, out);
+    compute_item<SPS, BT, 0, W>(r, la, out);
 #pragma unroll
     for (int b = 0; b < nvec(BT); ++b) red_add_f32(accp + (int64_t)b * Mpad, out[b]);
 }
@@ -550,40 +600,41 @@ __device__ __forceinline__ void preload_first(ItemRegs<SPS> &r, const uint8_t *p
 // in flight per SM to cover the L2 latency at full HBM rate).  A trip of the steady loop handles
 // kDepth items with every address a pointer plus an immediate; each warp also bulk-prefetches,
 // kPrefetchTrips trips ahead, its share of the kDepth*kWarps items the CTA reads per trip.
-template <int SPS, int BT>
+template <int SPS, int BT, int W = 32>
 __device__ __forceinline__ void process_rows(const uint8_t *pair_items, int rb_lo, int rb_hi,
                                              const LaneAddr<BT> &la, float *acc, int Mpad,
-                                             const ItemRegs<SPS> *pre = nullptr)   // pre: preload_first's result
+                                             const ItemRegs<SPS, W> *pre = nullptr)   // pre: preload_first's result
 {
-    constexpr int IB = ItemBytes<SPS>::value;
+    constexpr int IB = ItemBytes<SPS, W>::value;
     constexpr int kWarps = Cfg<BT>::kWarps;
     constexpr int STRIDE = kWarps * IB;                   // bytes between a warp's consecutive items
-    constexpr int SB = (SPS == 16) ? 4 : (SPS == 8) ? 8 : 16;   // scale bytes per lane (per plane)
+    constexpr int kSc = ItemRegs<SPS, W>::kSc;
+    constexpr int SB = kSc == 1 ? 4 : kSc == 2 ? 8 : 16;  // scale bytes per lane (per plane)
     constexpr int D = (SPS == 1) ? 1 : DepthFor<BT>::value;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int first = rb_lo + warp;
     if (first >= rb_hi) return;
     const int n = (rb_hi - first + kWarps - 1) / kWarps;  // items of this warp
-    const uint8_t *pl = pair_items + (int64_t)first * IB + lane * 16;
-    const uint8_t *ps = pair_items + (int64_t)first * IB + FB_ITEM_BITS_BYTES + lane * SB;
+    const uint8_t *pl = pair_items + (int64_t)first * IB + lane * (W < 16 ? W : 16);
+    const uint8_t *ps = pair_items + (int64_t)first * IB + 32 * W + lane * SB;
     // this warp's prefetch window inside the block of D*kWarps items the CTA consumes per trip
     const uint8_t *pp = pair_items + (int64_t)(rb_lo + D * warp) * IB + (int64_t)kPrefetchTrips * D * STRIDE;
     const uint8_t *pend = pair_items + (int64_t)rb_hi * IB;
     float *accp = acc + first * 32 + lane;
 
-    ItemRegs<SPS> r[D];
+    ItemRegs<SPS, W> r[D];
 #pragma unroll
     for (int d = 0; d < D - 1; ++d) {
         if (d == 0 && pre) r[0] = *pre;
-        else if (d < n) load_item<SPS>(r[d], pl, ps, d * STRIDE);
+        else if (d < n) load_item<SPS, W>(r[d], pl, ps, d * STRIDE);
     }
     // items t .. t+D-1 are looked up while items t+D-1 .. t+2D-2 are loaded (warp-uniform guards)
     for (int t = 0; t < n; t += D) {
         if (lane == 0 && pp + D * IB <= pend) prefetch_l2(pp, D * IB);
 #pragma unroll
         for (int d = 0; d < D; ++d) {
-            if (t + d + D - 1 < n) load_item<SPS>(r[(d + D - 1) % D], pl, ps, (d + D - 1) * STRIDE);
-            if (t + d < n) finish_item<SPS, BT>(r[d], la, accp + d * (kWarps * 32), Mpad);
+            if (t + d + D - 1 < n) load_item<SPS, W>(r[(d + D - 1) % D], pl, ps, (d + D - 1) * STRIDE);
+            if (t + d < n) finish_item<SPS, BT, W>(r[d], la, accp + d * (kWarps * 32), Mpad);
         }
         pl += D * STRIDE;
         ps += D * STRIDE;
@@ -592,14 +643,64 @@ __device__ __forceinline__ void process_rows(const uint8_t *pair_items, int rb_l
     }
 }
 
+// Row blocks of the narrow last pair of a salient region (W = 8 or 16 steps per item, one scale per step).  These
+// items are small, so a warp keeps the next one in flight while it looks the current one up (with a single item
+// in flight a warp pays a full load latency per item whatever its size, which makes a narrow item as slow as a
+// full one).
+template <int W, int BT>
+__device__ __forceinline__ void process_rows_narrow(const uint8_t *pair_items, int rb_lo, int rb_hi, const LaneAddr<BT> &la,
+                                                    float *acc, int Mpad)
+{
+    constexpr int IB = ItemBytes<1, W>::value;
+    constexpr int kWarps = Cfg<BT>::kWarps;
+    constexpr int STRIDE = kWarps * IB;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int first = rb_lo + warp;
+    if (first >= rb_hi) return;
+    const int n = (rb_hi - first + kWarps - 1) / kWarps;
+    const uint8_t *pl = pair_items + (int64_t)first * IB + lane * (W < 16 ? W : 16);
+    const uint8_t *ps = pair_items + (int64_t)first * IB + 32 * W + lane * 16;
+    const uint8_t *pend = pair_items + (int64_t)rb_hi * IB;
+    float *accp = acc + first * 32 + lane;
+    ItemRegs<1, W> cur, nxt;
+    load_item<1, W>(cur, pl, ps, 0);
+#pragma unroll 1
+    for (int t = 0; t < n; ++t) {
+        if (t + 1 < n) load_item<1, W>(nxt, pl, ps, STRIDE);
+        if (lane == 0 && pl + 3 * STRIDE < pend) prefetch_l2(pl - lane * (W < 16 ? W : 16) + 2 * STRIDE, IB);
+        finish_item<1, BT, W>(cur, la, accp, Mpad);
+        cur = nxt;
+        pl += STRIDE;
+        ps += STRIDE;
+        accp += kWarps * 32;
+    }
+}
+
 // The same for TWO pairs whose table sets are resident together (slots 0..31 and 32..63, 4-byte entries):
 // for every row block the lane looks up the item of the first pair, then the item of the second
 // (items_b = the second pair's items), adds the two row sums and issues ONE reduction -- half the
 // atomic traffic and half the per-item bookkeeping.  One item is always in flight ahead.
 // BT: 1 (one vector, fp32 entries) or 16 + 2 (two vectors, fp16 entries: the same 4-byte slots).
+// The first row block's two items of this warp's run (the loads process_rows2 would start with), requested ahead
+// of the wait for the predecessor and of the table build.
+template <int SPS, int BT>
+__device__ __forceinline__ void preload_first2(ItemRegs<SPS> &ra, ItemRegs<SPS> &rb, const uint8_t *items_a, const uint8_t *items_b,
+                                               int rb_lo, int rb_hi)
+{
+    constexpr int IB = ItemBytes<SPS>::value;
+    constexpr int SB = (SPS == 16) ? 4 : (SPS == 8) ? 8 : 16;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int first = rb_lo + warp;
+    if (first >= rb_hi) return;
+    const int64_t o_l = (int64_t)first * IB + lane * 16, o_s = (int64_t)first * IB + FB_ITEM_BITS_BYTES + lane * SB;
+    load_item<SPS>(ra, items_a + o_l, items_a + o_s, 0);
+    load_item<SPS>(rb, items_b + o_l, items_b + o_s, 0);
+}
+
 template <int SPS, int BT>
 __device__ __forceinline__ void process_rows2(const uint8_t *items_a, const uint8_t *items_b, int rb_lo, int rb_hi,
-                                              const LaneAddr<1> &la, float *acc, int Mpad)
+                                              const LaneAddr<1> &la, float *acc, int Mpad,
+                                              const ItemRegs<SPS> *pre_a = nullptr, const ItemRegs<SPS> *pre_b = nullptr)
 {
     static_assert(geom(BT) == 1, "two table sets side by side need 4-byte entries");
     // lookups of one 128-bit half of an item, added to the row sums of the batch vectors
@@ -635,8 +736,11 @@ __device__ __forceinline__ void process_rows2(const uint8_t *items_a, const uint
     // The last row block is peeled off: the steady state has no guards in it, and the prefetch is one
     // predicated instruction (guards cost about 20 instructions per item in moves, predicates and branches).
     ItemRegs<SPS> ra, rb;
-    load_item<SPS>(ra, pla, psa, 0);
-    load_item<SPS>(rb, plb, psb, 0);
+    if (pre_a) { ra = *pre_a; rb = *pre_b; }
+    else {
+        load_item<SPS>(ra, pla, psa, 0);
+        load_item<SPS>(rb, plb, psb, 0);
+    }
     const int n_pf = lane < 2 * LPI ? n - (kPrefetchTrips + 1) : 0;      // trips in which this lane prefetches
     for (int t = 0; t < n - 1; ++t) {
         prefetch_line_if(pp, t < n_pf);
@@ -681,32 +785,24 @@ __device__ __forceinline__ void prefetch_run_head(const uint8_t *pair_items, int
 }
 
 #ifdef FB_TRACE
-// Instrumented build only: per-CTA phase timestamps (globaltimer, ns) for the cycle breakdown.
-__device__ unsigned long long g_fb_trace[1024][12];
-__device__ __forceinline__ void trace(int slot)
-{
-    if (threadIdx.x == 0 && blockIdx.x < 1024) {
-        unsigned long long t;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-        g_fb_trace[blockIdx.x][slot] = t;
-    }
-}
+// Instrumented build only: per-CTA phase timestamps (globaltimer, ns) of the last eight launches.
+// Slots: 0 CTA start, 11 before / 1 after the wait for the predecessor, 3 end of the CTA's last layer;
+// accumulated durations: 7 share and layer set-up, 9 input fetch (incl. the wait), 8 barrier before a build,
+// 4 table build, 5 row loop, 10 tile counts, 6 reduction epilogue, 2 drawing a share.
+__device__ unsigned long long g_fb_trace[8][1024][12];
 __device__ __forceinline__ unsigned long long trace_now()
 {
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// accumulate the time since t0 into a per-CTA phase total
-__device__ __forceinline__ void trace_add(int slot, unsigned long long t0)
-{
-    if (threadIdx.x == 0 && blockIdx.x < 1024) g_fb_trace[blockIdx.x][slot] += trace_now() - t0;
-}
-#define FB_TRACE_AT(slot) trace(slot)
+#define FB_TRACE_ROW g_fb_trace[P.trace_slot & 7][blockIdx.x]
+#define FB_TRACE_ON (threadIdx.x == 0 && blockIdx.x < 1024)
+#define FB_TRACE_AT(slot) do { if (FB_TRACE_ON) FB_TRACE_ROW[slot] = trace_now(); } while (0)
 #define FB_TRACE_T0(var) unsigned long long var = trace_now()
-#define FB_TRACE_ADD(slot, var) trace_add(slot, var)
+#define FB_TRACE_ADD(slot, var) do { if (FB_TRACE_ON) FB_TRACE_ROW[slot] += trace_now() - var; } while (0)
 #define FB_TRACE_SET(var) var = trace_now()
-#define FB_TRACE_ZERO() do { if (threadIdx.x == 0 && blockIdx.x < 1024) { g_fb_trace[blockIdx.x][4] = 0; g_fb_trace[blockIdx.x][5] = 0; g_fb_trace[blockIdx.x][6] = 0; g_fb_trace[blockIdx.x][7] = 0; g_fb_trace[blockIdx.x][1] = 0; g_fb_trace[blockIdx.x][2] = 0; g_fb_trace[blockIdx.x][8] = 0; g_fb_trace[blockIdx.x][9] = 0; g_fb_trace[blockIdx.x][10] = 0; } } while (0)
+#define FB_TRACE_ZERO() do { if (FB_TRACE_ON) { for (int i_ = 1; i_ < 12; ++i_) FB_TRACE_ROW[i_] = 0; } } while (0)
 #else
 #define FB_TRACE_AT(slot)
 #define FB_TRACE_T0(var)
@@ -752,40 +848,58 @@ __device__ __forceinline__ void reduce_and_store(const LinearEntry &E, int nb, i
     const int ndone = done_list[kMaxTiles];
     if (ndone > 0) {
         __threadfence();
-        // all rows of all completed tiles in one flat loop of 4-row groups, four 128-bit loads in
+        // all rows of all completed tiles in one flat loop of 4-row groups, six 128-bit loads in
         // flight per thread (the accumulators live in L2; one round trip serves ~8K rows per CTA)
         const int gpt = E.tile_rb * 8;                 // 4-row groups per tile
         constexpr int NV = nvec(BT);
         const int total = ndone * gpt * NV;
-        constexpr int U = 4;
+        constexpr int U = 6;
+        const bool vec_ok = (E.ldy & 3) == 0;          // rows in groups of four stay 8 / 16-byte aligned in y
+        // group idx of the flat list -> batch vector and first row (done_list is small and lives in shared memory,
+        // so the decode is repeated after the loads instead of being kept in registers across them)
+        // (idx is in range) -> element offset of the group in the accumulators, or -1 for rows beyond the padding
+        auto decode = [&](int idx, int &bb, int &row) -> int {
+            const int li = idx / (gpt * NV), rem = idx - li * (gpt * NV);
+            bb = rem / gpt;
+            row = (done_list[li] * gpt + (rem - bb * gpt)) * 4;
+            return row < E.Mpad ? bb * E.Mpad + row : -1;
+        };
         for (int base = tid; base < total; base += U * kThreads) {
             float4 v[U];
-            float *a[U];
-            int row[U], bb[U];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                int idx = base + u * kThreads;
-                a[u] = nullptr;
-                if (idx < total) {
-                    int li = idx / (gpt * NV), rem = idx - li * (gpt * NV);
-                    bb[u] = rem / gpt;
-                    row[u] = (done_list[li] * gpt + (rem - bb[u] * gpt)) * 4;
-                    if (row[u] < E.Mpad) a[u] = E.acc + (int64_t)bb[u] * E.Mpad + row[u];
-                }
+                const int idx = base + u * kThreads;
+                int bb, row;
+                const int eoff = idx < total ? decode(idx, bb, row) : -1;
+                if (eoff >= 0) v[u] = __ldcg((const float4 *)(E.acc + eoff));
             }
 #pragma unroll
-            for (int u = 0; u < U; ++u) if (a[u]) v[u] = __ldcg((const float4 *)a[u]);
-#pragma unroll
             for (int u = 0; u < U; ++u) {
-                if (!a[u]) continue;
-                __stcg((float4 *)a[u], make_float4(0.f, 0.f, 0.f, 0.f));
-                if (bb[u] >= nb) continue;
+                const int idx = base + u * kThreads;
+                if (idx >= total) break;
+                int bb, row;
+                const int eoff = decode(idx, bb, row);
+                if (eoff < 0) continue;
+                __stcg((float4 *)(E.acc + eoff), make_float4(0.f, 0.f, 0.f, 0.f));
+                if (bb >= nb) continue;
                 const float e[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+                if (vec_ok && row + 3 < E.M) {
+                    if (y_fp32) {
+                        *(float4 *)((float *)E.y + (int64_t)bb * E.ldy + row) = v[u];
+                    } else {
+                        const __half2 lo = __floats2half2_rn(e[0], e[1]), hi = __floats2half2_rn(e[2], e[3]);
+                        uint2 pk;
+                        pk.x = *(const uint32_t *)&lo;
+                        pk.y = *(const uint32_t *)&hi;
+                        *(uint2 *)((__half *)E.y + (int64_t)bb * E.ldy + row) = pk;
+                    }
+                    continue;
+                }
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    if (row[u] + k >= E.M) break;
-                    if (y_fp32) ((float *)E.y)[(int64_t)bb[u] * E.ldy + row[u] + k] = e[k];
-                    else ((__half *)E.y)[(int64_t)bb[u] * E.ldy + row[u] + k] = __float2half_rn(e[k]);
+                    if (row + k >= E.M) break;
+                    if (y_fp32) ((float *)E.y)[(int64_t)bb * E.ldy + row + k] = e[k];
+                    else ((__half *)E.y)[(int64_t)bb * E.ldy + row + k] = __float2half_rn(e[k]);
                 }
             }
         }
@@ -794,11 +908,8 @@ __device__ __forceinline__ void reduce_and_store(const LinearEntry &E, int nb, i
     __syncthreads();       // done_list / tile_cnt are reused by the next entry
 }
 
-#ifndef FB_MINB
-#define FB_MINB 3
-#endif
 template <int SPS0, int SPS1, int BT, int NP>
-__global__ void __launch_bounds__(Cfg<BT>::kThreads, (geom(BT) == 1) ? FB_MINB : Cfg<BT>::kMinBlocks)
+__global__ void __launch_bounds__(Cfg<BT>::kThreads, Cfg<BT>::kMinBlocks)
 fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
 {
     constexpr int kThreads = Cfg<BT>::kThreads, kWarps = Cfg<BT>::kWarps;
@@ -808,9 +919,9 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
     if (smem_base > kTabBase) return;                                    // the host probes this first
     uint8_t *small = smem + (kTabBase - smem_base) + TabCfg<BT>::kTableBytes;
     float *abuf = (float *)small;
-    int *tile_cnt = (int *)(abuf + 256 * nvec(BT));
+    int *tile_cnt = (int *)(abuf + TabCfg<BT>::kScratchFloats);
     int *done_list = tile_cnt;                     // compacted in place over the counters
-    int *range = tile_cnt + kMaxTiles + 4;        // [0]: first item, [1]: end item of this CTA in the entry
+    int *range = tile_cnt + kMaxTiles + 4;        // [2]: the share a CTA has drawn
     LinearEntry *Es = (LinearEntry *)(range + 8);  // the current entry, copied once (128 bytes)
     static_assert(sizeof(LinearEntry) == 128, "entry copy below moves 32 words");
     static_assert(NP == 1 || geom(BT) == 1, "two table sets side by side need 4-byte table entries");
@@ -821,92 +932,59 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
 
     // Programmatic dependent launch: let the next kernel in the stream start its own prologue as soon
     // as SM resources free up; below, this kernel in turn waits for its predecessor only at the point
-    // where it first touches data the predecessor may have written (activations, workspace) -- the
-    // index arithmetic and the first L2 prefetches of the (static) weights run ahead of that.
+    // where it first touches data the predecessor may have written (activations, workspace) -- everything
+    // that reads the packed layer alone (share bounds, column tables, the first weight bytes and the L2
+    // prefetches behind them) runs ahead of that.
     asm volatile("griddepcontrol.launch_dependents;");
     bool predecessor_done = false;
 
     LaneAddr<BT> la;
     la.init(tid & 31);
 
-    const long long w0 = P.item_cost[0], w1 = P.item_cost[1];
-
-    // The first P.static_cost of the cost line is cut into one big share per CTA; the rest into small
-    // shares that CTAs draw from a counter when they finish (no CTA waits for another).  Co-resident
-    // CTAs do not progress at the same speed (the warp schedulers favour the older ones), so the
-    // quick ones pick up the small shares and the SM stays fully occupied until the end.
-    const int G = (int)gridDim.x;
+    // The host has cut the cost line of the launch: the first gridDim.x shares are dealt one per CTA; any
+    // further (small) shares are drawn from a counter by whichever CTA finishes first (no CTA waits for
+    // another).  Co-resident CTAs do not progress at the same speed (the warp schedulers favour the older
+    // ones), so the quick ones pick up the small shares and the SM stays fully occupied until the end.
     for (int share = blockIdx.x; share < P.nshares;) {
     FB_TRACE_T0(t_pro);
-    long long lo, hi;
-    if (share < G) {
-        lo = P.static_cost * (long long)share / G;
-        hi = P.static_cost * (long long)(share + 1) / G;
+    int e0, i0, e1, i1;
+    if (P.cuts) {
+        const int2 c0 = __ldg((const int2 *)P.cuts + share), c1 = __ldg((const int2 *)P.cuts + share + 1);
+        e0 = c0.x; i0 = c0.y; e1 = c1.x; i1 = c1.y;
     } else {
-        const long long rest = P.total_cost - P.static_cost;
-        const int j = share - G, nj = P.nshares - G;
-        lo = P.static_cost + rest * (long long)j / nj;
-        hi = P.static_cost + rest * (long long)(j + 1) / nj;
+        e0 = 0; e1 = 0;
+        i0 = P.single_cut[share];
+        i1 = P.single_cut[share + 1];
     }
 
-    // first entry that reaches past lo (CTA-uniform binary search over the prefix sums)
-    int e = 0;
-    if (P.table) {
-        int a = 0, b = P.n - 1;
-        while (a < b) {
-            int m = (a + b + 1) >> 1;
-            if (__ldg(&P.table[m].cost_begin) <= lo) a = m; else b = m - 1;
-        }
-        e = a;
-    }
-
-    for (; e < P.n; ++e) {
+    for (int e = e0; e <= e1; ++e) {
+        if (e == e1 && i1 == 0) break;             // the share ends where entry e1 begins (also: e1 == n)
         const LinearEntry *src = P.table ? P.table + e : &P.single;
-        if (src->cost_begin >= hi) break;
         if (tid < 32) ((uint32_t *)Es)[tid] = ((const uint32_t *)src)[tid];
         __syncthreads();
         const LinearEntry &E = *Es;
         // With NP == 2 region 0 is walked two pairs at a time, their table sets side by side (4-byte entries,
         // every entry with an even number of global pairs): a "work pair" is then a couple of pairs, a
-        // work row block their two items.  Costs per pair are unchanged, only the cut granularity doubles.
+        // work row block their two items.
         // (NP is a kernel template parameter: the host picks the two-pair kernel unless a CTA's share is
         // only a handful of items, where building two table sets per run costs more than the better row
         // loop gains.  Deciding it at run time was measured slower than either variant: both row loops in
         // one kernel cost registers.)
         const int wp0 = E.npairs[0] / NP;
         const int I0 = wp0 * E.nrb, I1 = E.npairs[1] * E.nrb;
-        if (tid == 0) {
-            // Cost line of this entry: every pair costs build_cost + nrb * item_cost of its region.
-            // The CTA owns the work row blocks whose start lies in [lo, hi); a cut inside the build
-            // part of a work pair goes to its first row block.
-            const long long Pc0 = NP * (P.build_cost + (long long)E.nrb * w0), Pc1 = P.build_cost + (long long)E.nrb * w1;
-            const long long T0 = (long long)wp0 * Pc0, T = T0 + (long long)E.npairs[1] * Pc1;
-            auto first_item = [&](long long pos) -> int {
-                if (pos <= 0) return 0;
-                if (pos >= T) return I0 + I1;
-                const bool reg1 = pos >= T0;
-                const long long rel = reg1 ? pos - T0 : pos, Pc = reg1 ? Pc1 : Pc0, w = reg1 ? w1 : NP * w0;
-                const long long pair = rel / Pc, within = rel - pair * Pc - (reg1 ? 1 : NP) * P.build_cost;
-                long long rb = within <= 0 ? 0 : (within + w - 1) / w;
-                if (rb > E.nrb) rb = E.nrb;
-                return (reg1 ? I0 : 0) + (int)(pair * E.nrb + rb);
-            };
-            range[0] = first_item(lo - E.cost_begin);
-            range[1] = first_item(hi - E.cost_begin);
-        }
+        // (the counters are next touched behind the barrier that precedes every table build)
         for (int t = tid; t < E.ntiles; t += kThreads) tile_cnt[t] = 0;
-        __syncthreads();
-        int cur = range[0];
-        const int end = range[1];
-        __syncthreads();                           // range[] is rewritten for the next entry
+        int cur = (e == e0) ? i0 : 0;
+        const int end = (e == e1) ? i1 : I0 + I1;
         FB_TRACE_ADD(7, t_pro);
-        if (cur >= end) { FB_TRACE_SET(t_pro); continue; }
+        if (cur >= end) { __syncthreads(); FB_TRACE_SET(t_pro); continue; }
 
         // a segment = the CTA's row blocks of one work pair
-        auto fetch_for = [&](int region, int pair, BuildInput<BT> &in) {
-            const uint8_t *desc = E.packed + E.off_coldesc + (size_t)((region ? E.npairs[0] : 0) + pair) * FB_PAIR_DESC_BYTES;
-            fetch_build_input<BT>(in, desc, E.x, E.ldx, P.nb, region ? -1 : (2 * pair) / E.Kb * 128,
-                                  (2 * pair + 1) / E.Kb * 128, E.N);
+        auto desc_of = [&](int region, int pair) {
+            return E.packed + E.off_coldesc + (size_t)((region ? E.npairs[0] : 0) + pair) * FB_PAIR_DESC_BYTES;
+        };
+        auto fetch_x_for = [&](int region, int pair, BuildInput<BT> &in) {
+            fetch_build_x<BT>(in, E.x, E.ldx, P.nb, region ? -1 : (2 * pair) / E.Kb * 128, (2 * pair + 1) / E.Kb * 128, E.N);
         };
         // With 16-byte entries one CTA owns the SM, so nothing covers the load latency of a build's inputs: the
         // inputs of the CTA's next pair are requested before the rows of the current one (+2 % at batch 8 with
@@ -922,9 +1000,12 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
             const int rb_hi = rb_lo + (seg_end - cur);
             const int np = region ? 1 : NP;                 // pairs walked together in this segment
             const int pair = wpair * np;
-            const int ib = region ? ItemBytes<SPS1>::value : ItemBytes<SPS0>::value;
-            const uint8_t *items = E.packed + E.off_items[region] + (size_t)pair * E.nrb * ib;
-            const uint8_t *items_b = items + (size_t)E.nrb * ib;
+            const int ib_full = region ? ItemBytes<SPS1>::value : ItemBytes<SPS0>::value;
+            // the last salient pair may be stored narrow: 8 or 16 steps per item instead of 32
+            const int steps = (SPS1 == 1 && region && pair == E.npairs[1] - 1) ? E.sal_last_w : 32;
+            const int ib = steps == 32 ? ib_full : 96 * steps;
+            const uint8_t *items = E.packed + E.off_items[region] + (size_t)pair * E.nrb * ib_full;
+            const uint8_t *items_b = items + (size_t)E.nrb * ib_full;
             const int pf_d = np == 2 ? 1 : (region ? SPS1 : SPS0) == 1 ? 1 : DepthFor<BT>::value;
             // weights start moving now.  The two-pair loop prefetches the trip two ahead, so its head covers
             // trips 0 and 1 (+2 %); longer heads were measured slower in every launch mode.
@@ -932,46 +1013,81 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
             prefetch_run_head(items, ib, pf_d, kWarps, rb_lo, rb_hi, head_trips);
             if (np == 2) prefetch_run_head(items_b, ib, pf_d, kWarps, rb_lo, rb_hi, head_trips);
 
-            if (!predecessor_done) {
-                asm volatile("griddepcontrol.wait;" ::: "memory");
-                predecessor_done = true;
+            if (!predecessor_done && P.head_bytes > 0) {
+                // EXPERIMENT: the start of the CTA's first run of items goes to L2 while the predecessor drains
+                const int seg_bytes = (rb_hi - rb_lo) * ib;
+                const int want = min(seg_bytes, P.head_bytes / np);
+                const int off = tid * 4096;
+                if (off < want) {
+                    const uint32_t nbytes = (uint32_t)min(4096, want - off);
+                    prefetch_l2(items + (size_t)rb_lo * ib + off, nbytes);
+                    if (np == 2) prefetch_l2(items_b + (size_t)rb_lo * ib + off, nbytes);
+                }
             }
-            FB_TRACE_T0(t_build);
-            __syncthreads();     // previous segment's lookups are done before the tables are overwritten
-            FB_TRACE_ADD(8, t_build);
             FB_TRACE_T0(t_fetch);
             // (fetching the next pair's inputs ahead of the lookups was measured 15 % slower: the extra
             // live registers push the lookup loop over the 80-register budget of 3 CTAs per SM)
             BuildInput<BT> bin, bin_b;
-            if constexpr (kNextInputsEarly) {
-                if (have_next) bin = bin_next; else fetch_for(region, pair, bin);
-            } else {
-                fetch_for(region, pair, bin);
-                if (np == 2) fetch_for(region, pair + 1, bin_b);
+            const bool reuse = kNextInputsEarly && have_next;
+            if (!reuse) {
+                fetch_build_desc<BT>(bin, desc_of(region, pair));
+                if (np == 2) fetch_build_desc<BT>(bin_b, desc_of(region, pair + 1));
             }
             // region 0, one pair at a time (short runs): first item in flight during the build.  (With two
             // pairs per row block the runs are long and the extra live registers cost more than they hide.)
-            ItemRegs<SPS0> pre;
+            ItemRegs<SPS0> pre, pre_b;
             if (NP == 1 && region == 0) preload_first<SPS0, BT>(pre, items, rb_lo, rb_hi);
+            const bool early2 = NP == 2 && region == 0 && P.early_items && !predecessor_done;    // EXPERIMENT
+            if constexpr (NP == 2 && geom(BT) == 1) {
+                if (early2) preload_first2<SPS0, BT>(pre, pre_b, items, items_b, rb_lo, rb_hi);
+            }
+
+            if (!predecessor_done) {
+                FB_TRACE_AT(11);
+                asm volatile("griddepcontrol.wait;" ::: "memory");
+                predecessor_done = true;
+                FB_TRACE_AT(1);
+            }
+            if constexpr (kNextInputsEarly) {
+                if (reuse) bin = bin_next; else fetch_x_for(region, pair, bin);
+            } else {
+                fetch_x_for(region, pair, bin);
+                if (np == 2) fetch_x_for(region, pair + 1, bin_b);
+            }
+            FB_TRACE_T0(t_build);
+            __syncthreads();     // previous segment's lookups are done before the tables are overwritten
+            FB_TRACE_ADD(8, t_build);
             FB_TRACE_ADD(9, t_fetch);
-            build_tables<BT>(bin, abuf);
-            if (np == 2) build_tables<BT>(bin_b, abuf, 128u);
+            if (np == 2) {
+                if constexpr (geom(BT) == 1) build_tables2<BT>(bin, bin_b, abuf);
+            } else {
+                build_tables<BT>(bin, abuf);
+            }
             // the column tables of the next run's pairs (1 KB each, read once per run: otherwise an HBM miss on the
             // serial path of the next build) start moving into L2 now (+0.5 to 0.8 % in every launch mode)
             if (tid < 8 * np && pair + np < E.npairs[region])
-                prefetch_line_if(E.packed + E.off_coldesc + (size_t)((region ? E.npairs[0] : 0) + pair + np) * FB_PAIR_DESC_BYTES + tid * 128, true);
+                prefetch_line_if(desc_of(region, pair + np) + tid * 128, true);
             if constexpr (kNextInputsEarly) {
                 // the CTA's next segment is the next pair of this entry's global region: its inputs start moving now
                 have_next = seg_end < end && seg_end < I0;
-                if (have_next) fetch_for(0, pair + 1, bin_next);
+                if (have_next) {
+                    fetch_build_desc<BT>(bin_next, desc_of(0, pair + 1));
+                    fetch_x_for(0, pair + 1, bin_next);
+                }
             }
             FB_TRACE_ADD(4, t_build);
             FB_TRACE_T0(t_rows);
             if (region == 0) {
-                if constexpr (NP == 2) process_rows2<SPS0, BT>(items, items_b, rb_lo, rb_hi, la, E.acc, E.Mpad);
+                if constexpr (NP == 2) {
+                    if (early2) process_rows2<SPS0, BT>(items, items_b, rb_lo, rb_hi, la, E.acc, E.Mpad, &pre, &pre_b);
+                    else process_rows2<SPS0, BT>(items, items_b, rb_lo, rb_hi, la, E.acc, E.Mpad);
+                }
                 else process_rows<SPS0, BT>(items, rb_lo, rb_hi, la, E.acc, E.Mpad, &pre);
-            } else {
+            } else if (steps == 32) {
                 process_rows<SPS1, BT>(items, rb_lo, rb_hi, la, E.acc, E.Mpad);
+            } else if constexpr (SPS1 == 1) {
+                if (steps == 16) process_rows_narrow<16, BT>(items, rb_lo, rb_hi, la, E.acc, E.Mpad);
+                else process_rows_narrow<8, BT>(items, rb_lo, rb_hi, la, E.acc, E.Mpad);
             }
 
             FB_TRACE_ADD(5, t_rows);
@@ -983,7 +1099,7 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
                 tile_cnt[t] += (b - a) * np;     // one thread per tile, segments are serial: no race
             }
             cur = seg_end;
-            FB_TRACE_ADD(1, t_cnt);
+            FB_TRACE_ADD(10, t_cnt);
         }
         FB_TRACE_T0(t_red);
         reduce_and_store<BT>(E, P.nb, P.y_fp32, tile_cnt, done_list);

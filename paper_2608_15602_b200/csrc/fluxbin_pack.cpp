@@ -4,6 +4,7 @@
 #include "fluxbin_internal.h"
 
 #include <algorithm>
+#include <cstdlib>
 #include <cstring>
 #include <vector>
 
@@ -61,6 +62,17 @@ static int salient_sps(int N, int g) { return (N / g == 1 && g % 128 == 0) ? 16 
 
 static int item_bytes_for(int sps) { return FB_ITEM_BITS_BYTES + 32 * 2 * (32 / sps); }
 
+// table slots of pair P (32, or fewer for a narrow last salient pair) and the bytes of one of its items
+static int pair_width(const FbHeader &h, int region, int P)
+{
+    return (region == 1 && h.sps[1] == 1 && P == h.npairs[1] - 1) ? h.sal_last_w : 32;
+}
+static int pair_item_bytes(const FbHeader &h, int region, int P)
+{
+    const int w = pair_width(h, region, P);
+    return w == 32 ? h.item_bytes[region] : 96 * w;
+}
+
 // Fill every header field.  n_svec < 0 selects the upper bound (salient map unknown).
 static void make_header(const fluxbin_layer_desc_t *d, int n_svec, int n_dead, FbHeader &h)
 {
@@ -76,6 +88,7 @@ static void make_header(const fluxbin_layer_desc_t *d, int n_svec, int n_dead, F
     int ng = d->N / d->g;
     h.sps[0] = gcd_int(d->g, 128) / 8;
     h.sps[1] = salient_sps(d->N, d->g);
+    h.sal_last_w = 32;
     int nblk = (d->N + 127) / 128;
     h.nunits[0] = nblk * d->Kb;
     h.npairs[0] = (h.nunits[0] + 1) / 2;
@@ -87,8 +100,19 @@ static void make_header(const fluxbin_layer_desc_t *d, int n_svec, int n_dead, F
         }
         h.n_sal_svec = n_svec;
         h.n_dead = n_dead;
-        h.nunits[1] = ((n_svec + 15) / 16) * h.Ks;
-        h.npairs[1] = (h.nunits[1] + 1) / 2;
+        if (h.sps[1] == 16) {
+            // one scale per (row, unit): every base's sub-vectors are padded to whole units of 16
+            h.nunits[1] = ((n_svec + 15) / 16) * h.Ks;
+            h.npairs[1] = (h.nunits[1] + 1) / 2;
+        } else {
+            // one scale per (row, sub-vector): the sub-vectors of all bases form one flat list of table slots
+            const int slots = n_svec * h.Ks;
+            h.nunits[1] = (slots + 15) / 16;
+            h.npairs[1] = (slots + 31) / 32;
+            const int last = slots - 32 * (h.npairs[1] - 1);
+            h.sal_last_w = last <= 8 ? 8 : last <= 16 ? 16 : 32;
+            if (getenv("FBX_NO_NARROW")) h.sal_last_w = 32;      // EXPERIMENT
+        }
     }
     h.item_bytes[0] = item_bytes_for(h.sps[0]);
     h.item_bytes[1] = item_bytes_for(h.sps[1]);
@@ -98,7 +122,8 @@ static void make_header(const fluxbin_layer_desc_t *d, int n_svec, int n_dead, F
     h.off_items[0] = off;
     off += (uint64_t)h.npairs[0] * h.nrb * h.item_bytes[0];
     h.off_items[1] = off;
-    off += (uint64_t)h.npairs[1] * h.nrb * h.item_bytes[1];
+    if (h.npairs[1] > 0)
+        off += (uint64_t)(h.npairs[1] - 1) * h.nrb * h.item_bytes[1] + (uint64_t)h.nrb * pair_item_bytes(h, 1, h.npairs[1] - 1);
     h.off_sal_idx = off;
     off += ((uint64_t)h.n_sal * 4 + 15) / 16 * 16;
     h.off_dead_ids = off;
@@ -134,23 +159,42 @@ fluxbin_status_t check_header(const void *p, size_t bytes, FbHeader &h)
     return FLUXBIN_OK;
 }
 
-// ---- sources of one unit: which canonical bits / scales / columns it covers -------------------
+// ---- what a table slot holds: which canonical bits / scales / columns it covers ------------------
 
-struct UnitSrc {
+struct SlotSrc {
     bool valid = false;
     bool salient = false;
     int k = 0;          // base
-    int blk = 0;        // global: 128-column block;  salient: first sub-vector index j*16
+    int sv = 0;         // global: sub-vector index (8 columns from sv * 8);  salient: index into the sub-vector list
 };
 
-static UnitSrc unit_src(const FbHeader &h, int region, int u)
+// table slot sigma (0..31) of pair P of a region; n_sv = salient sub-vectors per base
+static SlotSrc slot_src(const FbHeader &h, int region, int P, int sigma)
 {
-    UnitSrc s;
-    if (u >= h.nunits[region]) return s;
+    SlotSrc s;
+    if (region == 0) {
+        const int u = 2 * P + (sigma >> 4);
+        if (u >= h.nunits[0]) return s;
+        s.valid = true;
+        s.k = u % h.Kb;
+        s.sv = (u / h.Kb) * 16 + (sigma & 15);
+        if (s.sv * 8 >= h.N) s.valid = false;
+        return s;
+    }
+    s.salient = true;
+    if (h.sps[1] == 16) {
+        const int u = 2 * P + (sigma >> 4), upb = h.nunits[1] / h.Ks;
+        if (u >= h.nunits[1]) return s;
+        s.k = u / upb;
+        s.sv = (u % upb) * 16 + (sigma & 15);
+        s.valid = s.sv < h.n_sal_svec;
+        return s;
+    }
+    const int flat = 32 * P + (sigma & (pair_width(h, 1, P) - 1));       // a narrow pair repeats its live tables
+    if (flat >= h.n_sal_svec * h.Ks) return s;
     s.valid = true;
-    s.salient = region == 1;
-    if (region == 0) { s.blk = u / h.Kb; s.k = u % h.Kb; }
-    else { int upb = h.nunits[1] / h.Ks; s.k = u / upb; s.blk = (u % upb) * 16; }
+    s.k = flat / h.n_sal_svec;
+    s.sv = flat % h.n_sal_svec;
     return s;
 }
 
@@ -251,20 +295,16 @@ extern "C" fluxbin_status_t fluxbin_pack_host(const fluxbin_layer_desc_t *d, voi
         for (int P = 0; P < h.npairs[region]; ++P) {
             uint16_t *pd = cd + (size_t)((region ? h.npairs[0] : 0) + P) * (FB_PAIR_DESC_BYTES / 2);
             for (int sigma = 0; sigma < 32; ++sigma) {
-                UnitSrc us = unit_src(h, region, 2 * P + (sigma >> 4));
-                int t = sigma & 15;
+                const SlotSrc ss = slot_src(h, region, P, sigma);
                 for (int n = 0; n < 8; ++n) {
                     uint16_t xi = 0, al = 0;
-                    if (us.valid && !us.salient) {
-                        int col = us.blk * 128 + t * 8 + n;
-                        if (col < N) { xi = (uint16_t)col; al = d->col_scale[(size_t)us.k * N + col]; }
-                    } else if (us.valid) {
-                        int s = us.blk + t;
-                        if (s < (int)sv.size() && n < sv[s].w) {
-                            int v = sv[s].vstart + n;
-                            xi = (uint16_t)d->sal_idx[v];
-                            al = d->sal_col_scale[(size_t)us.k * n_sal + v];
-                        }
+                    if (ss.valid && !ss.salient) {
+                        int col = ss.sv * 8 + n;
+                        if (col < N) { xi = (uint16_t)col; al = d->col_scale[(size_t)ss.k * N + col]; }
+                    } else if (ss.valid && n < sv[ss.sv].w) {
+                        int v = sv[ss.sv].vstart + n;
+                        xi = (uint16_t)d->sal_idx[v];
+                        al = d->sal_col_scale[(size_t)ss.k * n_sal + v];
                     }
                     pd[(sigma * 8 + n) * 2 + 0] = xi;
                     pd[(sigma * 8 + n) * 2 + 1] = al;
@@ -274,57 +314,64 @@ extern "C" fluxbin_status_t fluxbin_pack_host(const fluxbin_layer_desc_t *d, voi
 
     // ---- items: weight bytes in lane-rotated order + row scales in step order
     for (int region = 0; region < 2; ++region) {
-        const int sps = h.sps[region], nseg = 32 / sps, ib = h.item_bytes[region];
+        const int sps = h.sps[region];
         const int64_t nitems = (int64_t)h.npairs[region] * h.nrb;
 #pragma omp parallel for schedule(static)
         for (int64_t it = 0; it < nitems; ++it) {
             const int P = (int)(it / h.nrb), rb = (int)(it % h.nrb);
-            uint8_t *item = base + h.off_items[region] + (uint64_t)it * ib;
-            uint16_t *sc = (uint16_t *)(item + FB_ITEM_BITS_BYTES);
-            UnitSrc us[2] = {unit_src(h, region, 2 * P), unit_src(h, region, 2 * P + 1)};
+            const int w = pair_width(h, region, P), nseg = w / sps;
+            uint8_t *item = base + h.off_items[region] + (uint64_t)P * h.nrb * h.item_bytes[region] + (uint64_t)rb * pair_item_bytes(h, region, P);
+            uint16_t *sc = (uint16_t *)(item + 32 * w);
+            SlotSrc ss[32];
+            for (int sigma = 0; sigma < 32; ++sigma) ss[sigma] = slot_src(h, region, P, sigma);
             for (int l = 0; l < 32; ++l) {
                 const int row = rb * 32 + l;
                 const bool live = row < M;
-                // the 16 table indices of this row for both units, in sub-vector order
-                alignas(16) uint8_t src[2][16];
-                uint16_t segscale[2][16];   // row scale per sub-vector (only segment starts are read)
-                for (int u = 0; u < 2; ++u) {
-                    std::memset(src[u], 0, 16);
-                    std::memset(segscale[u], 0, sizeof(segscale[u]));
-                    if (!live || !us[u].valid) continue;
-                    if (!us[u].salient) {
-                        const int colb = us[u].blk * 128;
+                // table index and row scale of this row for every table slot of the pair
+                alignas(16) uint8_t src[32];
+                uint16_t slotscale[32];
+                std::memset(src, 0, sizeof(src));
+                std::memset(slotscale, 0, sizeof(slotscale));
+                if (live && region == 0) {
+                    for (int u = 0; u < 2; ++u) {
+                        if (!ss[16 * u].valid) continue;
+                        const int k = ss[16 * u].k, colb = ss[16 * u].sv * 8;
                         const int nbytes = std::min(16, (N - colb) / 8);   // N % 32 == 0
-                        const uint8_t *r = (const uint8_t *)(d->bits + ((size_t)us[u].k * M + row) * nw);
-                        std::memcpy(src[u], r + colb / 8, nbytes);         // little-endian words: byte = 8 columns
-                        const uint16_t *rs = d->row_scale + ((size_t)us[u].k * M + row) * ng;
-                        for (int t = 0; t < nbytes; t += sps) segscale[u][t] = rs[(colb + t * 8) / g];
-                    } else {
-                        const uint32_t *r = d->sal_bits + ((size_t)us[u].k * M + row) * nws;
-                        const uint16_t *rs = d->sal_row_scale + ((size_t)us[u].k * M + row) * ng;
-                        for (int t = 0; t < 16 && us[u].blk + t < (int)sv.size(); ++t) {
-                            const SalSvec &q = sv[us[u].blk + t];
-                            src[u][t] = (uint8_t)extract_bits(r, q.vstart, q.w);
-                            segscale[u][t] = rs[q.G];
-                        }
+                        const uint8_t *r = (const uint8_t *)(d->bits + ((size_t)k * M + row) * nw);
+                        std::memcpy(src + 16 * u, r + colb / 8, nbytes);   // little-endian words: byte = 8 columns
+                        const uint16_t *rs = d->row_scale + ((size_t)k * M + row) * ng;
+                        for (int t = 0; t < nbytes; t += sps) slotscale[16 * u + t] = rs[(colb + t * 8) / g];
+                    }
+                } else if (live) {
+                    for (int sigma = 0; sigma < w; ++sigma) {
+                        if (!ss[sigma].valid) continue;
+                        const SalSvec &q = sv[ss[sigma].sv];
+                        const uint32_t *r = d->sal_bits + ((size_t)ss[sigma].k * M + row) * nws;
+                        src[sigma] = (uint8_t)extract_bits(r, q.vstart, q.w);
+                        slotscale[sigma] = d->sal_row_scale[((size_t)ss[sigma].k * M + row) * ng + q.G];
                     }
                 }
-                // lane l reads slot l ^ s at step s: unit u sits in half u ^ (l >> 4), and inside the
-                // half the byte of sub-vector t sits at position t ^ (l & 15)
-                for (int u = 0; u < 2; ++u) {
-                    uint64_t lo, hi;
-                    std::memcpy(&lo, src[u], 8);
-                    std::memcpy(&hi, src[u] + 8, 8);
-                    xor_permute16(lo, hi, l & 15);
-                    uint8_t *dst = item + (u ^ (l >> 4)) * 512 + l * 16;
-                    std::memcpy(dst, &lo, 8);
-                    std::memcpy(dst + 8, &hi, 8);
+                if (w == 32) {
+                    // lane l reads slot l ^ s at step s: unit u sits in half u ^ (l >> 4), and inside the
+                    // half the byte of sub-vector t sits at position t ^ (l & 15)
+                    for (int u = 0; u < 2; ++u) {
+                        uint64_t lo, hi;
+                        std::memcpy(&lo, src + 16 * u, 8);
+                        std::memcpy(&hi, src + 16 * u + 8, 8);
+                        xor_permute16(lo, hi, l & 15);
+                        uint8_t *dst = item + (u ^ (l >> 4)) * 512 + l * 16;
+                        std::memcpy(dst, &lo, 8);
+                        std::memcpy(dst + 8, &hi, 8);
+                    }
+                } else {
+                    // narrow item: w steps, the byte of step s is that of live slot (l ^ s) mod w
+                    for (int c = 0; c < w; ++c) item[l * w + c] = src[(l ^ c) & (w - 1)];
                 }
                 for (int j = 0; j < nseg; ++j) {
                     // the segment is the aligned block of sps sub-vectors around slot l ^ (j*sps); its
                     // scale is that of the block's first sub-vector (live sub-vectors form a prefix)
-                    int sigma = l ^ (j * sps);
-                    uint16_t v = segscale[sigma >> 4][(sigma & 15) / sps * sps];
+                    const int sigma = (l ^ (j * sps)) & (w - 1);
+                    const uint16_t v = slotscale[sigma / sps * sps];
                     if (nseg <= 8) sc[l * nseg + j] = v;
                     else sc[(j >> 3) * 256 + l * 8 + (j & 7)] = v;
                 }
@@ -384,75 +431,61 @@ extern "C" fluxbin_status_t fluxbin_unpack_host(const void *h_packed, size_t byt
     for (int region = 0; region < 2; ++region)
         for (int P = 0; P < h.npairs[region]; ++P) {
             const uint16_t *pd = cd + (size_t)((region ? h.npairs[0] : 0) + P) * (FB_PAIR_DESC_BYTES / 2);
-            for (int sigma = 0; sigma < 32; ++sigma) {
-                UnitSrc us = unit_src(h, region, 2 * P + (sigma >> 4));
-                if (!us.valid) continue;
-                int t = sigma & 15;
+            for (int sigma = 0; sigma < pair_width(h, region, P); ++sigma) {
+                const SlotSrc ss = slot_src(h, region, P, sigma);
+                if (!ss.valid) continue;
                 for (int n = 0; n < 8; ++n) {
                     uint16_t al = pd[(sigma * 8 + n) * 2 + 1];
-                    if (!us.salient) {
-                        int col = us.blk * 128 + t * 8 + n;
-                        if (col < N && col_scale) col_scale[(size_t)us.k * N + col] = al;
-                    } else {
-                        int s = us.blk + t;
-                        if (s < (int)sv.size() && n < sv[s].w && sal_col_scale)
-                            sal_col_scale[(size_t)us.k * n_sal + sv[s].vstart + n] = al;
+                    if (!ss.salient) {
+                        int col = ss.sv * 8 + n;
+                        if (col < N && col_scale) col_scale[(size_t)ss.k * N + col] = al;
+                    } else if (n < sv[ss.sv].w && sal_col_scale) {
+                        sal_col_scale[(size_t)ss.k * n_sal + sv[ss.sv].vstart + n] = al;
                     }
                 }
             }
         }
 
     for (int region = 0; region < 2; ++region) {
-        const int sps = h.sps[region], nseg = 32 / sps, ib = h.item_bytes[region];
-        const int64_t nitems = (int64_t)h.npairs[region] * h.nrb;
+        const int sps = h.sps[region];
         // rows of different items never overlap for global bits/scales; salient bits of one row are
         // touched by several pairs, so the salient region is processed pair-serially per row block
 #pragma omp parallel for schedule(static)
         for (int rb = 0; rb < h.nrb; ++rb)
             for (int P = 0; P < h.npairs[region]; ++P) {
-                const int64_t it = (int64_t)P * h.nrb + rb;
-                (void)nitems;
-                const uint8_t *item = base + h.off_items[region] + (uint64_t)it * ib;
-                const uint16_t *sc = (const uint16_t *)(item + FB_ITEM_BITS_BYTES);
-                UnitSrc us[2] = {unit_src(h, region, 2 * P), unit_src(h, region, 2 * P + 1)};
+                const int w = pair_width(h, region, P), nseg = w / sps;
+                const uint8_t *item = base + h.off_items[region] + (uint64_t)P * h.nrb * h.item_bytes[region] + (uint64_t)rb * pair_item_bytes(h, region, P);
+                const uint16_t *sc = (const uint16_t *)(item + 32 * w);
+                SlotSrc ss[32];
+                for (int sigma = 0; sigma < 32; ++sigma) ss[sigma] = slot_src(h, region, P, sigma);
                 for (int l = 0; l < 32; ++l) {
                     const int row = rb * 32 + l;
                     if (row >= M) continue;
-                    uint8_t src[2][16];
-                    uint16_t segscale[2][16];
-                    for (int s = 0; s < 32; ++s) {
-                        int sigma = l ^ s;
-                        src[sigma >> 4][sigma & 15] = item[(s >> 4) * 512 + l * 16 + (s & 15)];
+                    uint8_t src[32];
+                    uint16_t slotscale[32];
+                    for (int c = 0; c < w; ++c) {
+                        const int sigma = (l ^ c) & (w - 1);
+                        src[sigma] = (w == 32) ? item[(c >> 4) * 512 + l * 16 + (c & 15)] : item[l * w + c];
                     }
                     for (int j = 0; j < nseg; ++j) {
-                        int sigma0 = l ^ (j * sps);
-                        uint16_t v = (nseg <= 8) ? sc[l * nseg + j] : sc[(j >> 3) * 256 + l * 8 + (j & 7)];
-                        for (int q = 0; q < sps; ++q) {
-                            int sigma = sigma0 ^ q;      // the segment's sub-vectors: an aligned block of sps
-                            segscale[sigma >> 4][sigma & 15] = v;
-                        }
+                        const int sigma0 = (l ^ (j * sps)) & (w - 1);
+                        const uint16_t v = (nseg <= 8) ? sc[l * nseg + j] : sc[(j >> 3) * 256 + l * 8 + (j & 7)];
+                        for (int q = 0; q < sps; ++q) slotscale[sigma0 ^ q] = v;      // the segment's sub-vectors: an aligned block of sps
                     }
-                    for (int u = 0; u < 2; ++u) {
-                        if (!us[u].valid) continue;
-                        for (int t = 0; t < 16; ++t) {
-                            if (!us[u].salient) {
-                                int col0 = us[u].blk * 128 + t * 8;
-                                if (col0 >= N) continue;
-                                if (bits) {
-                                    uint8_t *r = (uint8_t *)(bits + ((size_t)us[u].k * M + row) * nw);
-                                    r[col0 >> 3] = src[u][t];     // little-endian words: byte col0/8
-                                }
-                                if (row_scale && col0 % g == 0)
-                                    row_scale[((size_t)us[u].k * M + row) * ng + col0 / g] = segscale[u][t];
-                            } else {
-                                int s = us[u].blk + t;
-                                if (s >= (int)sv.size()) continue;
-                                if (sal_bits)
-                                    deposit_bits(sal_bits + ((size_t)us[u].k * M + row) * nws, sv[s].vstart, sv[s].w,
-                                                 src[u][t]);
-                                if (sal_row_scale)
-                                    sal_row_scale[((size_t)us[u].k * M + row) * ng + sv[s].G] = segscale[u][t];
+                    for (int sigma = 0; sigma < w; ++sigma) {
+                        if (!ss[sigma].valid) continue;
+                        const int k = ss[sigma].k;
+                        if (!ss[sigma].salient) {
+                            const int col0 = ss[sigma].sv * 8;
+                            if (bits) {
+                                uint8_t *r = (uint8_t *)(bits + ((size_t)k * M + row) * nw);
+                                r[col0 >> 3] = src[sigma];     // little-endian words: byte col0/8
                             }
+                            if (row_scale && col0 % g == 0) row_scale[((size_t)k * M + row) * ng + col0 / g] = slotscale[sigma];
+                        } else {
+                            const SalSvec &q = sv[ss[sigma].sv];
+                            if (sal_bits) deposit_bits(sal_bits + ((size_t)k * M + row) * nws, q.vstart, q.w, src[sigma]);
+                            if (sal_row_scale) sal_row_scale[((size_t)k * M + row) * ng + q.G] = slotscale[sigma];
                         }
                     }
                 }

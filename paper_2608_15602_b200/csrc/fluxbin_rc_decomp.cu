@@ -8,14 +8,19 @@
 // contraction in it); one warp owns one (row, group) at a time, lane l the g/32 adjacent columns l*g/32 ... of
 // the group, so a row of a group is one 128-bit load per lane and a lane's signs are adjacent bits of one word.
 //
-//   init        one pass: greedy residual initialisation, all K bases of a (row, group) in registers
-//   per iteration, per base k:
-//     row pass  target = W - (other bases); a_r(k) by Eq. 5; with the new a_r the numerators of the column form
-//               of Eq. 5, reduced over the 64 rows of a CTA in shared memory, then one atomic per column and CTA
-//     col pass  a_c(k) = numerator / (sum_i a_r^2 + eps)   (B^2 = 1), accumulators re-zeroed
-//   sign pass   per element the tuple minimising |W - sum_k M(k) b_k| over all 2^K tuples, lowest index on ties,
-//               evaluated one base at a time with single roundings (M = a_r * a_c rounded once)
-//   final       scales rounded to fp16 (round to nearest even)
+// Passes over W per call: 1 + T * K.  Every pass is local to a warp's (row, group) except the column form of
+// Eq. 5, whose numerators are summed over all rows; so the steps are grouped into passes that end where that
+// sum is needed:
+//   first pass        greedy residual initialisation of all K bases, then the row form of Eq. 5 for base 1 and the
+//                     numerators of its column form
+//   per round, base k row form of Eq. 5 for base k (target = W - other bases) and the numerators of its column form
+//   end of a round    the joint sign update of Eq. 6 (all 2^K tuples per element, lowest index on ties, one base at
+//                     a time with single roundings) followed, in the same pass, by the next round's row form for
+//                     base 1, which needs nothing but the new signs
+//   column form       a_c(k) = numerator / (sum_i a_r^2 + eps): the numerators of a column group are reduced in
+//                     shared memory over the 64 rows of a CTA, then one atomic per column and CTA; the last CTA
+//                     to arrive at a group (a ticket per group) divides, stores and re-zeroes the accumulators
+// Scales are stored as fp32 (working copy) and, rounded to nearest even, as fp16 whenever they are written.
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -38,9 +43,12 @@ struct Args {
     uint32_t *bits;        // [K][M][N/32]
     float *ar;             // [K][M][NG]
     float *ac;             // [K][N]
+    uint16_t *ar16;        // the same, fp16 bit patterns
+    uint16_t *ac16;
     const float *live;     // [N] 1 = real column, 0 = padding column (W must be 0 there); nullptr: all real
-    float *colnum;         // [N]
-    float *colden;         // [2][NG], double buffered
+    float *colnum;         // [N]   numerators of the column form, zero between passes
+    float *colden;         // [NG]  sum of a_r^2 per group, zero between passes
+    unsigned *tickets;     // [NG]  CTAs of a group that have added their part, zero between passes
 };
 
 __device__ __forceinline__ float warp_sum(float v)
@@ -123,228 +131,233 @@ template <int C, int K> struct WarpRows {
 template <int C> __device__ __forceinline__ int word_of_lane(int lane) { return (lane * C) / 32; }
 template <int C> __device__ __forceinline__ bool stores_word(int lane) { return (lane % (32 / C)) == 0; }
 
-template <int C> __global__ void __launch_bounds__(kWarpsPerCta * 32) init_kernel(Args a)
+__device__ __forceinline__ uint16_t half_bits(float v) { return __half_as_ushort(__float2half_rn(v)); }
+
+enum PassMode {
+    kRow = 0,        // row form of Eq. 5 for base k (signs read from memory) + column numerators
+    kSignRow = 1,    // Eq. 6 for all bases, then the row form for base 0 with the new signs + column numerators
+    kSign = 2,       // Eq. 6 only (the last pass of a call)
+    kInitRow = 3,    // greedy initialisation, then the row form for base 0 + column numerators
+    kInit = 4        // greedy initialisation only (T == 0)
+};
+
+template <int C, int K, int MODE> __global__ void __launch_bounds__(kWarpsPerCta * 32) pass_kernel(Args a, int k_arg)
 {
+    constexpr bool kInitial = MODE == kInitRow || MODE == kInit;
+    constexpr bool kSearch = MODE == kSignRow || MODE == kSign;
+    constexpr bool kRowForm = MODE == kRow || MODE == kSignRow || MODE == kInitRow;
+    __shared__ float part[kWarpsPerCta][C * 32];
+    __shared__ float den_part[kWarpsPerCta];
+    __shared__ int is_last;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int G = blockIdx.x, row0 = blockIdx.y * kRowsPerCta + warp * kRowsPerWarp;
     const int nw = a.N / 32;
-    const int nrows = min(kRowsPerWarp, a.M - row0);
-    WarpRows<C, 1> in;                                                    // (only the W part is used here)
-    in.load_w(a, G, row0, nrows, lane);
-    // initial column scales: 1 on real columns, 0 on padding columns (which then stay 0 through every update:
-    // their numerators are sums of zeros); Eq. 5 with those scales divides by the number of real columns
-    float lv[C];
-#pragma unroll
-    for (int c = 0; c < C; ++c) lv[c] = 1.f;
-    if (a.live) load_cols<C>(lv, a.live + G * a.g + lane * C);
-    float nlive = 0.f;
-#pragma unroll
-    for (int c = 0; c < C; ++c) nlive += lv[c];
-    const float inv_n = 1.f / (warp_sum(nlive) + a.eps);
-#pragma unroll
-    for (int r = 0; r < kRowsPerWarp; ++r) {
-        const int i = row0 + r;
-        float R[C];
-#pragma unroll
-        for (int c = 0; c < C; ++c) R[c] = in.w[r][c];
-        for (int k = 0; k < a.K; ++k) {
-            float s = 0.f;
-#pragma unroll
-            for (int c = 0; c < C; ++c) s += fabsf(R[c]) * lv[c];
-            s = warp_sum(s) * inv_n;                                      // Eq. 5 with a_c = 1 on the real columns
-            uint32_t mine = 0u;
-#pragma unroll
-            for (int c = 0; c < C; ++c) {
-                const bool pos = R[c] >= 0.f;                             // sign(0) = +1
-                mine |= (pos ? 1u : 0u) << c;
-                const float step = s * lv[c];
-                R[c] = pos ? __fsub_rn(R[c], step) : __fadd_rn(R[c], step);
-            }
-            const uint32_t word = gather_word<C>(mine << ((lane * C) & 31));
-            if (stores_word<C>(lane) && r < nrows) a.bits[((size_t)k * a.M + i) * nw + G * C + word_of_lane<C>(lane)] = word;
-            if (lane == 0 && r < nrows) a.ar[((size_t)k * a.M + i) * a.NG + G] = s;
-        }
-    }
-}
+    const int nrows = max(0, min(kRowsPerWarp, a.M - row0));
+    const int k = MODE == kRow ? k_arg : 0;                // base of the row form
 
-__global__ void fill_kernel(float *p, float v, long long n)
-{
-    long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;
-    if (i < n) p[i] = v;
-}
-
-// dst[i] = src[i % n]: the live mask as the initial column scales of every base
-__global__ void tile_kernel(float *dst, const float *src, int n, long long total)
-{
-    long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;
-    if (i < total) dst[i] = src[i % n];
-}
-
-// Row form of Eq. 5 for base k, then the column form's numerators with the new row scale.
-template <int C, int K> __global__ void __launch_bounds__(kWarpsPerCta * 32) row_kernel(Args a, int k, int parity)
-{
-    __shared__ float part[kWarpsPerCta][C * 32];
-    __shared__ float den_part[kWarpsPerCta];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int G = blockIdx.x, row0 = blockIdx.y * kRowsPerCta + warp * kRowsPerWarp;
-    const int nrows = min(kRowsPerWarp, a.M - row0);
     WarpRows<C, K> in;
     in.load_w(a, G, row0, nrows, lane);
-    in.load_signs(a, G, row0, nrows, lane);
-    in.load_row_scales(a, G, row0, nrows, lane);
+    if constexpr (MODE == kRow) in.load_signs(a, G, row0, nrows, lane);
+    if constexpr (!kInitial) in.load_row_scales(a, G, row0, nrows, lane);
     float ack[K][C];                     // column scales of every base for this lane's columns
+    float lv[C];                         // live mask (initial column scales)
+    if constexpr (kInitial) {
+        // initial column scales: 1 on real columns, 0 on padding columns (which then stay 0 through every update:
+        // their numerators are sums of zeros); Eq. 5 with those scales divides by the number of real columns
+#pragma unroll
+        for (int c = 0; c < C; ++c) lv[c] = 1.f;
+        if (a.live) load_cols<C>(lv, a.live + G * a.g + lane * C);
+#pragma unroll
+        for (int q = 0; q < K; ++q)
+#pragma unroll
+            for (int c = 0; c < C; ++c) ack[q][c] = lv[c];
+    } else {
+#pragma unroll
+        for (int q = 0; q < K; ++q) load_cols<C>(ack[q], a.ac + (size_t)q * a.N + G * a.g + lane * C);
+    }
     float akc[C];                        // those of base k
 #pragma unroll
-    for (int q = 0; q < K; ++q) {
-        load_cols<C>(ack[q], a.ac + (size_t)q * a.N + G * a.g + lane * C);
+    for (int q = 0; q < K; ++q)
         if (q == k) {
 #pragma unroll
             for (int c = 0; c < C; ++c) akc[c] = ack[q][c];
         }
-    }
     float den_c = 0.f;
 #pragma unroll
     for (int c = 0; c < C; ++c) den_c += akc[c] * akc[c];
     den_c = warp_sum(den_c) + a.eps;                                      // sum_j (a_c B)^2 + eps, B^2 = 1
+    const float inv_den = 1.f / den_c;                                   // (initial pass: 1 / (live columns + eps))
     float colsum[C];
 #pragma unroll
     for (int c = 0; c < C; ++c) colsum[c] = 0.f;
     float ar2 = 0.f;
-    const float inv_den = 1.f / den_c;
+
 #pragma unroll
     for (int r = 0; r < kRowsPerWarp; ++r) {
-        // signs enter as a choice between +v and -v (one select, then a fused multiply-add): the passes are
-        // bound by issue slots as much as by memory, so the per-element instruction count matters
-        float t[C];
-        uint32_t sk = 0u;
+        const int i = row0 + r;
+        float arq[K];
+        uint32_t sg[K];                  // the C sign bits of this lane's columns, per base
+        if constexpr (kInitial) {
+            float R[C];
 #pragma unroll
-        for (int c = 0; c < C; ++c) t[c] = in.w[r][c];
+            for (int c = 0; c < C; ++c) R[c] = in.w[r][c];
 #pragma unroll
-        for (int q = 0; q < K; ++q) {
-            const float arq = in.ar(r, q);
-            const uint32_t sg = in.signs(r, q, lane);
-            if (q == k) sk = sg;
-            else {
+            for (int q = 0; q < K; ++q) {
+                float s = 0.f;
+#pragma unroll
+                for (int c = 0; c < C; ++c) s += fabsf(R[c]) * lv[c];
+                s = warp_sum(s) * inv_den;                                // Eq. 5 with a_c = 1 on the real columns
+                uint32_t mine = 0u;
+#pragma unroll
+                for (int c = 0; c < C; ++c) {
+                    const bool pos = R[c] >= 0.f;                         // sign(0) = +1
+                    mine |= (pos ? 1u : 0u) << c;
+                    const float step = s * lv[c];
+                    R[c] = pos ? __fsub_rn(R[c], step) : __fadd_rn(R[c], step);
+                }
+                sg[q] = mine;
+                arq[q] = s;
+                if (lane == 0 && r < nrows && (MODE == kInit || q != 0)) {       // base 0's scale is replaced just below
+                    a.ar[((size_t)q * a.M + i) * a.NG + G] = s;
+                    a.ar16[((size_t)q * a.M + i) * a.NG + G] = half_bits(s);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int q = 0; q < K; ++q) arq[q] = in.ar(r, q);
+            if constexpr (kSearch) {
+#pragma unroll
+                for (int q = 0; q < K; ++q) sg[q] = 0u;
+#pragma unroll
+                for (int c = 0; c < C; ++c) {
+                    const float x = in.w[r][c];
+                    float mag[K];
+#pragma unroll
+                    for (int q = 0; q < K; ++q) mag[q] = __fmul_rn(arq[q], ack[q][c]);        // rounded once
+                    int best = 0;
+                    float best_e = 0.f;
+#pragma unroll
+                    for (int t = 0; t < (1 << K); ++t) {
+                        float e = x;
+#pragma unroll
+                        for (int q = 0; q < K; ++q) e = ((t >> q) & 1) ? __fsub_rn(e, mag[q]) : __fadd_rn(e, mag[q]);
+                        e = fabsf(e);
+                        if (t == 0 || e < best_e) { best_e = e; best = t; }                   // lowest index wins ties
+                    }
+#pragma unroll
+                    for (int q = 0; q < K; ++q) sg[q] |= (uint32_t)((best >> q) & 1) << c;
+                }
+            } else {
+#pragma unroll
+                for (int q = 0; q < K; ++q) sg[q] = in.signs(r, q, lane);
+            }
+        }
+        if constexpr (kInitial || kSearch) {
+#pragma unroll
+            for (int q = 0; q < K; ++q) {
+                const uint32_t word = gather_word<C>((sg[q] & ((1u << C) - 1u)) << ((lane * C) & 31));
+                if (stores_word<C>(lane) && r < nrows) a.bits[((size_t)q * a.M + i) * nw + G * C + word_of_lane<C>(lane)] = word;
+            }
+        }
+        if constexpr (kRowForm) {
+            // signs enter as a choice between +v and -v (one select, then a fused multiply-add): the passes are
+            // bound by issue slots as much as by memory, so the per-element instruction count matters
+            float t[C];
+#pragma unroll
+            for (int c = 0; c < C; ++c) t[c] = in.w[r][c];
+#pragma unroll
+            for (int q = 0; q < K; ++q) {
+                if (q == k) continue;
 #pragma unroll
                 for (int c = 0; c < C; ++c)
-                    t[c] = fmaf(((sg >> c) & 1u) ? -arq : arq, ack[q][c], t[c]);          // what the other bases leave
+                    t[c] = fmaf(((sg[q] >> c) & 1u) ? -arq[q] : arq[q], ack[q][c], t[c]);     // what the other bases leave
             }
-        }
-        float num = 0.f;
+            uint32_t sk = 0u;
 #pragma unroll
-        for (int c = 0; c < C; ++c) num = fmaf(((sk >> c) & 1u) ? akc[c] : -akc[c], t[c], num);
-        const float arn = r < nrows ? warp_sum(num) * inv_den : 0.f;       // (r < nrows is warp-uniform)
-        if (lane == 0 && r < nrows) a.ar[((size_t)k * a.M + row0 + r) * a.NG + G] = arn;
-        ar2 = fmaf(arn, arn, ar2);
+            for (int q = 0; q < K; ++q) if (q == k) sk = sg[q];
+            float num = 0.f;
 #pragma unroll
-        for (int c = 0; c < C; ++c) colsum[c] = fmaf(((sk >> c) & 1u) ? arn : -arn, t[c], colsum[c]);
-    }
-#pragma unroll
-    for (int c = 0; c < C; ++c) part[warp][lane * C + c] = colsum[c];
-    if (lane == 0) den_part[warp] = ar2;
-    __syncthreads();
-    for (int j = threadIdx.x; j < C * 32; j += kWarpsPerCta * 32) {
-        float s = 0.f;
-#pragma unroll
-        for (int w = 0; w < kWarpsPerCta; ++w) s += part[w][j];
-        atomicAdd(a.colnum + G * a.g + j, s);
-    }
-    if (threadIdx.x == 0) {
-        float s = 0.f;
-        for (int w = 0; w < kWarpsPerCta; ++w) s += den_part[w];
-        atomicAdd(a.colden + (size_t)(parity & 1) * a.NG + G, s);
-    }
-}
-
-// Column form of Eq. 5: a_c(k)_j = numerator_j / (sum_i a_r_i^2 + eps); the accumulators go back to zero.
-// (the group denominators are double buffered: this pass reads buffer `parity` and clears the other one, which the
-// next row pass accumulates into -- no thread reads what another clears)
-__global__ void col_kernel(Args a, int k, int parity)
-{
-    const int j = blockIdx.x * blockDim.x + threadIdx.x;
-    if (j >= a.N) return;
-    a.ac[(size_t)k * a.N + j] = a.colnum[j] / (a.colden[(size_t)(parity & 1) * a.NG + j / a.g] + a.eps);
-    a.colnum[j] = 0.f;
-    if (j < a.NG) a.colden[(size_t)((parity + 1) & 1) * a.NG + j] = 0.f;
-}
-__global__ void zero_kernel(float *p, int n)
-{
-    const int j = blockIdx.x * blockDim.x + threadIdx.x;
-    if (j < n) p[j] = 0.f;
-}
-
-// Eq. 6 for every element.
-template <int C, int K> __global__ void __launch_bounds__(kWarpsPerCta * 32) sign_kernel(Args a)
-{
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int G = blockIdx.x, row0 = blockIdx.y * kRowsPerCta + warp * kRowsPerWarp;
-    const int nw = a.N / 32;
-    const int nrows = min(kRowsPerWarp, a.M - row0);
-    WarpRows<C, K> in;
-    in.load_w(a, G, row0, nrows, lane);
-    in.load_row_scales(a, G, row0, nrows, lane);
-    float ack[K][C];
-#pragma unroll
-    for (int q = 0; q < K; ++q) load_cols<C>(ack[q], a.ac + (size_t)q * a.N + G * a.g + lane * C);
-#pragma unroll
-    for (int r = 0; r < kRowsPerWarp; ++r) {
-        float arq[K];
-#pragma unroll
-        for (int q = 0; q < K; ++q) arq[q] = in.ar(r, q);
-        uint32_t mine[K];
-#pragma unroll
-        for (int q = 0; q < K; ++q) mine[q] = 0u;
-#pragma unroll
-        for (int c = 0; c < C; ++c) {
-            const float x = in.w[r][c];
-            float mag[K];
-#pragma unroll
-            for (int q = 0; q < K; ++q) mag[q] = __fmul_rn(arq[q], ack[q][c]);        // rounded once
-            int best = 0;
-            float best_e = 0.f;
-#pragma unroll
-            for (int t = 0; t < (1 << K); ++t) {
-                float e = x;
-#pragma unroll
-                for (int q = 0; q < K; ++q) e = ((t >> q) & 1) ? __fsub_rn(e, mag[q]) : __fadd_rn(e, mag[q]);
-                e = fabsf(e);
-                if (t == 0 || e < best_e) { best_e = e; best = t; }                   // lowest index wins ties
+            for (int c = 0; c < C; ++c) num = fmaf(((sk >> c) & 1u) ? akc[c] : -akc[c], t[c], num);
+            const float arn = r < nrows ? warp_sum(num) * inv_den : 0.f;   // (r < nrows is warp-uniform)
+            if (lane == 0 && r < nrows) {
+                a.ar[((size_t)k * a.M + i) * a.NG + G] = arn;
+                a.ar16[((size_t)k * a.M + i) * a.NG + G] = half_bits(arn);
             }
+            ar2 = fmaf(arn, arn, ar2);
 #pragma unroll
-            for (int q = 0; q < K; ++q) mine[q] |= (uint32_t)((best >> q) & 1) << c;
-        }
-#pragma unroll
-        for (int q = 0; q < K; ++q) {
-            const uint32_t word = gather_word<C>(mine[q] << ((lane * C) & 31));
-            if (stores_word<C>(lane) && r < nrows)
-                a.bits[((size_t)q * a.M + row0 + r) * nw + G * C + word_of_lane<C>(lane)] = word;
+            for (int c = 0; c < C; ++c) colsum[c] = fmaf(((sk >> c) & 1u) ? arn : -arn, t[c], colsum[c]);
         }
     }
-}
 
-__global__ void to_half_kernel(const float *src, uint16_t *dst, long long n)
-{
-    long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;
-    if (i < n) dst[i] = __half_as_ushort(__float2half_rn(src[i]));
+    if constexpr (MODE == kInit) {
+        // no update follows: the column scales are the initial ones
+        if (blockIdx.y == 0 && warp == 0) {
+#pragma unroll
+            for (int q = 0; q < K; ++q)
+#pragma unroll
+                for (int c = 0; c < C; ++c) {
+                    a.ac[(size_t)q * a.N + G * a.g + lane * C + c] = lv[c];
+                    a.ac16[(size_t)q * a.N + G * a.g + lane * C + c] = half_bits(lv[c]);
+                }
+        }
+    }
+    if constexpr (kRowForm) {
+#pragma unroll
+        for (int c = 0; c < C; ++c) part[warp][lane * C + c] = colsum[c];
+        if (lane == 0) den_part[warp] = ar2;
+        __syncthreads();
+        for (int j = threadIdx.x; j < C * 32; j += kWarpsPerCta * 32) {
+            float s = 0.f;
+#pragma unroll
+            for (int w = 0; w < kWarpsPerCta; ++w) s += part[w][j];
+            atomicAdd(a.colnum + G * a.g + j, s);
+        }
+        if (threadIdx.x == 0) {
+            float s = 0.f;
+            for (int w = 0; w < kWarpsPerCta; ++w) s += den_part[w];
+            atomicAdd(a.colden + G, s);
+        }
+        // Column form of Eq. 5 by the last CTA of the group to get here: a_c(k)_j = numerator_j / (sum_i a_r_i^2 + eps);
+        // the accumulators and the ticket go back to zero for the next pass.
+        __threadfence();
+        __syncthreads();
+        if (threadIdx.x == 0) is_last = (atomicAdd(a.tickets + G, 1u) == gridDim.y - 1);
+        __syncthreads();
+        if (is_last) {
+            __threadfence();
+            const float den = __ldcg(a.colden + G) + a.eps;
+            for (int j = threadIdx.x; j < C * 32; j += kWarpsPerCta * 32) {
+                const int col = G * a.g + j;
+                const float v = __ldcg(a.colnum + col) / den;
+                a.ac[(size_t)k * a.N + col] = v;
+                a.ac16[(size_t)k * a.N + col] = half_bits(v);
+                a.colnum[col] = 0.f;
+                if constexpr (MODE == kInitRow) {
+                    const float l = a.live ? a.live[col] : 1.f;
+                    for (int q = 1; q < K; ++q) {
+                        a.ac[(size_t)q * a.N + col] = l;
+                        a.ac16[(size_t)q * a.N + col] = half_bits(l);
+                    }
+                }
+            }
+            __syncthreads();
+            if (threadIdx.x == 0) { a.colden[G] = 0.f; a.tickets[G] = 0u; }
+        }
+    }
 }
 
 template <int C, int K> cudaError_t run(const Args &a, int T, cudaStream_t s)
 {
     const dim3 grid(a.NG, (a.M + kRowsPerCta - 1) / kRowsPerCta), block(kWarpsPerCta * 32);
-    const long long nac = (long long)a.K * a.N;
-    if (a.live) tile_kernel<<<(unsigned)((nac + 255) / 256), 256, 0, s>>>(a.ac, a.live, a.N, nac);
-    else fill_kernel<<<(unsigned)((nac + 255) / 256), 256, 0, s>>>(a.ac, 1.f, nac);
-    zero_kernel<<<(a.N + 255) / 256, 256, 0, s>>>(a.colnum, a.N);
-    zero_kernel<<<(2 * a.NG + 255) / 256, 256, 0, s>>>(a.colden, 2 * a.NG);
-    init_kernel<C><<<grid, block, 0, s>>>(a);
-    int parity = 0;
+    if (T == 0) {
+        pass_kernel<C, K, kInit><<<grid, block, 0, s>>>(a, 0);
+        return cudaGetLastError();
+    }
+    pass_kernel<C, K, kInitRow><<<grid, block, 0, s>>>(a, 0);
     for (int it = 0; it < T; ++it) {
-        for (int k = 0; k < a.K; ++k) {
-            row_kernel<C, K><<<grid, block, 0, s>>>(a, k, parity);
-            col_kernel<<<(a.N + 255) / 256, 256, 0, s>>>(a, k, parity);
-            parity ^= 1;
-        }
-        sign_kernel<C, K><<<grid, block, 0, s>>>(a);
+        for (int k = 1; k < a.K; ++k) pass_kernel<C, K, kRow><<<grid, block, 0, s>>>(a, k);
+        if (it + 1 < T) pass_kernel<C, K, kSignRow><<<grid, block, 0, s>>>(a, 0);
+        else pass_kernel<C, K, kSign><<<grid, block, 0, s>>>(a, 0);
     }
     return cudaGetLastError();
 }
@@ -358,7 +371,13 @@ extern "C" size_t fluxbin_rc_decomp_workspace_size(int32_t M, int32_t N, int32_t
 {
     if (M < 1 || N < 32 || g < 32 || K < 1 || K > rcd::kMaxK || N % g != 0) return 0;
     const size_t NG = (size_t)N / g;
-    return align256((size_t)K * M * NG * 4) + align256((size_t)K * N * 4) + align256((size_t)N * 4) + align256(2 * NG * 4);
+    return align256((size_t)K * M * NG * 4) + align256((size_t)K * N * 4) + align256((size_t)N * 4 + 2 * NG * 4);
+}
+
+extern "C" int32_t fluxbin_rc_decomp_passes(int32_t K, int32_t T)
+{
+    if (K < 1 || K > rcd::kMaxK || T < 0) return -1;
+    return 1 + T * K;
 }
 
 extern "C" fluxbin_status_t fluxbin_rc_decomp(const float *d_W, int64_t ldw, const float *d_col_live, int32_t M, int32_t N,
@@ -371,18 +390,23 @@ extern "C" fluxbin_status_t fluxbin_rc_decomp(const float *d_W, int64_t ldw, con
     if (M < 1 || N < 32 || N % 32 != 0 || g < 32 || g % 32 != 0 || N % g != 0 || ldw < N) return FLUXBIN_ERR_SHAPE;
     if (K < 1 || K > rcd::kMaxK || T < 0 || !(eps >= 0.f)) return FLUXBIN_ERR_RANGE;
     if (g != 32 && g != 64 && g != 128 && g != 256) return FLUXBIN_ERR_UNSUPPORTED;
-    if (((uintptr_t)d_workspace & 15) != 0 || ((uintptr_t)d_W & 15) != 0 || (ldw & 3) != 0 || ((uintptr_t)d_col_live & 15) != 0)
+    if (((uintptr_t)d_workspace & 15) != 0 || ((uintptr_t)d_W & 15) != 0 || (ldw & 3) != 0 || ((uintptr_t)d_col_live & 15) != 0 ||
+        ((uintptr_t)d_col_scale_f32 & 15) != 0)
         return FLUXBIN_ERR_ALIGNMENT;
     if (ws_bytes < fluxbin_rc_decomp_workspace_size(M, N, g, K)) return FLUXBIN_ERR_BUFFER_TOO_SMALL;
     cudaStream_t s = (cudaStream_t)cuda_stream;
     rcd::Args a;
     a.W = d_W; a.live = d_col_live; a.ldw = ldw; a.M = M; a.N = N; a.g = g; a.NG = N / g; a.K = K; a.eps = eps;
     a.bits = d_bits;
+    a.ar16 = d_row_scale; a.ac16 = d_col_scale;
     uint8_t *ws = (uint8_t *)d_workspace;
-    a.ar = (float *)ws;     ws += align256((size_t)K * M * a.NG * 4);
-    a.ac = (float *)ws;     ws += align256((size_t)K * N * 4);
-    a.colnum = (float *)ws; ws += align256((size_t)N * 4);
-    a.colden = (float *)ws;
+    // the fp32 working copies of the scales live in the caller's fp32 outputs when those are given
+    a.ar = d_row_scale_f32 ? d_row_scale_f32 : (float *)ws;     ws += align256((size_t)K * M * a.NG * 4);
+    a.ac = d_col_scale_f32 ? d_col_scale_f32 : (float *)ws;     ws += align256((size_t)K * N * 4);
+    a.colnum = (float *)ws;
+    a.colden = a.colnum + N;
+    a.tickets = (unsigned *)(a.colden + a.NG);
+    FB_CUDA(cudaMemsetAsync(a.colnum, 0, (size_t)N * 4 + 2 * (size_t)a.NG * 4, s));
     cudaError_t e = cudaErrorInvalidValue;
 #define RCD_K(CC) (K == 1 ? rcd::run<CC, 1>(a, T, s) : K == 2 ? rcd::run<CC, 2>(a, T, s) : K == 3 ? rcd::run<CC, 3>(a, T, s) : rcd::run<CC, 4>(a, T, s))
     switch (g / 32) {
@@ -393,12 +417,6 @@ extern "C" fluxbin_status_t fluxbin_rc_decomp(const float *d_W, int64_t ldw, con
     }
 #undef RCD_K
     if (e != cudaSuccess) return fb::record_cuda_error((int)e);
-    const long long nar = (long long)K * M * a.NG, nac = (long long)K * N;
-    rcd::to_half_kernel<<<(unsigned)((nar + 255) / 256), 256, 0, s>>>(a.ar, d_row_scale, nar);
-    rcd::to_half_kernel<<<(unsigned)((nac + 255) / 256), 256, 0, s>>>(a.ac, d_col_scale, nac);
-    if (d_row_scale_f32) FB_CUDA(cudaMemcpyAsync(d_row_scale_f32, a.ar, (size_t)nar * 4, cudaMemcpyDeviceToDevice, s));
-    if (d_col_scale_f32) FB_CUDA(cudaMemcpyAsync(d_col_scale_f32, a.ac, (size_t)nac * 4, cudaMemcpyDeviceToDevice, s));
-    FB_CUDA(cudaGetLastError());
     return FLUXBIN_OK;
 }
 

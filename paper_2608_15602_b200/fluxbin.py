@@ -34,6 +34,7 @@ class LayerDesc(ctypes.Structure):
 
 EXPORTS = ["fluxbin_packed_size", "fluxbin_validate", "fluxbin_pack_host", "fluxbin_unpack_host",
            "fluxbin_packed_dims", "fluxbin_pack", "fluxbin_attach", "fluxbin_unpack", "fluxbin_weight_dims",
+           "fluxbin_weight_device", "fluxbin_debug_cut_shares",
            "fluxbin_workspace_size", "fluxbin_workspace_init", "fluxbin_linear", "fluxbin_debug_tables",
            "fluxbin_num_table_sets", "fluxbin_num_launches", "fluxbin_free", "fluxbin_status_string",
            "fluxbin_last_cuda_error", "fluxbin_plan_table_bytes", "fluxbin_plan_workspace_bytes",
@@ -63,12 +64,15 @@ def _lib():
         lib.fluxbin_attach.restype, lib.fluxbin_attach.argtypes = ctypes.c_int, [vp, sz, vp, sz, ctypes.POINTER(vp)]
         lib.fluxbin_unpack.restype, lib.fluxbin_unpack.argtypes = ctypes.c_int, [vp, dp, vp]
         lib.fluxbin_weight_dims.restype, lib.fluxbin_weight_dims.argtypes = ctypes.c_int, [vp, dp]
+        lib.fluxbin_weight_device.restype, lib.fluxbin_weight_device.argtypes = i32, [vp]
         lib.fluxbin_workspace_size.restype, lib.fluxbin_workspace_size.argtypes = sz, [vp, i32]
         lib.fluxbin_workspace_init.restype, lib.fluxbin_workspace_init.argtypes = ctypes.c_int, [vp, sz, vp]
         lib.fluxbin_linear.restype = ctypes.c_int
         lib.fluxbin_linear.argtypes = [vp, vp, i32, i64, vp, i32, i64, vp, sz, vp]
         lib.fluxbin_debug_tables.restype = ctypes.c_int
         lib.fluxbin_debug_tables.argtypes = [vp, vp, i32, vp, vp, vp, vp]
+        lib.fluxbin_debug_cut_shares.restype = ctypes.c_int
+        lib.fluxbin_debug_cut_shares.argtypes = [i32, ctypes.POINTER(vp), i32, i32, i32, i32, i32, vp, vp]
         lib.fluxbin_num_table_sets.restype, lib.fluxbin_num_table_sets.argtypes = i32, [vp]
         lib.fluxbin_num_launches.restype, lib.fluxbin_num_launches.argtypes = i32, [vp, i32]
         lib.fluxbin_set_table_format.restype, lib.fluxbin_set_table_format.argtypes = ctypes.c_int, [vp, i32]
@@ -193,6 +197,9 @@ class Weight:
     def workspace_size(self, B: int) -> int:
         return int(_lib().fluxbin_workspace_size(self.handle, B))
 
+    def device(self) -> int:
+        return int(_lib().fluxbin_weight_device(self.handle))
+
     def num_table_sets(self) -> int:
         return int(_lib().fluxbin_num_table_sets(self.handle))
 
@@ -287,6 +294,18 @@ def debug_tables(w: Weight, d_x: int, pair: int, d_tables: int, stream: int = 0)
     _check(_lib().fluxbin_debug_tables(w.handle, d_x, pair, d_tables, cols.ctypes.data, alpha.ctypes.data, stream),
            "fluxbin_debug_tables")
     return cols, alpha
+
+
+def debug_cut_shares(headers, mode: int, pairs_per_row_block: int, grid: int, nshares: int, static_percent: int = 100):
+    """fluxbin_debug_cut_shares: (cuts int32 [nshares + 1][2], work items per layer) for packed-layer headers
+    (uint8 arrays of at least 256 bytes each).  Host only."""
+    n = len(headers)
+    cuts = np.zeros((nshares + 1, 2), np.int32)
+    items = np.zeros(n, np.int32)
+    hp = _arr(ctypes.c_void_p, [h.ctypes.data for h in headers])
+    _check(_lib().fluxbin_debug_cut_shares(n, hp, mode, pairs_per_row_block, grid, nshares, static_percent,
+                                           cuts.ctypes.data, items.ctypes.data), "fluxbin_debug_cut_shares")
+    return cuts, items
 
 
 class Plan:

@@ -43,6 +43,17 @@ class FluxBinLinear:
             self.weight.set_table_format(fluxbin.TABLES_FP16)
         self.packed_bytes = int(self.buffer.numel())
 
+    def clone(self) -> "FluxBinLinear":
+        """The same packed layer in a device buffer of its own (a device-to-device copy plus fluxbin_attach)."""
+        c = object.__new__(FluxBinLinear)
+        c.device = self.device
+        c.buffer = self.buffer.clone()
+        header = self.buffer[:256].cpu().numpy()
+        c.weight = fluxbin.attach(header, c.buffer.data_ptr(), int(c.buffer.numel()), buffer=c.buffer)
+        c.weight.set_table_format(self.weight.table_format())
+        c.M, c.N, c.packed_bytes = self.M, self.N, self.packed_bytes
+        return c
+
     def workspace(self, B: int) -> Workspace:
         return Workspace(self.weight.workspace_size(B), self.device)
 

@@ -5,13 +5,13 @@ import struct
 
 import numpy as np
 
-HEADER_FMT = "<II18i7Q"
+HEADER_FMT = "<II20i7Q"
 
 
 def parse_header(buf):
     f = struct.unpack_from(HEADER_FMT, buf.tobytes()[:256])
     names = ["magic", "version", "M", "N", "Kb", "Ks", "g", "n_sal", "Mpad", "nrb", "sps0", "sps1", "nunits0",
-             "nunits1", "npairs0", "npairs1", "item_bytes0", "item_bytes1", "n_sal_svec", "n_dead",
+             "nunits1", "npairs0", "npairs1", "item_bytes0", "item_bytes1", "n_sal_svec", "n_dead", "sal_last_w", "reserved0",
              "off_coldesc", "off_items0", "off_items1", "off_sal_idx", "off_dead_ids", "off_dead_scales",
              "total_bytes"]
     return dict(zip(names, f))
@@ -30,20 +30,27 @@ def emulate_linear(buf, x_bits):
     signs = np.array([[1.0 if (p >> n) & 1 else -1.0 for n in range(8)] for p in range(256)])   # [256][8]
     lanes = np.arange(32)
     for region in (0, 1):
-        npairs, sps, ib = h[f"npairs{region}"], h[f"sps{region}"], h[f"item_bytes{region}"]
-        nseg = 32 // sps
+        npairs, sps, ib_full = h[f"npairs{region}"], h[f"sps{region}"], h[f"item_bytes{region}"]
         for P in range(npairs):
+            # the last salient pair may be narrow: w = 8 or 16 steps per item instead of 32 (all 32 table slots
+            # are still built; the column table repeats the live ones)
+            w = h["sal_last_w"] if (region == 1 and sps == 1 and P == npairs - 1) else 32
+            ib = ib_full if w == 32 else 96 * w
+            nseg = w // sps
             off = h["off_coldesc"] + ((h["npairs0"] if region else 0) + P) * 1024
             cd = buf[off:off + 1024].view(np.uint16).reshape(32, 8, 2)
             a = xs[:, cd[:, :, 0].astype(np.int64)] * _f16(cd[:, :, 1])[None]      # [B][32][8]
             tables = np.einsum("bsn,pn->bsp", a, signs)                              # [B][32][256]
             for rb in range(h["nrb"]):
-                ioff = h[f"off_items{region}"] + (P * h["nrb"] + rb) * ib
+                ioff = h[f"off_items{region}"] + P * h["nrb"] * ib_full + rb * ib
                 item = buf[ioff:ioff + ib]
-                sc = item[1024:].view(np.uint16)
-                for s in range(32):
+                sc = item[32 * w:].view(np.uint16)
+                for s in range(w):
                     sigma = lanes ^ s
-                    byte = item[(s >> 4) * 512 + lanes * 16 + (s & 15)].astype(np.int64)
+                    if w == 32:
+                        byte = item[(s >> 4) * 512 + lanes * 16 + (s & 15)].astype(np.int64)
+                    else:
+                        byte = item[lanes * w + s].astype(np.int64)
                     j = s // sps
                     if nseg <= 8:
                         scale = _f16(sc[lanes * nseg + j])

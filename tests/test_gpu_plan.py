@@ -135,16 +135,17 @@ def test_plan_rejects_mixed_scale_formats_and_bad_buffers(fb):
     x = torch.zeros((1, 256), dtype=torch.float16, device="cuda")
     ya = torch.zeros((1, 64), dtype=torch.float16, device="cuda")
     yb = torch.zeros((1, 64), dtype=torch.float16, device="cuda")
-    table = torch.zeros(1024, dtype=torch.uint8, device="cuda")
+    tb = fluxbin.plan_table_bytes(2, 1)
+    table = torch.zeros(tb, dtype=torch.uint8, device="cuda")
     ws = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
     args = ([x.data_ptr()] * 2, [256, 256], [ya.data_ptr(), yb.data_ptr()], [64, 64], 1, False)
-    st, _ = fluxbin.plan_create_status([a.weight, b.weight], *args, table.data_ptr(), 1024, ws.data_ptr(), 1 << 16)
+    st, _ = fluxbin.plan_create_status([a.weight, b.weight], *args, table.data_ptr(), tb, ws.data_ptr(), 1 << 16)
     assert st == 7
-    st, _ = fluxbin.plan_create_status([a.weight, a.weight], *args, table.data_ptr(), 100, ws.data_ptr(), 1 << 16)
+    st, _ = fluxbin.plan_create_status([a.weight, a.weight], *args, table.data_ptr(), tb - 1, ws.data_ptr(), 1 << 16)
     assert st == 5
-    st, _ = fluxbin.plan_create_status([a.weight, a.weight], *args, table.data_ptr(), 1024, ws.data_ptr(), 64)
+    st, _ = fluxbin.plan_create_status([a.weight, a.weight], *args, table.data_ptr(), tb, ws.data_ptr(), 64)
     assert st == 5
-    st, h = fluxbin.plan_create_status([a.weight, a.weight], *args, table.data_ptr(), 1024, ws.data_ptr(), 1 << 16)
+    st, h = fluxbin.plan_create_status([a.weight, a.weight], *args, table.data_ptr(), tb, ws.data_ptr(), 1 << 16)
     assert st == 0
     fluxbin.library().fluxbin_plan_free(h)
 

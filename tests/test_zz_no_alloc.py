@@ -64,3 +64,25 @@ def test_noalloc_rejects_layers_beyond_the_fixed_scratch():
     assert st == 5 and "too small" in fluxbin.status_string(st)
     assert fluxbin.linear_noalloc_status(lin.weight, x.data_ptr(), 1, 32, y.data_ptr(), False, 140000) == 0  # batch 1 fits
     torch.cuda.synchronize()
+
+
+def test_noalloc_row_limits_follow_the_accumulator_rows_of_the_batch():
+    """The scratch holds one fp32 accumulator row per vector of a chunk: four rows from batch 3 with fp32 table
+    entries, eight from batch 5 with fp16 entries.  Status checks only: calls just above a limit are rejected
+    before anything is put on the stream, calls just below it are accepted."""
+    from paper_2608_15602_b200 import build
+    build.build()
+    from paper_2608_15602_b200 import fluxbin, layer
+    cap = fluxbin.noalloc_capacity()
+    for rows, B, fp16_tables, fits in [(65000, 4, False, True), (66000, 4, False, False),
+                                       (32400, 8, True, True), (33000, 8, True, False), (65000, 8, False, True)]:
+        lin = layer.FluxBinLinear(synth.make_linear(6, rows, rows, 32, 1, 0, 32), fp16_tables=fp16_tables)
+        assert (lin.weight.workspace_size(B) <= cap) == fits, (rows, B, fp16_tables)
+        x = torch.zeros((B, 32), dtype=torch.float16, device="cuda")
+        y = torch.zeros((B, rows), dtype=torch.float16, device="cuda")
+        st = fluxbin.linear_noalloc_status(lin.weight, x.data_ptr(), B, 32, y.data_ptr(), False, rows)
+        assert st == (0 if fits else 5), (rows, B, fp16_tables, st)
+        # argument errors are reported before the scratch is cleared
+        assert fluxbin.linear_noalloc_status(lin.weight, x.data_ptr(), B, 16, y.data_ptr(), False, rows) == 3
+        assert fluxbin.linear_noalloc_status(lin.weight, x.data_ptr() + 2, B, 32, y.data_ptr(), False, rows) == 6
+    torch.cuda.synchronize()
