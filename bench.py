@@ -565,7 +565,7 @@ def section_rc_decomp(shapes=((4096, 4096), (8192, 8192)), K=2, T=10, g=128):
         b.record()
         torch.cuda.synchronize()
         ms = a.elapsed_time(b) / (reps * copies)
-        passes = 1 + T * (K + 1)                     # initialisation + per round: one row pass per base, one sign pass
+        passes = fluxbin.rc_decomp_passes(K, T)
         rows.append({"shape": f"{M}x{N}", "g": g, "K": K, "T": T, "ms_per_call": round(ms, 4), "passes_over_W": passes,
                      "us_per_pass": round(ms * 1e3 / passes, 2), "GBps_of_W": round(4.0 * M * N * passes / (ms * 1e-3) / 1e9, 1),
                      "copies": copies})

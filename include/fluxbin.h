@@ -333,12 +333,17 @@ void fluxbin_plan_free(fluxbin_plan_t *plan);
  *   d_bits         device out, uint32 [K][M][N/32]: bit (j % 32) of word j/32 is 1 <=> B_ij = +1
  *   d_row_scale    device out, fp16 bit patterns [K][M][N/g]   } the canonical layout of a layer description,
  *   d_col_scale    device out, fp16 bit patterns [K][N]        } rounded to nearest even
- *   d_row_scale_f32, d_col_scale_f32   optional device out (NULL to skip): the same scales before rounding
+ *   d_row_scale_f32, d_col_scale_f32   optional device out (NULL to skip): the same scales before rounding; when given
+ *                  they serve as the working copies during the call (d_col_scale_f32 16-byte aligned)
  *   d_workspace    device scratch of fluxbin_rc_decomp_workspace_size() bytes, 16-byte aligned, any contents
  * All arithmetic is fp32.  Asynchronous on cuda_stream; allocates nothing; caller owns every buffer.
  * Errors: NULL / SHAPE / RANGE / UNSUPPORTED (other g) / ALIGNMENT / BUFFER_TOO_SMALL before any launch, CUDA.
  */
 size_t fluxbin_rc_decomp_workspace_size(int32_t M, int32_t N, int32_t g, int32_t K);   /* 0 on invalid arguments */
+/* Passes over W one call makes (each reads the fp32 matrix once): 1 + T * K -- the initialisation runs in the same
+ * pass as the first row-scale update, and the sign update of a round in the same pass as the next round's first
+ * row-scale update.  -1 on invalid arguments. */
+int32_t fluxbin_rc_decomp_passes(int32_t K, int32_t T);
 fluxbin_status_t fluxbin_rc_decomp(const float *d_W, int64_t ldw, const float *d_col_live, int32_t M, int32_t N, int32_t g,
                                    int32_t K, int32_t T, float eps, uint32_t *d_bits, uint16_t *d_row_scale, uint16_t *d_col_scale,
                                    float *d_row_scale_f32, float *d_col_scale_f32, void *d_workspace, size_t ws_bytes,
@@ -362,6 +367,49 @@ fluxbin_status_t fluxbin_rc_salient_residual(const float *d_W, int64_t ldw, int3
                                              const float *d_col_scale_f32, const int32_t *d_sal_idx, const int32_t *d_pos,
                                              int32_t n_sal, float *d_P, int64_t ldp, int32_t ncols_p, float *d_live,
                                              void *cuda_stream);
+
+/*
+ * The canonical salient arrays from the outputs of the salient refinement (Algorithm 2, step 3).  The refinement
+ * ran fluxbin_rc_decomp on the padded matrix fluxbin_rc_salient_residual wrote: one block of `width` columns per
+ * row-scale group that holds salient columns (nblocks blocks; block b belongs to group d_block_group[b]; virtual
+ * column v sits in column d_pos[v]).  This call gathers the sign bits of the virtual columns into the dense VCM
+ * matrix (Eq. 12), scatters the blocks' row scales to their groups (zero for groups without salient columns) and
+ * gathers the column scales (Eq. 13), rounding the scales to fp16 (to nearest even) on the device.
+ *
+ *   d_bits_p            device uint32 [Ks][M][width * nblocks / 32]   } as fluxbin_rc_decomp wrote them for the
+ *   d_row_scale_p_f32   device fp32 [Ks][M][nblocks]                   } padded matrix (g = width)
+ *   d_col_scale_p_f32   device fp32 [Ks][width * nblocks]              }
+ *   d_pos, d_block_group   device int32 [n_sal], [nblocks]
+ *   d_sal_bits          device out uint32 [Ks][M][ceil(n_sal / 32)]: bit v % 32 of word v / 32 = virtual column v
+ *   d_sal_row_scale     device out fp16 bits [Ks][M][N / g];  d_sal_col_scale  device out fp16 bits [Ks][n_sal]
+ *   d_sal_row_scale_f32, d_sal_col_scale_f32   optional device out (NULL to skip): the same before rounding
+ * Asynchronous on cuda_stream; allocates nothing.  Errors: NULL / SHAPE / RANGE / CUDA.
+ */
+fluxbin_status_t fluxbin_rc_salient_collect(const uint32_t *d_bits_p, const float *d_row_scale_p_f32,
+                                            const float *d_col_scale_p_f32, const int32_t *d_pos,
+                                            const int32_t *d_block_group, int32_t M, int32_t N, int32_t g, int32_t Ks,
+                                            int32_t n_sal, int32_t width, int32_t nblocks, uint32_t *d_sal_bits,
+                                            uint16_t *d_sal_row_scale, uint16_t *d_sal_col_scale,
+                                            float *d_sal_row_scale_f32, float *d_sal_col_scale_f32, void *cuda_stream);
+
+/*
+ * fluxbin_pack for canonical arrays that already live in DEVICE memory (the outputs of fluxbin_rc_decomp and
+ * fluxbin_rc_salient_collect): the same packed bytes as fluxbin_pack_host (VCM, Def. 3.5), written by kernels, so
+ * the arrays never cross host memory.
+ *
+ *   d_desc        HOST struct whose dimensions are as usual and whose array pointers are DEVICE memory in the
+ *                 canonical layout (sal_idx included)
+ *   h_sal_idx     HOST copy of the salient map [n_sal] (the header and the virtual-column structure are functions
+ *                 of it); NULL when there is no salient branch
+ *   d_packed      DEVICE buffer of at least fluxbin_packed_size bytes (computed with h_sal_idx), 16-byte aligned
+ *   d_workspace   DEVICE scratch of fluxbin_pack_device_workspace_size(N, g, n_sal) bytes, 16-byte aligned
+ * The stream is synchronised before returning.  On success *out receives a handle that borrows d_packed.
+ * Errors: as fluxbin_pack.
+ */
+size_t fluxbin_pack_device_workspace_size(int32_t N, int32_t g, int32_t n_sal);     /* 0 on invalid arguments */
+fluxbin_status_t fluxbin_pack_device(const fluxbin_layer_desc_t *d_desc, const int32_t *h_sal_idx, void *d_packed,
+                                     size_t d_bytes, void *d_workspace, size_t ws_bytes, void *cuda_stream,
+                                     fluxbin_weight_t **out);
 
 #ifdef __cplusplus
 }

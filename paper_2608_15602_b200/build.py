@@ -8,7 +8,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_PKG, "csrc")
 LIB_DIR = os.path.join(_PKG, "lib")
 LIB_PATH = os.environ.get("FLUXBIN_LIB") or os.path.join(LIB_DIR, "libfluxbin.so")
-SOURCES = ["fluxbin_api.cu", "fluxbin_pack.cpp", "fluxbin_noalloc.cu", "fluxbin_rc_decomp.cu"]
+SOURCES = ["fluxbin_api.cu", "fluxbin_pack.cpp", "fluxbin_pack_device.cu", "fluxbin_noalloc.cu", "fluxbin_rc_decomp.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC,-fopenmp", "-shared"]
 

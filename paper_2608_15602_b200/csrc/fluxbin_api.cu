@@ -357,11 +357,15 @@ static void item_costs(int sps0, int sps1, int cost[2])
     cost[1] = (sps1 == sps0) ? 2 : 4;
 }
 
-// an item of the last salient pair costs in proportion to its steps when that pair is stored narrow
+// An item of a narrow last salient pair (8 or 16 steps instead of 32) is costed like a full one: the loop for items
+// with one scale per sub-vector keeps a single item in flight per warp (a full one fills 24 registers), so an item
+// takes a load latency whatever its size.  (Measured: costing it by its bytes left the CTAs that own the narrow
+// pair with twice the items and made one-launch-per-group runs 5 % slower; a two-deep loop for the narrow items
+// cost the whole kernel spills.)
 static int last_salient_item_cost(const FbHeader &h, int cost1)
 {
-    const int c = (h.sps[1] == 1) ? cost1 * h.sal_last_w / 32 : cost1;
-    return c > 0 ? c : 1;
+    (void)h;
+    return cost1;
 }
 
 static long long entry_cost(const FbHeader &h, int sps1, int build_cost)
@@ -404,21 +408,14 @@ static cudaError_t launch_shape(int dev, int mode, int s0, int s1, long long tot
         slot.store(occ, std::memory_order_relaxed);
     }
     long long grid = (long long)num_sms * occ;
-    {   // EXPERIMENT
-        static const int small_per_sm = getenv("FBX_SMALL_PER_SM") ? atoi(getenv("FBX_SMALL_PER_SM")) : 0;
-        static const long long small_thresh = getenv("FBX_SMALL_THRESH") ? atoll(getenv("FBX_SMALL_THRESH")) : 0;
-        if (small_per_sm > 0 && total_cost / grid < small_thresh && small_per_sm < occ) grid = (long long)num_sms * small_per_sm;
-    }
     if (items < grid) grid = items;
     if (grid > kMaxGrid) grid = kMaxGrid;
     if (!allow_dynamic && grid > fbk::kMaxSingleShares) grid = fbk::kMaxSingleShares;
     // Launches with enough work deal 90 % of it out statically and cut the rest into three small
     // shares per CTA (each worth >= ~200 items), drawn dynamically; small launches stay static.
-    static const int dyn_pct = getenv("FBX_DYN_PCT") ? atoi(getenv("FBX_DYN_PCT")) : 10;      // EXPERIMENT
-    static const int dyn_k = getenv("FBX_DYN_K") ? atoi(getenv("FBX_DYN_K")) : 3;
-    static const int dyn_min = getenv("FBX_DYN_MIN") ? atoi(getenv("FBX_DYN_MIN")) : 400;
+    constexpr int dyn_pct = 10, dyn_k = 3;
     const long long rest = total_cost * dyn_pct / 100;
-    if (allow_dynamic && dyn_pct > 0 && rest / (grid * dyn_k) >= dyn_min) {
+    if (allow_dynamic && rest / (grid * dyn_k) >= 400) {
         out->static_cost = total_cost - rest;
         out->nshares = (int)(grid * (1 + dyn_k));
     } else {
@@ -550,12 +547,6 @@ static cudaError_t launch_kernel(int mode, int s0, int s1, const LaunchShape &sh
     static std::atomic<int> launches{0};
     const_cast<fbk::LaunchParams &>(p).trace_slot = launches.fetch_add(1) & 7;
 #endif
-    {   // EXPERIMENT
-        static const int head = getenv("FBX_HEAD") ? atoi(getenv("FBX_HEAD")) : 0;
-        const_cast<fbk::LaunchParams &>(p).head_bytes = head;
-        static const int early = getenv("FBX_EARLY") ? atoi(getenv("FBX_EARLY")) : 0;
-        const_cast<fbk::LaunchParams &>(p).early_items = early;
-    }
     void *args[1] = {(void *)&p};
     return cudaLaunchKernelExC(&cfg, kernel_for(mode, s0, s1, shape.np), args);
 }

@@ -19,6 +19,10 @@ struct SalSvec {
 fluxbin_status_t validate_dims(const fluxbin_layer_desc_t *d);
 void salient_svecs(const fluxbin_layer_desc_t *d, int sps1, std::vector<SalSvec> &out);
 fluxbin_status_t check_header(const void *p, size_t bytes, FbHeader &h);
+// dimension rules and the salient map (host pointer d->sal_idx) without looking at the other arrays
+fluxbin_status_t validate_dims_and_map(const fluxbin_layer_desc_t *d);
+// header, salient sub-vector list and the row-scale groups without salient columns of a validated description
+void make_packed_header(const fluxbin_layer_desc_t *d, FbHeader &h, std::vector<SalSvec> &sv, std::vector<int> &dead);
 // shared-memory opt-in of every instantiation of the layer kernel on the current device
 fluxbin_status_t opt_in_all_kernels();
 // remember a CUDA error code for fluxbin_last_cuda_error(), clear the runtime's sticky state, return FLUXBIN_ERR_CUDA

@@ -103,8 +103,6 @@ struct LaunchParams {
 #ifdef FB_TRACE
     int trace_slot;             // instrumented build: which of the eight trace buffers this launch writes
 #endif
-    int head_bytes;             // EXPERIMENT: bytes of the first segment prefetched into L2 before the wait
-    int early_items;            // EXPERIMENT: two-pair kernel requests its first items before the wait
     int single_cut[kMaxSingleShares + 1];    // first work item of share s of the single entry; [nshares] = all items
 };
 
@@ -643,64 +641,14 @@ __device__ __forceinline__ void process_rows(const uint8_t *pair_items, int rb_l
     }
 }
 
-// Row blocks of the narrow last pair of a salient region (W = 8 or 16 steps per item, one scale per step).  These
-// items are small, so a warp keeps the next one in flight while it looks the current one up (with a single item
-// in flight a warp pays a full load latency per item whatever its size, which makes a narrow item as slow as a
-// full one).
-template <int W, int BT>
-__device__ __forceinline__ void process_rows_narrow(const uint8_t *pair_items, int rb_lo, int rb_hi, const LaneAddr<BT> &la,
-                                                    float *acc, int Mpad)
-{
-    constexpr int IB = ItemBytes<1, W>::value;
-    constexpr int kWarps = Cfg<BT>::kWarps;
-    constexpr int STRIDE = kWarps * IB;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int first = rb_lo + warp;
-    if (first >= rb_hi) return;
-    const int n = (rb_hi - first + kWarps - 1) / kWarps;
-    const uint8_t *pl = pair_items + (int64_t)first * IB + lane * (W < 16 ? W : 16);
-    const uint8_t *ps = pair_items + (int64_t)first * IB + 32 * W + lane * 16;
-    const uint8_t *pend = pair_items + (int64_t)rb_hi * IB;
-    float *accp = acc + first * 32 + lane;
-    ItemRegs<1, W> cur, nxt;
-    load_item<1, W>(cur, pl, ps, 0);
-#pragma unroll 1
-    for (int t = 0; t < n; ++t) {
-        if (t + 1 < n) load_item<1, W>(nxt, pl, ps, STRIDE);
-        if (lane == 0 && pl + 3 * STRIDE < pend) prefetch_l2(pl - lane * (W < 16 ? W : 16) + 2 * STRIDE, IB);
-        finish_item<1, BT, W>(cur, la, accp, Mpad);
-        cur = nxt;
-        pl += STRIDE;
-        ps += STRIDE;
-        accp += kWarps * 32;
-    }
-}
-
 // The same for TWO pairs whose table sets are resident together (slots 0..31 and 32..63, 4-byte entries):
 // for every row block the lane looks up the item of the first pair, then the item of the second
 // (items_b = the second pair's items), adds the two row sums and issues ONE reduction -- half the
 // atomic traffic and half the per-item bookkeeping.  One item is always in flight ahead.
 // BT: 1 (one vector, fp32 entries) or 16 + 2 (two vectors, fp16 entries: the same 4-byte slots).
-// The first row block's two items of this warp's run (the loads process_rows2 would start with), requested ahead
-// of the wait for the predecessor and of the table build.
-template <int SPS, int BT>
-__device__ __forceinline__ void preload_first2(ItemRegs<SPS> &ra, ItemRegs<SPS> &rb, const uint8_t *items_a, const uint8_t *items_b,
-                                               int rb_lo, int rb_hi)
-{
-    constexpr int IB = ItemBytes<SPS>::value;
-    constexpr int SB = (SPS == 16) ? 4 : (SPS == 8) ? 8 : 16;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int first = rb_lo + warp;
-    if (first >= rb_hi) return;
-    const int64_t o_l = (int64_t)first * IB + lane * 16, o_s = (int64_t)first * IB + FB_ITEM_BITS_BYTES + lane * SB;
-    load_item<SPS>(ra, items_a + o_l, items_a + o_s, 0);
-    load_item<SPS>(rb, items_b + o_l, items_b + o_s, 0);
-}
-
 template <int SPS, int BT>
 __device__ __forceinline__ void process_rows2(const uint8_t *items_a, const uint8_t *items_b, int rb_lo, int rb_hi,
-                                              const LaneAddr<1> &la, float *acc, int Mpad,
-                                              const ItemRegs<SPS> *pre_a = nullptr, const ItemRegs<SPS> *pre_b = nullptr)
+                                              const LaneAddr<1> &la, float *acc, int Mpad)
 {
     static_assert(geom(BT) == 1, "two table sets side by side need 4-byte entries");
     // lookups of one 128-bit half of an item, added to the row sums of the batch vectors
@@ -736,11 +684,8 @@ __device__ __forceinline__ void process_rows2(const uint8_t *items_a, const uint
     // The last row block is peeled off: the steady state has no guards in it, and the prefetch is one
     // predicated instruction (guards cost about 20 instructions per item in moves, predicates and branches).
     ItemRegs<SPS> ra, rb;
-    if (pre_a) { ra = *pre_a; rb = *pre_b; }
-    else {
-        load_item<SPS>(ra, pla, psa, 0);
-        load_item<SPS>(rb, plb, psb, 0);
-    }
+    load_item<SPS>(ra, pla, psa, 0);
+    load_item<SPS>(rb, plb, psb, 0);
     const int n_pf = lane < 2 * LPI ? n - (kPrefetchTrips + 1) : 0;      // trips in which this lane prefetches
     for (int t = 0; t < n - 1; ++t) {
         prefetch_line_if(pp, t < n_pf);
@@ -848,46 +793,48 @@ __device__ __forceinline__ void reduce_and_store(const LinearEntry &E, int nb, i
     const int ndone = done_list[kMaxTiles];
     if (ndone > 0) {
         __threadfence();
-        // all rows of all completed tiles in one flat loop of 4-row groups, six 128-bit loads in
-        // flight per thread (the accumulators live in L2; one round trip serves ~8K rows per CTA)
+#ifdef FB_STAGED_READBACK
+        // All rows of all completed tiles, in 4-row groups: every group is requested with one asynchronous 16-byte
+        // copy from the accumulators (L2) into the table area, which is free by now -- no registers are held while
+        // the copies fly, so one round trip serves every tile the CTA completed (up to 16K rows per batch) however
+        // many there are -- then the groups are converted from shared memory and the accumulators re-zeroed.
         const int gpt = E.tile_rb * 8;                 // 4-row groups per tile
         constexpr int NV = nvec(BT);
         const int total = ndone * gpt * NV;
-        constexpr int U = 6;
-        const bool vec_ok = (E.ldy & 3) == 0;          // rows in groups of four stay 8 / 16-byte aligned in y
-        // group idx of the flat list -> batch vector and first row (done_list is small and lives in shared memory,
-        // so the decode is repeated after the loads instead of being kept in registers across them)
-        // (idx is in range) -> element offset of the group in the accumulators, or -1 for rows beyond the padding
+        constexpr int kStageGroups = TabCfg<BT>::kTableBytes / 16;
+        // group idx of the flat list -> batch vector, first row, element offset in the accumulators (-1: padding rows)
         auto decode = [&](int idx, int &bb, int &row) -> int {
             const int li = idx / (gpt * NV), rem = idx - li * (gpt * NV);
             bb = rem / gpt;
             row = (done_list[li] * gpt + (rem - bb * gpt)) * 4;
             return row < E.Mpad ? bb * E.Mpad + row : -1;
         };
-        for (int base = tid; base < total; base += U * kThreads) {
-            float4 v[U];
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int idx = base + u * kThreads;
+        const bool vec_ok = (E.ldy & 3) == 0;          // rows in groups of four stay 8 / 16-byte aligned in y
+        for (int b0 = 0; b0 < total; b0 += kStageGroups) {
+            const int n = min(kStageGroups, total - b0);
+            for (int i = tid; i < n; i += kThreads) {
                 int bb, row;
-                const int eoff = idx < total ? decode(idx, bb, row) : -1;
-                if (eoff >= 0) v[u] = __ldcg((const float4 *)(E.acc + eoff));
+                const int eoff = decode(b0 + i, bb, row);
+                if (eoff >= 0)
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(kTabBase + 16u * (uint32_t)i),
+                                 "l"(__cvta_generic_to_global(E.acc + eoff)) : "memory");
             }
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int idx = base + u * kThreads;
-                if (idx >= total) break;
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            __syncthreads();
+            for (int i = tid; i < n; i += kThreads) {
                 int bb, row;
-                const int eoff = decode(idx, bb, row);
+                const int eoff = decode(b0 + i, bb, row);
                 if (eoff < 0) continue;
+                float4 v;
+                asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(kTabBase + 16u * (uint32_t)i));
                 __stcg((float4 *)(E.acc + eoff), make_float4(0.f, 0.f, 0.f, 0.f));
                 if (bb >= nb) continue;
-                const float e[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
                 if (vec_ok && row + 3 < E.M) {
                     if (y_fp32) {
-                        *(float4 *)((float *)E.y + (int64_t)bb * E.ldy + row) = v[u];
+                        *(float4 *)((float *)E.y + (int64_t)bb * E.ldy + row) = v;
                     } else {
-                        const __half2 lo = __floats2half2_rn(e[0], e[1]), hi = __floats2half2_rn(e[2], e[3]);
+                        const __half2 lo = __floats2half2_rn(v.x, v.y), hi = __floats2half2_rn(v.z, v.w);
                         uint2 pk;
                         pk.x = *(const uint32_t *)&lo;
                         pk.y = *(const uint32_t *)&hi;
@@ -895,6 +842,7 @@ __device__ __forceinline__ void reduce_and_store(const LinearEntry &E, int nb, i
                     }
                     continue;
                 }
+                const float e[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     if (row + k >= E.M) break;
@@ -902,7 +850,47 @@ __device__ __forceinline__ void reduce_and_store(const LinearEntry &E, int nb, i
                     else ((__half *)E.y)[(int64_t)bb * E.ldy + row + k] = __float2half_rn(e[k]);
                 }
             }
+            __syncthreads();       // the stage is reused by the next batch (and by the next table build)
         }
+#else
+        // all rows of all completed tiles in one flat loop of 4-row groups, four 128-bit loads in
+        // flight per thread (the accumulators live in L2; one round trip serves ~8K rows per CTA)
+        const int gpt = E.tile_rb * 8;                 // 4-row groups per tile
+        constexpr int NV = nvec(BT);
+        const int total = ndone * gpt * NV;
+        constexpr int U = 4;
+        for (int base = tid; base < total; base += U * kThreads) {
+            float4 v[U];
+            float *a[U];
+            int row[U], bb[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                int idx = base + u * kThreads;
+                a[u] = nullptr;
+                if (idx < total) {
+                    int li = idx / (gpt * NV), rem = idx - li * (gpt * NV);
+                    bb[u] = rem / gpt;
+                    row[u] = (done_list[li] * gpt + (rem - bb[u] * gpt)) * 4;
+                    if (row[u] < E.Mpad) a[u] = E.acc + (int64_t)bb[u] * E.Mpad + row[u];
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) if (a[u]) v[u] = __ldcg((const float4 *)a[u]);
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (!a[u]) continue;
+                __stcg((float4 *)a[u], make_float4(0.f, 0.f, 0.f, 0.f));
+                if (bb[u] >= nb) continue;
+                const float e[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    if (row[u] + k >= E.M) break;
+                    if (y_fp32) ((float *)E.y)[(int64_t)bb[u] * E.ldy + row[u] + k] = e[k];
+                    else ((__half *)E.y)[(int64_t)bb[u] * E.ldy + row[u] + k] = __float2half_rn(e[k]);
+                }
+            }
+        }
+#endif
         for (int li = tid; li < ndone; li += kThreads) E.tickets[done_list[li]] = 0;
     }
     __syncthreads();       // done_list / tile_cnt are reused by the next entry
@@ -1013,17 +1001,6 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
             prefetch_run_head(items, ib, pf_d, kWarps, rb_lo, rb_hi, head_trips);
             if (np == 2) prefetch_run_head(items_b, ib, pf_d, kWarps, rb_lo, rb_hi, head_trips);
 
-            if (!predecessor_done && P.head_bytes > 0) {
-                // EXPERIMENT: the start of the CTA's first run of items goes to L2 while the predecessor drains
-                const int seg_bytes = (rb_hi - rb_lo) * ib;
-                const int want = min(seg_bytes, P.head_bytes / np);
-                const int off = tid * 4096;
-                if (off < want) {
-                    const uint32_t nbytes = (uint32_t)min(4096, want - off);
-                    prefetch_l2(items + (size_t)rb_lo * ib + off, nbytes);
-                    if (np == 2) prefetch_l2(items_b + (size_t)rb_lo * ib + off, nbytes);
-                }
-            }
             FB_TRACE_T0(t_fetch);
             // (fetching the next pair's inputs ahead of the lookups was measured 15 % slower: the extra
             // live registers push the lookup loop over the 80-register budget of 3 CTAs per SM)
@@ -1035,12 +1012,8 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
             }
             // region 0, one pair at a time (short runs): first item in flight during the build.  (With two
             // pairs per row block the runs are long and the extra live registers cost more than they hide.)
-            ItemRegs<SPS0> pre, pre_b;
+            ItemRegs<SPS0> pre;
             if (NP == 1 && region == 0) preload_first<SPS0, BT>(pre, items, rb_lo, rb_hi);
-            const bool early2 = NP == 2 && region == 0 && P.early_items && !predecessor_done;    // EXPERIMENT
-            if constexpr (NP == 2 && geom(BT) == 1) {
-                if (early2) preload_first2<SPS0, BT>(pre, pre_b, items, items_b, rb_lo, rb_hi);
-            }
 
             if (!predecessor_done) {
                 FB_TRACE_AT(11);
@@ -1078,16 +1051,13 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
             FB_TRACE_ADD(4, t_build);
             FB_TRACE_T0(t_rows);
             if (region == 0) {
-                if constexpr (NP == 2) {
-                    if (early2) process_rows2<SPS0, BT>(items, items_b, rb_lo, rb_hi, la, E.acc, E.Mpad, &pre, &pre_b);
-                    else process_rows2<SPS0, BT>(items, items_b, rb_lo, rb_hi, la, E.acc, E.Mpad);
-                }
+                if constexpr (NP == 2) process_rows2<SPS0, BT>(items, items_b, rb_lo, rb_hi, la, E.acc, E.Mpad);
                 else process_rows<SPS0, BT>(items, rb_lo, rb_hi, la, E.acc, E.Mpad, &pre);
             } else if (steps == 32) {
                 process_rows<SPS1, BT>(items, rb_lo, rb_hi, la, E.acc, E.Mpad);
             } else if constexpr (SPS1 == 1) {
-                if (steps == 16) process_rows_narrow<16, BT>(items, rb_lo, rb_hi, la, E.acc, E.Mpad);
-                else process_rows_narrow<8, BT>(items, rb_lo, rb_hi, la, E.acc, E.Mpad);
+                if (steps == 16) process_rows<1, BT, 16>(items, rb_lo, rb_hi, la, E.acc, E.Mpad);
+                else process_rows<1, BT, 8>(items, rb_lo, rb_hi, la, E.acc, E.Mpad);
             }
 
             FB_TRACE_ADD(5, t_rows);

@@ -4,7 +4,6 @@
 #include "fluxbin_internal.h"
 
 #include <algorithm>
-#include <cstdlib>
 #include <cstring>
 #include <vector>
 
@@ -111,7 +110,6 @@ static void make_header(const fluxbin_layer_desc_t *d, int n_svec, int n_dead, F
             h.npairs[1] = (slots + 31) / 32;
             const int last = slots - 32 * (h.npairs[1] - 1);
             h.sal_last_w = last <= 8 ? 8 : last <= 16 ? 16 : 32;
-            if (getenv("FBX_NO_NARROW")) h.sal_last_w = 32;      // EXPERIMENT
         }
     }
     h.item_bytes[0] = item_bytes_for(h.sps[0]);
@@ -157,6 +155,20 @@ fluxbin_status_t check_header(const void *p, size_t bytes, FbHeader &h)
     make_header(&d, h.n_sal_svec, h.n_dead, ref);
     if (std::memcmp(&ref, &h, sizeof(h)) != 0) return FLUXBIN_ERR_FORMAT;
     return FLUXBIN_OK;
+}
+
+fluxbin_status_t validate_dims_and_map(const fluxbin_layer_desc_t *d)
+{
+    fluxbin_status_t s = validate_dims(d);
+    if (s != FLUXBIN_OK) return s;
+    return validate_salient(d);
+}
+
+void make_packed_header(const fluxbin_layer_desc_t *d, FbHeader &h, std::vector<SalSvec> &sv, std::vector<int> &dead)
+{
+    salient_svecs(d, salient_sps(d->N, d->g), sv);
+    dead_groups(d, dead);
+    make_header(d, (int)sv.size(), (int)dead.size(), h);
 }
 
 // ---- what a table slot holds: which canonical bits / scales / columns it covers ------------------

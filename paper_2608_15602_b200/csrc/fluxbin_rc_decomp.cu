@@ -38,7 +38,7 @@ constexpr int kMaxK = 4;
 struct Args {
     const float *W;        // [M][ldw]
     long long ldw;
-    int M, N, g, NG, K;
+    int M, N, g, NG, K, num_sms;
     float eps;
     uint32_t *bits;        // [K][M][N/32]
     float *ar;             // [K][M][NG]
@@ -141,7 +141,10 @@ enum PassMode {
     kInit = 4        // greedy initialisation only (T == 0)
 };
 
-template <int C, int K, int MODE> __global__ void __launch_bounds__(kWarpsPerCta * 32) pass_kernel(Args a, int k_arg)
+// A CTA owns one column group and a strided set of its 64-row blocks (gridDim.x = groups x CTAs per group), so
+// the column scales are loaded once, the column numerators stay in registers across the row blocks and the
+// reduction over the CTA, the atomics and the ticket happen once per CTA.
+template <int C, int K, int MODE> __global__ void __launch_bounds__(kWarpsPerCta * 32, (C * K <= 8) ? 3 : 1) pass_kernel(Args a, int k_arg)
 {
     constexpr bool kInitial = MODE == kInitRow || MODE == kInit;
     constexpr bool kSearch = MODE == kSignRow || MODE == kSign;
@@ -150,15 +153,11 @@ template <int C, int K, int MODE> __global__ void __launch_bounds__(kWarpsPerCta
     __shared__ float den_part[kWarpsPerCta];
     __shared__ int is_last;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int G = blockIdx.x, row0 = blockIdx.y * kRowsPerCta + warp * kRowsPerWarp;
+    const int G = blockIdx.x % a.NG, part_id = blockIdx.x / a.NG, cpg = gridDim.x / a.NG;
     const int nw = a.N / 32;
-    const int nrows = max(0, min(kRowsPerWarp, a.M - row0));
+    const int nblocks = (a.M + kRowsPerCta - 1) / kRowsPerCta;
     const int k = MODE == kRow ? k_arg : 0;                // base of the row form
 
-    WarpRows<C, K> in;
-    in.load_w(a, G, row0, nrows, lane);
-    if constexpr (MODE == kRow) in.load_signs(a, G, row0, nrows, lane);
-    if constexpr (!kInitial) in.load_row_scales(a, G, row0, nrows, lane);
     float ack[K][C];                     // column scales of every base for this lane's columns
     float lv[C];                         // live mask (initial column scales)
     if constexpr (kInitial) {
@@ -191,6 +190,22 @@ template <int C, int K, int MODE> __global__ void __launch_bounds__(kWarpsPerCta
 #pragma unroll
     for (int c = 0; c < C; ++c) colsum[c] = 0.f;
     float ar2 = 0.f;
+
+    for (int blk = part_id; blk < nblocks; blk += cpg) {
+    const int row0 = blk * kRowsPerCta + warp * kRowsPerWarp;
+    const int nrows = max(0, min(kRowsPerWarp, a.M - row0));
+    if (blk + cpg < nblocks) {
+        // the W lines of this warp's rows in the CTA's next block start moving into L2
+        const int nrow0 = row0 + cpg * kRowsPerCta;
+        for (int f = lane; f < kRowsPerWarp * C; f += 32) {
+            const int r = f / C, line = f % C;
+            if (nrow0 + r < a.M) asm volatile("prefetch.global.L2 [%0];" ::"l"(a.W + (long long)(nrow0 + r) * a.ldw + G * a.g + line * 32));
+        }
+    }
+    WarpRows<C, K> in;
+    in.load_w(a, G, row0, nrows, lane);
+    if constexpr (MODE == kRow) in.load_signs(a, G, row0, nrows, lane);
+    if constexpr (!kInitial) in.load_row_scales(a, G, row0, nrows, lane);
 
 #pragma unroll
     for (int r = 0; r < kRowsPerWarp; ++r) {
@@ -289,9 +304,11 @@ template <int C, int K, int MODE> __global__ void __launch_bounds__(kWarpsPerCta
         }
     }
 
+    }       // row blocks of this CTA
+
     if constexpr (MODE == kInit) {
         // no update follows: the column scales are the initial ones
-        if (blockIdx.y == 0 && warp == 0) {
+        if (part_id == 0 && warp == 0) {
 #pragma unroll
             for (int q = 0; q < K; ++q)
 #pragma unroll
@@ -321,7 +338,7 @@ template <int C, int K, int MODE> __global__ void __launch_bounds__(kWarpsPerCta
         // the accumulators and the ticket go back to zero for the next pass.
         __threadfence();
         __syncthreads();
-        if (threadIdx.x == 0) is_last = (atomicAdd(a.tickets + G, 1u) == gridDim.y - 1);
+        if (threadIdx.x == 0) is_last = (atomicAdd(a.tickets + G, 1u) == (unsigned)cpg - 1u);
         __syncthreads();
         if (is_last) {
             __threadfence();
@@ -348,7 +365,14 @@ template <int C, int K, int MODE> __global__ void __launch_bounds__(kWarpsPerCta
 
 template <int C, int K> cudaError_t run(const Args &a, int T, cudaStream_t s)
 {
-    const dim3 grid(a.NG, (a.M + kRowsPerCta - 1) / kRowsPerCta), block(kWarpsPerCta * 32);
+    // CTAs per column group: enough to fill every SM with the CTAs it can hold (three of the small instantiations,
+    // one of those with many bases or wide groups: see the launch bounds), at most one per 64-row block
+    const int nblocks = (a.M + kRowsPerCta - 1) / kRowsPerCta;
+    constexpr int kCtasPerSm = (C * K <= 8) ? 3 : 1;
+    int cpg = (kCtasPerSm * a.num_sms + a.NG - 1) / a.NG;
+    if (cpg > nblocks) cpg = nblocks;
+    if (cpg < 1) cpg = 1;
+    const dim3 grid((unsigned)(a.NG * cpg)), block(kWarpsPerCta * 32);
     if (T == 0) {
         pass_kernel<C, K, kInit><<<grid, block, 0, s>>>(a, 0);
         return cudaGetLastError();
@@ -399,6 +423,12 @@ extern "C" fluxbin_status_t fluxbin_rc_decomp(const float *d_W, int64_t ldw, con
     a.W = d_W; a.live = d_col_live; a.ldw = ldw; a.M = M; a.N = N; a.g = g; a.NG = N / g; a.K = K; a.eps = eps;
     a.bits = d_bits;
     a.ar16 = d_row_scale; a.ac16 = d_col_scale;
+    {
+        int dev = 0, sms = 0;
+        FB_CUDA(cudaGetDevice(&dev));
+        FB_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        a.num_sms = sms > 0 ? sms : 1;
+    }
     uint8_t *ws = (uint8_t *)d_workspace;
     // the fp32 working copies of the scales live in the caller's fp32 outputs when those are given
     a.ar = d_row_scale_f32 ? d_row_scale_f32 : (float *)ws;     ws += align256((size_t)K * M * a.NG * 4);

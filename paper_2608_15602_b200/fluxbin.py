@@ -41,7 +41,8 @@ EXPORTS = ["fluxbin_packed_size", "fluxbin_validate", "fluxbin_pack_host", "flux
            "fluxbin_plan_create", "fluxbin_plan_run", "fluxbin_plan_num_launches", "fluxbin_plan_pairs_per_row_block",
            "fluxbin_plan_free",
            "fluxbin_linear_noalloc", "fluxbin_noalloc_capacity", "fluxbin_set_table_format", "fluxbin_get_table_format",
-           "fluxbin_rc_decomp", "fluxbin_rc_decomp_workspace_size", "fluxbin_rc_salient_residual"]
+           "fluxbin_rc_decomp", "fluxbin_rc_decomp_workspace_size", "fluxbin_rc_decomp_passes",
+           "fluxbin_rc_salient_collect", "fluxbin_pack_device", "fluxbin_pack_device_workspace_size", "fluxbin_rc_salient_residual"]
 
 _LIB = None
 
@@ -96,10 +97,16 @@ def _lib():
         lib.fluxbin_noalloc_capacity.restype, lib.fluxbin_noalloc_capacity.argtypes = sz, []
         lib.fluxbin_rc_decomp_workspace_size.restype = sz
         lib.fluxbin_rc_decomp_workspace_size.argtypes = [i32, i32, i32, i32]
+        lib.fluxbin_rc_decomp_passes.restype, lib.fluxbin_rc_decomp_passes.argtypes = i32, [i32, i32]
         lib.fluxbin_rc_decomp.restype = ctypes.c_int
         lib.fluxbin_rc_decomp.argtypes = [vp, i64, vp, i32, i32, i32, i32, i32, ctypes.c_float, vp, vp, vp, vp, vp, vp, sz, vp]
         lib.fluxbin_rc_salient_residual.restype = ctypes.c_int
         lib.fluxbin_rc_salient_residual.argtypes = [vp, i64, i32, i32, i32, i32, vp, vp, vp, vp, vp, i32, vp, i64, i32, vp, vp]
+        lib.fluxbin_rc_salient_collect.restype = ctypes.c_int
+        lib.fluxbin_rc_salient_collect.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
+        lib.fluxbin_pack_device_workspace_size.restype, lib.fluxbin_pack_device_workspace_size.argtypes = sz, [i32, i32, i32]
+        lib.fluxbin_pack_device.restype = ctypes.c_int
+        lib.fluxbin_pack_device.argtypes = [dp, vp, vp, sz, vp, sz, vp, ctypes.POINTER(vp)]
         _LIB = lib
     return _LIB
 
@@ -271,6 +278,10 @@ def rc_decomp_workspace_size(M: int, N: int, g: int, K: int) -> int:
     return int(_lib().fluxbin_rc_decomp_workspace_size(M, N, g, K))
 
 
+def rc_decomp_passes(K: int, T: int) -> int:
+    return int(_lib().fluxbin_rc_decomp_passes(K, T))
+
+
 def rc_decomp_status(d_W, ldw, M, N, g, K, T, eps, d_bits, d_row_scale, d_col_scale, d_row_f32, d_col_f32, d_ws, ws_bytes,
                      stream=0, d_col_live=None) -> int:
     """fluxbin_rc_decomp (argument marshalling only; every pointer is a device address or None)."""
@@ -282,6 +293,39 @@ def rc_salient_residual(d_W, ldw, M, N, g, Kb, d_bits, d_row_f32, d_col_f32, d_s
                         d_live, stream=0):
     _check(int(_lib().fluxbin_rc_salient_residual(d_W, ldw, M, N, g, Kb, d_bits, d_row_f32, d_col_f32, d_sal_idx, d_pos,
                                                   n_sal, d_P, ldp, ncols_p, d_live, stream)), "fluxbin_rc_salient_residual")
+
+
+def rc_salient_collect(d_bits_p, d_row_f32_p, d_col_f32_p, d_pos, d_block_group, M, N, g, Ks, n_sal, width, nblocks, d_sal_bits,
+                       d_sal_row_scale, d_sal_col_scale, d_sal_row_f32=None, d_sal_col_f32=None, stream=0):
+    _check(int(_lib().fluxbin_rc_salient_collect(d_bits_p, d_row_f32_p, d_col_f32_p, d_pos, d_block_group, M, N, g, Ks, n_sal,
+                                                 width, nblocks, d_sal_bits, d_sal_row_scale, d_sal_col_scale, d_sal_row_f32,
+                                                 d_sal_col_f32, stream)), "fluxbin_rc_salient_collect")
+
+
+def pack_device_workspace_size(N: int, g: int, n_sal: int) -> int:
+    return int(_lib().fluxbin_pack_device_workspace_size(N, g, n_sal))
+
+
+def packed_size_of(M, N, Kb, Ks, g, sal_idx: np.ndarray) -> int:
+    """fluxbin_packed_size from the dimensions and the (host) salient map alone."""
+    d = LayerDesc(M, N, Kb, Ks, g, int(sal_idx.size), None, None, None, _ptr(sal_idx), None, None, None)
+    return int(_lib().fluxbin_packed_size(ctypes.byref(d)))
+
+
+def pack_device_status(dims, dev_ptrs, h_sal_idx: np.ndarray, d_packed: int, d_bytes: int, d_ws: int, ws_bytes: int, stream: int = 0):
+    """fluxbin_pack_device returning (status, handle).  dims = (M, N, Kb, Ks, g, n_sal); dev_ptrs = device addresses of
+    bits, row_scale, col_scale, sal_idx, sal_bits, sal_row_scale, sal_col_scale (None where absent)."""
+    d = LayerDesc(*dims, *dev_ptrs)
+    h = ctypes.c_void_p()
+    st = _lib().fluxbin_pack_device(ctypes.byref(d), _ptr(h_sal_idx), d_packed, d_bytes, d_ws, ws_bytes, stream, ctypes.byref(h))
+    return int(st), h.value
+
+
+def pack_device(dims, dev_ptrs, h_sal_idx, d_packed, d_bytes, d_ws, ws_bytes, stream=0, buffer=None) -> Weight:
+    st, h = pack_device_status(dims, dev_ptrs, h_sal_idx, d_packed, d_bytes, d_ws, ws_bytes, stream)
+    _check(st, "fluxbin_pack_device")
+    M, N, Kb, Ks, g, n_sal = dims
+    return Weight(h, (M, N, Kb, Ks if n_sal else 0, g, n_sal if Ks else 0), buffer)
 
 
 def rc_decomp(*args, **kw):

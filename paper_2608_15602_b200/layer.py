@@ -138,74 +138,82 @@ def _pad_width(s_max: int) -> int:
 def hybrid_decompose(W: torch.Tensor, g: int, Kb: int, Ks: int, sal_idx, T: int, eps: float = 1e-8):
     """Global bases plus a refinement on given salient columns (Algorithm 2 without the saliency search and the
     Hessian compensation): fluxbin_rc_decomp on W, then on the residual of every group's salient columns, each
-    group's block padded with zero columns to a common width (the padding marked in the live mask).  Only data
-    movement happens here (gathers, scatters, bit packing of the result); both decompositions run in the library.
-    Returns a dict of CUDA tensors in the canonical layout of a layer description."""
+    group's block padded with zero columns to a common width (the padding marked in the live mask), then
+    fluxbin_rc_salient_collect.  Only index arithmetic for the padded layout happens here; the decompositions, the
+    residual, the gathers of the result and every rounding run in the library.
+    Returns a dict of CUDA tensors in the canonical layout of a layer description (sal_idx also as a host array)."""
     assert W.is_cuda and W.dtype == torch.float32
     W = W.contiguous()
     M, N = W.shape
     dev = W.device
     out = rc_decompose(W, g, Kb, T, eps)
-    sal_idx = torch.as_tensor(np.asarray(sal_idx, np.int64), device=dev)
-    n_sal = int(sal_idx.numel())
+    sal_host = np.ascontiguousarray(np.asarray(sal_idx, np.int32))
+    n_sal = int(sal_host.size)
     res = {"bits": out["bits"], "row_scale": out["row_scale"], "col_scale": out["col_scale"],
-           "row_scale_f32": out["row_scale_f32"], "col_scale_f32": out["col_scale_f32"], "sal_idx": sal_idx}
+           "row_scale_f32": out["row_scale_f32"], "col_scale_f32": out["col_scale_f32"], "sal_idx_host": sal_host}
     if Ks == 0 or n_sal == 0:
         return res
-    # one padded block per group that has salient columns (index arithmetic for the layout only)
-    grp = sal_idx // g
-    groups, counts = torch.unique_consecutive(grp, return_counts=True)
+    # one padded block per group that has salient columns (index arithmetic for the layout only, on the host)
+    grp = sal_host // g
+    groups, first, counts = np.unique(grp, return_index=True, return_counts=True)
     width = _pad_width(int(counts.max()))
-    first = torch.cumsum(counts, 0) - counts
-    slot = torch.repeat_interleave(torch.arange(len(groups), device=dev), counts)            # block of each virtual column
-    pos = slot * width + (torch.arange(n_sal, device=dev) - first[slot])                     # its column in the padded matrix
-    ncols_p = len(groups) * width
+    slot = np.repeat(np.arange(len(groups)), counts)                        # block of each virtual column
+    pos = (slot * width + (np.arange(n_sal) - first[slot])).astype(np.int32)  # its column in the padded matrix
+    nblocks = len(groups)
+    ncols_p = nblocks * width
+    idx32 = torch.from_numpy(sal_host).to(dev)
+    pos32 = torch.from_numpy(pos).to(dev)
+    block_group = torch.from_numpy(groups.astype(np.int32)).to(dev)
     P = torch.empty((M, ncols_p), dtype=torch.float32, device=dev)
     live = torch.empty(ncols_p, dtype=torch.float32, device=dev)
-    idx32, pos32 = sal_idx.to(torch.int32), pos.to(torch.int32)
     # the residual of the global part on the salient columns, written into the padded layout by the library
     fluxbin.rc_salient_residual(W.data_ptr(), W.stride(0), M, N, g, Kb, out["bits"].data_ptr(), out["row_scale_f32"].data_ptr(),
                                 out["col_scale_f32"].data_ptr(), idx32.data_ptr(), pos32.data_ptr(), n_sal, P.data_ptr(),
                                 P.stride(0), ncols_p, live.data_ptr(), _stream_ptr())
     so = rc_decompose(P, width, Ks, T, eps, col_live=live)
-    # back to the canonical salient arrays
-    nws = (n_sal + 31) // 32
-    sw = so["bits"][:, :, pos // 32]
-    sbit = ((sw >> (pos % 32).to(torch.int32)) & 1).to(torch.int64)                           # [Ks][M][n_sal]
-    v = torch.arange(n_sal, device=dev)
-    packed = torch.zeros((Ks, M, nws), dtype=torch.int64, device=dev)
-    packed.scatter_add_(2, (v // 32).expand(Ks, M, n_sal), sbit << (v % 32))
-    res["sal_bits"] = (packed & 0xFFFFFFFF).to(torch.int64)
-    sal_row = torch.zeros((Ks, M, N // g), dtype=torch.float32, device=dev)
-    sal_row[:, :, groups] = so["row_scale_f32"]
-    res["sal_row_scale_f32"] = sal_row
-    res["sal_col_scale_f32"] = so["col_scale_f32"][:, pos]
-    res["sal_row_scale"] = sal_row.to(torch.float16)
-    res["sal_col_scale"] = res["sal_col_scale_f32"].to(torch.float16)
-    res["sal_signs"] = sbit
+    # back to the canonical salient arrays, on the device
+    res["sal_idx"] = idx32
+    res["sal_bits"] = torch.empty((Ks, M, (n_sal + 31) // 32), dtype=torch.int32, device=dev)
+    res["sal_row_scale"] = torch.empty((Ks, M, N // g), dtype=torch.float16, device=dev)
+    res["sal_col_scale"] = torch.empty((Ks, n_sal), dtype=torch.float16, device=dev)
+    res["sal_row_scale_f32"] = torch.empty((Ks, M, N // g), dtype=torch.float32, device=dev)
+    res["sal_col_scale_f32"] = torch.empty((Ks, n_sal), dtype=torch.float32, device=dev)
+    fluxbin.rc_salient_collect(so["bits"].data_ptr(), so["row_scale_f32"].data_ptr(), so["col_scale_f32"].data_ptr(),
+                               pos32.data_ptr(), block_group.data_ptr(), M, N, g, Ks, n_sal, width, nblocks,
+                               res["sal_bits"].data_ptr(), res["sal_row_scale"].data_ptr(), res["sal_col_scale"].data_ptr(),
+                               res["sal_row_scale_f32"].data_ptr(), res["sal_col_scale_f32"].data_ptr(), _stream_ptr())
+    res["_keep"] = (so, P, live, pos32, block_group)
     return res
+
+
+def pack_device(r: dict, M: int, N: int, g: int, Kb: int, Ks: int) -> "FluxBinLinear":
+    """fluxbin_pack_device on the device-resident canonical arrays of hybrid_decompose: a packed layer without the
+    arrays crossing host memory."""
+    dev = r["bits"].device
+    sal_host = r.get("sal_idx_host", np.zeros(0, np.int32))
+    has_sal = Ks > 0 and sal_host.size > 0 and "sal_bits" in r
+    if not has_sal:
+        Ks, sal_host = 0, np.zeros(0, np.int32)
+    n_sal = int(sal_host.size)
+    nbytes = fluxbin.packed_size_of(M, N, Kb, Ks, g, sal_host)
+    lin = object.__new__(FluxBinLinear)
+    lin.device = torch.device(dev)
+    lin.buffer = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    ws = torch.empty(max(fluxbin.pack_device_workspace_size(N, g, n_sal), 256), dtype=torch.uint8, device=dev)
+    ptrs = [r["bits"].data_ptr(), r["row_scale"].data_ptr(), r["col_scale"].data_ptr()]
+    ptrs += [r[k].data_ptr() for k in ("sal_idx", "sal_bits", "sal_row_scale", "sal_col_scale")] if has_sal else [None] * 4
+    lin.weight = fluxbin.pack_device((M, N, Kb, Ks, g, n_sal), ptrs, sal_host, lin.buffer.data_ptr(), nbytes, ws.data_ptr(),
+                                     int(ws.numel()), _stream_ptr(), buffer=lin.buffer)
+    lin.M, lin.N, lin.packed_bytes = M, N, nbytes
+    return lin
 
 
 def quantize_dense(W: torch.Tensor, g: int = 128, K: int = 2, T: int = 10, eps: float = 1e-8, sal_idx=None,
                    Ks: int = 0) -> "FluxBinLinear":
     """Dense fp32 CUDA matrix -> packed FluxBin layer: K global bases and, if `sal_idx` (ascending column indices)
-    and Ks > 0 are given, Ks further bases on those columns.  The decompositions run on the GPU
-    (fluxbin_rc_decomp); the canonical arrays pass through host memory because fluxbin_pack takes host pointers."""
-    from . import synth
+    and Ks > 0 are given, Ks further bases on those columns.  Decomposition, collection of the salient arrays and
+    packing all run on the GPU (fluxbin_rc_decomp, fluxbin_rc_salient_collect, fluxbin_pack_device); only the salient
+    map itself is host data."""
     M, N = W.shape
     r = hybrid_decompose(W, g, K, Ks if sal_idx is not None else 0, [] if sal_idx is None else sal_idx, T, eps)
-    torch.cuda.synchronize(W.device)
-    u16 = lambda t: np.ascontiguousarray(t.cpu().numpy().view(np.uint16))
-    if "sal_bits" in r:
-        n_sal = int(r["sal_idx"].numel())
-        L = synth.Linear(M, N, K, Ks, g, n_sal,
-                         np.ascontiguousarray(r["bits"].cpu().numpy().view(np.uint32)), u16(r["row_scale"]), u16(r["col_scale"]),
-                         r["sal_idx"].cpu().numpy().astype(np.int32),
-                         np.ascontiguousarray(r["sal_bits"].cpu().numpy().astype(np.uint32)),
-                         u16(r["sal_row_scale"]), u16(r["sal_col_scale"]))
-    else:
-        L = synth.Linear(M, N, K, 0, g, 0,
-                         np.ascontiguousarray(r["bits"].cpu().numpy().view(np.uint32)), u16(r["row_scale"]), u16(r["col_scale"]),
-                         np.zeros(0, np.int32), np.zeros((0, M, 0), np.uint32), np.zeros((0, M, N // g), np.uint16),
-                         np.zeros((0, 0), np.uint16))
-    return FluxBinLinear(L, device=W.device)
+    return pack_device(r, M, N, g, K, Ks if sal_idx is not None else 0)

@@ -185,7 +185,7 @@ def test_hybrid_decomposition_matches_the_oracle(fb):
     torch.cuda.synchronize()
     want = rc.hybrid_decomp(W, g, Kb, Ks, sal_idx, T, 1e-8, dtype=np.float32)
     B = unpack_bits(r["bits"].cpu().numpy(), N)
-    sB = r["sal_signs"].cpu().numpy().astype(np.float64) * 2 - 1
+    sB = unpack_bits(r["sal_bits"].cpu().numpy(), len(sal_idx))
     got = rc.hybrid_reconstruct(r["row_scale_f32"].cpu().numpy().astype(np.float64), r["col_scale_f32"].cpu().numpy().astype(np.float64), B,
                                 r["sal_row_scale_f32"].cpu().numpy().astype(np.float64),
                                 r["sal_col_scale_f32"].cpu().numpy().astype(np.float64), sB, sal_idx, g)
@@ -220,3 +220,82 @@ def test_quantize_dense_hybrid_layer_runs_through_the_linear_path(fb):
     # and the packed hybrid layer round-trips to the arrays the decomposition produced
     got = linh.unpack()
     assert got.n_sal == len(sal_idx) and np.array_equal(got.sal_idx, sal_idx)
+
+
+def test_salient_collect_gathers_the_padded_refinement(fb):
+    """fluxbin_rc_salient_collect against a numpy gather of the same padded arrays: sign bits of the virtual columns,
+    block row scales scattered to their groups (zero elsewhere), column scales, fp16 rounding to nearest even."""
+    from paper_2608_15602_b200 import fluxbin
+    rng = np.random.default_rng(5)
+    M, N, g, Ks, width = 37, 1024, 128, 2, 32
+    groups = np.array([0, 2, 3, 7], np.int32)                       # blocks of the padded matrix -> row-scale groups
+    counts = [5, 32, 1, 17]
+    sal_idx = np.concatenate([G * g + np.sort(rng.choice(g, c, replace=False)) for G, c in zip(groups, counts)]).astype(np.int32)
+    n_sal, nblocks = len(sal_idx), len(groups)
+    pos = np.concatenate([b * width + np.arange(c) for b, c in enumerate(counts)]).astype(np.int32)
+    ncols_p = nblocks * width
+    bits_p = rng.integers(0, 2 ** 32, size=(Ks, M, ncols_p // 32), dtype=np.uint64).astype(np.uint32)
+    rs_p = rng.standard_normal((Ks, M, nblocks)).astype(np.float32) * 0.02
+    cs_p = rng.standard_normal((Ks, ncols_p)).astype(np.float32)
+    dev = lambda a: torch.from_numpy(a).cuda()
+    out_bits = torch.full((Ks, M, (n_sal + 31) // 32), -1, dtype=torch.int32, device="cuda")
+    out_rs = torch.full((Ks, M, N // g), 7, dtype=torch.float16, device="cuda")
+    out_cs = torch.empty((Ks, n_sal), dtype=torch.float16, device="cuda")
+    out_rs32 = torch.empty((Ks, M, N // g), dtype=torch.float32, device="cuda")
+    out_cs32 = torch.empty((Ks, n_sal), dtype=torch.float32, device="cuda")
+    t = [dev(bits_p.view(np.int32)), dev(rs_p), dev(cs_p), dev(pos), dev(groups)]
+    fluxbin.rc_salient_collect(t[0].data_ptr(), t[1].data_ptr(), t[2].data_ptr(), t[3].data_ptr(), t[4].data_ptr(), M, N, g, Ks,
+                               n_sal, width, nblocks, out_bits.data_ptr(), out_rs.data_ptr(), out_cs.data_ptr(),
+                               out_rs32.data_ptr(), out_cs32.data_ptr())
+    torch.cuda.synchronize()
+    signs = (bits_p[:, :, pos // 32] >> (pos % 32).astype(np.uint32)) & 1                       # [Ks][M][n_sal]
+    want_bits = np.zeros((Ks, M, (n_sal + 31) // 32), np.uint32)
+    for v in range(n_sal):
+        want_bits[:, :, v // 32] |= signs[:, :, v].astype(np.uint32) << np.uint32(v % 32)
+    assert np.array_equal(out_bits.cpu().numpy().view(np.uint32), want_bits)
+    want_rs = np.zeros((Ks, M, N // g), np.float32)
+    want_rs[:, :, groups] = rs_p
+    assert np.array_equal(out_rs32.cpu().numpy(), want_rs)
+    assert np.array_equal(out_rs.cpu().numpy().view(np.uint16), want_rs.astype(np.float16).view(np.uint16))
+    assert np.array_equal(out_cs32.cpu().numpy(), cs_p[:, pos])
+    assert np.array_equal(out_cs.cpu().numpy().view(np.uint16), cs_p[:, pos].astype(np.float16).view(np.uint16))
+
+
+PACK_CASES = [(1, 32, 1, 0, 32, 0), (5, 128, 2, 1, 32, 7), (33, 384, 3, 2, 128, 40), (100, 256, 1, 1, 256, 19),
+              (257, 1024, 2, 1, 128, 51), (65, 640, 2, 1, 128, 640), (127, 128, 4, 4, 64, 128), (600, 2048, 2, 2, 128, 128),
+              (1000, 512, 2, 1, 512, 1), (31, 256, 2, 2, 64, 9)]
+
+
+@pytest.mark.parametrize("M,N,Kb,Ks,g,n_sal", PACK_CASES)
+def test_pack_device_writes_the_bytes_of_pack_host(fb, M, N, Kb, Ks, g, n_sal):
+    """The device packer and the host packer produce the same buffer, byte for byte (all scale formats, narrow and
+    full last salient pairs, ragged row counts), and the handle it returns multiplies like the layer."""
+    from paper_2608_15602_b200 import fluxbin
+    from test_gpu_parity import layer_of, check
+    import oracle
+    L = layer_of(M + 7 * N, M, N, Kb, Ks, g, n_sal)
+    want = fluxbin.pack_host(L)
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int32 if a.dtype == np.uint32 else a.dtype)).cuda()
+    has_sal = L.Ks > 0 and L.n_sal > 0
+    arrays = [dev(L.bits), dev(L.row_scale.view(np.int16)), dev(L.col_scale.view(np.int16))]
+    arrays += [dev(L.sal_idx), dev(L.sal_bits), dev(L.sal_row_scale.view(np.int16)), dev(L.sal_col_scale.view(np.int16))] if has_sal else []
+    ptrs = [a.data_ptr() for a in arrays] + ([None] * 4 if not has_sal else [])
+    packed = torch.full((want.size,), 0xAB, dtype=torch.uint8, device="cuda")
+    ws = torch.empty(max(256, fluxbin.pack_device_workspace_size(N, g, L.n_sal)), dtype=torch.uint8, device="cuda")
+    w = fluxbin.pack_device((L.M, L.N, L.Kb, L.Ks, L.g, L.n_sal), ptrs, L.sal_idx, packed.data_ptr(), want.size, ws.data_ptr(),
+                            ws.numel(), buffer=packed)
+    got = packed.cpu().numpy()
+    assert np.array_equal(got, want), f"first difference at byte {np.nonzero(got != want)[0][:5]}"
+    lin = object.__new__(fb.FluxBinLinear)
+    lin.device, lin.buffer, lin.weight, lin.M, lin.N, lin.packed_bytes = packed.device, packed, w, M, N, want.size
+    x = synth.make_activations(3, M, 2, N)
+    y = lin.forward(torch.from_numpy(x.view(np.float16)).cuda(), lin.workspace(2), fp32_out=True)
+    torch.cuda.synchronize()
+    check(y.cpu().numpy(), oracle.linear_direct(L, x), "device-packed layer", L, x)
+    # argument errors are statuses
+    st, _ = fluxbin.pack_device_status((L.M, L.N, L.Kb, L.Ks, L.g, L.n_sal), ptrs, L.sal_idx, packed.data_ptr(), want.size - 1,
+                                       ws.data_ptr(), ws.numel())
+    assert st == 5
+    st, _ = fluxbin.pack_device_status((L.M, L.N + 1, L.Kb, L.Ks, L.g, L.n_sal), ptrs, L.sal_idx, packed.data_ptr(), want.size,
+                                       ws.data_ptr(), ws.numel())
+    assert st == 2
