@@ -295,6 +295,27 @@ fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_t *const *w
                                      void *cuda_stream, fluxbin_plan_t **out);
 
 /*
+ * A plan with gated pairs: for each of the n_gated pairs {gate member, up member} in gate_up (HOST int32
+ * [n_gated][2]) the plan writes  y = silu(What_gate x_gate) * (What_up x_up),  silu(t) = t / (1 + exp(-t)), into
+ * the gate member's d_y instead of the two separate outputs (the gated feed-forward block of a decoder layer:
+ * gate and up projections read the same input and only their product is needed).  The paper runs its linears as
+ * separate kernels (Experimental Setup); here the CTA that completes a tile of rows of both layers converts both
+ * accumulator tiles at once, so the two fp16 intermediates never reach memory.  Both sums are complete fp32
+ * results of Eq. 10 when they are combined; the product is formed in fp32 and rounded once.
+ * The two members of a pair must have the same number of rows (else FLUXBIN_ERR_SHAPE); a member belongs to at most
+ * one pair and the indices must be valid (else FLUXBIN_ERR_RANGE); d_y / ldy of an up member are ignored (may be
+ * NULL / 0).  Everything else as fluxbin_plan_create.
+ */
+fluxbin_status_t fluxbin_plan_create_gated(int32_t n, const fluxbin_weight_t *const *w,
+                                           const uint16_t *const *d_x, const int64_t *ldx,
+                                           void *const *d_y, const int64_t *ldy,
+                                           const int32_t *gate_up, int32_t n_gated,
+                                           int32_t B, int32_t y_is_fp32,
+                                           void *d_table, size_t table_bytes,
+                                           void *d_workspace, size_t ws_bytes,
+                                           void *cuda_stream, fluxbin_plan_t **out);
+
+/*
  * Launch the plan on cuda_stream: asynchronous, no allocation, no synchronisation (capturable).
  * Runs of plans that share a workspace must be ordered on one stream.
  */

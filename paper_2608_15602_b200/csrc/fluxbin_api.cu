@@ -556,11 +556,12 @@ static void fill_entry(fbk::LinearEntry &E, const fluxbin_weight_t *w, const uin
 {
     E.packed = (const uint8_t *)w->d_packed;
     E.x = x; E.y = y; E.acc = acc; E.tickets = tickets;
-    E.ldx = ldx; E.ldy = ldy; E.reserved0 = 0;
+    E.ldx = ldx; E.ldy = ldy; E.acc2 = nullptr;
     E.off_coldesc = w->h.off_coldesc; E.off_items[0] = w->h.off_items[0]; E.off_items[1] = w->h.off_items[1];
-    E.M = w->h.M; E.N = w->h.N; E.Kb = w->h.Kb; E.Mpad = w->h.Mpad; E.nrb = w->h.nrb;
+    E.M = w->h.M; E.N = w->h.N; E.Kb = w->h.Kb; E.nrb = w->h.nrb;
     E.npairs[0] = w->h.npairs[0]; E.npairs[1] = w->h.npairs[1];
-    E.tile_rb = w->tile_rb; E.ntiles = w->ntiles; E.sal_last_w = w->h.sal_last_w;
+    E.arrivals = w->h.npairs[0] + w->h.npairs[1];
+    E.tile_rb = w->tile_rb; E.ntiles = w->ntiles; E.flags = w->h.sal_last_w;
 }
 
 // The launch shape and the share bounds of a one-layer launch in a given mode depend on the layer alone: they are
@@ -689,25 +690,38 @@ extern "C" size_t fluxbin_plan_workspace_bytes(int32_t n, const fluxbin_weight_t
     return total + 256;      // + the launch counters
 }
 
-extern "C" fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_t *const *w,
-                                                const uint16_t *const *d_x, const int64_t *ldx,
-                                                void *const *d_y, const int64_t *ldy,
-                                                int32_t B, int32_t y_is_fp32,
-                                                void *d_table, size_t table_bytes,
-                                                void *d_workspace, size_t ws_bytes,
-                                                void *cuda_stream, fluxbin_plan_t **out)
+// gate_up: n_gated pairs {gate member, up member} whose outputs are combined as silu(gate) * up into the gate's y
+static fluxbin_status_t plan_create_impl(int32_t n, const fluxbin_weight_t *const *w,
+                                         const uint16_t *const *d_x, const int64_t *ldx,
+                                         void *const *d_y, const int64_t *ldy,
+                                         const int32_t *gate_up, int32_t n_gated,
+                                         int32_t B, int32_t y_is_fp32,
+                                         void *d_table, size_t table_bytes,
+                                         void *d_workspace, size_t ws_bytes,
+                                         void *cuda_stream, fluxbin_plan_t **out)
 {
     if (!out) return FLUXBIN_ERR_NULL;
     *out = nullptr;
     if (!w || !d_x || !ldx || !d_y || !ldy || !d_table || !d_workspace) return FLUXBIN_ERR_NULL;
-    if (n < 1 || B < 1) return FLUXBIN_ERR_RANGE;
+    if (n < 1 || B < 1 || n_gated < 0 || (n_gated > 0 && !gate_up)) return n_gated > 0 && !gate_up ? FLUXBIN_ERR_NULL : FLUXBIN_ERR_RANGE;
+    std::vector<int> role((size_t)n, 0), partner((size_t)n, -1);
+    for (int p = 0; p < n_gated; ++p) {
+        const int g = gate_up[2 * p], u = gate_up[2 * p + 1];
+        if (g < 0 || g >= n || u < 0 || u >= n || g == u) return FLUXBIN_ERR_RANGE;
+        if (role[(size_t)g] || role[(size_t)u]) return FLUXBIN_ERR_RANGE;          // a member belongs to at most one pair
+        if (!w[g] || !w[u]) return FLUXBIN_ERR_NULL;
+        if (w[g]->h.M != w[u]->h.M) return FLUXBIN_ERR_SHAPE;                     // the two outputs are multiplied row by row
+        role[(size_t)g] = 1; role[(size_t)u] = 2;
+        partner[(size_t)g] = u; partner[(size_t)u] = g;
+    }
     if ((((uintptr_t)d_table) & 15) || (((uintptr_t)d_workspace) & 15)) return FLUXBIN_ERR_ALIGNMENT;
     if (table_bytes < fluxbin_plan_table_bytes(n, B)) return FLUXBIN_ERR_BUFFER_TOO_SMALL;
     int sps1 = 0;
     for (int i = 0; i < n; ++i) {
-        if (!w[i] || !d_x[i] || !d_y[i]) return FLUXBIN_ERR_NULL;
-        if (ldx[i] < w[i]->h.N || ldy[i] < w[i]->h.M) return FLUXBIN_ERR_RANGE;
-        if ((((uintptr_t)d_x[i]) & 15) || (((uintptr_t)d_y[i]) & 15)) return FLUXBIN_ERR_ALIGNMENT;
+        const bool has_y = role[(size_t)i] != 2;              // the up member of a gated pair writes into the gate's y
+        if (!w[i] || !d_x[i] || (has_y && !d_y[i])) return FLUXBIN_ERR_NULL;
+        if (ldx[i] < w[i]->h.N || (has_y && ldy[i] < w[i]->h.M)) return FLUXBIN_ERR_RANGE;
+        if ((((uintptr_t)d_x[i]) & 15) || (has_y && (((uintptr_t)d_y[i]) & 15))) return FLUXBIN_ERR_ALIGNMENT;
         if (w[i]->device != w[0]->device) return FLUXBIN_ERR_UNSUPPORTED;      // all members on one device
         if (w[i]->h.sps[0] != w[0]->h.sps[0]) return FLUXBIN_ERR_UNSUPPORTED;
         if (w[i]->table_format != w[0]->table_format) return FLUXBIN_ERR_UNSUPPORTED;
@@ -758,13 +772,24 @@ extern "C" fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_
         for (int i = 0; i < n; ++i) {
             float *acc = (float *)ws;
             unsigned *tickets = (unsigned *)(ws + acc_bytes(w[i], bt));
-            fill_entry(entries[i], w[i], d_x[i] + (int64_t)b0 * ldx[i], ldx[i], (uint8_t *)d_y[i] + (size_t)b0 * ldy[i] * ysz,
-                       ldy[i], acc, tickets);
+            const int yi = role[(size_t)i] == 2 ? partner[(size_t)i] : i;      // whose output buffer this member writes
+            fill_entry(entries[i], w[i], d_x[i] + (int64_t)b0 * ldx[i], ldx[i], (uint8_t *)d_y[yi] + (size_t)b0 * ldy[yi] * ysz,
+                       ldy[yi], acc, tickets);
             cost_begin[(size_t)i] = cost;
             cost += entry_cost(w[i]->h, sps1, m.build_cost);
             ws += entry_ws_bytes(w[i], bt);
         }
         cost_begin[(size_t)n] = cost;
+        for (int i = 0; i < n; ++i) {
+            if (!role[(size_t)i]) continue;
+            // the two layers of a gated pair count their arrivals on one set of tickets (the gate's) and see each
+            // other's accumulators: whoever completes a row tile of both writes silu(gate) * up
+            const int j = partner[(size_t)i], g = role[(size_t)i] == 1 ? i : j;
+            entries[i].acc2 = entries[j].acc;
+            entries[i].tickets = entries[g].tickets;
+            entries[i].arrivals = w[i]->h.npairs[0] + w[i]->h.npairs[1] + w[j]->h.npairs[0] + w[j]->h.npairs[1];
+            entries[i].flags |= role[(size_t)i] << 8;
+        }
         cudaError_t e = launch_shape(dev, pc.mode, sps0, sps1, cost, w[0]->num_sms, items, couple_cost, true, &pc.shape);
         if (e != cudaSuccess) { delete p; return cuda_fail(e); }
         m.np = pc.shape.np;
@@ -784,6 +809,31 @@ extern "C" fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_
     p->d_counters = (unsigned *)((uint8_t *)d_workspace + fluxbin_plan_workspace_bytes(n, w, B) - 256);
     *out = p;
     return FLUXBIN_OK;
+}
+
+extern "C" fluxbin_status_t fluxbin_plan_create(int32_t n, const fluxbin_weight_t *const *w,
+                                                const uint16_t *const *d_x, const int64_t *ldx,
+                                                void *const *d_y, const int64_t *ldy,
+                                                int32_t B, int32_t y_is_fp32,
+                                                void *d_table, size_t table_bytes,
+                                                void *d_workspace, size_t ws_bytes,
+                                                void *cuda_stream, fluxbin_plan_t **out)
+{
+    return plan_create_impl(n, w, d_x, ldx, d_y, ldy, nullptr, 0, B, y_is_fp32, d_table, table_bytes, d_workspace, ws_bytes,
+                            cuda_stream, out);
+}
+
+extern "C" fluxbin_status_t fluxbin_plan_create_gated(int32_t n, const fluxbin_weight_t *const *w,
+                                                      const uint16_t *const *d_x, const int64_t *ldx,
+                                                      void *const *d_y, const int64_t *ldy,
+                                                      const int32_t *gate_up, int32_t n_gated,
+                                                      int32_t B, int32_t y_is_fp32,
+                                                      void *d_table, size_t table_bytes,
+                                                      void *d_workspace, size_t ws_bytes,
+                                                      void *cuda_stream, fluxbin_plan_t **out)
+{
+    return plan_create_impl(n, w, d_x, ldx, d_y, ldy, gate_up, n_gated, B, y_is_fp32, d_table, table_bytes, d_workspace, ws_bytes,
+                            cuda_stream, out);
 }
 
 extern "C" fluxbin_status_t fluxbin_plan_run(const fluxbin_plan_t *plan, void *cuda_stream)

@@ -72,14 +72,19 @@ struct LinearEntry {
     const uint16_t *x;       // [B][ldx] fp16
     void *y;                 // [B][ldy] fp16 or fp32
     float *acc;              // [BT][Mpad] split-K accumulators, zero on entry and on exit
-    unsigned *tickets;       // [ntiles] arrival counters, zero on entry and on exit
+    unsigned *tickets;       // [ntiles] arrival counters, zero on entry and on exit (shared by the two layers of a gated pair)
     long long ldx, ldy;
-    long long reserved0;
+    float *acc2;             // gated pair: the partner layer's accumulators, else nullptr
     unsigned long long off_coldesc, off_items[2];
-    int M, N, Kb, Mpad, nrb;
+    int M, N, Kb, nrb;       // rows are padded to Mpad = nrb * 32
     int npairs[2];
+    int arrivals;            // (pair, row block) items that complete one row block: npairs[0] + npairs[1], plus the partner's in a gated pair
     int tile_rb, ntiles;
-    int sal_last_w;          // table slots of the last salient pair (32; 16 or 8: stored narrow)
+    int flags;               // bits 0..7: table slots of the last salient pair (32; 16 or 8: stored narrow); bits 8..9: role in a
+                             // gated pair (0 none, 1 gate: y = silu(this) * partner, 2 up: y = silu(partner) * this)
+    __host__ __device__ int mpad() const { return nrb * 32; }
+    __host__ __device__ int sal_last_w() const { return flags & 0xff; }
+    __host__ __device__ int role() const { return (flags >> 8) & 3; }
 };
 
 // Where a share of a launch begins: layer `entry`, work item `item` of it (a work item is one row block of one
@@ -765,7 +770,7 @@ __device__ __forceinline__ void reduce_and_store(const LinearEntry &E, int nb, i
     constexpr int kThreads = Cfg<BT>::kThreads;
     __threadfence();
     __syncthreads();
-    const int npairs = E.npairs[0] + E.npairs[1];
+    const int npairs = E.arrivals;
     for (int t = tid; t < E.ntiles; t += kThreads) {
         int c = tile_cnt[t];
         int last = 0;
@@ -793,7 +798,6 @@ __device__ __forceinline__ void reduce_and_store(const LinearEntry &E, int nb, i
     const int ndone = done_list[kMaxTiles];
     if (ndone > 0) {
         __threadfence();
-#ifdef FB_STAGED_READBACK
         // All rows of all completed tiles, in 4-row groups: every group is requested with one asynchronous 16-byte
         // copy from the accumulators (L2) into the table area, which is free by now -- no registers are held while
         // the copies fly, so one round trip serves every tile the CTA completed (up to 16K rows per batch) however
@@ -801,13 +805,15 @@ __device__ __forceinline__ void reduce_and_store(const LinearEntry &E, int nb, i
         const int gpt = E.tile_rb * 8;                 // 4-row groups per tile
         constexpr int NV = nvec(BT);
         const int total = ndone * gpt * NV;
-        constexpr int kStageGroups = TabCfg<BT>::kTableBytes / 16;
+        // a gated pair stages the partner layer's groups behind its own (half the groups per batch)
+        const int role = E.role();
+        const int kStageGroups = role ? TabCfg<BT>::kTableBytes / 32 : TabCfg<BT>::kTableBytes / 16;
         // group idx of the flat list -> batch vector, first row, element offset in the accumulators (-1: padding rows)
         auto decode = [&](int idx, int &bb, int &row) -> int {
             const int li = idx / (gpt * NV), rem = idx - li * (gpt * NV);
             bb = rem / gpt;
             row = (done_list[li] * gpt + (rem - bb * gpt)) * 4;
-            return row < E.Mpad ? bb * E.Mpad + row : -1;
+            return row < E.mpad() ? bb * E.mpad() + row : -1;
         };
         const bool vec_ok = (E.ldy & 3) == 0;          // rows in groups of four stay 8 / 16-byte aligned in y
         for (int b0 = 0; b0 < total; b0 += kStageGroups) {
@@ -815,9 +821,13 @@ __device__ __forceinline__ void reduce_and_store(const LinearEntry &E, int nb, i
             for (int i = tid; i < n; i += kThreads) {
                 int bb, row;
                 const int eoff = decode(b0 + i, bb, row);
-                if (eoff >= 0)
+                if (eoff >= 0) {
                     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(kTabBase + 16u * (uint32_t)i),
                                  "l"(__cvta_generic_to_global(E.acc + eoff)) : "memory");
+                    if (role)
+                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(kTabBase + 16u * (uint32_t)(kStageGroups + i)),
+                                     "l"(__cvta_generic_to_global(E.acc2 + eoff)) : "memory");
+                }
             }
             asm volatile("cp.async.commit_group;" ::: "memory");
             asm volatile("cp.async.wait_group 0;" ::: "memory");
@@ -829,6 +839,17 @@ __device__ __forceinline__ void reduce_and_store(const LinearEntry &E, int nb, i
                 float4 v;
                 asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(kTabBase + 16u * (uint32_t)i));
                 __stcg((float4 *)(E.acc + eoff), make_float4(0.f, 0.f, 0.f, 0.f));
+                if (role) {
+                    // SiLU-gated product of the two layers of the pair: y = silu(gate) * up, in fp32
+                    float4 p;
+                    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(p.x), "=f"(p.y), "=f"(p.z), "=f"(p.w) : "r"(kTabBase + 16u * (uint32_t)(kStageGroups + i)));
+                    __stcg((float4 *)(E.acc2 + eoff), make_float4(0.f, 0.f, 0.f, 0.f));
+                    const float4 g = role == 1 ? v : p, u = role == 1 ? p : v;
+                    v.x = g.x / (1.f + expf(-g.x)) * u.x;
+                    v.y = g.y / (1.f + expf(-g.y)) * u.y;
+                    v.z = g.z / (1.f + expf(-g.z)) * u.z;
+                    v.w = g.w / (1.f + expf(-g.w)) * u.w;
+                }
                 if (bb >= nb) continue;
                 if (vec_ok && row + 3 < E.M) {
                     if (y_fp32) {
@@ -852,45 +873,6 @@ __device__ __forceinline__ void reduce_and_store(const LinearEntry &E, int nb, i
             }
             __syncthreads();       // the stage is reused by the next batch (and by the next table build)
         }
-#else
-        // all rows of all completed tiles in one flat loop of 4-row groups, four 128-bit loads in
-        // flight per thread (the accumulators live in L2; one round trip serves ~8K rows per CTA)
-        const int gpt = E.tile_rb * 8;                 // 4-row groups per tile
-        constexpr int NV = nvec(BT);
-        const int total = ndone * gpt * NV;
-        constexpr int U = 4;
-        for (int base = tid; base < total; base += U * kThreads) {
-            float4 v[U];
-            float *a[U];
-            int row[U], bb[U];
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                int idx = base + u * kThreads;
-                a[u] = nullptr;
-                if (idx < total) {
-                    int li = idx / (gpt * NV), rem = idx - li * (gpt * NV);
-                    bb[u] = rem / gpt;
-                    row[u] = (done_list[li] * gpt + (rem - bb[u] * gpt)) * 4;
-                    if (row[u] < E.Mpad) a[u] = E.acc + (int64_t)bb[u] * E.Mpad + row[u];
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < U; ++u) if (a[u]) v[u] = __ldcg((const float4 *)a[u]);
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                if (!a[u]) continue;
-                __stcg((float4 *)a[u], make_float4(0.f, 0.f, 0.f, 0.f));
-                if (bb[u] >= nb) continue;
-                const float e[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    if (row[u] + k >= E.M) break;
-                    if (y_fp32) ((float *)E.y)[(int64_t)bb[u] * E.ldy + row[u] + k] = e[k];
-                    else ((__half *)E.y)[(int64_t)bb[u] * E.ldy + row[u] + k] = __float2half_rn(e[k]);
-                }
-            }
-        }
-#endif
         for (int li = tid; li < ndone; li += kThreads) E.tickets[done_list[li]] = 0;
     }
     __syncthreads();       // done_list / tile_cnt are reused by the next entry
@@ -990,7 +972,7 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
             const int pair = wpair * np;
             const int ib_full = region ? ItemBytes<SPS1>::value : ItemBytes<SPS0>::value;
             // the last salient pair may be stored narrow: 8 or 16 steps per item instead of 32
-            const int steps = (SPS1 == 1 && region && pair == E.npairs[1] - 1) ? E.sal_last_w : 32;
+            const int steps = (SPS1 == 1 && region && pair == E.npairs[1] - 1) ? E.sal_last_w() : 32;
             const int ib = steps == 32 ? ib_full : 96 * steps;
             const uint8_t *items = E.packed + E.off_items[region] + (size_t)pair * E.nrb * ib_full;
             const uint8_t *items_b = items + (size_t)E.nrb * ib_full;
@@ -1051,13 +1033,13 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
             FB_TRACE_ADD(4, t_build);
             FB_TRACE_T0(t_rows);
             if (region == 0) {
-                if constexpr (NP == 2) process_rows2<SPS0, BT>(items, items_b, rb_lo, rb_hi, la, E.acc, E.Mpad);
-                else process_rows<SPS0, BT>(items, rb_lo, rb_hi, la, E.acc, E.Mpad, &pre);
+                if constexpr (NP == 2) process_rows2<SPS0, BT>(items, items_b, rb_lo, rb_hi, la, E.acc, E.mpad());
+                else process_rows<SPS0, BT>(items, rb_lo, rb_hi, la, E.acc, E.mpad(), &pre);
             } else if (steps == 32) {
-                process_rows<SPS1, BT>(items, rb_lo, rb_hi, la, E.acc, E.Mpad);
+                process_rows<SPS1, BT>(items, rb_lo, rb_hi, la, E.acc, E.mpad());
             } else if constexpr (SPS1 == 1) {
-                if (steps == 16) process_rows<1, BT, 16>(items, rb_lo, rb_hi, la, E.acc, E.Mpad);
-                else process_rows<1, BT, 8>(items, rb_lo, rb_hi, la, E.acc, E.Mpad);
+                if (steps == 16) process_rows<1, BT, 16>(items, rb_lo, rb_hi, la, E.acc, E.mpad());
+                else process_rows<1, BT, 8>(items, rb_lo, rb_hi, la, E.acc, E.mpad());
             }
 
             FB_TRACE_ADD(5, t_rows);

@@ -18,8 +18,11 @@
 //                     a time with single roundings) followed, in the same pass, by the next round's row form for
 //                     base 1, which needs nothing but the new signs
 //   column form       a_c(k) = numerator / (sum_i a_r^2 + eps): the numerators of a column group are reduced in
-//                     shared memory over the 64 rows of a CTA, then one atomic per column and CTA; the last CTA
-//                     to arrive at a group (a ticket per group) divides, stores and re-zeroes the accumulators
+//                     shared memory over the 64 rows of a CTA, then one atomic per column and CTA; a small kernel
+//                     behind the pass divides, stores and re-zeroes the accumulators.  (Folding that into the pass
+//                     -- a ticket per group, the last CTA divides -- was measured slower: every CTA then ends with
+//                     a fence and an atomic round trip, about 2 us of a 5 us CTA lifetime, 38 instead of ~30 us per
+//                     pass at 4096 x 4096; CTAs that loop over several row blocks were slower still, 46 us.)
 // Scales are stored as fp32 (working copy) and, rounded to nearest even, as fp16 whenever they are written.
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
@@ -38,7 +41,7 @@ constexpr int kMaxK = 4;
 struct Args {
     const float *W;        // [M][ldw]
     long long ldw;
-    int M, N, g, NG, K, num_sms;
+    int M, N, g, NG, K;
     float eps;
     uint32_t *bits;        // [K][M][N/32]
     float *ar;             // [K][M][NG]
@@ -46,9 +49,8 @@ struct Args {
     uint16_t *ar16;        // the same, fp16 bit patterns
     uint16_t *ac16;
     const float *live;     // [N] 1 = real column, 0 = padding column (W must be 0 there); nullptr: all real
-    float *colnum;         // [N]   numerators of the column form, zero between passes
-    float *colden;         // [NG]  sum of a_r^2 per group, zero between passes
-    unsigned *tickets;     // [NG]  CTAs of a group that have added their part, zero between passes
+    float *colnum;         // [N]      numerators of the column form, zero between passes
+    float *colden;         // [2][NG]  sum of a_r^2 per group, double buffered (see col_kernel)
 };
 
 __device__ __forceinline__ float warp_sum(float v)
@@ -141,23 +143,23 @@ enum PassMode {
     kInit = 4        // greedy initialisation only (T == 0)
 };
 
-// A CTA owns one column group and a strided set of its 64-row blocks (gridDim.x = groups x CTAs per group), so
-// the column scales are loaded once, the column numerators stay in registers across the row blocks and the
-// reduction over the CTA, the atomics and the ticket happen once per CTA.
-template <int C, int K, int MODE> __global__ void __launch_bounds__(kWarpsPerCta * 32, (C * K <= 8) ? 3 : 1) pass_kernel(Args a, int k_arg)
+template <int C, int K, int MODE> __global__ void __launch_bounds__(kWarpsPerCta * 32) pass_kernel(Args a, int k_arg, int parity)
 {
     constexpr bool kInitial = MODE == kInitRow || MODE == kInit;
     constexpr bool kSearch = MODE == kSignRow || MODE == kSign;
     constexpr bool kRowForm = MODE == kRow || MODE == kSignRow || MODE == kInitRow;
     __shared__ float part[kWarpsPerCta][C * 32];
     __shared__ float den_part[kWarpsPerCta];
-    __shared__ int is_last;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int G = blockIdx.x % a.NG, part_id = blockIdx.x / a.NG, cpg = gridDim.x / a.NG;
+    const int G = blockIdx.x, row0 = blockIdx.y * kRowsPerCta + warp * kRowsPerWarp;
     const int nw = a.N / 32;
-    const int nblocks = (a.M + kRowsPerCta - 1) / kRowsPerCta;
+    const int nrows = max(0, min(kRowsPerWarp, a.M - row0));
     const int k = MODE == kRow ? k_arg : 0;                // base of the row form
 
+    WarpRows<C, K> in;
+    in.load_w(a, G, row0, nrows, lane);
+    if constexpr (MODE == kRow) in.load_signs(a, G, row0, nrows, lane);
+    if constexpr (!kInitial) in.load_row_scales(a, G, row0, nrows, lane);
     float ack[K][C];                     // column scales of every base for this lane's columns
     float lv[C];                         // live mask (initial column scales)
     if constexpr (kInitial) {
@@ -190,22 +192,6 @@ template <int C, int K, int MODE> __global__ void __launch_bounds__(kWarpsPerCta
 #pragma unroll
     for (int c = 0; c < C; ++c) colsum[c] = 0.f;
     float ar2 = 0.f;
-
-    for (int blk = part_id; blk < nblocks; blk += cpg) {
-    const int row0 = blk * kRowsPerCta + warp * kRowsPerWarp;
-    const int nrows = max(0, min(kRowsPerWarp, a.M - row0));
-    if (blk + cpg < nblocks) {
-        // the W lines of this warp's rows in the CTA's next block start moving into L2
-        const int nrow0 = row0 + cpg * kRowsPerCta;
-        for (int f = lane; f < kRowsPerWarp * C; f += 32) {
-            const int r = f / C, line = f % C;
-            if (nrow0 + r < a.M) asm volatile("prefetch.global.L2 [%0];" ::"l"(a.W + (long long)(nrow0 + r) * a.ldw + G * a.g + line * 32));
-        }
-    }
-    WarpRows<C, K> in;
-    in.load_w(a, G, row0, nrows, lane);
-    if constexpr (MODE == kRow) in.load_signs(a, G, row0, nrows, lane);
-    if constexpr (!kInitial) in.load_row_scales(a, G, row0, nrows, lane);
 
 #pragma unroll
     for (int r = 0; r < kRowsPerWarp; ++r) {
@@ -304,11 +290,9 @@ template <int C, int K, int MODE> __global__ void __launch_bounds__(kWarpsPerCta
         }
     }
 
-    }       // row blocks of this CTA
-
     if constexpr (MODE == kInit) {
         // no update follows: the column scales are the initial ones
-        if (part_id == 0 && warp == 0) {
+        if (blockIdx.y == 0 && warp == 0) {
 #pragma unroll
             for (int q = 0; q < K; ++q)
 #pragma unroll
@@ -332,56 +316,59 @@ template <int C, int K, int MODE> __global__ void __launch_bounds__(kWarpsPerCta
         if (threadIdx.x == 0) {
             float s = 0.f;
             for (int w = 0; w < kWarpsPerCta; ++w) s += den_part[w];
-            atomicAdd(a.colden + G, s);
+            atomicAdd(a.colden + (size_t)(parity & 1) * a.NG + G, s);
         }
-        // Column form of Eq. 5 by the last CTA of the group to get here: a_c(k)_j = numerator_j / (sum_i a_r_i^2 + eps);
-        // the accumulators and the ticket go back to zero for the next pass.
-        __threadfence();
-        __syncthreads();
-        if (threadIdx.x == 0) is_last = (atomicAdd(a.tickets + G, 1u) == (unsigned)cpg - 1u);
-        __syncthreads();
-        if (is_last) {
-            __threadfence();
-            const float den = __ldcg(a.colden + G) + a.eps;
-            for (int j = threadIdx.x; j < C * 32; j += kWarpsPerCta * 32) {
-                const int col = G * a.g + j;
-                const float v = __ldcg(a.colnum + col) / den;
-                a.ac[(size_t)k * a.N + col] = v;
-                a.ac16[(size_t)k * a.N + col] = half_bits(v);
-                a.colnum[col] = 0.f;
-                if constexpr (MODE == kInitRow) {
-                    const float l = a.live ? a.live[col] : 1.f;
-                    for (int q = 1; q < K; ++q) {
-                        a.ac[(size_t)q * a.N + col] = l;
-                        a.ac16[(size_t)q * a.N + col] = half_bits(l);
-                    }
-                }
-            }
-            __syncthreads();
-            if (threadIdx.x == 0) { a.colden[G] = 0.f; a.tickets[G] = 0u; }
+    }
+}
+
+// Column form of Eq. 5 behind a pass: a_c(k)_j = numerator_j / (sum_i a_r_i^2 + eps), fp32 and fp16; the accumulators go
+// back to zero.  The group denominators are double buffered: this kernel reads buffer `parity` and clears the other
+// one, which the next pass accumulates into -- no thread reads what another clears.  init_rest: the first pass
+// of a call also gives the bases it did not update their initial column scales (the live mask).
+__global__ void col_kernel(Args a, int k, int parity, int init_rest)
+{
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= a.N) return;
+    const float v = a.colnum[j] / (a.colden[(size_t)(parity & 1) * a.NG + j / a.g] + a.eps);
+    a.ac[(size_t)k * a.N + j] = v;
+    a.ac16[(size_t)k * a.N + j] = half_bits(v);
+    a.colnum[j] = 0.f;
+    if (j < a.NG) a.colden[(size_t)((parity + 1) & 1) * a.NG + j] = 0.f;
+    if (init_rest) {
+        const float l = a.live ? a.live[j] : 1.f;
+        for (int q = 0; q < a.K; ++q) {
+            if (q == k) continue;
+            a.ac[(size_t)q * a.N + j] = l;
+            a.ac16[(size_t)q * a.N + j] = half_bits(l);
         }
     }
 }
 
 template <int C, int K> cudaError_t run(const Args &a, int T, cudaStream_t s)
 {
-    // CTAs per column group: enough to fill every SM with the CTAs it can hold (three of the small instantiations,
-    // one of those with many bases or wide groups: see the launch bounds), at most one per 64-row block
-    const int nblocks = (a.M + kRowsPerCta - 1) / kRowsPerCta;
-    constexpr int kCtasPerSm = (C * K <= 8) ? 3 : 1;
-    int cpg = (kCtasPerSm * a.num_sms + a.NG - 1) / a.NG;
-    if (cpg > nblocks) cpg = nblocks;
-    if (cpg < 1) cpg = 1;
-    const dim3 grid((unsigned)(a.NG * cpg)), block(kWarpsPerCta * 32);
+    const dim3 grid(a.NG, (a.M + kRowsPerCta - 1) / kRowsPerCta), block(kWarpsPerCta * 32);
+    const unsigned colgrid = (unsigned)((a.N + 255) / 256);
     if (T == 0) {
-        pass_kernel<C, K, kInit><<<grid, block, 0, s>>>(a, 0);
+        pass_kernel<C, K, kInit><<<grid, block, 0, s>>>(a, 0, 0);
         return cudaGetLastError();
     }
-    pass_kernel<C, K, kInitRow><<<grid, block, 0, s>>>(a, 0);
+    int parity = 0;
+    pass_kernel<C, K, kInitRow><<<grid, block, 0, s>>>(a, 0, parity);
+    col_kernel<<<colgrid, 256, 0, s>>>(a, 0, parity, 1);
+    parity ^= 1;
     for (int it = 0; it < T; ++it) {
-        for (int k = 1; k < a.K; ++k) pass_kernel<C, K, kRow><<<grid, block, 0, s>>>(a, k);
-        if (it + 1 < T) pass_kernel<C, K, kSignRow><<<grid, block, 0, s>>>(a, 0);
-        else pass_kernel<C, K, kSign><<<grid, block, 0, s>>>(a, 0);
+        for (int k = 1; k < a.K; ++k) {
+            pass_kernel<C, K, kRow><<<grid, block, 0, s>>>(a, k, parity);
+            col_kernel<<<colgrid, 256, 0, s>>>(a, k, parity, 0);
+            parity ^= 1;
+        }
+        if (it + 1 < T) {
+            pass_kernel<C, K, kSignRow><<<grid, block, 0, s>>>(a, 0, parity);
+            col_kernel<<<colgrid, 256, 0, s>>>(a, 0, parity, 0);
+            parity ^= 1;
+        } else {
+            pass_kernel<C, K, kSign><<<grid, block, 0, s>>>(a, 0, parity);
+        }
     }
     return cudaGetLastError();
 }
@@ -423,19 +410,12 @@ extern "C" fluxbin_status_t fluxbin_rc_decomp(const float *d_W, int64_t ldw, con
     a.W = d_W; a.live = d_col_live; a.ldw = ldw; a.M = M; a.N = N; a.g = g; a.NG = N / g; a.K = K; a.eps = eps;
     a.bits = d_bits;
     a.ar16 = d_row_scale; a.ac16 = d_col_scale;
-    {
-        int dev = 0, sms = 0;
-        FB_CUDA(cudaGetDevice(&dev));
-        FB_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-        a.num_sms = sms > 0 ? sms : 1;
-    }
     uint8_t *ws = (uint8_t *)d_workspace;
     // the fp32 working copies of the scales live in the caller's fp32 outputs when those are given
     a.ar = d_row_scale_f32 ? d_row_scale_f32 : (float *)ws;     ws += align256((size_t)K * M * a.NG * 4);
     a.ac = d_col_scale_f32 ? d_col_scale_f32 : (float *)ws;     ws += align256((size_t)K * N * 4);
     a.colnum = (float *)ws;
     a.colden = a.colnum + N;
-    a.tickets = (unsigned *)(a.colden + a.NG);
     FB_CUDA(cudaMemsetAsync(a.colnum, 0, (size_t)N * 4 + 2 * (size_t)a.NG * 4, s));
     cudaError_t e = cudaErrorInvalidValue;
 #define RCD_K(CC) (K == 1 ? rcd::run<CC, 1>(a, T, s) : K == 2 ? rcd::run<CC, 2>(a, T, s) : K == 3 ? rcd::run<CC, 3>(a, T, s) : rcd::run<CC, 4>(a, T, s))

@@ -38,7 +38,7 @@ EXPORTS = ["fluxbin_packed_size", "fluxbin_validate", "fluxbin_pack_host", "flux
            "fluxbin_workspace_size", "fluxbin_workspace_init", "fluxbin_linear", "fluxbin_debug_tables",
            "fluxbin_num_table_sets", "fluxbin_num_launches", "fluxbin_free", "fluxbin_status_string",
            "fluxbin_last_cuda_error", "fluxbin_plan_table_bytes", "fluxbin_plan_workspace_bytes",
-           "fluxbin_plan_create", "fluxbin_plan_run", "fluxbin_plan_num_launches", "fluxbin_plan_pairs_per_row_block",
+           "fluxbin_plan_create", "fluxbin_plan_create_gated", "fluxbin_plan_run", "fluxbin_plan_num_launches", "fluxbin_plan_pairs_per_row_block",
            "fluxbin_plan_free",
            "fluxbin_linear_noalloc", "fluxbin_noalloc_capacity", "fluxbin_set_table_format", "fluxbin_get_table_format",
            "fluxbin_rc_decomp", "fluxbin_rc_decomp_workspace_size", "fluxbin_rc_decomp_passes",
@@ -88,6 +88,10 @@ def _lib():
         lib.fluxbin_plan_create.argtypes = [i32, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(i64),
                                             ctypes.POINTER(vp), ctypes.POINTER(i64), i32, i32, vp, sz, vp, sz, vp,
                                             ctypes.POINTER(vp)]
+        lib.fluxbin_plan_create_gated.restype = ctypes.c_int
+        lib.fluxbin_plan_create_gated.argtypes = [i32, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(i64),
+                                                  ctypes.POINTER(vp), ctypes.POINTER(i64), ctypes.POINTER(i32), i32, i32, i32, vp, sz,
+                                                  vp, sz, vp, ctypes.POINTER(vp)]
         lib.fluxbin_plan_run.restype, lib.fluxbin_plan_run.argtypes = ctypes.c_int, [vp, vp]
         lib.fluxbin_plan_num_launches.restype, lib.fluxbin_plan_num_launches.argtypes = i32, [vp]
         lib.fluxbin_plan_pairs_per_row_block.restype, lib.fluxbin_plan_pairs_per_row_block.argtypes = i32, [vp]
@@ -405,7 +409,24 @@ def plan_create_status(weights, d_x, ldx, d_y, ldy, B, y_is_fp32, d_table, table
     return int(st), h.value
 
 
-def plan_create(weights, d_x, ldx, d_y, ldy, B, y_is_fp32, d_table, table_bytes, d_ws, ws_bytes, stream=0, keep=None):
-    st, h = plan_create_status(weights, d_x, ldx, d_y, ldy, B, y_is_fp32, d_table, table_bytes, d_ws, ws_bytes, stream)
-    _check(st, "fluxbin_plan_create")
+def plan_create_gated_status(weights, d_x, ldx, d_y, ldy, gate_up, B, y_is_fp32, d_table, table_bytes, d_ws, ws_bytes, stream=0):
+    """fluxbin_plan_create_gated returning (status, handle); gate_up = list of (gate member, up member)."""
+    n = len(weights)
+    h = ctypes.c_void_p()
+    flat = [int(v) for pair in gate_up for v in pair]
+    st = _lib().fluxbin_plan_create_gated(n, _arr(ctypes.c_void_p, [w.handle for w in weights]),
+                                          _arr(ctypes.c_void_p, list(d_x)), _arr(ctypes.c_int64, list(ldx)),
+                                          _arr(ctypes.c_void_p, list(d_y)), _arr(ctypes.c_int64, list(ldy)),
+                                          _arr(ctypes.c_int32, flat) if flat else None, len(gate_up),
+                                          B, 1 if y_is_fp32 else 0, d_table, table_bytes, d_ws, ws_bytes, stream, ctypes.byref(h))
+    return int(st), h.value
+
+
+def plan_create(weights, d_x, ldx, d_y, ldy, B, y_is_fp32, d_table, table_bytes, d_ws, ws_bytes, stream=0, keep=None, gate_up=None):
+    if gate_up:
+        st, h = plan_create_gated_status(weights, d_x, ldx, d_y, ldy, gate_up, B, y_is_fp32, d_table, table_bytes, d_ws, ws_bytes, stream)
+        _check(st, "fluxbin_plan_create_gated")
+    else:
+        st, h = plan_create_status(weights, d_x, ldx, d_y, ldy, B, y_is_fp32, d_table, table_bytes, d_ws, ws_bytes, stream)
+        _check(st, "fluxbin_plan_create")
     return Plan(h, (list(weights), keep))

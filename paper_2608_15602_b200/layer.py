@@ -76,25 +76,29 @@ class FluxBinPlan:
     """Several independent layers run in one persistent launch (fluxbin_plan_*).
 
     `members` is a list of (FluxBinLinear, x, y) with x fp16 [B][>=N] and y [B][M] CUDA tensors that
-    stay alive and in place for the life of the plan (the pointers are captured at creation)."""
+    stay alive and in place for the life of the plan (the pointers are captured at creation).
+    `gate_up`: list of (gate member, up member) index pairs whose outputs are combined as silu(gate) * up into the
+    gate member's y (fluxbin_plan_create_gated); the y of an up member may be None."""
 
-    def __init__(self, members, device="cuda"):
+    def __init__(self, members, device="cuda", gate_up=None):
         self.members = list(members)
         lins = [m[0] for m in self.members]
         xs = [m[1] for m in self.members]
         ys = [m[2] for m in self.members]
         B = xs[0].shape[0]
         assert all(x.shape[0] == B and x.dtype == torch.float16 and x.stride(1) == 1 for x in xs)
-        fp32 = ys[0].dtype == torch.float32
-        assert all((y.dtype == torch.float32) == fp32 and y.shape[0] == B for y in ys)
+        first_y = next(y for y in ys if y is not None)
+        fp32 = first_y.dtype == torch.float32
+        assert all(y is None or ((y.dtype == torch.float32) == fp32 and y.shape[0] == B) for y in ys)
         weights = [l.weight for l in lins]
         tbytes = fluxbin.plan_table_bytes(len(lins), B)
         self.table = torch.empty(max(tbytes, 16), dtype=torch.uint8, device=device)
         self.ws = Workspace(fluxbin.plan_workspace_bytes(weights, B), device)
         self.plan = fluxbin.plan_create(weights, [x.data_ptr() for x in xs], [x.stride(0) for x in xs],
-                                        [y.data_ptr() for y in ys], [y.stride(0) for y in ys], B, fp32,
+                                        [None if y is None else y.data_ptr() for y in ys],
+                                        [0 if y is None else y.stride(0) for y in ys], B, fp32,
                                         self.table.data_ptr(), tbytes, self.ws.tensor.data_ptr(), self.ws.nbytes,
-                                        _stream_ptr(), keep=(self.members, self.table, self.ws))
+                                        _stream_ptr(), keep=(self.members, self.table, self.ws), gate_up=gate_up)
         self.B = B
 
     def run(self, stream=None):

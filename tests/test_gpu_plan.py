@@ -185,3 +185,70 @@ def test_large_plans_cut_a_rest_with_dead_vectors_once_more(fb, B, fp16, launche
             check(got, want, f"B={B} rep {rep}")
         # the four members hold the same layer: same weights, different activations -> rows must differ between members
         assert not torch.equal(members[0][2], members[1][2])
+
+
+@pytest.mark.parametrize("B,fp32", [(1, True), (1, False), (3, True), (8, False)])
+def test_gated_pairs_write_silu_gate_times_up(fb, B, fp32):
+    """fluxbin_plan_create_gated: y = silu(W_gate x) * (W_up x) written once by whoever completes a row tile of both
+    layers, against the oracle's two results combined in fp64; an unpaired member of the same plan is unaffected and
+    the workspace (both layers' accumulators, the shared tickets) comes back zeroed."""
+    specs = [(11008, 4096, 2, 1, 128, 205), (11008, 4096, 2, 1, 128, 205),      # gate, up of a 7B-shaped block
+             (300, 1024, 2, 1, 128, 51),                                         # an ordinary member in between
+             (777, 512, 2, 0, 128, 0), (777, 512, 3, 2, 128, 40)]                # a ragged pair with different base counts
+    Ls = [layer_of(500 + i, *sp) for i, sp in enumerate(specs)]
+    xs = [synth.make_activations(31, 0, B, 4096), None, synth.make_activations(31, 2, B, 1024),
+          synth.make_activations(31, 3, B, 512), synth.make_activations(31, 4, B, 512)]
+    xs[1] = xs[0]                                                                # gate and up read the same input
+    lins = [fb.FluxBinLinear(L) for L in Ls]
+    xt = [torch.from_numpy(x.view(np.float16)).cuda() for x in xs]
+    dt = torch.float32 if fp32 else torch.float16
+    ys = [torch.full((B, L.M), float("nan"), dtype=dt, device="cuda") for L in Ls]
+    gate_up = [(0, 1), (4, 3)]                                                   # second pair: member 4 gates member 3
+    members = [(lins[i], xt[i], None if i in (1, 3) else ys[i]) for i in range(5)]
+    plan = fb.FluxBinPlan(members, gate_up=gate_up)
+    want = [oracle.linear_direct(L, x) for L, x in zip(Ls, xs)]
+    silu = lambda t: t / (1.0 + np.exp(-t))
+    for rep in range(2):
+        for i in (0, 2, 4):
+            ys[i].fill_(float("nan"))
+        plan.run()
+        torch.cuda.synchronize()
+        assert int(plan.ws.tensor.count_nonzero()) == 0, "plan workspace must be left zeroed"
+        got = [y.float().cpu().numpy() for y in ys]
+        tol = dict() if fp32 else dict()
+        for g, u in gate_up:
+            expect = silu(want[g]) * want[u]
+            if fp32:
+                check(got[g], expect, f"gated pair ({g},{u}) B={B} run {rep}")
+            else:
+                y = got[g].astype(np.float64)
+                for b in range(B):
+                    rms = np.sqrt(np.mean(expect[b] ** 2))
+                    assert np.linalg.norm(y[b] - expect[b]) / np.linalg.norm(expect[b]) <= 1e-3
+                    assert (np.abs(y[b] - expect[b]) / np.maximum(np.abs(expect[b]), 1e-2 * rms)).max() <= 5e-3 + 2.0 ** -11
+        if fp32:
+            check(got[2], want[2], "unpaired member")
+        assert np.isnan(ys[1].float().cpu().numpy()).all() and np.isnan(ys[3].float().cpu().numpy()).all(), "up members have no output"
+
+
+def test_gated_plan_argument_errors(fb):
+    from paper_2608_15602_b200 import fluxbin
+    a = fb.FluxBinLinear(layer_of(1, 64, 256, 2, 0, 128, 0))
+    b = fb.FluxBinLinear(layer_of(2, 64, 256, 2, 0, 128, 0))
+    c = fb.FluxBinLinear(layer_of(3, 96, 256, 2, 0, 128, 0))           # another row count
+    x = torch.zeros((1, 256), dtype=torch.float16, device="cuda")
+    y = torch.zeros((1, 96), dtype=torch.float16, device="cuda")
+    tb = fluxbin.plan_table_bytes(3, 1)
+    table = torch.zeros(tb, dtype=torch.uint8, device="cuda")
+    ws = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+    ws_args = (1, False, table.data_ptr(), tb, ws.data_ptr(), 1 << 16)
+    ptrs = ([x.data_ptr()] * 3, [256] * 3, [y.data_ptr(), None, y.data_ptr()], [96, 0, 96])
+    W = [a.weight, b.weight, c.weight]
+    assert fluxbin.plan_create_gated_status(W, *ptrs, [(0, 2)], *ws_args)[0] == 2        # 64 rows against 96
+    assert fluxbin.plan_create_gated_status(W, *ptrs, [(0, 0)], *ws_args)[0] == 3        # a member with itself
+    assert fluxbin.plan_create_gated_status(W, *ptrs, [(0, 1), (1, 2)], *ws_args)[0] == 3  # member 1 twice
+    assert fluxbin.plan_create_gated_status(W, *ptrs, [(0, 5)], *ws_args)[0] == 3        # no such member
+    assert fluxbin.plan_create_gated_status(W, *ptrs, [(1, 0)], *ws_args)[0] == 1        # the gate (member 1) has no output buffer
+    st, h = fluxbin.plan_create_gated_status(W, *ptrs, [(0, 1)], *ws_args)
+    assert st == 0
+    fluxbin.library().fluxbin_plan_free(h)
