@@ -135,6 +135,13 @@ template <int C> __device__ __forceinline__ bool stores_word(int lane) { return 
 
 __device__ __forceinline__ uint16_t half_bits(float v) { return __half_as_ushort(__float2half_rn(v)); }
 
+// v with its sign flipped when bit c of `bits` is set: a shift and one three-input logic operation, where a select
+// between v and -v costs a bit test, a compare and the select (the passes are bound by issue slots).
+__device__ __forceinline__ float flip_if_bit(float v, uint32_t bits, int c)       // c: compile-time after unrolling
+{
+    return __uint_as_float(__float_as_uint(v) ^ ((bits << (31 - c)) & 0x80000000u));
+}
+
 enum PassMode {
     kRow = 0,        // row form of Eq. 5 for base k (signs read from memory) + column numerators
     kSignRow = 1,    // Eq. 6 for all bases, then the row form for base 0 with the new signs + column numerators
@@ -156,8 +163,15 @@ template <int C, int K, int MODE> __global__ void __launch_bounds__(kWarpsPerCta
     const int nrows = max(0, min(kRowsPerWarp, a.M - row0));
     const int k = MODE == kRow ? k_arg : 0;                // base of the row form
 
+    // Programmatic dependent launch: the next kernel of the call may become resident while this one drains, and this
+    // one requests its W values -- which no kernel of the call writes -- before it waits for its predecessor;
+    // everything a predecessor wrote (signs, scales, zeroed accumulators) is read, and everything is written, after
+    // the wait.  The first pass of a call waits first: whatever produced W may still be running.
+    asm volatile("griddepcontrol.launch_dependents;");
     WarpRows<C, K> in;
+    if constexpr (kInitial) asm volatile("griddepcontrol.wait;" ::: "memory");
     in.load_w(a, G, row0, nrows, lane);
+    if constexpr (!kInitial) asm volatile("griddepcontrol.wait;" ::: "memory");
     if constexpr (MODE == kRow) in.load_signs(a, G, row0, nrows, lane);
     if constexpr (!kInitial) in.load_row_scales(a, G, row0, nrows, lane);
     float ack[K][C];                     // column scales of every base for this lane's columns
@@ -192,6 +206,7 @@ template <int C, int K, int MODE> __global__ void __launch_bounds__(kWarpsPerCta
 #pragma unroll
     for (int c = 0; c < C; ++c) colsum[c] = 0.f;
     float ar2 = 0.f;
+    float arn_mine = 0.f;                // lane r: the new row scale of row r
 
 #pragma unroll
     for (int r = 0; r < kRowsPerWarp; ++r) {
@@ -261,8 +276,8 @@ template <int C, int K, int MODE> __global__ void __launch_bounds__(kWarpsPerCta
             }
         }
         if constexpr (kRowForm) {
-            // signs enter as a choice between +v and -v (one select, then a fused multiply-add): the passes are
-            // bound by issue slots as much as by memory, so the per-element instruction count matters
+            // signs enter as a flip of the sign bit of one factor ((-a) * t and a * (-t) round alike, so which
+            // factor carries the sign does not change a result)
             float t[C];
 #pragma unroll
             for (int c = 0; c < C; ++c) t[c] = in.w[r][c];
@@ -271,22 +286,29 @@ template <int C, int K, int MODE> __global__ void __launch_bounds__(kWarpsPerCta
                 if (q == k) continue;
 #pragma unroll
                 for (int c = 0; c < C; ++c)
-                    t[c] = fmaf(((sg[q] >> c) & 1u) ? -arq[q] : arq[q], ack[q][c], t[c]);     // what the other bases leave
+                    t[c] = fmaf(flip_if_bit(arq[q], sg[q], c), ack[q][c], t[c]);      // what the other bases leave
             }
-            uint32_t sk = 0u;
+            uint32_t nsk = 0u;
 #pragma unroll
-            for (int q = 0; q < K; ++q) if (q == k) sk = sg[q];
+            for (int q = 0; q < K; ++q) if (q == k) nsk = ~sg[q];
             float num = 0.f;
 #pragma unroll
-            for (int c = 0; c < C; ++c) num = fmaf(((sk >> c) & 1u) ? akc[c] : -akc[c], t[c], num);
-            const float arn = r < nrows ? warp_sum(num) * inv_den : 0.f;   // (r < nrows is warp-uniform)
-            if (lane == 0 && r < nrows) {
-                a.ar[((size_t)k * a.M + i) * a.NG + G] = arn;
-                a.ar16[((size_t)k * a.M + i) * a.NG + G] = half_bits(arn);
+            for (int c = 0; c < C; ++c) {
+                t[c] = flip_if_bit(t[c], nsk, c);                                      // B_k * target
+                num = fmaf(akc[c], t[c], num);
             }
+            const float arn = warp_sum(num) * inv_den;                                 // rows past M: W = 0 there, so 0
+            if (lane == r) arn_mine = arn;
             ar2 = fmaf(arn, arn, ar2);
 #pragma unroll
-            for (int c = 0; c < C; ++c) colsum[c] = fmaf(((sk >> c) & 1u) ? arn : -arn, t[c], colsum[c]);
+            for (int c = 0; c < C; ++c) colsum[c] = fmaf(arn, t[c], colsum[c]);
+        }
+    }
+    if constexpr (kRowForm) {
+        // lane r holds the new row scale of row r: one store per lane instead of eight by lane 0
+        if (lane < nrows) {
+            a.ar[((size_t)k * a.M + row0 + lane) * a.NG + G] = arn_mine;
+            a.ar16[((size_t)k * a.M + row0 + lane) * a.NG + G] = half_bits(arn_mine);
         }
     }
 
@@ -327,6 +349,8 @@ template <int C, int K, int MODE> __global__ void __launch_bounds__(kWarpsPerCta
 // of a call also gives the bases it did not update their initial column scales (the live mask).
 __global__ void col_kernel(Args a, int k, int parity, int init_rest)
 {
+    asm volatile("griddepcontrol.launch_dependents;");
+    asm volatile("griddepcontrol.wait;" ::: "memory");          // the pass before this has added all its numerators
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= a.N) return;
     const float v = a.colnum[j] / (a.colden[(size_t)(parity & 1) * a.NG + j / a.g] + a.eps);
@@ -344,33 +368,53 @@ __global__ void col_kernel(Args a, int k, int parity, int init_rest)
     }
 }
 
+// launch with the programmatic-dependent-launch attribute (see pass_kernel)
+template <typename... KArgs, typename... Args2>
+static cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t s, Args2... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 template <int C, int K> cudaError_t run(const Args &a, int T, cudaStream_t s)
 {
     const dim3 grid(a.NG, (a.M + kRowsPerCta - 1) / kRowsPerCta), block(kWarpsPerCta * 32);
-    const unsigned colgrid = (unsigned)((a.N + 255) / 256);
+    const dim3 colgrid((unsigned)((a.N + 255) / 256)), colblock(256);
+    cudaError_t e;
+#define RCD_LAUNCH(...) do { e = launch_pdl(__VA_ARGS__); if (e != cudaSuccess) return e; } while (0)
     if (T == 0) {
-        pass_kernel<C, K, kInit><<<grid, block, 0, s>>>(a, 0, 0);
-        return cudaGetLastError();
+        RCD_LAUNCH(pass_kernel<C, K, kInit>, grid, block, s, a, 0, 0);
+        return cudaSuccess;
     }
     int parity = 0;
-    pass_kernel<C, K, kInitRow><<<grid, block, 0, s>>>(a, 0, parity);
-    col_kernel<<<colgrid, 256, 0, s>>>(a, 0, parity, 1);
+    RCD_LAUNCH(pass_kernel<C, K, kInitRow>, grid, block, s, a, 0, parity);
+    RCD_LAUNCH(col_kernel, colgrid, colblock, s, a, 0, parity, 1);
     parity ^= 1;
     for (int it = 0; it < T; ++it) {
         for (int k = 1; k < a.K; ++k) {
-            pass_kernel<C, K, kRow><<<grid, block, 0, s>>>(a, k, parity);
-            col_kernel<<<colgrid, 256, 0, s>>>(a, k, parity, 0);
+            RCD_LAUNCH(pass_kernel<C, K, kRow>, grid, block, s, a, k, parity);
+            RCD_LAUNCH(col_kernel, colgrid, colblock, s, a, k, parity, 0);
             parity ^= 1;
         }
         if (it + 1 < T) {
-            pass_kernel<C, K, kSignRow><<<grid, block, 0, s>>>(a, 0, parity);
-            col_kernel<<<colgrid, 256, 0, s>>>(a, 0, parity, 0);
+            RCD_LAUNCH(pass_kernel<C, K, kSignRow>, grid, block, s, a, 0, parity);
+            RCD_LAUNCH(col_kernel, colgrid, colblock, s, a, 0, parity, 0);
             parity ^= 1;
         } else {
-            pass_kernel<C, K, kSign><<<grid, block, 0, s>>>(a, 0, parity);
+            RCD_LAUNCH(pass_kernel<C, K, kSign>, grid, block, s, a, 0, parity);
         }
     }
-    return cudaGetLastError();
+#undef RCD_LAUNCH
+    return cudaSuccess;
 }
 
 } // namespace rcd
