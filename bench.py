@@ -24,6 +24,7 @@ Beside the headline the line carries (rank 0, one GPU; --sections picks them):
   configs     the smaller workloads (one layer, hybrid layer, 7B set, 13B set) in linear / group / stack mode
               as rotations of copies larger than L2, and the batched cases of the workloads
   variants    the paper's deployed formats at the shapes of its per-operator latency table, one chained call each
+  mu_sweep    sub-vector size 4 against 8 on the 7B-shaped set at batch 1, 4, 8 (the paper's sub-vector-size table)
   rc_decomp   the decomposition step (Algorithm 3) on dense matrices
   cpu_baseline, context_dense_fp16_gemv
 
@@ -51,7 +52,7 @@ from paper_2608_15602_b200 import synth  # noqa: E402
 METRIC = "decode_linear_stack_effective_hbm_gbps_batch1"
 UNIT = "GB/s"
 L2_BYTES = 126e6
-ALL_SECTIONS = ["group_mode", "sustained", "configs", "variants", "rc_decomp", "context", "cpu_baseline"]
+ALL_SECTIONS = ["group_mode", "sustained", "configs", "variants", "mu_sweep", "rc_decomp", "context", "cpu_baseline"]
 
 
 def algorithmic_bytes(M, N, Kb, Ks, g, n_sal, B):
@@ -145,15 +146,15 @@ class Stack:
     members: list of (FluxBinLinear, canonical dims, x fp16 bits [B][N]); `names` the linears of one layer / set in
     order, `nl` how many such layers the members hold (member index = layer * len(names) + linear)."""
 
-    def __init__(self, members, names, nl, B, fp16_tables=False):
+    def __init__(self, members, names, nl, B, fp16_tables=False, mu4=False):
         import torch
         from paper_2608_15602_b200 import fluxbin, layer as fb_layer
-        self.names, self.nl, self.B, self.fp16 = names, nl, B, bool(fp16_tables and B > 1)
+        self.names, self.nl, self.B, self.fp16, self.mu4 = names, nl, B, bool(fp16_tables and B > 1), bool(mu4)
         self.linears = [m[0] for m in members]
         self.dims = [m[1] for m in members]
         self._fmt_before = [l.weight.table_format() for l in self.linears]
         for l in self.linears:                      # workspaces and plans are sized after the format is set
-            l.weight.set_table_format(fluxbin.TABLES_FP16 if self.fp16 else fluxbin.TABLES_FP32)
+            l.weight.set_table_format(fluxbin.TABLES_FP32_MU4 if self.mu4 else fluxbin.TABLES_FP16 if self.fp16 else fluxbin.TABLES_FP32)
         self.alg_bytes = [algorithmic_bytes(*d, B) for d in self.dims]
         self.eff_flops = sum(2.0 * d[0] * (d[1] + d[5]) * B for d in self.dims)
         self.lookups = sum(d[2] * d[0] * (d[1] // 8) + d[3] * d[0] * ((d[5] + 7) // 8) for d in self.dims)   # one per weight byte
@@ -286,7 +287,7 @@ def build_config_stack(config, nl, B, g=128, fp16_tables=False):
     return Stack(generate_members(jobs, make, fp16_tables), [n for n, _, _ in lins], nl, B, fp16_tables)
 
 
-def build_rotation(make_layers, names, B, fp16_tables=False):
+def build_rotation(make_layers, names, B, fp16_tables=False, mu4=False):
     """A rotation of copies of one set of layers, enough of them that a step streams more than four times L2.
     The set is generated and packed once; the copies are device-side clones at their own addresses (what the
     memory system sees is the same as with independently seeded copies: every copy is read once per step)."""
@@ -300,7 +301,7 @@ def build_rotation(make_layers, names, B, fp16_tables=False):
     members = list(base)
     for _ in range(copies - 1):
         members += [(m[0].clone(), m[1], m[2]) for m in base]
-    return Stack(members, names, copies, B, fp16_tables)
+    return Stack(members, names, copies, B, fp16_tables, mu4)
 
 
 def lookup_ceiling(stack, ms_per_step, launches_per_step, mhz, launch="stack"):
@@ -317,7 +318,7 @@ def lookup_ceiling(stack, ms_per_step, launches_per_step, mhz, launch="stack"):
         first = 2 if (big and not fp16 and rest == 3) else 4 if (big and fp16 and rest in (5, 6)) else rest
         chunks += [first] + ([rest - first] if first < rest else [])
     assert len(chunks) == launches_per_step or launch != "stack"
-    entry_bytes = sum((2 if (fp16 and nb >= 2) else 4) * nvec(nb) for nb in chunks)
+    entry_bytes = sum((2 if (fp16 and nb >= 2) else 4) * nvec(nb) for nb in chunks) * (2 if stack.mu4 else 1)   # mu = 4: two lookups per byte
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     smem_peak = sms * 128 * mhz * 1e6 / 1e9                     # GB/s at 128 B/clk/SM
     smem_achieved = stack.lookups * entry_bytes / (ms_per_step * 1e-3) / 1e9
@@ -426,7 +427,7 @@ def summarize(stack, runner, total_ms, step_ms, steps, peak, per="linear"):
     n_lin = len(stack.linears)
     gbps = nbytes / (ms * 1e-3) / 1e9
     out = {"launch": runner.launch, "launches_per_step": runner.launches_per_step, "batch": stack.B,
-           "table_entries": "fp16" if stack.fp16 else "fp32", "GBps": round(gbps, 1), "frac_of_measured_peak": round(gbps / peak, 4),
+           "table_entries": "fp32, mu = 4" if stack.mu4 else "fp16" if stack.fp16 else "fp32", "GBps": round(gbps, 1), "frac_of_measured_peak": round(gbps / peak, 4),
            "frac_of_8TBps": round(gbps / 8000.0, 4), "us_per_linear": round(ms * 1e3 / n_lin, 3),
            "us_per_set": round(ms * 1e3 / stack.nl, 3), "ms_per_step": round(ms, 4),
            "step_ms_min": round(min(step_ms), 4), "copies_or_layers": stack.nl,
@@ -530,6 +531,40 @@ def section_variants(stream, peak, steps=10, warmup=3):
     return {"rows": rows, "how": "batch 1; linear = dependent calls chained on one stream (the per-operator latency the paper's "
             "table reports, its kernels on A100: 41-252 us), stack = the same copies as one plan (throughput); effective_tflops = "
             "2 M (N + n_sal) / t as in the paper"}
+
+
+def section_mu_sweep(stream, peak, steps=10, warmup=3):
+    """Sub-vector size mu = 4 against mu = 8 on the LLaMA-2-7B-shaped set in the 2b-g128 format at batch 1, 4 and 8
+    (the paper's sub-vector-size table): shared-memory bytes of the lookup tables a CTA holds, and throughput."""
+    import torch
+    lins = synth.LLAMA2_7B
+    names = [n for n, _, _ in lins]
+    rows = []
+    for B in (1, 4, 8):
+        def make_layers(B=B):
+            return [(synth.make_linear(9, li, M, N, 2, 0, 128), synth.make_activations(9, li, B, N)) for li, (_, M, N) in enumerate(lins)]
+
+        for mu in (4, 8):
+            st = build_rotation(make_layers, names, B, mu4=(mu == 4))
+            for launch in ("group", "stack"):
+                r = st.runner(launch, stream)
+                total, step_ms = r.time(steps, warmup)
+                row = summarize(st, r, total, step_ms, steps, peak)
+                nb = min(B, 4)                                               # vectors per launch (fp32 entries: chunks of four)
+                nvec = 1 if nb == 1 else 2 if nb == 2 else 4
+                rows.append({"mu": mu, "batch": B, "launch": launch, "launches_per_step": row["launches_per_step"],
+                             "table_KB_per_table_set": (2 * 16 if mu == 4 else 256) * 32 * 4 * nvec // 1024,
+                             "GBps": row["GBps"], "frac_of_measured_peak": row["frac_of_measured_peak"],
+                             "us_per_set": row["us_per_set"], "sets_per_s": round(1e6 / row["us_per_set"], 1),
+                             "lookup_ceiling_frac_at_1965MHz": row.get("lookup_ceiling_frac_at_1965MHz")})
+                del r
+            st.restore_formats()
+            del st
+            torch.cuda.empty_cache()
+    return {"rows": rows, "how": "fp32 table entries, the same packed layers for both sub-vector sizes; a table set serves 256 columns "
+            "(32 slots of 8 columns: mu = 8 one 256-entry table per slot, mu = 4 two 16-entry tables per slot) for the vectors of one launch "
+            "(chunks of up to four); group = one plan per dependency group, stack = one plan for all copies; sets_per_s = passes over "
+            "the seven linears of one decoder layer per second"}
 
 
 def section_rc_decomp(shapes=((4096, 4096), (8192, 8192)), K=2, T=10, g=128):
@@ -762,7 +797,7 @@ def main():
             "config": {"workload": f"config {args.config}: Llama-2-70B-shaped decode linear stack" if args.config == 4
                        else f"config {args.config}: {nl} independently seeded copies of the layer/set per step",
                        "layers": nl, "linears_per_step": len(stack.linears), "batch": B,
-                       "table_entries": "fp16" if stack.fp16 else "fp32",
+                       "table_entries": "fp32, mu = 4" if stack.mu4 else "fp16" if stack.fp16 else "fp32",
                        "Kb": 2, "Ks": 0 if args.config == 0 else 1, "salient_frac": 0.0 if args.config == 0 else 0.05,
                        "g": args.g or "N", "packed_bytes_resident": stack.packed_bytes, "algorithmic_bytes_per_step": bytes_per_step,
                        "l2": "inputs larger than L2 (weights streamed once per step)" if stack.packed_bytes > 4e8
@@ -834,6 +869,8 @@ def main():
             line["configs"] = section_configs(stack, stream, peak)
         if "variants" in sections:
             line["variants"] = section_variants(stream, peak)
+        if "mu_sweep" in sections:
+            line["mu_sweep"] = section_mu_sweep(stream, peak)
         if "rc_decomp" in sections:
             line["rc_decomp"] = section_rc_decomp()
         if "context" in sections:

@@ -150,14 +150,23 @@ int32_t fluxbin_weight_device(const fluxbin_weight_t *w);
  *                                  cancelling) sum.  Entries beyond the fp16 range (|sum of 8 fused activations|
  *                                  > 65504) become infinite and tiny ones lose bits below 6e-8: meant for
  *                                  normalised activations.
+ *   FLUXBIN_TABLES_FP32_MU4        sub-vectors of mu = 4 columns instead of 8 (the paper's sub-vector-size study,
+ *                                  "Impact of Sub-vector Size" and its table): every byte of weight bits indexes
+ *                                  two 16-entry fp32 tables (Eq. 14 with mu = 4) instead of one 256-entry table, so
+ *                                  the tables of 256 columns take 4 KB per batch vector instead of 32 KB and the
+ *                                  lookups and their additions double.  The packed layer is the same; results agree with the
+ *                                  mu = 8 path up to fp32 rounding order.  B runs in chunks of up to 4 vectors, and
+ *                                  a single vector uses these tables too.  Only for layers whose row-scale groups
+ *                                  are a multiple of 128 columns (FLUXBIN_ERR_UNSUPPORTED otherwise).
  *
- * A single vector (B == 1, or a trailing chunk of one) always uses fp32 entries.  The setting is read by
+ * With the first two formats a single vector (B == 1, or a trailing chunk of one) always uses fp32 entries of mu = 8.  The setting is read by
  * fluxbin_workspace_size, fluxbin_num_launches, fluxbin_linear and fluxbin_plan_create (all members of a plan
  * must agree, else FLUXBIN_ERR_UNSUPPORTED); change it only between those calls, and size workspaces after
  * it.  Returns FLUXBIN_ERR_RANGE for an unknown format.  fluxbin_get_table_format: the setting, -1 on NULL.
  */
 #define FLUXBIN_TABLES_FP32 0
 #define FLUXBIN_TABLES_FP16 1
+#define FLUXBIN_TABLES_FP32_MU4 2
 fluxbin_status_t fluxbin_set_table_format(fluxbin_weight_t *w, int32_t format);
 int32_t fluxbin_get_table_format(const fluxbin_weight_t *w);
 

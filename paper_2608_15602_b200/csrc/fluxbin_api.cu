@@ -192,7 +192,10 @@ extern "C" int32_t fluxbin_num_table_sets(const fluxbin_weight_t *w) { return w 
 extern "C" fluxbin_status_t fluxbin_set_table_format(fluxbin_weight_t *w, int32_t format)
 {
     if (!w) return FLUXBIN_ERR_NULL;
-    if (format != FLUXBIN_TABLES_FP32 && format != FLUXBIN_TABLES_FP16) return FLUXBIN_ERR_RANGE;
+    if (format != FLUXBIN_TABLES_FP32 && format != FLUXBIN_TABLES_FP16 && format != FLUXBIN_TABLES_FP32_MU4) return FLUXBIN_ERR_RANGE;
+    // the mu = 4 kernels exist for row-scale groups of a multiple of 128 columns (the configurations of the paper's
+    // sub-vector-size study)
+    if (format == FLUXBIN_TABLES_FP32_MU4 && w->h.sps[0] != 16) return FLUXBIN_ERR_UNSUPPORTED;
     w->table_format = format;
     return FLUXBIN_OK;
 }
@@ -205,7 +208,11 @@ extern "C" int32_t fluxbin_get_table_format(const fluxbin_weight_t *w) { return 
 // entry.  A single vector always uses fp32 entries (nothing to share a word with).
 static int chunk_size(int fmt) { return fmt == FLUXBIN_TABLES_FP16 ? 8 : 4; }
 static int nvec_for(int nb) { return nb == 1 ? 1 : nb == 2 ? 2 : nb <= 4 ? 4 : 8; }
-static int mode_for(int nb, int fmt) { return (fmt == FLUXBIN_TABLES_FP16 && nb >= 2) ? 16 + nvec_for(nb) : nvec_for(nb); }
+static int mode_for(int nb, int fmt)
+{
+    if (fmt == FLUXBIN_TABLES_FP32_MU4) return 32 + nvec_for(nb);
+    return (fmt == FLUXBIN_TABLES_FP16 && nb >= 2) ? 16 + nvec_for(nb) : nvec_for(nb);
+}
 static int ws_bt(int B, int fmt) { return nvec_for(B < chunk_size(fmt) ? B : chunk_size(fmt)); }   // accumulator rows per layer
 
 // The chunks of a batch of B vectors, largest first: full chunks, then the rest.  A rest that would run with
@@ -272,12 +279,12 @@ extern "C" fluxbin_status_t fluxbin_workspace_init(void *d_workspace, size_t byt
 
 // ---- the layer ------------------------------------------------------------------------------------
 
-// The kernel instantiation for a launch mode (1, 2, 4 vectors with fp32 tables, 16 + (2, 4, 8) with fp16 tables),
-// a row-scale format class (sub-vectors per scale segment of the global / salient region) and the number of
+// The kernel instantiation for a launch mode (1, 2, 4 vectors with fp32 tables, 16 + (2, 4, 8) with fp16 tables,
+// 32 + (1, 2, 4) with fp32 tables of mu = 4 sub-vectors), a row-scale format class (sub-vectors per scale segment of the global / salient region) and the number of
 // pairs walked per row block (2 exists for the modes with 4-byte table entries: 1 and 16 + 2).
 template <int S0, int S1, int BT> static const void *kernel_of(int np)
 {
-    if constexpr (fbk::geom(BT) == 1) {
+    if constexpr (fbk::geom(BT) == 1 && !fbk::mu4(BT)) {
         if (np == 2) return (const void *)fbk::fluxbin_linear_kernel<S0, S1, BT, 2>;
     }
     return (const void *)fbk::fluxbin_linear_kernel<S0, S1, BT, 1>;
@@ -289,9 +296,18 @@ template <int BT> static const void *kernel_of_bt(int s0, int s1, int np)
     if (s0 == 8) return kernel_of<8, 1, BT>(np);
     return kernel_of<4, 1, BT>(np);
 }
+template <int BT> static const void *kernel_of_mu4(int s0, int s1)
+{
+    if (s0 == 16 && s1 == 16) return kernel_of<16, 16, BT>(1);
+    if (s0 == 16) return kernel_of<16, 1, BT>(1);
+    return nullptr;                     // fluxbin_set_table_format refuses the other classes
+}
 static const void *kernel_for(int mode, int s0, int s1, int np)
 {
     switch (mode) {
+    case 32 + 1: return kernel_of_mu4<32 + 1>(s0, s1);
+    case 32 + 2: return kernel_of_mu4<32 + 2>(s0, s1);
+    case 32 + 4: return kernel_of_mu4<32 + 4>(s0, s1);
     case 1: return kernel_of_bt<1>(s0, s1, np);
     case 2: return kernel_of_bt<2>(s0, s1, np);
     case 4: return kernel_of_bt<4>(s0, s1, np);
@@ -301,7 +317,12 @@ static const void *kernel_for(int mode, int s0, int s1, int np)
     }
     return nullptr;
 }
-static int mode_index(int mode) { return mode == 1 ? 0 : mode == 2 ? 1 : mode == 4 ? 2 : mode == 16 + 2 ? 3 : mode == 16 + 4 ? 4 : 5; }
+constexpr int kNumModes = 9;
+static int mode_index(int mode)
+{
+    if (mode >= 32) return mode == 32 + 1 ? 6 : mode == 32 + 2 ? 7 : 8;
+    return mode == 1 ? 0 : mode == 2 ? 1 : mode == 4 ? 2 : mode == 16 + 2 ? 3 : mode == 16 + 4 ? 4 : 5;
+}
 static int class_index(int s0, int s1) { return (s0 == 16 && s1 == 16) ? 0 : s0 == 16 ? 1 : s0 == 8 ? 2 : 3; }
 static int threads_for(int mode) { return fbk::geom(mode) == 4 ? 512 : 256; }
 static size_t smem_for(int mode)      // the scratch beside the tables grows with the vectors of the mode
@@ -313,18 +334,23 @@ static size_t smem_for(int mode)      // the scratch beside the tables grows wit
     case 16 + 2: return fbk::smem_bytes<16 + 2>();
     case 16 + 4: return fbk::smem_bytes<16 + 4>();
     case 16 + 8: return fbk::smem_bytes<16 + 8>();
+    case 32 + 1: return fbk::smem_bytes<32 + 1>();
+    case 32 + 2: return fbk::smem_bytes<32 + 2>();
+    case 32 + 4: return fbk::smem_bytes<32 + 4>();
     }
     return 0;
 }
 
 fluxbin_status_t fb::opt_in_all_kernels()
 {
-    static const int modes[6] = {1, 2, 4, 16 + 2, 16 + 4, 16 + 8};
+    static const int modes[kNumModes] = {1, 2, 4, 16 + 2, 16 + 4, 16 + 8, 32 + 1, 32 + 2, 32 + 4};
     static const int cls[4][2] = {{16, 16}, {16, 1}, {8, 1}, {4, 1}};
     for (int m : modes)
         for (auto &c : cls)
-            for (int np = 1; np <= (fbk::geom(m) == 1 ? 2 : 1); ++np)
-                FB_CUDA(cudaFuncSetAttribute(kernel_for(m, c[0], c[1], np), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_for(m)));
+            for (int np = 1; np <= ((fbk::geom(m) == 1 && !fbk::mu4(m)) ? 2 : 1); ++np) {
+                const void *k = kernel_for(m, c[0], c[1], np);
+                if (k) FB_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_for(m)));
+            }
     return FLUXBIN_OK;
 }
 
@@ -337,8 +363,12 @@ constexpr int kBuildCost = 44;
 // a build (more vectors per entry, conversions) does not: measured 44 / 66 / 88 / 132 -> 3.29 / 3.47 / 3.51 / 3.46
 // TB/s at batch 4 and 1.73 / 1.81 / 1.81 / 1.81 at batch 8.  (With fp32 entries, batch 2 and 4: no effect.)
 constexpr int kBuildCostHalfWide = 88;
+// mu = 4: a table set has 32 rows of entries instead of 256 and an item twice the lookups, so a build is worth far
+// fewer items (the dependent loads and the two barriers remain).
+constexpr int kBuildCostMu4 = 12;
 static int build_cost_for(int mode)
 {
+    if (fbk::mu4(mode)) return kBuildCostMu4;
     return (mode == 16 + 4 || mode == 16 + 8) ? kBuildCostHalfWide : kBuildCost;    // two vectors in fp16 entries: 36 / 44 / 56 / 66 all within 1 %
 }
 // The reduction epilogue a CTA runs when it leaves an entry (fence, tickets, read-back of the tiles it
@@ -397,7 +427,7 @@ static cudaError_t launch_shape(int dev, int mode, int s0, int s1, long long tot
                                 long long couple_cost, bool allow_dynamic, LaunchShape *out)
 {
     // resident CTAs per SM of an instantiation, per device (0 = not asked yet; racing threads store the same value)
-    static std::atomic<int> occ_of[kMaxDevices][6][4];
+    static std::atomic<int> occ_of[kMaxDevices][kNumModes][4];
     std::atomic<int> &slot = occ_of[dev][mode_index(mode)][class_index(s0, s1)];
     int occ = slot.load(std::memory_order_relaxed);
     if (occ == 0) {
@@ -425,7 +455,7 @@ static cudaError_t launch_shape(int dev, int mode, int s0, int s1, long long tot
     out->grid = (int)grid;
     // two pairs per row block when every layer allows it (couple_cost > 0: even pair counts everywhere) and a
     // CTA's share is large enough to pay for the second table build
-    out->np = (fbk::geom(mode) == 1 && couple_cost > 0 && out->static_cost / grid >= kCoupleMinShare) ? 2 : 1;
+    out->np = (fbk::geom(mode) == 1 && !fbk::mu4(mode) && couple_cost > 0 && out->static_cost / grid >= kCoupleMinShare) ? 2 : 1;
     return cudaSuccess;
 }
 

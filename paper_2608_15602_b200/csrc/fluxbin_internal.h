@@ -49,8 +49,8 @@ struct fluxbin_weight {
     int num_sms;
     int tile_rb;  // row blocks (of 32 rows) per arrival-counter tile
     int ntiles;
-    int table_format;   // FLUXBIN_TABLES_FP32 / _FP16: how batched launches (B >= 2) hold their table entries
-    mutable std::atomic<fb::SingleLaunch *> single[6];   // per launch mode, made on first use, owned by the handle
+    int table_format;   // FLUXBIN_TABLES_FP32 / _FP16 / _FP32_MU4: how launches hold their table entries
+    mutable std::atomic<fb::SingleLaunch *> single[9];   // per launch mode, made on first use, owned by the handle
 };
 
 #endif

@@ -41,10 +41,14 @@ namespace fbk {
 // The template parameter BT of everything below is a launch MODE: 1, 2 or 4 = that many batch vectors per
 // launch with fp32 table entries (the precision the paper's shared-memory model states); 16 + n (n = 2, 4, 8)
 // = n batch vectors with fp16 table entries, two vectors per 32-bit word -- half the shared-memory bytes per
-// lookup, which is what bounds the batched path.  Sums still accumulate in fp32.
+// lookup, which is what bounds the batched path.  Sums still accumulate in fp32.  32 + n (n = 1, 2, 4) = n batch
+// vectors with fp32 entries and sub-vectors of mu = 4 columns (the paper's sub-vector-size study): every byte of
+// weight bits then indexes two 16-entry tables (its low and its high four columns) instead of one 256-entry table,
+// so a table set (256 columns) shrinks from 32 KB to 4 KB per vector and the lookups double.  The packed layer is the same.
 __host__ __device__ constexpr int nvec(int BT) { return BT & 15; }               // batch vectors per launch
-__host__ __device__ constexpr bool half_tables(int BT) { return BT >= 16; }
-__host__ __device__ constexpr int geom(int BT) { return half_tables(BT) ? nvec(BT) / 2 : BT; }   // 32-bit words per table entry
+__host__ __device__ constexpr bool half_tables(int BT) { return (BT & 16) != 0; }
+__host__ __device__ constexpr bool mu4(int BT) { return (BT & 32) != 0; }
+__host__ __device__ constexpr int geom(int BT) { return half_tables(BT) ? nvec(BT) / 2 : nvec(BT); }   // 32-bit words per table entry
 
 // Threads per CTA: 8 warps with 4- or 8-byte entries (3 or 2 CTAs per SM); with 16-byte entries the
 // tables fill 128 KB, one CTA owns the SM and runs 16 warps.
@@ -159,13 +163,15 @@ __device__ __forceinline__ uint32_t ldg_stream_u32(const void *p)
 template <int BT> struct Vec { float v[nvec(BT)]; };
 
 // HALF selects the table set inside the 256-byte p-rows: slots 0..31 or (4-byte entries only) slots 32..63.
-template <int BT, int HALF> __device__ __forceinline__ Vec<BT> lds_entry(uint32_t addr)
+// HI (mu = 4 only) selects the tables of a byte's high four columns: p-rows 16..31 instead of 0..15.
+template <int BT, int HALF, int HI = 0> __device__ __forceinline__ Vec<BT> lds_entry(uint32_t addr)
 {
     Vec<BT> r;
-    // addr is an offset from the table base; base and half ride in the immediate
-    if constexpr (BT == 1) asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(r.v[0]) : "r"(addr), "n"(kTabBase + HALF * 128));
-    else if constexpr (BT == 2) asm volatile("ld.shared.v2.f32 {%0,%1}, [%2+%3];" : "=f"(r.v[0]), "=f"(r.v[1]) : "r"(addr), "n"(kTabBase));
-    else asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4+%5];" : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3]) : "r"(addr), "n"(kTabBase));
+    // addr is an offset from the table base; base, half and row offset ride in the immediate
+    constexpr uint32_t kBase = kTabBase + HI * (16u << 8);
+    if constexpr (geom(BT) == 1) asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(r.v[0]) : "r"(addr), "n"(kBase + HALF * 128));
+    else if constexpr (geom(BT) == 2) asm volatile("ld.shared.v2.f32 {%0,%1}, [%2+%3];" : "=f"(r.v[0]), "=f"(r.v[1]) : "r"(addr), "n"(kBase));
+    else asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4+%5];" : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3]) : "r"(addr), "n"(kBase));
     return r;
 }
 
@@ -311,6 +317,32 @@ __device__ __forceinline__ void enumerate_tables(const float *abuf, uint32_t hal
     const int tid = threadIdx.x;
     constexpr int NV = nvec(BT);
     const int lane = tid & 31, warp = tid >> 5;
+    if constexpr (mu4(BT)) {
+        // mu = 4: two 16-entry tables per slot -- p-rows 0..15 index columns 0..3 of the slot's eight, p-rows 16..31
+        // columns 4..7 (Eq. 14 with mu = 4); a warp fills whole p-rows, one entry (all vectors) per lane and row.
+        static_assert(!half_tables(BT) && NV <= 4, "mu = 4 runs with fp32 entries");
+        float a[8][NV];
+#pragma unroll
+        for (int n = 0; n < 8; ++n)
+#pragma unroll
+            for (int b = 0; b < NV; ++b) a[n][b] = abuf[abuf_index<BT>(lane, n, b)];
+#pragma unroll 1
+        for (int p = warp; p < 32; p += Cfg<BT>::kWarps) {
+            float v[NV];
+#pragma unroll
+            for (int b = 0; b < NV; ++b) {
+                float sum = 0.f;
+#pragma unroll
+                for (int n = 3; n >= 0; --n) {
+                    const float an = (p & 16) ? a[4 + n][b] : a[n][b];
+                    sum += ((p >> n) & 1) ? an : -an;
+                }
+                v[b] = sum;
+            }
+            sts_entry<NV>(half_off | TabCfg<BT>::lane_const((uint32_t)lane) | ((uint32_t)p << 8), v);
+        }
+        return;
+    }
     // EB entries at a time: the high index bits fix a base value, the low LB bits are enumerated by
     // doubling (entry p | 2^n = entry p + 2 a_n), one add per entry.  Up to four batch vectors of an entry are
     // stored with one instruction (with four, blocks of 8 entries keep the registers in bounds).  With eight
@@ -480,6 +512,10 @@ template <> struct LaneAddr<4> {
 template <> struct LaneAddr<16 + 2> : LaneAddr<1> {};
 template <> struct LaneAddr<16 + 4> : LaneAddr<2> {};
 template <> struct LaneAddr<16 + 8> : LaneAddr<4> {};
+// mu = 4: the same slots, the table index is a nibble of the weight byte (masked out before the PRMT)
+template <> struct LaneAddr<32 + 1> : LaneAddr<1> {};
+template <> struct LaneAddr<32 + 2> : LaneAddr<2> {};
+template <> struct LaneAddr<32 + 4> : LaneAddr<4> {};
 
 // Two alternating partial sums per vector shorten the dependency chain of a segment's adds; with four or more
 // vectors the adds of one lookup already space out each vector's chain (+1-5 % without the split there).
@@ -503,6 +539,18 @@ __device__ __forceinline__ void compute_item(const ItemRegs<SPS, W> &r, const La
 #pragma unroll
             for (int q = 0; q < SPS; ++q) {
                 const int s = j * SPS + q;
+                if constexpr (mu4(BT)) {
+                    // the byte's low and high four columns: two lookups (the masks are shared by the four steps of a word)
+                    const uint32_t lo = w[s >> 2] & 0x0f0f0f0fu, hi = (w[s >> 2] >> 4) & 0x0f0f0f0fu;
+                    const Vec<BT> e0 = lds_entry<BT, HALF, 0>(la.addr(s, lo));
+                    const Vec<BT> e1 = lds_entry<BT, HALF, 1>(la.addr(s, hi));
+#pragma unroll
+                    for (int b = 0; b < NV; ++b) {
+                        s0[b] += e0.v[b];
+                        if (NV < kSplitBelowVectors) s1[b] += e1.v[b]; else s0[b] += e1.v[b];
+                    }
+                    continue;
+                }
                 const uint32_t addr = la.addr(s, w[s >> 2]);
                 if constexpr (half_tables(BT)) {
                     uint32_t e[geom(BT)];
@@ -895,7 +943,9 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
     LinearEntry *Es = (LinearEntry *)(range + 8);  // the current entry, copied once (128 bytes)
     static_assert(sizeof(LinearEntry) == 128, "entry copy below moves 32 words");
     static_assert(NP == 1 || geom(BT) == 1, "two table sets side by side need 4-byte table entries");
-    static_assert(BT == 1 || BT == 2 || BT == 4 || BT == 16 + 2 || BT == 16 + 4 || BT == 16 + 8, "launch mode");
+    static_assert(BT == 1 || BT == 2 || BT == 4 || BT == 16 + 2 || BT == 16 + 4 || BT == 16 + 8 || BT == 32 + 1 || BT == 32 + 2 ||
+                  BT == 32 + 4, "launch mode");
+    static_assert(NP == 1 || !mu4(BT), "mu = 4 walks one pair per row block");
     const int tid = threadIdx.x;
     FB_TRACE_AT(0);
     FB_TRACE_ZERO();

@@ -183,7 +183,7 @@ def unpack_host(buf: np.ndarray):
     return out
 
 
-TABLES_FP32, TABLES_FP16 = 0, 1
+TABLES_FP32, TABLES_FP16, TABLES_FP32_MU4 = 0, 1, 2
 
 
 class Weight:
@@ -218,7 +218,8 @@ class Weight:
         return int(_lib().fluxbin_num_launches(self.handle, B))
 
     def set_table_format(self, fmt: int) -> None:
-        """TABLES_FP32 (default) or TABLES_FP16 entries for batched launches; size workspaces afterwards."""
+        """TABLES_FP32 (default) or TABLES_FP16 entries for batched launches, or TABLES_FP32_MU4 (16-entry tables of
+        sub-vectors of four columns, every launch); size workspaces afterwards."""
         _check(_lib().fluxbin_set_table_format(self.handle, fmt), "fluxbin_set_table_format")
 
     def table_format(self) -> int:
