@@ -275,7 +275,7 @@ def generate_members(jobs, make, fp16_tables=False):
     return members
 
 
-def build_config_stack(config, nl, B, g=128, fp16_tables=False):
+def build_config_stack(config, nl, B, g=128, fp16_tables=False, mu4=False):
     """Workload `config` with nl independently seeded layers / sets (config 4: the layers of the stack)."""
     lins, _ = synth.config_linears(config)
     jobs = [(layer, li) for layer in range(nl) for li in range(len(lins))]
@@ -284,7 +284,7 @@ def build_config_stack(config, nl, B, g=128, fp16_tables=False):
         layer, li = job
         return synth.make_config_linear(config, layer, li, g=(g or lins[li][2])), synth.make_config_activations(config, layer, li, B)
 
-    return Stack(generate_members(jobs, make, fp16_tables), [n for n, _, _ in lins], nl, B, fp16_tables)
+    return Stack(generate_members(jobs, make, fp16_tables), [n for n, _, _ in lins], nl, B, fp16_tables, mu4)
 
 
 def build_rotation(make_layers, names, B, fp16_tables=False, mu4=False):
@@ -623,6 +623,8 @@ def main():
     ap.add_argument("--batch", type=int, default=1)
     ap.add_argument("--fp16-tables", action="store_true",
                     help="batched launches keep their lookup tables in fp16 (fluxbin_set_table_format); no effect at batch 1")
+    ap.add_argument("--mu", type=int, default=8, choices=[4, 8],
+                    help="sub-vector size: 8 (default) or 4 (fluxbin_set_table_format FLUXBIN_TABLES_FP32_MU4: 16-entry tables, twice the lookups)")
     ap.add_argument("--g", type=int, default=128, help="columns per row-scale group; 0 = one scale per row (g = N)")
     ap.add_argument("--no-graph", action="store_true", help="plain launches instead of a CUDA graph replay")
     ap.add_argument("--launch", default="stack", choices=["linear", "group", "layer", "stack"],
@@ -659,7 +661,7 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
-    default_workload = (args.config == 4 and args.layers is None and args.batch == 1 and args.g == 128 and args.launch == "stack")
+    default_workload = (args.config == 4 and args.layers is None and args.batch == 1 and args.g == 128 and args.launch == "stack" and args.mu == 8)
     if args.sections is None:
         sections = list(ALL_SECTIONS) if (default_workload and world == 1) else ["context", "cpu_baseline"]
     else:
@@ -691,7 +693,7 @@ def main():
 
     # ---- build the resident stack: generate (threads) -> pack on the host -> upload ----------------
     t_setup = time.perf_counter()
-    stack = build_config_stack(args.config, nl, B, g=args.g, fp16_tables=args.fp16_tables)
+    stack = build_config_stack(args.config, nl, B, g=args.g, fp16_tables=args.fp16_tables, mu4=(args.mu == 4))
     setup_s = time.perf_counter() - t_setup
     stream = torch.cuda.Stream()
     runner = stack.runner(args.launch, stream, graph=not args.no_graph)
