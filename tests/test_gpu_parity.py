@@ -182,6 +182,17 @@ def test_llama70b_shapes_batch1(fb, li):
     check(run(fb, L, x), oracle.linear_direct(L, x), f"70B linear {li}", L, x)
 
 
+@pytest.mark.parametrize("B", [1, 3])
+def test_widest_layer(fb, B):
+    """N = 65536, the widest layer the 16-bit column indices of the packed column tables allow: 512 global units
+    (the longest K split there is) and salient columns at both ends of the index range."""
+    N = 65536
+    idx = np.array([0, 1, 127, 128, 40000, 65407, 65408, 65534, 65535], dtype=np.int32)
+    L = synth.make_linear(91, 5, 70, N, 1, 2, 128, idx)
+    x = synth.make_activations(91, 6, B, N)
+    check(run(fb, L, x), oracle.linear_direct(L, x), f"N = 65536, B = {B}", L, x)
+
+
 def test_fp16_output_is_rounded_fp32_result(fb):
     L = synth.make_config_linear(1, 0, 0)
     x = synth.make_config_activations(1, 0, 0, 2)

@@ -263,7 +263,7 @@ def test_salient_collect_gathers_the_padded_refinement(fb):
 
 PACK_CASES = [(1, 32, 1, 0, 32, 0), (5, 128, 2, 1, 32, 7), (33, 384, 3, 2, 128, 40), (100, 256, 1, 1, 256, 19),
               (257, 1024, 2, 1, 128, 51), (65, 640, 2, 1, 128, 640), (127, 128, 4, 4, 64, 128), (600, 2048, 2, 2, 128, 128),
-              (1000, 512, 2, 1, 512, 1), (31, 256, 2, 2, 64, 9)]
+              (1000, 512, 2, 1, 512, 1), (31, 256, 2, 2, 64, 9), (40, 65536, 1, 1, 128, 300)]      # last: the widest layer
 
 
 @pytest.mark.parametrize("M,N,Kb,Ks,g,n_sal", PACK_CASES)

@@ -91,6 +91,22 @@ def test_packed_layout_walk_matches_oracle(M, N, Kb, Ks, g, n_sal):
     assert np.all(np.abs(got - want) <= 1e-12 * bound + 1e-300)
 
 
+def test_widest_layer_layout_walk():
+    """N = 65536 (the limit of the 16-bit column indices), salient columns at both ends of the index range."""
+    N = 65536
+    idx = np.array([0, 1, 127, 128, 40000, 65407, 65408, 65534, 65535], dtype=np.int32)
+    L = synth.make_linear(91, 5, 70, N, 1, 2, 128, idx)
+    x = synth.make_activations(91, 6, 2, N)
+    want = oracle.linear_direct(L, x)
+    buf = fluxbin.pack_host(L)
+    got = emulate_linear(buf, x)
+    bound = np.abs(x.view(np.float16).astype(np.float64)) @ np.abs(oracle.dense_weight(L)).T
+    assert np.all(np.abs(got - want) <= 1e-12 * bound + 1e-300)
+    U = fluxbin.unpack_host(buf)
+    for f in FIELDS:
+        assert np.array_equal(getattr(L, f), getattr(U, f)), f
+
+
 def test_validation_statuses():
     L = layer(1, 8, 128, 2, 1, 32, 5)
     assert fluxbin.validate(L) == 0
