@@ -410,11 +410,13 @@ static long long entry_cost(const FbHeader &h, int sps1, int build_cost)
 }
 
 // The two-pairs-per-row-block kernel pays two table builds per run of rows but has the better row loop (one
-// reduction per two items, loads requested half an item earlier).  Measured on B200 (batch 1): it wins as soon
-// as a CTA's share is worth about 30 plain items (cost 60) -- +11 % with one launch per 70B linear, +15 % with
-// one per dependency group, +21 % with one per layer -- and loses below that (4096 x 4096 alone, 18 items per
-// CTA: 6.7 -> 7.7 us per call).
-constexpr long long kCoupleMinShare = 60;
+// reduction per two items, loads requested half an item earlier).  Measured on B200 (batch 1) against the one-pair
+// kernel with its first item in flight during the build: it wins once a CTA's share is worth about 200 to 270 plain
+// items (cost 400 to 540: the {gate, up} launch of a 70B-shaped layer, one launch per layer, one plan for a stack)
+// and loses below that -- with the threshold at 60 instead of 400 the 7B-shaped set ran 7 % slower with one launch
+// per dependency group (5.43 against 5.05 us per linear), the 13B-shaped set 5 %, the 70B-shaped layers 2 %; with
+// it at 1000 the 70B-shaped groups lose 1.4 %, at 3000 one launch per layer loses 7 %.
+constexpr long long kCoupleMinShare = 400;
 
 // How a launch is cut: grid size, the statically dealt part of the cost line, the number of shares, and
 // how many pairs the kernel walks per row block (2: the two-pairs-per-row-block kernel).

@@ -182,7 +182,7 @@ def test_long_plan_of_two_vectors_runs_the_two_pair_kernel(fb):
     enough work per CTA runs the variant that keeps two table sets resident (g = 128 and g = 64 formats)."""
     for g, shapes in ((128, [(256, 4096), (250, 4096), (512, 4096), (96, 8192)]), (64, [(300, 2048), (512, 4096)])):
         members, cases = [], []
-        for i in range(72):
+        for i in range(120):
             M, N = shapes[i % len(shapes)]
             L = layer_of(700 + i, M, N, 2, 1, g, int(round(0.05 * N)))
             x = synth.make_activations(19, i, 2, N)

@@ -100,7 +100,7 @@ def test_long_plan_runs_the_two_pair_kernel(fb):
     plan of the same members launches the one-pair variant.  Both must match the oracle on every output."""
     shapes = [(256, 4096), (250, 4096), (512, 4096), (96, 8192)]
     members, wants = [], []
-    for i in range(72):
+    for i in range(120):
         M, N = shapes[i % len(shapes)]
         n_sal = int(round(0.05 * N))
         L = layer_of(500 + i, M, N, 2, 1, 128, n_sal)
