@@ -251,7 +251,8 @@ fluxbin_status_t fluxbin_debug_tables(const fluxbin_weight_t *w, const uint16_t 
  * `nshares - grid` small ones drawn dynamically from the last (100 - static_percent) % of the cost.
  *
  *   h_headers            HOST array of n pointers, each to the first 256 bytes of a packed layer
- *   mode                 launch mode: 1, 2, 4 vectors with fp32 table entries, 16 + (2, 4, 8) with fp16 entries
+ *   mode                 launch mode: 1, 2, 4 vectors with fp32 table entries, 16 + (2, 4, 8) with fp16 entries,
+ *                        32 + (1, 2, 4) with fp32 entries of mu = 4 tables
  *   pairs_per_row_block  1 or 2 (2 needs an even number of global pairs in every layer)
  *   out_cuts             HOST int32 [nshares + 1][2]: {layer, work item} where share s begins; the last is {n, 0}
  *   out_work_items       HOST int32 [n] or NULL: work items of each layer
@@ -335,7 +336,7 @@ int32_t fluxbin_plan_num_launches(const fluxbin_plan_t *plan);
 
 /* Introspection: how many table sets (pairs of 16-sub-vector units) the kernel of the plan's first launch keeps
  * resident per row block -- 2 when every member has an even number of global pairs, the table entries are 4 bytes
- * (batch 1, or batch 2 with fp16 entries) and each CTA's share of the plan is worth at least about 30 items (then
+ * (batch 1, or batch 2 with fp16 entries) and each CTA's share of the plan is worth at least about 200 items (then
  * two pairs' row sums share one reduction, stage (iii)), else 1.
  * Both variants compute the same sums (Eq. 15) in a different order.  -1 on NULL. */
 int32_t fluxbin_plan_pairs_per_row_block(const fluxbin_plan_t *plan);

@@ -986,8 +986,8 @@ fluxbin_linear_kernel(const __grid_constant__ LaunchParams P)
         // With NP == 2 region 0 is walked two pairs at a time, their table sets side by side (4-byte entries,
         // every entry with an even number of global pairs): a "work pair" is then a couple of pairs, a
         // work row block their two items.
-        // (NP is a kernel template parameter: the host picks the two-pair kernel unless a CTA's share is
-        // only a handful of items, where building two table sets per run costs more than the better row
+        // (NP is a kernel template parameter: the host picks the two-pair kernel when a CTA's share is worth
+        // a couple of hundred items; below that building two table sets per run costs more than the better row
         // loop gains.  Deciding it at run time was measured slower than either variant: both row loops in
         // one kernel cost registers.)
         const int wp0 = E.npairs[0] / NP;
